@@ -1,0 +1,158 @@
+/*
+ * GranQ CPU oracle (TEST INFRASTRUCTURE; see granq_oracle.h).
+ *
+ * Build: gcc -O2 -std=c11 -ffp-contract=off -fno-fast-math -shared -fPIC
+ * Everything is `float`: no double intermediates, no fused multiply-add, default
+ * rounding mode (round-to-nearest-even).  Loops are the definitions written out.
+ */
+#include "granq_oracle.h"
+
+#include <math.h>
+#include <stddef.h>
+#include <string.h>
+
+/* ---- bf16 <-> fp32 (bit patterns) ------------------------------------------------ */
+
+static float bf16_widen(uint16_t h) {
+    uint32_t u = (uint32_t)h << 16;
+    float f;
+    memcpy(&f, &u, 4);
+    return f;
+}
+
+/* round-to-nearest-even on the 16 discarded mantissa bits; inputs are finite */
+static uint16_t bf16_narrow(float f) {
+    uint32_t u;
+    memcpy(&u, &f, 4);
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7FFFu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+static float load_elem(const void* p, int dtype, int64_t i) {
+    if (dtype == GRANQ_ORACLE_BF16) return bf16_widen(((const uint16_t*)p)[i]);
+    return ((const float*)p)[i];
+}
+
+static void store_elem(void* p, int dtype, int64_t i, float v) {
+    if (dtype == GRANQ_ORACLE_BF16) ((uint16_t*)p)[i] = bf16_narrow(v);
+    else ((float*)p)[i] = v;
+}
+
+/* ---- geometry: activation decomposition (Eq. 4) ---------------------------------- */
+
+typedef struct { int64_t outer, C, inner; } geom_t;
+
+static int make_geom(const int64_t dims[4], int axis, int mode, geom_t* g) {
+    if (!dims || axis < 0 || axis > 3 || mode < 0 || mode > 2) return -1;
+    for (int d = 0; d < 4; ++d) if (dims[d] <= 0) return -1;
+    g->outer = 1; g->inner = 1;
+    for (int d = 0; d < axis; ++d) g->outer *= dims[d];
+    for (int d = axis + 1; d < 4; ++d) g->inner *= dims[d];
+    g->C = dims[axis];
+    return 0;
+}
+
+/* group of the element at (o, c, *) */
+static int64_t group_of(const geom_t* g, int mode, int64_t o, int64_t c) {
+    if (mode == GRANQ_ORACLE_GROUP_CHANNEL) return c;
+    if (mode == GRANQ_ORACLE_GROUP_SAMPLE_CHANNEL) return o * g->C + c;
+    return 0;
+}
+
+int64_t granq_oracle_num_groups(const int64_t dims[4], int channel_axis, int group_mode) {
+    geom_t g;
+    if (make_geom(dims, channel_axis, group_mode, &g)) return -1;
+    if (group_mode == GRANQ_ORACLE_GROUP_CHANNEL) return g.C;
+    if (group_mode == GRANQ_ORACLE_GROUP_SAMPLE_CHANNEL) return g.outer * g.C;
+    return 1;
+}
+
+/* ---- Eq. 4: per-group min / max --------------------------------------------------- */
+
+int granq_oracle_range(const void* x, int dtype, const int64_t dims[4], int channel_axis,
+                       int group_mode, float* lo, float* hi) {
+    geom_t g;
+    if (!x || !lo || !hi || make_geom(dims, channel_axis, group_mode, &g)) return -1;
+    int64_t G = granq_oracle_num_groups(dims, channel_axis, group_mode);
+    for (int64_t k = 0; k < G; ++k) { lo[k] = INFINITY; hi[k] = -INFINITY; }
+    for (int64_t o = 0; o < g.outer; ++o)
+        for (int64_t c = 0; c < g.C; ++c) {
+            int64_t k = group_of(&g, group_mode, o, c);
+            for (int64_t i = 0; i < g.inner; ++i) {
+                float v = load_elem(x, dtype, (o * g.C + c) * g.inner + i);
+                if (!isfinite(v)) return -2;
+                if (v < lo[k]) lo[k] = v;
+                if (v > hi[k]) hi[k] = v;
+            }
+        }
+    for (int64_t k = 0; k < G; ++k) { lo[k] += 0.0f; hi[k] += 0.0f; } /* -0 -> +0 */
+    return 0;
+}
+
+/* ---- Eq. 2 / Eq. 5: scale and zero-point ------------------------------------------ */
+
+static void scale_zero(float lo, float hi, int bits, float* s_out, float* z_out) {
+    float qmax = (float)((1 << bits) - 1);
+    float s = (hi - lo) / qmax;      /* one subtract, one true division */
+    if (!(s >= 1e-8f)) s = 1e-8f;    /* degenerate-range floor */
+    float z = rintf((-lo) / s);      /* true division, round-half-to-even */
+    *s_out = s;
+    *z_out = z + 0.0f;               /* -0 -> +0 */
+}
+
+int granq_oracle_params(const float* lo, const float* hi, int64_t G, int bits, float* s, float* z) {
+    if (!lo || !hi || !s || !z || G <= 0 || bits < 1 || bits > 8) return -1;
+    for (int64_t k = 0; k < G; ++k) scale_zero(lo[k], hi[k], bits, &s[k], &z[k]);
+    return 0;
+}
+
+/* ---- Eq. 1, clamp, Eq. 6, STE ------------------------------------------------------ */
+
+int granq_oracle_fakequant(const void* x, const void* gy, int dtype, const int64_t dims[4],
+                           int channel_axis, int group_mode, int bits,
+                           const float* lo, const float* hi,
+                           void* y, void* gx, uint8_t* codes, uint8_t* mask, float* s, float* z) {
+    geom_t g;
+    if (!x || !y || !lo || !hi || bits < 1 || bits > 8) return -1;
+    if ((gy == NULL) != (gx == NULL)) return -1;
+    if (make_geom(dims, channel_axis, group_mode, &g)) return -1;
+    const float qmax = (float)((1 << bits) - 1);
+    for (int64_t o = 0; o < g.outer; ++o)
+        for (int64_t c = 0; c < g.C; ++c) {
+            int64_t k = group_of(&g, group_mode, o, c);
+            float sk, zk;
+            scale_zero(lo[k], hi[k], bits, &sk, &zk);
+            if (s) s[k] = sk;
+            if (z) z[k] = zk;
+            for (int64_t i = 0; i < g.inner; ++i) {
+                int64_t e = (o * g.C + c) * g.inner + i;
+                float v = load_elem(x, dtype, e);
+                float t = v / sk;                  /* Eq. 1: true division          */
+                float u = t + zk;                  /*        separate addition      */
+                float r = rintf(u);                /*        round-half-to-even     */
+                float q = fminf(fmaxf(r, 0.0f), qmax);     /* clamp to [0, 2^b - 1] */
+                int inside = (r >= 0.0f) && (r <= qmax);   /* clamp inactive        */
+                float d = q - zk;                  /* Eq. 6: subtract zero-point    */
+                float yv = sk * d;                 /*        multiply by the scale  */
+                store_elem(y, dtype, e, yv);
+                if (codes) codes[e] = (uint8_t)q;
+                if (mask) mask[e] = (uint8_t)inside;
+                if (gx) {
+                    float gv = load_elem(gy, dtype, e);
+                    store_elem(gx, dtype, e, inside ? gv : 0.0f);  /* STE: pass or zero */
+                }
+            }
+        }
+    return 0;
+}
+
+int granq_oracle_fused(const void* x, const void* gy, int dtype, const int64_t dims[4],
+                       int channel_axis, int group_mode, int bits,
+                       void* y, void* gx, float* lo, float* hi,
+                       uint8_t* codes, uint8_t* mask, float* s, float* z) {
+    int rc = granq_oracle_range(x, dtype, dims, channel_axis, group_mode, lo, hi);
+    if (rc) return rc;
+    return granq_oracle_fakequant(x, gy, dtype, dims, channel_axis, group_mode, bits,
+                                  lo, hi, y, gx, codes, mask, s, z);
+}

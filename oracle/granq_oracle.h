@@ -1,0 +1,72 @@
+/*
+ * GranQ channel-wise activation fake-quantization: CPU oracle (TEST INFRASTRUCTURE).
+ *
+ * A plain, slow, single-threaded restatement of the paper's definitions, used only
+ * to check the CUDA library and to serve as the timed CPU baseline.  It shares no
+ * code with the CUDA path and must never be called from the product path.
+ *
+ * What it computes, group by group and element by element, in IEEE fp32 with
+ * round-to-nearest-even and no fused multiply-add:
+ *   activation decomposition + per-group range .......... Eq. 4, Algorithm 1 (range step)
+ *   scale and zero-point ................................ Eq. 2 / Eq. 5
+ *   integer mapping  x_q = round(x / s + z) ............. Eq. 1, Algorithm 1 (quantize step)
+ *   dequantize / pre-scale  s * (x_q - z) ............... Eq. 6, Algorithm 1 (pre-scale step)
+ *   straight-through-estimator backward ................. Section 2.1 (named only)
+ *
+ * Readings taken where the paper is silent (all listed again in the design notes):
+ *   - rounding is round-half-to-even;
+ *   - the rounded value is clamped to [0, 2^b - 1] before dequantization;
+ *   - a degenerate range is floored: s = max(s, 1e-8);
+ *   - the backward mask is 1 exactly where the clamp was inactive;
+ *   - with a batch axis, one group is one channel over (n, h, w) (GROUP_CHANNEL);
+ *     the per-sample reading of Eq. 4 is GROUP_SAMPLE_CHANNEL; the layer-wise
+ *     baseline is GROUP_TENSOR.
+ *
+ * Every function is pinned by tests that do not call the oracle to produce the
+ * expected value (hand-worked cases, closed forms, exact rational arithmetic,
+ * invariants): no part is "parity unpinned".
+ *
+ * All pointers are host memory.  Tensors are contiguous row-major dims[4].
+ * dtype 0 = fp32 (float), 1 = bf16 (uint16_t bit patterns, widened exactly on
+ * read, narrowed round-to-nearest-even on write).
+ */
+#ifndef GRANQ_ORACLE_H
+#define GRANQ_ORACLE_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum { GRANQ_ORACLE_F32 = 0, GRANQ_ORACLE_BF16 = 1 };
+enum { GRANQ_ORACLE_GROUP_CHANNEL = 0, GRANQ_ORACLE_GROUP_SAMPLE_CHANNEL = 1, GRANQ_ORACLE_GROUP_TENSOR = 2 };
+
+/* Number of groups G for the given geometry; -1 on invalid arguments. */
+int64_t granq_oracle_num_groups(const int64_t dims[4], int channel_axis, int group_mode);
+
+/* Eq. 4: lo[g] = min, hi[g] = max over the members of group g (-0 canonicalised to +0).
+ * Returns 0, or -1 on invalid arguments, or -2 if a non-finite input is met. */
+int granq_oracle_range(const void* x, int dtype, const int64_t dims[4], int channel_axis,
+                       int group_mode, float* lo, float* hi);
+
+/* Eq. 2 / Eq. 5 for G groups. */
+int granq_oracle_params(const float* lo, const float* hi, int64_t G, int bits, float* s, float* z);
+
+/* Eq. 1 + clamp + Eq. 6 + STE mask with a GIVEN range (lo, hi per group).
+ * gy/gx may both be NULL (forward only); codes, mask, s, z may be NULL. */
+int granq_oracle_fakequant(const void* x, const void* gy, int dtype, const int64_t dims[4],
+                           int channel_axis, int group_mode, int bits,
+                           const float* lo, const float* hi,
+                           void* y, void* gx, uint8_t* codes, uint8_t* mask, float* s, float* z);
+
+/* Range from the tensor itself, then fakequant: the whole hot path. lo/hi are outputs. */
+int granq_oracle_fused(const void* x, const void* gy, int dtype, const int64_t dims[4],
+                       int channel_axis, int group_mode, int bits,
+                       void* y, void* gx, float* lo, float* hi,
+                       uint8_t* codes, uint8_t* mask, float* s, float* z);
+
+#ifdef __cplusplus
+}
+#endif
+#endif

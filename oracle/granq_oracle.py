@@ -1,0 +1,174 @@
+"""ctypes front end of the GranQ CPU oracle (TEST INFRASTRUCTURE).
+
+Only tests, the smoke check and the benchmark's CPU-baseline leg may import this
+module; the product path never does.  It compiles ``granq_oracle.c`` with gcc into
+``libgranq_oracle.so`` beside the source when the library is missing or older than
+its sources, and marshals numpy arrays to the C functions.  No arithmetic of the
+method lives here.
+
+fp32 tensors are ``float32`` arrays; bf16 tensors are ``uint16`` arrays holding the
+bit patterns.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+from dataclasses import dataclass
+from typing import Optional
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = [os.path.join(_HERE, "granq_oracle.c"), os.path.join(_HERE, "granq_oracle.h")]
+_LIB = os.path.join(_HERE, "libgranq_oracle.so")
+
+F32, BF16 = 0, 1
+GROUP_CHANNEL, GROUP_SAMPLE_CHANNEL, GROUP_TENSOR = 0, 1, 2
+
+CFLAGS = ["-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC"]
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (a second or so); returns the library path."""
+    stale = force or not os.path.exists(_LIB) or any(
+        os.path.getmtime(s) > os.path.getmtime(_LIB) for s in _SRC)
+    if stale:
+        tmp = _LIB + f".tmp{os.getpid()}"
+        subprocess.check_call(["gcc", *CFLAGS, "-o", tmp, _SRC[0], "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    global _lib
+    if _lib is None:
+        L = ctypes.CDLL(build())
+        vp, i64p, fp, u8p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.c_void_p, ctypes.c_void_p
+        ci = ctypes.c_int
+        L.granq_oracle_num_groups.restype = ctypes.c_int64
+        L.granq_oracle_num_groups.argtypes = [i64p, ci, ci]
+        L.granq_oracle_range.restype = ci
+        L.granq_oracle_range.argtypes = [vp, ci, i64p, ci, ci, fp, fp]
+        L.granq_oracle_params.restype = ci
+        L.granq_oracle_params.argtypes = [fp, fp, ctypes.c_int64, ci, fp, fp]
+        L.granq_oracle_fakequant.restype = ci
+        L.granq_oracle_fakequant.argtypes = [vp, vp, ci, i64p, ci, ci, ci, fp, fp, vp, vp, u8p, u8p, fp, fp]
+        L.granq_oracle_fused.restype = ci
+        L.granq_oracle_fused.argtypes = [vp, vp, ci, i64p, ci, ci, ci, vp, vp, fp, fp, u8p, u8p, fp, fp]
+        _lib = L
+    return _lib
+
+
+def _dims(shape):
+    if len(shape) != 4:
+        raise ValueError("oracle tensors are 4-d")
+    return (ctypes.c_int64 * 4)(*[int(d) for d in shape])
+
+
+def _dtype_of(a: np.ndarray) -> int:
+    if a.dtype == np.float32:
+        return F32
+    if a.dtype == np.uint16:
+        return BF16
+    raise TypeError(f"oracle takes float32 or uint16(bf16 bits), got {a.dtype}")
+
+
+def _p(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _check(rc: int, what: str):
+    if rc != 0:
+        raise RuntimeError(f"{what} failed with code {rc}")
+
+
+@dataclass
+class FakeQuantResult:
+    y: np.ndarray
+    gx: Optional[np.ndarray]
+    lo: np.ndarray
+    hi: np.ndarray
+    s: np.ndarray
+    z: np.ndarray
+    codes: np.ndarray
+    mask: np.ndarray
+
+
+def num_groups(shape, channel_axis: int = 1, group_mode: int = GROUP_CHANNEL) -> int:
+    g = lib().granq_oracle_num_groups(_dims(shape), channel_axis, group_mode)
+    if g < 0:
+        raise ValueError("invalid geometry")
+    return int(g)
+
+
+def range_(x: np.ndarray, channel_axis: int = 1, group_mode: int = GROUP_CHANNEL):
+    """Per-group (lo, hi): Eq. 4."""
+    x = np.ascontiguousarray(x)
+    G = num_groups(x.shape, channel_axis, group_mode)
+    lo = np.empty(G, np.float32)
+    hi = np.empty(G, np.float32)
+    _check(lib().granq_oracle_range(_p(x), _dtype_of(x), _dims(x.shape), channel_axis, group_mode,
+                                    _p(lo), _p(hi)), "granq_oracle_range")
+    return lo, hi
+
+
+def params(lo: np.ndarray, hi: np.ndarray, bits: int):
+    """Per-group (s, z): Eq. 2 / Eq. 5."""
+    lo = np.ascontiguousarray(lo, np.float32)
+    hi = np.ascontiguousarray(hi, np.float32)
+    s = np.empty_like(lo)
+    z = np.empty_like(lo)
+    _check(lib().granq_oracle_params(_p(lo), _p(hi), lo.size, bits, _p(s), _p(z)), "granq_oracle_params")
+    return s, z
+
+
+def fakequant(x: np.ndarray, bits: int, lo: np.ndarray, hi: np.ndarray, gy: Optional[np.ndarray] = None,
+              channel_axis: int = 1, group_mode: int = GROUP_CHANNEL) -> FakeQuantResult:
+    """Quantize -> clamp -> dequantize (+ STE backward when gy is given) with a given range."""
+    x = np.ascontiguousarray(x)
+    G = num_groups(x.shape, channel_axis, group_mode)
+    lo = np.ascontiguousarray(lo, np.float32)
+    hi = np.ascontiguousarray(hi, np.float32)
+    if lo.size != G or hi.size != G:
+        raise ValueError("range vectors must have one entry per group")
+    if gy is not None:
+        gy = np.ascontiguousarray(gy)
+        if gy.shape != x.shape or gy.dtype != x.dtype:
+            raise ValueError("gy must match x")
+    y = np.empty_like(x)
+    gx = None if gy is None else np.empty_like(x)
+    codes = np.empty(x.shape, np.uint8)
+    mask = np.empty(x.shape, np.uint8)
+    s = np.empty(G, np.float32)
+    z = np.empty(G, np.float32)
+    _check(lib().granq_oracle_fakequant(_p(x), _p(gy), _dtype_of(x), _dims(x.shape), channel_axis, group_mode,
+                                        bits, _p(lo), _p(hi), _p(y), _p(gx), _p(codes), _p(mask), _p(s), _p(z)),
+           "granq_oracle_fakequant")
+    return FakeQuantResult(y, gx, lo, hi, s, z, codes, mask)
+
+
+def fused(x: np.ndarray, bits: int, gy: Optional[np.ndarray] = None, channel_axis: int = 1,
+          group_mode: int = GROUP_CHANNEL, want_codes: bool = True) -> FakeQuantResult:
+    """The whole hot path: range from x itself, then fakequant (+ backward when gy is given)."""
+    x = np.ascontiguousarray(x)
+    G = num_groups(x.shape, channel_axis, group_mode)
+    if gy is not None:
+        gy = np.ascontiguousarray(gy)
+        if gy.shape != x.shape or gy.dtype != x.dtype:
+            raise ValueError("gy must match x")
+    y = np.empty_like(x)
+    gx = None if gy is None else np.empty_like(x)
+    codes = np.empty(x.shape, np.uint8) if want_codes else None
+    mask = np.empty(x.shape, np.uint8) if want_codes else None
+    lo = np.empty(G, np.float32)
+    hi = np.empty(G, np.float32)
+    s = np.empty(G, np.float32)
+    z = np.empty(G, np.float32)
+    _check(lib().granq_oracle_fused(_p(x), _p(gy), _dtype_of(x), _dims(x.shape), channel_axis, group_mode, bits,
+                                    _p(y), _p(gx), _p(lo), _p(hi), _p(codes), _p(mask), _p(s), _p(z)),
+           "granq_oracle_fused")
+    return FakeQuantResult(y, gx, lo, hi, s, z, codes, mask)
