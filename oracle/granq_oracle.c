@@ -131,7 +131,10 @@ int granq_oracle_fakequant(const void* x, const void* gy, int dtype, const int64
                 float t = v / sk;                  /* Eq. 1: true division          */
                 float u = t + zk;                  /*        separate addition      */
                 float r = rintf(u);                /*        round-half-to-even     */
-                float q = fminf(fmaxf(r, 0.0f), qmax);     /* clamp to [0, 2^b - 1] */
+                float q = r;                       /* clamp to [0, 2^b - 1]         */
+                if (q < 0.0f) q = 0.0f;
+                if (q > qmax) q = qmax;
+                q += 0.0f;                         /* an integer code has no -0     */
                 int inside = (r >= 0.0f) && (r <= qmax);   /* clamp inactive        */
                 float d = q - zk;                  /* Eq. 6: subtract zero-point    */
                 float yv = sk * d;                 /*        multiply by the scale  */
