@@ -1,0 +1,206 @@
+/*
+ * granq.h - C ABI of the GranQ channel-wise activation fake-quantization library
+ * for NVIDIA B200 (sm_100a).
+ *
+ * The library implements one data-parallel path of GranQ (arXiv 2503.18339):
+ *   1. activation decomposition and per-group range ............ Eq. 4, Algorithm 1 (range step)
+ *   2. scale and zero-point for b bits ........................... Eq. 2 / Eq. 5
+ *   3. quantize -> clamp -> dequantize ("pre-scaling") ........... Eq. 1, Eq. 6, Algorithm 1
+ *   4. straight-through-estimator backward ....................... Section 2.1
+ *
+ * Arithmetic (identical for every entry point), per group g with members x_i, in IEEE
+ * fp32, round-to-nearest-even, no fused multiply-add:
+ *     lo = min x_i, hi = max x_i                 (-0 reported as +0)
+ *     s  = max((hi - lo) / (2^b - 1), 1e-8)      z = round(-lo / s)
+ *     r  = round(x_i / s + z)                    code = clamp(r, 0, 2^b - 1)
+ *     y_i  = s * (code - z)                      mask_i = (0 <= r <= 2^b - 1)
+ *     gx_i = mask_i ? gy_i : 0
+ * round() is round-half-to-even.  The clamp, the 1e-8 floor, the tie rule and the mask
+ * are this library's reading of points the paper leaves open.
+ *
+ * Tensors.  Contiguous row-major dims[4] (NCHW for activations), element type fp32 or
+ * bf16.  `channel_axis` (0..3) selects the channel dimension; with outer = product of the
+ * dims before it, C = dims[channel_axis], inner = product of the dims after it:
+ *     GRANQ_GROUP_CHANNEL        one group per channel, reduced over everything else
+ *                                (batch included: "per channel at the batch level") G = C
+ *     GRANQ_GROUP_SAMPLE_CHANNEL Eq. 4 applied to each sample: G = outer * C, group index
+ *                                o * C + c
+ *     GRANQ_GROUP_TENSOR         layer-wise baseline: G = 1
+ * bf16 inputs are widened exactly, all arithmetic is fp32, y / gx are narrowed with
+ * round-to-nearest-even; lo, hi, s, z are always fp32.
+ *
+ * Memory.  Unless a parameter is documented as HOST memory, every pointer is DEVICE
+ * memory owned by the caller, valid until the stream has passed the call.  The library
+ * never allocates or frees device memory and keeps no results between calls; scratch comes
+ * from the caller's `workspace` (at least granq_workspace_bytes(), 256-byte aligned,
+ * contents irrelevant on entry, overwritten by the call).  Outputs must not overlap
+ * inputs.  Inputs must be finite (NaN / Inf give unspecified results, never a fault).
+ *
+ * Execution.  All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*;
+ * NULL = the default stream); no entry point synchronises with the host except
+ * granq_fakequant_fused_host() and granq_workspace_status().  Results are bit-identical
+ * from run to run.
+ *
+ * Errors.  Every function returning int returns a granq_status code.  Argument errors
+ * (null required pointer, bits outside 1..8, non-positive dim, more than 2^40 elements,
+ * bad enum, workspace too small or misaligned) are detected on the host before anything
+ * is launched and leave all outputs untouched.  CUDA launch errors are returned as
+ * GRANQ_ERR_CUDA.  The on-chip-staged plan of granq_fakequant_fused() contains bounded
+ * device-side waits; should one run out (it cannot unless the GPU is preempted for
+ * seconds) the kernel stops, outputs are unspecified, and granq_workspace_status()
+ * reports GRANQ_ERR_TIMEOUT.
+ */
+#ifndef GRANQ_H
+#define GRANQ_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum granq_status {
+    GRANQ_OK = 0,
+    GRANQ_ERR_INVALID_ARG = 1,
+    GRANQ_ERR_UNSUPPORTED = 2,
+    GRANQ_ERR_WORKSPACE = 3,
+    GRANQ_ERR_CUDA = 4,
+    GRANQ_ERR_TIMEOUT = 5
+};
+
+enum granq_dtype { GRANQ_F32 = 0, GRANQ_BF16 = 1 };
+
+enum granq_group { GRANQ_GROUP_CHANNEL = 0, GRANQ_GROUP_SAMPLE_CHANNEL = 1, GRANQ_GROUP_TENSOR = 2 };
+
+/* flags (bitwise or).  The plan-forcing flags exist so that every execution plan can be
+ * checked and measured on the same input; results do not depend on the plan. */
+enum granq_flags {
+    GRANQ_FLAG_NONE = 0,
+    GRANQ_FLAG_FORCE_TWO_PASS = 1u,  /* fused: range launch + quantize launch (x is read twice)      */
+    GRANQ_FLAG_FORCE_NAIVE = 2u,     /* fused: host loop over channels, three launches per channel -
+                                        the "conventional" scalar-loop scheme of Section 5.3.2       */
+    GRANQ_FLAG_FORCE_STAGED = 4u     /* fused: on-chip-staged persistent kernel or GRANQ_ERR_UNSUPPORTED */
+};
+
+/* Human-readable name of a status code (static storage, never NULL). */
+const char* granq_status_string(int status);
+
+/* Number of groups G for a geometry, or -1 if the arguments are invalid. */
+int64_t granq_num_groups(const int64_t dims[4], int channel_axis, int group);
+
+/* Bytes of scratch every entry point that takes a workspace needs for this geometry
+ * (0 if the arguments are invalid). */
+size_t granq_workspace_bytes(int dtype, const int64_t dims[4], int channel_axis, int group);
+
+/*
+ * Eq. 4 / Algorithm 1 (range step): min_out[g], max_out[g] for g in [0, G).
+ *   x          in   E elements of `dtype`
+ *   min_out    out  G floats        max_out   out  G floats
+ */
+int granq_range(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                float* min_out, float* max_out,
+                void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream);
+
+/*
+ * Eq. 1 + clamp + Eq. 6 with a range supplied by the caller (for instance one measured on
+ * another batch): y = s * (clamp(round(x / s + z)) - z), with s, z from Eq. 2 / Eq. 5.
+ *   min_in, max_in  in   G floats each
+ *   y               out  E elements of `dtype`
+ *   codes_opt       out  E bytes, the integer codes (NULL to skip)
+ *   scale_opt, zp_opt out G floats each (NULL to skip)
+ */
+int granq_fakequant_fwd(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                        int bits, const float* min_in, const float* max_in,
+                        void* y, uint8_t* codes_opt, float* scale_opt, float* zp_opt,
+                        uint32_t flags, void* cuda_stream);
+
+/*
+ * Straight-through-estimator backward (Section 2.1): gx = gy where the forward clamp was
+ * inactive for x, else 0.  The range, scale and zero-point are treated as constants.
+ *   gy, x      in   E elements each       gx   out  E elements
+ *   mask_opt   out  E bytes of 0/1 (NULL to skip)
+ */
+int granq_fakequant_bwd(const void* gy, const void* x, int dtype, const int64_t dims[4], int channel_axis,
+                        int group, int bits, const float* min_in, const float* max_in,
+                        void* gx, uint8_t* mask_opt, uint32_t flags, void* cuda_stream);
+
+/*
+ * The whole path in one call (Algorithm 1, range step through pre-scale step, plus the
+ * backward): range of x itself -> scale / zero-point -> y, and gx when gy_opt is given.
+ * Where a channel group fits in the GPU's shared memory the tensor is read from HBM once.
+ *   x                 in   E elements          gy_opt   in   E elements or NULL (forward only)
+ *   y                 out  E elements          gx_opt   out  E elements (required iff gy_opt)
+ *   min_out, max_out  out  G floats each (required)
+ *   codes_opt, mask_opt    E bytes each or NULL;  scale_opt, zp_opt  G floats each or NULL
+ */
+int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const int64_t dims[4],
+                          int channel_axis, int group, int bits,
+                          void* y, void* gx_opt, float* min_out, float* max_out,
+                          uint8_t* codes_opt, uint8_t* mask_opt, float* scale_opt, float* zp_opt,
+                          void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream);
+
+/*
+ * Status word the staged plan leaves in the workspace.  Synchronises `cuda_stream`, then
+ * returns GRANQ_OK, GRANQ_ERR_TIMEOUT (a bounded device-side wait ran out), or
+ * GRANQ_ERR_CUDA.  `workspace` is the pointer given to the preceding call.
+ */
+int granq_workspace_status(const void* workspace, void* cuda_stream);
+
+/* Bytes of device memory granq_fakequant_fused_host() needs as its arena. */
+size_t granq_host_arena_bytes(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward);
+
+/*
+ * granq_fakequant_fused() for tensors that live in HOST memory (pinned memory makes the
+ * copies asynchronous and fast; pageable memory works).  x_host / gy_host_opt are copied
+ * into `device_arena`, the fused path runs there, and y / gx / min / max (and scale / zp
+ * when asked for) are copied back; the call returns after `cuda_stream` has drained, so
+ * the host outputs are valid on return.
+ *   x_host, gy_host_opt, y_host, gx_host_opt, min_host, max_host, scale_host_opt,
+ *   zp_host_opt          HOST memory, sizes as for granq_fakequant_fused()
+ *   device_arena         DEVICE memory, 256-byte aligned, >= granq_host_arena_bytes()
+ */
+int granq_fakequant_fused_host(const void* x_host, const void* gy_host_opt, int dtype, const int64_t dims[4],
+                               int channel_axis, int group, int bits,
+                               void* y_host, void* gx_host_opt, float* min_host, float* max_host,
+                               float* scale_host_opt, float* zp_host_opt,
+                               void* device_arena, size_t arena_bytes, uint32_t flags, void* cuda_stream);
+
+/*
+ * Plan that granq_fakequant_fused() would take for this geometry and flags on the current
+ * device: 0 = two-pass, 1 = naive per-channel loop, 2 = on-chip staged; negative = -status.
+ * `launches_out` (HOST, may be NULL) receives the number of kernel launches of that plan.
+ */
+int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,
+                     uint32_t flags, int* launches_out);
+
+/*
+ * Host-only query: how the staged plan would cut this tensor on a device with `sm_count`
+ * SMs and `smem_bytes` of shared memory per CTA (no counterpart in the paper).
+ * out = { CTAs, threads per CTA, buffers per CTA, shared-memory bytes per CTA,
+ *         16-byte units per buffer, channels per wave, units per chunk, number of waves }.
+ * Returns GRANQ_ERR_UNSUPPORTED when the geometry does not qualify for staging.
+ */
+int granq_staged_geometry(int dtype, const int64_t dims[4], int channel_axis, int group, int sm_count,
+                          int smem_bytes, int64_t out[8]);
+
+/*
+ * Planner overrides for tests and tuning (no counterpart in the paper).  Process-wide and
+ * not thread-safe; value 0 restores the automatic choice.  They change how the staged plan
+ * cuts a tensor into waves and chunks, never its results.
+ */
+enum granq_knob {
+    GRANQ_KNOB_STAGED_DEPTH = 0,          /* shared-memory buffers per CTA (1..3)                  */
+    GRANQ_KNOB_STAGED_MAX_BUF_UNITS = 1,  /* cap on 16-byte units per buffer (forces small waves)  */
+    GRANQ_KNOB_STAGED_GRID = 2,           /* cap on the number of CTAs                             */
+    GRANQ_KNOB_SPIN_LIMIT = 3,            /* iteration limit of the wait on a wave's arrival count */
+    GRANQ_KNOB_TEST_EXTRA_ARRIVALS = 4    /* test hook: a wave waits for this many arrivals more
+                                             than the grid provides, so the bounded wait runs out
+                                             and the call ends with GRANQ_ERR_TIMEOUT              */
+};
+int granq_tune(int knob, int value);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRANQ_H */

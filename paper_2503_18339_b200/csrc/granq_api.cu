@@ -1,0 +1,306 @@
+// C ABI of the GranQ library: argument validation, reduction of (dims, channel axis, group
+// mode) to channel-group geometry, plan selection and launches.  See include/granq.h.
+#include "../../include/granq.h"
+
+#include "granq_internal.h"
+
+using namespace granq;
+
+namespace {
+
+constexpr int64_t kMaxElements = 1ll << 40;
+
+StagedTuning g_tune = {0, 0, 0, 0, 0};
+
+bool make_geom(const int64_t dims[4], int axis, int group, Geom& g, int64_t& G) {
+    if (!dims || axis < 0 || axis > 3 || group < 0 || group > 2) return false;
+    int64_t E = 1;
+    for (int d = 0; d < 4; ++d) {
+        if (dims[d] <= 0 || dims[d] > kMaxElements) return false;
+        if (E > kMaxElements / dims[d]) return false;
+        E *= dims[d];
+    }
+    if (E > kMaxElements) return false;
+    int64_t outer = 1, inner = 1;
+    for (int d = 0; d < axis; ++d) outer *= dims[d];
+    for (int d = axis + 1; d < 4; ++d) inner *= dims[d];
+    const int64_t C = dims[axis];
+    g.E = E;
+    if (group == GRANQ_GROUP_CHANNEL) {
+        g.outer = outer; g.C = C; g.inner = inner;
+    } else if (group == GRANQ_GROUP_SAMPLE_CHANNEL) {
+        g.outer = 1; g.C = outer * C; g.inner = inner;
+    } else {
+        g.outer = 1; g.C = 1; g.inner = E;
+    }
+    G = g.C;
+    return true;
+}
+
+bool dtype_ok(int dtype) { return dtype == GRANQ_F32 || dtype == GRANQ_BF16; }
+size_t elt_size(int dtype) { return dtype == GRANQ_F32 ? 4 : 2; }
+
+bool overlaps(const void* a, size_t na, const void* b, size_t nb) {
+    if (!a || !b) return false;
+    const char* pa = (const char*)a;
+    const char* pb = (const char*)b;
+    return pa < pb + nb && pb < pa + na;
+}
+
+int check_workspace(const void* ws, size_t bytes, int64_t G) {
+    if (!ws || ((uintptr_t)ws & 255) != 0) return GRANQ_ERR_WORKSPACE;
+    if (bytes < workspace_bytes_for(G)) return GRANQ_ERR_WORKSPACE;
+    return GRANQ_OK;
+}
+
+int cuda_status(cudaError_t e) { return e == cudaSuccess ? GRANQ_OK : GRANQ_ERR_CUDA; }
+
+enum { PLAN_TWO_PASS = 0, PLAN_NAIVE = 1, PLAN_STAGED = 2 };
+
+// plan of the fused entry point; `plan_out` is filled when the staged plan is taken
+int choose_plan(int dtype, const Geom& g, const QuantIO& io, uint32_t flags, StagedPlan* plan_out) {
+    if (flags & GRANQ_FLAG_FORCE_NAIVE) return PLAN_NAIVE;
+    if (flags & GRANQ_FLAG_FORCE_TWO_PASS) return PLAN_TWO_PASS;
+    int dev = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess) return -GRANQ_ERR_CUDA;
+    StagedPlan p = plan_staged(dtype, g, io, dev, g_tune);
+    if (p.ok) {
+        if (plan_out) *plan_out = p;
+        return PLAN_STAGED;
+    }
+    if (flags & GRANQ_FLAG_FORCE_STAGED) return -GRANQ_ERR_UNSUPPORTED;
+    return PLAN_TWO_PASS;
+}
+
+size_t align256(size_t v) { return (v + 255) & ~(size_t)255; }
+
+}  // namespace
+
+extern "C" {
+
+const char* granq_status_string(int status) {
+    switch (status) {
+        case GRANQ_OK: return "ok";
+        case GRANQ_ERR_INVALID_ARG: return "invalid argument";
+        case GRANQ_ERR_UNSUPPORTED: return "unsupported geometry or plan";
+        case GRANQ_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case GRANQ_ERR_CUDA: return "CUDA error";
+        case GRANQ_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        default: return "unknown status";
+    }
+}
+
+int64_t granq_num_groups(const int64_t dims[4], int channel_axis, int group) {
+    Geom g;
+    int64_t G;
+    if (!make_geom(dims, channel_axis, group, g, G)) return -1;
+    return G;
+}
+
+size_t granq_workspace_bytes(int dtype, const int64_t dims[4], int channel_axis, int group) {
+    Geom g;
+    int64_t G;
+    if (!dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G)) return 0;
+    return workspace_bytes_for(G);
+}
+
+int granq_range(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group, float* min_out,
+                float* max_out, void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream) {
+    (void)flags;
+    Geom g;
+    int64_t G;
+    if (!x || !min_out || !max_out || !dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G))
+        return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
+    if (int rc = check_workspace(workspace, workspace_bytes, G)) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    Workspace ws = carve_workspace(workspace, G);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
+    if (e == cudaSuccess) e = launch_range_flat(x, dtype, g, ws.kmin, ws.kmax, st);
+    if (e == cudaSuccess) e = launch_finalize_range(ws.kmin, ws.kmax, G, min_out, max_out, 0, nullptr, nullptr, st);
+    return cuda_status(e);
+}
+
+int granq_fakequant_fwd(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group, int bits,
+                        const float* min_in, const float* max_in, void* y, uint8_t* codes_opt, float* scale_opt,
+                        float* zp_opt, uint32_t flags, void* cuda_stream) {
+    (void)flags;
+    Geom g;
+    int64_t G;
+    if (!x || !y || !min_in || !max_in || bits < 1 || bits > 8 || !dtype_ok(dtype) ||
+        !make_geom(dims, channel_axis, group, g, G))
+        return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
+    const size_t nb = (size_t)g.E * elt_size(dtype);
+    if (overlaps(x, nb, y, nb)) return GRANQ_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    QuantIO io{x, nullptr, y, nullptr, codes_opt, nullptr};
+    cudaError_t e = launch_quant_flat(io, MODE_FWD, dtype, g, bits, min_in, max_in, st);
+    if (e == cudaSuccess && (scale_opt || zp_opt)) e = launch_params(min_in, max_in, G, bits, scale_opt, zp_opt, st);
+    return cuda_status(e);
+}
+
+int granq_fakequant_bwd(const void* gy, const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                        int bits, const float* min_in, const float* max_in, void* gx, uint8_t* mask_opt,
+                        uint32_t flags, void* cuda_stream) {
+    (void)flags;
+    Geom g;
+    int64_t G;
+    if (!gy || !x || !gx || !min_in || !max_in || bits < 1 || bits > 8 || !dtype_ok(dtype) ||
+        !make_geom(dims, channel_axis, group, g, G))
+        return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
+    const size_t nb = (size_t)g.E * elt_size(dtype);
+    if (overlaps(x, nb, gx, nb) || overlaps(gy, nb, gx, nb)) return GRANQ_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    QuantIO io{x, gy, nullptr, gx, nullptr, mask_opt};
+    return cuda_status(launch_quant_flat(io, MODE_BWD, dtype, g, bits, min_in, max_in, st));
+}
+
+int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const int64_t dims[4], int channel_axis,
+                          int group, int bits, void* y, void* gx_opt, float* min_out, float* max_out,
+                          uint8_t* codes_opt, uint8_t* mask_opt, float* scale_opt, float* zp_opt, void* workspace,
+                          size_t workspace_bytes, uint32_t flags, void* cuda_stream) {
+    Geom g;
+    int64_t G;
+    if (!x || !y || !min_out || !max_out || bits < 1 || bits > 8 || !dtype_ok(dtype) ||
+        !make_geom(dims, channel_axis, group, g, G))
+        return GRANQ_ERR_INVALID_ARG;
+    if ((gy_opt == nullptr) != (gx_opt == nullptr)) return GRANQ_ERR_INVALID_ARG;
+    if (mask_opt && !gy_opt) return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
+    const size_t nb = (size_t)g.E * elt_size(dtype);
+    if (overlaps(x, nb, y, nb) || overlaps(x, nb, gx_opt, nb) || overlaps(gy_opt, nb, y, nb) ||
+        overlaps(gy_opt, nb, gx_opt, nb) || overlaps(y, nb, gx_opt, nb))
+        return GRANQ_ERR_INVALID_ARG;
+    if (int rc = check_workspace(workspace, workspace_bytes, G)) return rc;
+
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const int mode = gy_opt ? MODE_BOTH : MODE_FWD;
+    QuantIO io{x, gy_opt, y, gx_opt, codes_opt, mask_opt};
+    StagedPlan sp{};
+    const int plan = choose_plan(dtype, g, io, flags, &sp);
+    if (plan < 0) return -plan;
+
+    Workspace ws = carve_workspace(workspace, G);
+    cudaError_t e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
+    if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+    if (plan == PLAN_STAGED) {
+        e = launch_staged(sp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
+    } else if (plan == PLAN_NAIVE) {
+        e = launch_naive(io, mode, dtype, g, bits, ws.kmin, ws.kmax, min_out, max_out, st, nullptr);
+        if (e == cudaSuccess && (scale_opt || zp_opt))
+            e = launch_params(min_out, max_out, G, bits, scale_opt, zp_opt, st);
+    } else {
+        e = launch_range_flat(x, dtype, g, ws.kmin, ws.kmax, st);
+        if (e == cudaSuccess)
+            e = launch_finalize_range(ws.kmin, ws.kmax, G, min_out, max_out, bits, scale_opt, zp_opt, st);
+        if (e == cudaSuccess) e = launch_quant_flat(io, mode, dtype, g, bits, min_out, max_out, st);
+    }
+    return cuda_status(e);
+}
+
+int granq_workspace_status(const void* workspace, void* cuda_stream) {
+    if (!workspace) return GRANQ_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    uint32_t word = 0;
+    if (cudaMemcpyAsync(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        return GRANQ_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return GRANQ_ERR_CUDA;
+    return word == 0 ? GRANQ_OK : (word == GRANQ_ERR_TIMEOUT ? GRANQ_ERR_TIMEOUT : GRANQ_ERR_CUDA);
+}
+
+// arena layout: x | gy | y | gx | lo | hi | s | z | workspace, each piece 256-byte aligned
+size_t granq_host_arena_bytes(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward) {
+    Geom g;
+    int64_t G;
+    if (!dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G)) return 0;
+    const size_t nb = align256((size_t)g.E * elt_size(dtype));
+    return nb * (with_backward ? 4 : 2) + 4 * align256((size_t)G * 4) + workspace_bytes_for(G);
+}
+
+int granq_fakequant_fused_host(const void* x_host, const void* gy_host_opt, int dtype, const int64_t dims[4],
+                               int channel_axis, int group, int bits, void* y_host, void* gx_host_opt,
+                               float* min_host, float* max_host, float* scale_host_opt, float* zp_host_opt,
+                               void* device_arena, size_t arena_bytes, uint32_t flags, void* cuda_stream) {
+    Geom g;
+    int64_t G;
+    if (!x_host || !y_host || !min_host || !max_host || !dtype_ok(dtype) ||
+        !make_geom(dims, channel_axis, group, g, G))
+        return GRANQ_ERR_INVALID_ARG;
+    if ((gy_host_opt == nullptr) != (gx_host_opt == nullptr)) return GRANQ_ERR_INVALID_ARG;
+    const int bwd = gy_host_opt ? 1 : 0;
+    if (!device_arena || ((uintptr_t)device_arena & 255) ||
+        arena_bytes < granq_host_arena_bytes(dtype, dims, channel_axis, group, bwd))
+        return GRANQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const size_t raw = (size_t)g.E * elt_size(dtype), nb = align256(raw), gb = align256((size_t)G * 4);
+    char* p = (char*)device_arena;
+    char* dx = p; p += nb;
+    char* dgy = nullptr; if (bwd) { dgy = p; p += nb; }
+    char* dy = p; p += nb;
+    char* dgx = nullptr; if (bwd) { dgx = p; p += nb; }
+    float* dlo = (float*)p; p += gb;
+    float* dhi = (float*)p; p += gb;
+    float* ds = (float*)p; p += gb;
+    float* dz = (float*)p; p += gb;
+    void* ws = p;
+    if (cudaMemcpyAsync(dx, x_host, raw, cudaMemcpyHostToDevice, st) != cudaSuccess) return GRANQ_ERR_CUDA;
+    if (bwd && cudaMemcpyAsync(dgy, gy_host_opt, raw, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return GRANQ_ERR_CUDA;
+    int rc = granq_fakequant_fused(dx, dgy, dtype, dims, channel_axis, group, bits, dy, dgx, dlo, dhi, nullptr,
+                                   nullptr, scale_host_opt ? ds : nullptr, zp_host_opt ? dz : nullptr, ws,
+                                   workspace_bytes_for(G), flags, cuda_stream);
+    if (rc != GRANQ_OK) return rc;
+    cudaError_t e = cudaMemcpyAsync(y_host, dy, raw, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && bwd) e = cudaMemcpyAsync(gx_host_opt, dgx, raw, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(min_host, dlo, (size_t)G * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess) e = cudaMemcpyAsync(max_host, dhi, (size_t)G * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && scale_host_opt)
+        e = cudaMemcpyAsync(scale_host_opt, ds, (size_t)G * 4, cudaMemcpyDeviceToHost, st);
+    if (e == cudaSuccess && zp_host_opt) e = cudaMemcpyAsync(zp_host_opt, dz, (size_t)G * 4, cudaMemcpyDeviceToHost, st);
+    if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+    return granq_workspace_status(ws, cuda_stream);
+}
+
+int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,
+                     uint32_t flags, int* launches_out) {
+    Geom g;
+    int64_t G;
+    if (!dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G)) return -GRANQ_ERR_INVALID_ARG;
+    (void)with_backward;
+    QuantIO io{};   // null pointers: alignment is assumed
+    const int plan = choose_plan(dtype, g, io, flags, nullptr);
+    if (launches_out) {
+        if (plan == PLAN_STAGED) *launches_out = 1;
+        else if (plan == PLAN_NAIVE) *launches_out = (int)(3 * g.C);
+        else if (plan == PLAN_TWO_PASS) *launches_out = 3;
+    }
+    return plan;
+}
+
+int granq_staged_geometry(int dtype, const int64_t dims[4], int channel_axis, int group, int sm_count,
+                          int smem_bytes, int64_t out[8]) {
+    Geom g;
+    int64_t G;
+    if (!out || !dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G)) return GRANQ_ERR_INVALID_ARG;
+    QuantIO io{};
+    StagedPlan p = plan_staged_on(dtype, g, io, sm_count, smem_bytes, g_tune);
+    if (!p.ok) return GRANQ_ERR_UNSUPPORTED;
+    out[0] = p.grid; out[1] = p.threads; out[2] = p.depth; out[3] = p.smem_bytes;
+    out[4] = p.buf_units; out[5] = p.cw; out[6] = p.cu; out[7] = p.nwaves;
+    return GRANQ_OK;
+}
+
+int granq_tune(int knob, int value) {
+    switch (knob) {
+        case GRANQ_KNOB_STAGED_DEPTH: g_tune.depth = value; return GRANQ_OK;
+        case GRANQ_KNOB_STAGED_MAX_BUF_UNITS: g_tune.max_buf_units = value; return GRANQ_OK;
+        case GRANQ_KNOB_STAGED_GRID: g_tune.grid = value; return GRANQ_OK;
+        case GRANQ_KNOB_SPIN_LIMIT: g_tune.spin_limit = value; return GRANQ_OK;
+        case GRANQ_KNOB_TEST_EXTRA_ARRIVALS: g_tune.extra_arrivals = value; return GRANQ_OK;
+        default: return GRANQ_ERR_INVALID_ARG;
+    }
+}
+
+}  // extern "C"

@@ -1,0 +1,203 @@
+// Device-side building blocks shared by the GranQ kernels: ordered keys for min/max,
+// the per-element quantizer arithmetic, 128-bit element packs, fast integer division and
+// the warp-level run accumulator of the range reduction.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace granq {
+
+// ---------------------------------------------------------------------------------------
+// Ordered keys.  enc() maps a float to an unsigned integer with the same ordering, so an
+// unsigned max over enc(x) is the float max and an unsigned max over ~enc(x) is the float
+// min.  0 is the identity of both reductions (no finite float encodes to 0 or ~0).
+// ---------------------------------------------------------------------------------------
+__host__ __device__ __forceinline__ uint32_t enc_bits(uint32_t b) {
+    return b ^ ((uint32_t)((int32_t)b >> 31) | 0x80000000u);
+}
+__device__ __forceinline__ uint32_t enc(float f) { return enc_bits(__float_as_uint(f)); }
+__device__ __forceinline__ float dec(uint32_t k) {
+    uint32_t b = (k & 0x80000000u) ? (k ^ 0x80000000u) : ~k;
+    return __uint_as_float(b);
+}
+// key pair -> (lo, hi), with -0 canonicalised to +0
+__device__ __forceinline__ void keys_to_range(uint32_t kmin, uint32_t kmax, float& lo, float& hi) {
+    lo = __fadd_rn(dec(~kmin), 0.0f);
+    hi = __fadd_rn(dec(kmax), 0.0f);
+}
+
+// ---------------------------------------------------------------------------------------
+// Quantizer arithmetic (Eq. 1, 2, 5, 6).  Every operation is an explicitly rounded fp32
+// intrinsic, so the compiler can neither contract multiply-adds nor replace the divisions.
+// ---------------------------------------------------------------------------------------
+struct QParam {
+    float s, z;
+};
+
+__device__ __forceinline__ QParam make_qparam(float lo, float hi, float qmax) {
+    QParam p;
+    float s = __fdiv_rn(__fsub_rn(hi, lo), qmax);
+    p.s = fmaxf(s, 1e-8f);
+    p.z = __fadd_rn(rintf(__fdiv_rn(-lo, p.s)), 0.0f);
+    return p;
+}
+
+// Rounds u = x / s + z to the nearest integer (ties to even) and clamps it to [0, qmax].
+// The value is first clamped to [-1, qmax + 1]: rounding is monotone and the bounds are
+// integers, so this changes neither the clamped code nor whether the clamp was active, and
+// it makes the add/subtract of 1.5 * 2^23 an exact round-half-to-even (|u| < 2^22) that
+// never yields -0.
+__device__ __forceinline__ float quant_one(float x, QParam p, float qmax, float& y, bool& inside) {
+    const float kMagic = 12582912.0f;  // 1.5 * 2^23
+    float t = __fdiv_rn(x, p.s);
+    float u = __fadd_rn(t, p.z);
+    float uc = fminf(fmaxf(u, -1.0f), __fadd_rn(qmax, 1.0f));
+    float r = __fsub_rn(__fadd_rn(uc, kMagic), kMagic);
+    float q = fminf(fmaxf(r, 0.0f), qmax);
+    inside = (r == q);
+    y = __fmul_rn(p.s, __fsub_rn(q, p.z));
+    return q;
+}
+
+// ---------------------------------------------------------------------------------------
+// 16-byte packs of elements.
+// ---------------------------------------------------------------------------------------
+template <typename T>
+struct Pack;
+
+template <>
+struct Pack<float> {
+    static constexpr int V = 4;
+    uint4 raw;
+    __device__ __forceinline__ float get(int i) const { return __uint_as_float((&raw.x)[i]); }
+    __device__ __forceinline__ void set(int i, float v) { (&raw.x)[i] = __float_as_uint(v); }
+};
+
+template <>
+struct Pack<__nv_bfloat16> {
+    static constexpr int V = 8;
+    uint4 raw;
+    __device__ __forceinline__ float get(int i) const {
+        uint32_t w = (&raw.x)[i >> 1];
+        uint32_t b = (i & 1) ? (w & 0xFFFF0000u) : (w << 16);
+        return __uint_as_float(b);
+    }
+    __device__ __forceinline__ void set(int i, float v) {
+        uint32_t h = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v));
+        uint32_t& w = (&raw.x)[i >> 1];
+        w = (i & 1) ? ((w & 0x0000FFFFu) | (h << 16)) : ((w & 0xFFFF0000u) | h);
+    }
+};
+
+__device__ __forceinline__ float load_scalar(const float* p) { return __ldg(p); }
+__device__ __forceinline__ float load_scalar(const __nv_bfloat16* p) {
+    return __uint_as_float((uint32_t)__ldg(reinterpret_cast<const unsigned short*>(p)) << 16);
+}
+__device__ __forceinline__ void store_scalar(float* p, float v) { *p = v; }
+__device__ __forceinline__ void store_scalar(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+
+// streaming 128-bit global accesses: data that is touched once should not displace anything
+__device__ __forceinline__ uint4 ld_stream_16(const void* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream_16(void* p, uint4 v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w)
+                 : "memory");
+}
+
+// ---------------------------------------------------------------------------------------
+// Division of n < 2^31 by a run-time constant d (1 <= d < 2^31): q = (n * M) >> (31 + l)
+// with l = ceil(log2 d), M = floor(2^(31+l) / d) + 1.
+// ---------------------------------------------------------------------------------------
+struct FastDiv {
+    uint32_t d, M, sh;
+    __host__ __device__ __forceinline__ uint32_t div(uint32_t n) const {
+        return (uint32_t)(((uint64_t)n * (uint64_t)M) >> sh);
+    }
+    __host__ __device__ __forceinline__ void divmod(uint32_t n, uint32_t& q, uint32_t& r) const {
+        q = div(n);
+        r = n - q * d;
+    }
+};
+
+inline FastDiv make_fastdiv(uint32_t d) {
+    FastDiv f;
+    f.d = d;
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;
+    f.M = (uint32_t)(((1ull << (31 + l)) / d) + 1ull);
+    f.sh = 31 + l;
+    return f;
+}
+
+constexpr uint32_t kNoGroup = 0xFFFFFFFFu;
+constexpr uint32_t kFullMask = 0xFFFFFFFFu;
+
+// ---------------------------------------------------------------------------------------
+// Warp-level run accumulator for per-group min/max (Eq. 4).
+// A warp walks memory in order, so the group of its elements changes rarely.  While all
+// lanes see the same group the partial min/max stay in registers; a change of group (or
+// a warp that straddles several groups) is resolved with warp reductions on the ordered
+// keys and one pair of atomics per group.
+// ---------------------------------------------------------------------------------------
+struct WarpRun {
+    uint32_t g, kmn, kmx;
+};
+
+__device__ __forceinline__ void run_flush(WarpRun& r, uint32_t* kmin, uint32_t* kmax) {
+    if (r.g != kNoGroup) {
+        uint32_t a = __reduce_max_sync(kFullMask, r.kmn);
+        uint32_t b = __reduce_max_sync(kFullMask, r.kmx);
+        if ((threadIdx.x & 31) == 0) {
+            atomicMax(kmin + r.g, a);
+            atomicMax(kmax + r.g, b);
+        }
+    }
+    r.g = kNoGroup;
+    r.kmn = 0;
+    r.kmx = 0;
+}
+
+// must be called by all 32 lanes of a warp
+__device__ __forceinline__ void run_add(WarpRun& r, bool valid, uint32_t g, uint32_t mn, uint32_t mx,
+                                        uint32_t* kmin, uint32_t* kmax) {
+    uint32_t pending = __ballot_sync(kFullMask, valid);
+    if (!pending) return;
+    const int lane = threadIdx.x & 31;
+    uint32_t first = __shfl_sync(kFullMask, g, __ffs(pending) - 1);
+    bool uniform = __all_sync(kFullMask, !valid || g == first);
+    if (!valid) {
+        mn = 0;
+        mx = 0;
+    }
+    if (uniform) {
+        if (first != r.g) {
+            run_flush(r, kmin, kmax);
+            r.g = first;
+        }
+        r.kmn = max(r.kmn, mn);
+        r.kmx = max(r.kmx, mx);
+        return;
+    }
+    run_flush(r, kmin, kmax);
+    while (pending) {
+        int src = __ffs(pending) - 1;
+        uint32_t cur = __shfl_sync(kFullMask, g, src);
+        bool mine = valid && g == cur;
+        uint32_t a = __reduce_max_sync(kFullMask, mine ? mn : 0u);
+        uint32_t b = __reduce_max_sync(kFullMask, mine ? mx : 0u);
+        if (lane == src) {
+            atomicMax(kmin + cur, a);
+            atomicMax(kmax + cur, b);
+        }
+        pending &= ~__ballot_sync(kFullMask, mine);
+    }
+}
+
+}  // namespace granq

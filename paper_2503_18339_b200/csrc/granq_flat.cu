@@ -1,0 +1,401 @@
+// Generic GranQ kernels: they accept any geometry and any pointer alignment and make no
+// assumption about what fits on chip.  The fused two-pass plan is
+//   range_flat_kernel (Eq. 4)  ->  finalize_range_kernel (Eq. 5)  ->  quant_flat_kernel (Eq. 1, 6, STE)
+// and the stand-alone entry points (range / forward / backward) use the same kernels.
+// Also here: the "conventional" per-channel loop the paper measures against (Section 5.3.2).
+#include "granq_internal.h"
+
+namespace granq {
+
+namespace {
+
+constexpr int kThreads = 256;
+constexpr uint32_t kTile = 8192;          // elements per CTA tile
+constexpr int kUnroll = 4;                // 16-byte loads in flight per thread
+constexpr uint32_t kTableMax = 1026;      // planes of one tile whose (s, z) are tabled in shared memory
+
+struct FlatGeom {
+    int64_t E, inner, C, ntiles;
+    FastDiv div_inner, div_C;   // valid when the divisor is < 2^30
+    int inner_big, C_big;       // divisor >= 2^30: at most one wrap inside a tile
+};
+
+FlatGeom make_flat(const Geom& g) {
+    FlatGeom f;
+    f.E = g.E;
+    f.inner = g.inner;
+    f.C = g.C;
+    f.ntiles = (g.E + kTile - 1) / kTile;
+    f.inner_big = g.inner >= (1ll << 30);
+    f.C_big = g.C >= (1ll << 30);
+    f.div_inner = make_fastdiv(f.inner_big ? 1u : (uint32_t)g.inner);
+    f.div_C = make_fastdiv(f.C_big ? 1u : (uint32_t)g.C);
+    return f;
+}
+
+// Position of a tile's first element: plane remainder and group of its first plane.
+struct TileBase {
+    int64_t rem;      // e0 % inner
+    uint32_t c;       // (e0 / inner) % C
+};
+
+__device__ __forceinline__ TileBase tile_base(const FlatGeom& g, int64_t e0) {
+    TileBase b;
+    int64_t p = e0 / g.inner;
+    b.rem = e0 - p * g.inner;
+    b.c = (uint32_t)(p % g.C);
+    return b;
+}
+
+// plane offset (relative to the tile's first plane) of the element k elements into the tile
+__device__ __forceinline__ uint32_t plane_offset(const FlatGeom& g, const TileBase& b, uint32_t k) {
+    if (g.inner_big) return (b.rem + (int64_t)k >= g.inner) ? 1u : 0u;
+    return g.div_inner.div((uint32_t)b.rem + k);
+}
+// group of the plane `q` planes after the tile's first plane
+__device__ __forceinline__ uint32_t group_at(const FlatGeom& g, const TileBase& b, uint32_t q) {
+    if (g.C_big) {
+        int64_t v = (int64_t)b.c + q;
+        return (uint32_t)(v >= g.C ? v - g.C : v);
+    }
+    uint32_t v = b.c + q, quo, r;
+    g.div_C.divmod(v, quo, r);
+    return r;
+}
+
+// ---- Eq. 4: range ------------------------------------------------------------------------------
+// V = elements per load: a 16-byte pack when planes and pointers allow it, else 1.
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads) range_flat_kernel(const T* __restrict__ x, FlatGeom g,
+                                                              uint32_t* __restrict__ kmin,
+                                                              uint32_t* __restrict__ kmax) {
+    __shared__ TileBase s_base;
+    WarpRun run{kNoGroup, 0u, 0u};
+    for (int64_t tile = blockIdx.x; tile < g.ntiles; tile += gridDim.x) {
+        const int64_t e0 = tile * (int64_t)kTile;
+        const uint32_t ne = (uint32_t)min((int64_t)kTile, g.E - e0);
+        __syncthreads();
+        if (threadIdx.x == 0) s_base = tile_base(g, e0);
+        __syncthreads();
+        const TileBase base = s_base;
+        for (uint32_t k0 = 0; k0 < ne; k0 += kThreads * V * kUnroll) {
+            uint32_t mn[kUnroll], mx[kUnroll], k[kUnroll];
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) {
+                k[j] = k0 + (j * kThreads + threadIdx.x) * V;
+                mn[j] = 0;
+                mx[j] = 0;
+                if (k[j] < ne) {
+                    if constexpr (V == 1) {
+                        uint32_t e = enc(load_scalar(x + e0 + k[j]));
+                        mn[j] = ~e;
+                        mx[j] = e;
+                    } else {
+                        Pack<T> p;
+                        p.raw = *reinterpret_cast<const uint4*>(x + e0 + k[j]);
+#pragma unroll
+                        for (int i = 0; i < V; ++i) {
+                            uint32_t e = enc(p.get(i));
+                            mn[j] = max(mn[j], ~e);
+                            mx[j] = max(mx[j], e);
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) {
+                bool valid = k[j] < ne;
+                uint32_t grp = valid ? group_at(g, base, plane_offset(g, base, k[j])) : kNoGroup;
+                run_add(run, valid, grp, mn[j], mx[j], kmin, kmax);
+            }
+        }
+    }
+    run_flush(run, kmin, kmax);
+}
+
+__global__ void finalize_range_kernel(const uint32_t* __restrict__ kmin, const uint32_t* __restrict__ kmax,
+                                      int64_t G, float* __restrict__ lo, float* __restrict__ hi, int bits,
+                                      float* __restrict__ s_opt, float* __restrict__ z_opt) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= G) return;
+    float l, h;
+    keys_to_range(kmin[i], kmax[i], l, h);
+    lo[i] = l;
+    hi[i] = h;
+    if (bits > 0) {
+        QParam p = make_qparam(l, h, (float)((1 << bits) - 1));
+        if (s_opt) s_opt[i] = p.s;
+        if (z_opt) z_opt[i] = p.z;
+    }
+}
+
+__global__ void params_kernel(const float* __restrict__ lo, const float* __restrict__ hi, int64_t G, int bits,
+                              float* __restrict__ s_opt, float* __restrict__ z_opt) {
+    int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    if (i >= G) return;
+    QParam p = make_qparam(__fadd_rn(lo[i], 0.0f), __fadd_rn(hi[i], 0.0f), (float)((1 << bits) - 1));
+    if (s_opt) s_opt[i] = p.s;
+    if (z_opt) z_opt[i] = p.z;
+}
+
+__device__ __forceinline__ uint32_t pack4(const uint8_t* b) {
+    return (uint32_t)b[0] | ((uint32_t)b[1] << 8) | ((uint32_t)b[2] << 16) | ((uint32_t)b[3] << 24);
+}
+
+// ---- Eq. 1, clamp, Eq. 6, STE: elementwise pass with a given per-group range ----------------------
+template <typename T, int V, int MODE>
+__global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restrict__ x, const T* __restrict__ gy,
+                                                              T* __restrict__ y, T* __restrict__ gx,
+                                                              uint8_t* __restrict__ codes,
+                                                              uint8_t* __restrict__ mask, FlatGeom g, float qmax,
+                                                              const float* __restrict__ lo,
+                                                              const float* __restrict__ hi) {
+    __shared__ TileBase s_base;
+    __shared__ QParam s_tab[kTableMax];
+    constexpr bool kFwd = (MODE & MODE_FWD) != 0, kBwd = (MODE & MODE_BWD) != 0;
+    for (int64_t tile = blockIdx.x; tile < g.ntiles; tile += gridDim.x) {
+        const int64_t e0 = tile * (int64_t)kTile;
+        const uint32_t ne = (uint32_t)min((int64_t)kTile, g.E - e0);
+        __syncthreads();
+        if (threadIdx.x == 0) s_base = tile_base(g, e0);
+        __syncthreads();
+        const TileBase base = s_base;
+        const uint32_t nplanes = plane_offset(g, base, ne - 1) + 1;
+        const bool tabled = nplanes <= kTableMax;
+        if (tabled) {
+            for (uint32_t q = threadIdx.x; q < nplanes; q += kThreads) {
+                uint32_t grp = group_at(g, base, q);
+                s_tab[q] = make_qparam(__fadd_rn(lo[grp], 0.0f), __fadd_rn(hi[grp], 0.0f), qmax);
+            }
+            __syncthreads();
+        }
+        for (uint32_t k0 = 0; k0 < ne; k0 += kThreads * V * kUnroll) {
+            uint32_t k[kUnroll];
+            Pack<T> px[kUnroll], pg[kUnroll];
+            float sx[kUnroll], sg[kUnroll];
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) {
+                k[j] = k0 + (j * kThreads + threadIdx.x) * V;
+                if (k[j] < ne) {
+                    if constexpr (V == 1) {
+                        sx[j] = load_scalar(x + e0 + k[j]);
+                        if constexpr (kBwd) sg[j] = load_scalar(gy + e0 + k[j]);
+                    } else {
+                        px[j].raw = ld_stream_16(x + e0 + k[j]);
+                        if constexpr (kBwd) pg[j].raw = ld_stream_16(gy + e0 + k[j]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < kUnroll; ++j) {
+                if (k[j] >= ne) continue;
+                const uint32_t q = plane_offset(g, base, k[j]);
+                QParam p;
+                if (tabled) {
+                    p = s_tab[q];
+                } else {
+                    uint32_t grp = group_at(g, base, q);
+                    p = make_qparam(__fadd_rn(lo[grp], 0.0f), __fadd_rn(hi[grp], 0.0f), qmax);
+                }
+                const int64_t e = e0 + k[j];
+                if constexpr (V == 1) {
+                    float yv;
+                    bool in;
+                    float code = quant_one(sx[j], p, qmax, yv, in);
+                    if constexpr (kFwd) {
+                        store_scalar(y + e, yv);
+                        if (codes) codes[e] = (uint8_t)code;
+                    }
+                    if constexpr (kBwd) {
+                        store_scalar(gx + e, in ? sg[j] : 0.0f);
+                        if (mask) mask[e] = in ? 1 : 0;
+                    }
+                } else {
+                    Pack<T> py, pgx;
+                    uint8_t cb[V], mb[V];
+#pragma unroll
+                    for (int i = 0; i < V; ++i) {
+                        float yv;
+                        bool in;
+                        float code = quant_one(px[j].get(i), p, qmax, yv, in);
+                        py.set(i, yv);
+                        cb[i] = (uint8_t)code;
+                        mb[i] = in ? 1 : 0;
+                        if constexpr (kBwd) pgx.set(i, in ? pg[j].get(i) : 0.0f);
+                    }
+                    if constexpr (kFwd) {
+                        st_stream_16(y + e, py.raw);
+                        if (codes) {
+#pragma unroll
+                            for (int i = 0; i < V; i += 4) *reinterpret_cast<uint32_t*>(codes + e + i) = pack4(cb + i);
+                        }
+                    }
+                    if constexpr (kBwd) {
+                        st_stream_16(gx + e, pgx.raw);
+                        if (mask) {
+#pragma unroll
+                            for (int i = 0; i < V; i += 4) *reinterpret_cast<uint32_t*>(mask + e + i) = pack4(mb + i);
+                        }
+                    }
+                }
+            }
+        }
+    }
+}
+
+// ---- the "conventional" per-channel scheme (Section 5.3.2): one group per launch ------------------
+template <typename T, bool IS_MAX>
+__global__ void __launch_bounds__(kThreads) naive_extreme_kernel(const T* __restrict__ x, Geom g, int64_t c,
+                                                                 uint32_t* __restrict__ key) {
+    uint32_t acc = 0;
+    for (int64_t o = blockIdx.x; o < g.outer; o += gridDim.x) {
+        const T* plane = x + (o * g.C + c) * g.inner;
+        for (int64_t i = threadIdx.x; i < g.inner; i += kThreads) {
+            uint32_t e = enc(load_scalar(plane + i));
+            acc = max(acc, IS_MAX ? e : ~e);
+        }
+    }
+    acc = __reduce_max_sync(kFullMask, acc);
+    if ((threadIdx.x & 31) == 0) atomicMax(key, acc);
+}
+
+template <typename T, int MODE>
+__global__ void __launch_bounds__(kThreads) naive_quant_kernel(const T* __restrict__ x, const T* __restrict__ gy,
+                                                               T* __restrict__ y, T* __restrict__ gx,
+                                                               uint8_t* __restrict__ codes,
+                                                               uint8_t* __restrict__ mask, Geom g, int64_t c,
+                                                               float qmax, const uint32_t* __restrict__ kmin,
+                                                               const uint32_t* __restrict__ kmax,
+                                                               float* __restrict__ lo_out,
+                                                               float* __restrict__ hi_out) {
+    constexpr bool kFwd = (MODE & MODE_FWD) != 0, kBwd = (MODE & MODE_BWD) != 0;
+    float lo, hi;
+    keys_to_range(kmin[c], kmax[c], lo, hi);
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        lo_out[c] = lo;
+        hi_out[c] = hi;
+    }
+    const QParam p = make_qparam(lo, hi, qmax);
+    for (int64_t o = blockIdx.x; o < g.outer; o += gridDim.x) {
+        const int64_t b = (o * g.C + c) * g.inner;
+        for (int64_t i = threadIdx.x; i < g.inner; i += kThreads) {
+            float yv;
+            bool in;
+            float code = quant_one(load_scalar(x + b + i), p, qmax, yv, in);
+            if constexpr (kFwd) {
+                store_scalar(y + b + i, yv);
+                if (codes) codes[b + i] = (uint8_t)code;
+            }
+            if constexpr (kBwd) {
+                store_scalar(gx + b + i, in ? load_scalar(gy + b + i) : 0.0f);
+                if (mask) mask[b + i] = in ? 1 : 0;
+            }
+        }
+    }
+}
+
+bool aligned16(const void* p) { return p == nullptr || ((uintptr_t)p & 15) == 0; }
+
+int flat_grid(const FlatGeom& f) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    int64_t cap = (int64_t)sms * 8;
+    return (int)(f.ntiles < cap ? f.ntiles : cap);
+}
+
+template <typename T>
+cudaError_t range_flat_t(const void* x, const Geom& g, uint32_t* kmin, uint32_t* kmax, cudaStream_t st) {
+    FlatGeom f = make_flat(g);
+    constexpr int VF = Pack<T>::V;
+    bool vec = aligned16(x) && (g.inner % VF == 0);
+    int grid = flat_grid(f);
+    if (vec)
+        range_flat_kernel<T, VF><<<grid, kThreads, 0, st>>>((const T*)x, f, kmin, kmax);
+    else
+        range_flat_kernel<T, 1><<<grid, kThreads, 0, st>>>((const T*)x, f, kmin, kmax);
+    return cudaGetLastError();
+}
+
+template <typename T, int MODE>
+cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float* lo, const float* hi,
+                         cudaStream_t st) {
+    FlatGeom f = make_flat(g);
+    constexpr int VF = Pack<T>::V;
+    bool vec = (g.inner % VF == 0) && aligned16(io.x) && aligned16(io.gy) && aligned16(io.y) && aligned16(io.gx) &&
+               ((uintptr_t)io.codes % 4 == 0) && ((uintptr_t)io.mask % 4 == 0);
+    int grid = flat_grid(f);
+    float qmax = (float)((1 << bits) - 1);
+    if (vec)
+        quant_flat_kernel<T, VF, MODE><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
+                                                                  (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
+    else
+        quant_flat_kernel<T, 1, MODE><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
+                                                                 (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
+    return cudaGetLastError();
+}
+
+template <typename T, int MODE>
+cudaError_t naive_t(const QuantIO& io, const Geom& g, int bits, uint32_t* kmin, uint32_t* kmax, float* lo,
+                    float* hi, cudaStream_t st, int* launches) {
+    int grid = (int)(g.outer < 1024 ? g.outer : 1024);
+    float qmax = (float)((1 << bits) - 1);
+    int n = 0;
+    for (int64_t c = 0; c < g.C; ++c) {
+        naive_extreme_kernel<T, false><<<grid, kThreads, 0, st>>>((const T*)io.x, g, c, kmin + c);
+        naive_extreme_kernel<T, true><<<grid, kThreads, 0, st>>>((const T*)io.x, g, c, kmax + c);
+        naive_quant_kernel<T, MODE><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
+                                                               (T*)io.gx, io.codes, io.mask, g, c, qmax, kmin,
+                                                               kmax, lo, hi);
+        n += 3;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+    }
+    if (launches) *launches = n;
+    return cudaSuccess;
+}
+
+}  // namespace
+
+cudaError_t launch_range_flat(const void* x, int dtype, const Geom& g, uint32_t* kmin, uint32_t* kmax,
+                              cudaStream_t st) {
+    return dtype == 0 ? range_flat_t<float>(x, g, kmin, kmax, st) : range_flat_t<__nv_bfloat16>(x, g, kmin, kmax, st);
+}
+
+cudaError_t launch_finalize_range(const uint32_t* kmin, const uint32_t* kmax, int64_t G, float* lo, float* hi,
+                                  int bits, float* s_opt, float* z_opt, cudaStream_t st) {
+    int grid = (int)((G + 255) / 256);
+    finalize_range_kernel<<<grid, 256, 0, st>>>(kmin, kmax, G, lo, hi, bits, s_opt, z_opt);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_params(const float* lo, const float* hi, int64_t G, int bits, float* s_opt, float* z_opt,
+                          cudaStream_t st) {
+    int grid = (int)((G + 255) / 256);
+    params_kernel<<<grid, 256, 0, st>>>(lo, hi, G, bits, s_opt, z_opt);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_quant_flat(const QuantIO& io, int mode, int dtype, const Geom& g, int bits, const float* lo,
+                              const float* hi, cudaStream_t st) {
+    if (dtype == 0) {
+        if (mode == MODE_FWD) return quant_flat_t<float, MODE_FWD>(io, g, bits, lo, hi, st);
+        if (mode == MODE_BWD) return quant_flat_t<float, MODE_BWD>(io, g, bits, lo, hi, st);
+        return quant_flat_t<float, MODE_BOTH>(io, g, bits, lo, hi, st);
+    }
+    if (mode == MODE_FWD) return quant_flat_t<__nv_bfloat16, MODE_FWD>(io, g, bits, lo, hi, st);
+    if (mode == MODE_BWD) return quant_flat_t<__nv_bfloat16, MODE_BWD>(io, g, bits, lo, hi, st);
+    return quant_flat_t<__nv_bfloat16, MODE_BOTH>(io, g, bits, lo, hi, st);
+}
+
+cudaError_t launch_naive(const QuantIO& io, int mode, int dtype, const Geom& g, int bits, uint32_t* kmin,
+                         uint32_t* kmax, float* lo, float* hi, cudaStream_t st, int* launches) {
+    if (dtype == 0) {
+        if (mode == MODE_FWD) return naive_t<float, MODE_FWD>(io, g, bits, kmin, kmax, lo, hi, st, launches);
+        return naive_t<float, MODE_BOTH>(io, g, bits, kmin, kmax, lo, hi, st, launches);
+    }
+    if (mode == MODE_FWD) return naive_t<__nv_bfloat16, MODE_FWD>(io, g, bits, kmin, kmax, lo, hi, st, launches);
+    return naive_t<__nv_bfloat16, MODE_BOTH>(io, g, bits, kmin, kmax, lo, hi, st, launches);
+}
+
+}  // namespace granq

@@ -1,0 +1,100 @@
+// Host-side declarations shared by the translation units of the GranQ library.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "granq_device.cuh"
+
+namespace granq {
+
+// A tensor reduced to channel-group form: element e lies in plane p = e / inner and in
+// group p % C.  Sample-channel grouping is (outer = 1, C = outer * C); tensor grouping is
+// (outer = 1, C = 1, inner = E).
+struct Geom {
+    int64_t E;      // elements
+    int64_t outer;  // slabs
+    int64_t C;      // groups (< 2^31)
+    int64_t inner;  // contiguous elements of one (slab, group) plane
+};
+
+// Workspace layout (all plans): a 256-byte header whose first word is the device status,
+// then G min-keys, G max-keys, then G + 1 wave arrival counters.
+constexpr size_t kWsHeaderBytes = 256;
+struct Workspace {
+    uint32_t* status;
+    uint32_t* kmin;
+    uint32_t* kmax;
+    uint32_t* counters;
+    size_t clear_bytes;  // bytes from the start that must be zero before a launch
+};
+inline size_t workspace_bytes_for(int64_t G) {
+    size_t b = kWsHeaderBytes + (size_t)G * 8 + ((size_t)G + 1) * 4;
+    return (b + 255) & ~(size_t)255;
+}
+inline Workspace carve_workspace(void* ws, int64_t G) {
+    Workspace w;
+    char* p = (char*)ws;
+    w.status = (uint32_t*)p;
+    w.kmin = (uint32_t*)(p + kWsHeaderBytes);
+    w.kmax = w.kmin + G;
+    w.counters = w.kmax + G;
+    w.clear_bytes = kWsHeaderBytes + (size_t)G * 8 + ((size_t)G + 1) * 4;
+    return w;
+}
+
+enum { MODE_FWD = 1, MODE_BWD = 2, MODE_BOTH = 3 };
+
+struct QuantIO {
+    const void* x;
+    const void* gy;   // MODE_BWD / MODE_BOTH
+    void* y;          // MODE_FWD / MODE_BOTH
+    void* gx;         // MODE_BWD / MODE_BOTH
+    uint8_t* codes;   // optional
+    uint8_t* mask;    // optional
+};
+
+// ---- generic ("flat") kernels: any geometry, any alignment --------------------------------
+// keys must be zero on entry; accumulates ordered min/max keys per group
+cudaError_t launch_range_flat(const void* x, int dtype, const Geom& g, uint32_t* kmin, uint32_t* kmax,
+                              cudaStream_t st);
+// keys -> lo / hi (and s / z when bits > 0 and the pointers are given)
+cudaError_t launch_finalize_range(const uint32_t* kmin, const uint32_t* kmax, int64_t G, float* lo, float* hi,
+                                  int bits, float* s_opt, float* z_opt, cudaStream_t st);
+// lo / hi -> s / z
+cudaError_t launch_params(const float* lo, const float* hi, int64_t G, int bits, float* s_opt, float* z_opt,
+                          cudaStream_t st);
+// elementwise quantize / backward with a per-group range in lo / hi
+cudaError_t launch_quant_flat(const QuantIO& io, int mode, int dtype, const Geom& g, int bits, const float* lo,
+                              const float* hi, cudaStream_t st);
+// the "conventional" scheme: a host loop over groups with three launches each
+cudaError_t launch_naive(const QuantIO& io, int mode, int dtype, const Geom& g, int bits, uint32_t* kmin,
+                         uint32_t* kmax, float* lo, float* hi, cudaStream_t st, int* launches);
+
+// ---- on-chip staged persistent kernel ------------------------------------------------------
+struct StagedPlan {
+    bool ok;
+    int grid, threads, depth;      // CTAs, threads per CTA, buffers per CTA
+    uint32_t smem_bytes;           // dynamic shared memory per CTA
+    uint32_t buf_units;            // 16-byte units per buffer
+    uint32_t cw;                   // channels per wave
+    uint32_t cu;                   // units per chunk
+    uint32_t nwaves;
+};
+// Test / tuning overrides of the planner (0 = automatic).
+struct StagedTuning {
+    int depth;            // force the number of buffers per CTA (1..3)
+    int max_buf_units;    // cap on 16-byte units per buffer (forces many small waves)
+    int grid;             // cap on the number of CTAs
+    int spin_limit;       // iteration limit of the wait on a wave's arrival count
+    int extra_arrivals;   // test hook: arrivals a wave waits for beyond the grid size (never come)
+};
+StagedPlan plan_staged(int dtype, const Geom& g, const QuantIO& io, int device, const StagedTuning& tune);
+StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_count, int smem_optin,
+                          const StagedTuning& tune);
+cudaError_t launch_staged(const StagedPlan& plan, const QuantIO& io, int mode, int dtype, const Geom& g, int bits,
+                          const Workspace& ws, float* lo, float* hi, float* s_opt, float* z_opt,
+                          const StagedTuning& tune, cudaStream_t st);
+
+}  // namespace granq
