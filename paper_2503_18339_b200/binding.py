@@ -1,0 +1,295 @@
+"""Thin ctypes binding of libgranq.so (include/granq.h): argument marshalling only.
+
+PyTorch supplies device memory and the CUDA stream; every step of the path runs in the
+library's kernels.  There is no fallback: if the shared library is missing, or a tensor is
+not a contiguous CUDA tensor, the call raises.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from dataclasses import dataclass
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libgranq.so")
+
+F32, BF16 = 0, 1
+GROUP_CHANNEL, GROUP_SAMPLE_CHANNEL, GROUP_TENSOR = 0, 1, 2
+FLAG_FORCE_TWO_PASS, FLAG_FORCE_NAIVE, FLAG_FORCE_STAGED = 1, 2, 4
+PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED = 0, 1, 2
+KNOB_STAGED_DEPTH, KNOB_STAGED_MAX_BUF_UNITS, KNOB_STAGED_GRID, KNOB_SPIN_LIMIT, KNOB_TEST_EXTRA_ARRIVALS = range(5)
+OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
+
+EXPORTS = [
+    "granq_status_string", "granq_num_groups", "granq_workspace_bytes", "granq_range",
+    "granq_fakequant_fwd", "granq_fakequant_bwd", "granq_fakequant_fused", "granq_workspace_status",
+    "granq_host_arena_bytes", "granq_fakequant_fused_host", "granq_fused_plan", "granq_staged_geometry",
+    "granq_tune",
+]
+
+
+class GranqError(RuntimeError):
+    def __init__(self, status: int, what: str):
+        self.status = status
+        super().__init__(f"{what}: {status_string(status)} (status {status})")
+
+
+_lib = None
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded shared library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(LIB_PATH):
+            raise RuntimeError(
+                f"{LIB_PATH} is missing: build it with `python -m paper_2503_18339_b200.build` "
+                "(needs nvcc); there is no fallback path")
+        L = ctypes.CDLL(LIB_PATH)
+        vp, i64p, ci, u32, sz = (ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.c_int, ctypes.c_uint32,
+                                 ctypes.c_size_t)
+        L.granq_status_string.restype = ctypes.c_char_p
+        L.granq_status_string.argtypes = [ci]
+        L.granq_num_groups.restype = ctypes.c_int64
+        L.granq_num_groups.argtypes = [i64p, ci, ci]
+        L.granq_workspace_bytes.restype = sz
+        L.granq_workspace_bytes.argtypes = [ci, i64p, ci, ci]
+        L.granq_range.restype = ci
+        L.granq_range.argtypes = [vp, ci, i64p, ci, ci, vp, vp, vp, sz, u32, vp]
+        L.granq_fakequant_fwd.restype = ci
+        L.granq_fakequant_fwd.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, u32, vp]
+        L.granq_fakequant_bwd.restype = ci
+        L.granq_fakequant_bwd.argtypes = [vp, vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, u32, vp]
+        L.granq_fakequant_fused.restype = ci
+        L.granq_fakequant_fused.argtypes = [vp, vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz,
+                                            u32, vp]
+        L.granq_workspace_status.restype = ci
+        L.granq_workspace_status.argtypes = [vp, vp]
+        L.granq_host_arena_bytes.restype = sz
+        L.granq_host_arena_bytes.argtypes = [ci, i64p, ci, ci, ci]
+        L.granq_fakequant_fused_host.restype = ci
+        L.granq_fakequant_fused_host.argtypes = [vp, vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, sz, u32,
+                                                 vp]
+        L.granq_fused_plan.restype = ci
+        L.granq_fused_plan.argtypes = [ci, i64p, ci, ci, ci, u32, ctypes.POINTER(ci)]
+        L.granq_staged_geometry.restype = ci
+        L.granq_staged_geometry.argtypes = [ci, i64p, ci, ci, ci, ci, i64p]
+        L.granq_tune.restype = ci
+        L.granq_tune.argtypes = [ci, ci]
+        _lib = L
+    return _lib
+
+
+def status_string(status: int) -> str:
+    return lib().granq_status_string(int(status)).decode()
+
+
+def _check(rc: int, what: str) -> None:
+    if rc != OK:
+        raise GranqError(rc, what)
+
+
+def _dims(shape):
+    if len(shape) != 4:
+        raise ValueError("granq tensors are 4-d (NCHW)")
+    return (ctypes.c_int64 * 4)(*[int(d) for d in shape])
+
+
+def _dtype(t: torch.Tensor) -> int:
+    if t.dtype == torch.float32:
+        return F32
+    if t.dtype == torch.bfloat16:
+        return BF16
+    raise TypeError(f"granq supports float32 and bfloat16 tensors, got {t.dtype}")
+
+
+def _dev(t: Optional[torch.Tensor], name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if not t.is_cuda:
+        raise ValueError(f"{name} must be a CUDA tensor (there is no CPU path)")
+    if not t.is_contiguous():
+        raise ValueError(f"{name} must be contiguous")
+    return t.data_ptr()
+
+
+def _host(t: Optional[torch.Tensor], name: str) -> Optional[int]:
+    if t is None:
+        return None
+    if t.is_cuda or not t.is_contiguous():
+        raise ValueError(f"{name} must be a contiguous host tensor")
+    return t.data_ptr()
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        return torch.cuda.current_stream().cuda_stream
+    return stream.cuda_stream if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def num_groups(shape, channel_axis: int = 1, group: int = GROUP_CHANNEL) -> int:
+    g = lib().granq_num_groups(_dims(shape), channel_axis, group)
+    if g < 0:
+        raise ValueError("invalid geometry")
+    return int(g)
+
+
+def workspace_bytes(dtype: int, shape, channel_axis: int = 1, group: int = GROUP_CHANNEL) -> int:
+    return int(lib().granq_workspace_bytes(dtype, _dims(shape), channel_axis, group))
+
+
+def make_workspace(x: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL) -> torch.Tensor:
+    n = workspace_bytes(_dtype(x), x.shape, channel_axis, group)
+    return torch.empty(n, dtype=torch.uint8, device=x.device)
+
+
+def tune(knob: int, value: int) -> None:
+    _check(lib().granq_tune(knob, value), "granq_tune")
+
+
+def fused_plan(dtype: int, shape, channel_axis: int = 1, group: int = GROUP_CHANNEL, with_backward: bool = True,
+               flags: int = 0):
+    """(plan, launches) the fused entry point would take for this geometry on the current device."""
+    n = ctypes.c_int(0)
+    p = lib().granq_fused_plan(dtype, _dims(shape), channel_axis, group, int(with_backward), flags, ctypes.byref(n))
+    if p < 0:
+        raise GranqError(-p, "granq_fused_plan")
+    return p, n.value
+
+
+def staged_geometry(dtype: int, shape, channel_axis: int = 1, group: int = GROUP_CHANNEL, sm_count: int = 148,
+                    smem_bytes: int = 232448):
+    """Host-only: wave / chunk geometry of the staged plan, or None if the geometry does not qualify."""
+    out = (ctypes.c_int64 * 8)()
+    rc = lib().granq_staged_geometry(dtype, _dims(shape), channel_axis, group, sm_count, smem_bytes, out)
+    if rc == ERR_UNSUPPORTED:
+        return None
+    _check(rc, "granq_staged_geometry")
+    keys = ["grid", "threads", "depth", "smem_bytes", "buf_units", "cw", "cu", "nwaves"]
+    return dict(zip(keys, [int(v) for v in out]))
+
+
+@dataclass
+class FakeQuantOut:
+    y: Optional[torch.Tensor] = None
+    gx: Optional[torch.Tensor] = None
+    lo: Optional[torch.Tensor] = None
+    hi: Optional[torch.Tensor] = None
+    s: Optional[torch.Tensor] = None
+    z: Optional[torch.Tensor] = None
+    codes: Optional[torch.Tensor] = None
+    mask: Optional[torch.Tensor] = None
+    workspace: Optional[torch.Tensor] = None
+
+
+def granq_range(x: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL, lo: torch.Tensor = None,
+                hi: torch.Tensor = None, workspace: torch.Tensor = None, flags: int = 0, stream=None):
+    """Per-group (lo, hi) of x: Eq. 4."""
+    G = num_groups(x.shape, channel_axis, group)
+    lo = torch.empty(G, dtype=torch.float32, device=x.device) if lo is None else lo
+    hi = torch.empty(G, dtype=torch.float32, device=x.device) if hi is None else hi
+    ws = make_workspace(x, channel_axis, group) if workspace is None else workspace
+    _check(lib().granq_range(_dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, _dev(lo, "lo"),
+                             _dev(hi, "hi"), _dev(ws, "workspace"), ws.numel(), flags, _stream(stream)),
+           "granq_range")
+    return lo, hi
+
+
+def granq_fakequant_fwd(x: torch.Tensor, bits: int, lo: torch.Tensor, hi: torch.Tensor, channel_axis: int = 1,
+                        group: int = GROUP_CHANNEL, y: torch.Tensor = None, want_codes: bool = False,
+                        want_params: bool = False, flags: int = 0, stream=None) -> FakeQuantOut:
+    """Quantize -> clamp -> dequantize with a given per-group range: Eq. 1, 2, 6."""
+    G = num_groups(x.shape, channel_axis, group)
+    o = FakeQuantOut(lo=lo, hi=hi)
+    o.y = torch.empty_like(x) if y is None else y
+    if want_codes:
+        o.codes = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+    if want_params:
+        o.s = torch.empty(G, dtype=torch.float32, device=x.device)
+        o.z = torch.empty(G, dtype=torch.float32, device=x.device)
+    _check(lib().granq_fakequant_fwd(_dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, bits,
+                                     _dev(lo, "lo"), _dev(hi, "hi"), _dev(o.y, "y"), _dev(o.codes, "codes"),
+                                     _dev(o.s, "s"), _dev(o.z, "z"), flags, _stream(stream)),
+           "granq_fakequant_fwd")
+    return o
+
+
+def granq_fakequant_bwd(gy: torch.Tensor, x: torch.Tensor, bits: int, lo: torch.Tensor, hi: torch.Tensor,
+                        channel_axis: int = 1, group: int = GROUP_CHANNEL, gx: torch.Tensor = None,
+                        want_mask: bool = False, flags: int = 0, stream=None) -> FakeQuantOut:
+    """Straight-through-estimator backward with a given per-group range."""
+    if gy.shape != x.shape or gy.dtype != x.dtype:
+        raise ValueError("gy must match x")
+    o = FakeQuantOut(lo=lo, hi=hi)
+    o.gx = torch.empty_like(x) if gx is None else gx
+    if want_mask:
+        o.mask = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+    _check(lib().granq_fakequant_bwd(_dev(gy, "gy"), _dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group,
+                                     bits, _dev(lo, "lo"), _dev(hi, "hi"), _dev(o.gx, "gx"), _dev(o.mask, "mask"),
+                                     flags, _stream(stream)),
+           "granq_fakequant_bwd")
+    return o
+
+
+def granq_fakequant_fused(x: torch.Tensor, bits: int, gy: torch.Tensor = None, channel_axis: int = 1,
+                          group: int = GROUP_CHANNEL, out: FakeQuantOut = None, want_codes: bool = False,
+                          want_mask: bool = False, want_params: bool = False, flags: int = 0,
+                          stream=None) -> FakeQuantOut:
+    """Range of x itself -> scale / zero-point -> y (and gx when gy is given), in one call.
+
+    `out` may carry preallocated tensors (y, gx, lo, hi, s, z, codes, mask, workspace);
+    whatever is missing is allocated here.
+    """
+    if gy is not None and (gy.shape != x.shape or gy.dtype != x.dtype):
+        raise ValueError("gy must match x")
+    G = num_groups(x.shape, channel_axis, group)
+    o = out if out is not None else FakeQuantOut()
+    dev = x.device
+    if o.y is None:
+        o.y = torch.empty_like(x)
+    if gy is not None and o.gx is None:
+        o.gx = torch.empty_like(x)
+    if o.lo is None:
+        o.lo = torch.empty(G, dtype=torch.float32, device=dev)
+    if o.hi is None:
+        o.hi = torch.empty(G, dtype=torch.float32, device=dev)
+    if want_params and o.s is None:
+        o.s = torch.empty(G, dtype=torch.float32, device=dev)
+        o.z = torch.empty(G, dtype=torch.float32, device=dev)
+    if want_codes and o.codes is None:
+        o.codes = torch.empty(x.shape, dtype=torch.uint8, device=dev)
+    if want_mask and gy is not None and o.mask is None:
+        o.mask = torch.empty(x.shape, dtype=torch.uint8, device=dev)
+    if o.workspace is None:
+        o.workspace = make_workspace(x, channel_axis, group)
+    _check(lib().granq_fakequant_fused(
+        _dev(x, "x"), _dev(gy, "gy"), _dtype(x), _dims(x.shape), channel_axis, group, bits,
+        _dev(o.y, "y"), _dev(o.gx if gy is not None else None, "gx"), _dev(o.lo, "lo"), _dev(o.hi, "hi"),
+        _dev(o.codes, "codes"), _dev(o.mask if gy is not None else None, "mask"), _dev(o.s, "s"), _dev(o.z, "z"),
+        _dev(o.workspace, "workspace"), o.workspace.numel(), flags, _stream(stream)), "granq_fakequant_fused")
+    return o
+
+
+def workspace_status(workspace: torch.Tensor, stream=None) -> int:
+    """Synchronises the stream and returns the device status word of the last staged call."""
+    return int(lib().granq_workspace_status(_dev(workspace, "workspace"), _stream(stream)))
+
+
+def host_arena_bytes(dtype: int, shape, channel_axis: int = 1, group: int = GROUP_CHANNEL,
+                     with_backward: bool = True) -> int:
+    return int(lib().granq_host_arena_bytes(dtype, _dims(shape), channel_axis, group, int(with_backward)))
+
+
+def granq_fakequant_fused_host(x: torch.Tensor, bits: int, gy: torch.Tensor, y: torch.Tensor, gx: torch.Tensor,
+                               lo: torch.Tensor, hi: torch.Tensor, arena: torch.Tensor, channel_axis: int = 1,
+                               group: int = GROUP_CHANNEL, s: torch.Tensor = None, z: torch.Tensor = None,
+                               flags: int = 0, stream=None) -> None:
+    """Fused path on HOST tensors (pinned memory recommended); `arena` is device scratch of
+    host_arena_bytes() bytes.  Returns when the host outputs are valid."""
+    _check(lib().granq_fakequant_fused_host(
+        _host(x, "x"), _host(gy, "gy"), _dtype(x), _dims(x.shape), channel_axis, group, bits,
+        _host(y, "y"), _host(gx, "gx"), _host(lo, "lo"), _host(hi, "hi"), _host(s, "s"), _host(z, "z"),
+        _dev(arena, "arena"), arena.numel(), flags, _stream(stream)), "granq_fakequant_fused_host")

@@ -1,0 +1,159 @@
+"""Host-only checks of the C ABI: the library builds, loads, exports every symbol that
+include/granq.h declares, rejects bad arguments before anything is launched, and plans the
+staged kernel's waves within the shared-memory budget."""
+import ctypes
+import os
+import random
+import re
+
+import pytest
+
+from paper_2503_18339_b200 import build as granq_build
+from paper_2503_18339_b200 import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def lib():
+    granq_build.build()
+    from paper_2503_18339_b200 import binding
+    return binding.lib()
+
+
+def declared_functions():
+    text = open(os.path.join(ROOT, "include", "granq.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(granq_[a-z_0-9]+)\s*\(", text)))
+
+
+def test_every_declared_symbol_is_exported(lib):
+    from paper_2503_18339_b200 import binding
+    names = declared_functions()
+    assert len(names) >= 13
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(binding.EXPORTS) == names
+
+
+def test_status_strings(lib):
+    from paper_2503_18339_b200 import binding
+    seen = {binding.status_string(i) for i in range(6)}
+    assert len(seen) == 6 and binding.status_string(99) == "unknown status"
+
+
+def test_geometry_queries(lib):
+    from paper_2503_18339_b200 import binding as b
+    shape = (8, 16, 7, 7)
+    assert b.num_groups(shape, 1, b.GROUP_CHANNEL) == 16
+    assert b.num_groups(shape, 1, b.GROUP_SAMPLE_CHANNEL) == 128
+    assert b.num_groups(shape, 1, b.GROUP_TENSOR) == 1
+    assert b.num_groups(shape, 0, b.GROUP_CHANNEL) == 8
+    assert b.workspace_bytes(b.F32, shape) % 256 == 0 and b.workspace_bytes(b.F32, shape) >= 256 + 16 * 12
+    assert b.workspace_bytes(7, shape) == 0
+    with pytest.raises(ValueError):
+        b.num_groups((8, 0, 7, 7))
+    with pytest.raises(ValueError):
+        b.num_groups((8, 16, 7, 7), channel_axis=4)
+    with pytest.raises(ValueError):
+        b.num_groups((1 << 20, 1 << 20, 2, 1))       # more than 2^40 elements
+
+
+def test_argument_errors_are_detected_before_any_launch(lib):
+    """Null pointers, bad bit-widths, bad enums and a missing workspace never reach the GPU
+    (this runs on a machine without one)."""
+    from paper_2503_18339_b200 import binding as b
+    dims = (ctypes.c_int64 * 4)(2, 3, 4, 4)
+    fake = ctypes.c_void_p(256 * 1024)                # never dereferenced on the host
+    far = ctypes.c_void_p(256 * 1024 * 1024)
+    r = lib.granq_range(None, b.F32, dims, 1, 0, fake, fake, fake, 4096, 0, None)
+    assert r == b.ERR_INVALID_ARG
+    r = lib.granq_range(fake, b.F32, dims, 1, 0, fake, fake, None, 0, 0, None)
+    assert r == b.ERR_WORKSPACE
+    r = lib.granq_range(fake, b.F32, dims, 1, 0, fake, fake, ctypes.c_void_p(256 * 1024 + 8), 4096, 0, None)
+    assert r == b.ERR_WORKSPACE                       # misaligned workspace
+    r = lib.granq_range(fake, b.F32, dims, 1, 0, fake, fake, fake, 64, 0, None)
+    assert r == b.ERR_WORKSPACE                       # too small
+    for bits in (0, 9, -1):
+        r = lib.granq_fakequant_fwd(fake, b.F32, dims, 1, 0, bits, fake, fake, far, None, None, None, 0, None)
+        assert r == b.ERR_INVALID_ARG
+    r = lib.granq_fakequant_fwd(fake, 5, dims, 1, 0, 4, fake, fake, far, None, None, None, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # bad dtype
+    r = lib.granq_fakequant_fwd(fake, b.F32, dims, 1, 3, 4, fake, fake, far, None, None, None, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # bad group mode
+    r = lib.granq_fakequant_fwd(fake, b.F32, dims, 1, 0, 4, fake, fake, fake, None, None, None, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # y overlaps x
+    r = lib.granq_fakequant_bwd(fake, far, b.F32, dims, 1, 0, 4, fake, fake, None, None, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # gx missing
+    # fused: gy without gx, mask without gy
+    r = lib.granq_fakequant_fused(fake, far, b.F32, dims, 1, 0, 4, ctypes.c_void_p(3 << 28), None, fake, fake,
+                                  None, None, None, None, fake, 4096, 0, None)
+    assert r == b.ERR_INVALID_ARG
+    r = lib.granq_fakequant_fused(fake, None, b.F32, dims, 1, 0, 4, far, None, fake, fake,
+                                  None, fake, None, None, fake, 4096, 0, None)
+    assert r == b.ERR_INVALID_ARG
+    assert lib.granq_tune(99, 0) == b.ERR_INVALID_ARG
+    assert lib.granq_workspace_status(None, None) == b.ERR_INVALID_ARG
+
+
+def test_binding_refuses_cpu_tensors(lib):
+    import torch
+    from paper_2503_18339_b200 import binding as b
+    x = torch.zeros(2, 3, 4, 4)
+    with pytest.raises(ValueError):
+        b.granq_fakequant_fused(x, 4, out=b.FakeQuantOut(
+            y=torch.empty_like(x), lo=torch.empty(3), hi=torch.empty(3), workspace=torch.empty(4096, dtype=torch.uint8)))
+
+
+def _check_geometry(shape, dt, grp, geo):
+    n, c, h, w = shape
+    V = 4 if dt == 0 else 8
+    outer, groups = (n, c) if grp == 0 else (1, n * c)
+    inner = h * w
+    cw, cu, nw = geo["cw"], geo["cu"], geo["nwaves"]
+    assert geo["smem_bytes"] <= 232448 and 1 <= geo["depth"] <= 3
+    assert (nw - 1) * cw < groups <= nw * cw
+    if nw > 1:
+        assert (cw * inner) % V == 0                       # every wave's slab starts on a 16-byte boundary
+    for ch in ({cw, groups - (nw - 1) * cw} if nw > 1 else {groups}):
+        units = ch * inner // V
+        cps = -(-units // cu)
+        nk = -(-outer * cps // geo["grid"])
+        assert nk * cu <= geo["buf_units"], (shape, geo, nk)
+
+
+def test_staged_plan_fits_the_shared_memory_budget_for_every_workload(lib):
+    from paper_2503_18339_b200 import binding as b
+    for cfg in range(1, 6):
+        for spec in wl.config_tensors(cfg):
+            for dt in ([b.F32, b.BF16] if cfg == 5 else [b.F32]):
+                for grp in (b.GROUP_CHANNEL, b.GROUP_SAMPLE_CHANNEL):
+                    geo = b.staged_geometry(dt, spec.shape, 1, grp)
+                    assert geo is not None, (spec.name, dt, grp)
+                    _check_geometry(spec.shape, dt, grp, geo)
+
+
+def test_staged_plan_under_forced_small_buffers(lib):
+    from paper_2503_18339_b200 import binding as b
+    rnd = random.Random(1)
+    planned = 0
+    try:
+        for _ in range(1500):
+            shape = (rnd.randint(1, 9), rnd.randint(1, 40), rnd.choice([1, 2, 4, 7, 8, 14, 28]),
+                     rnd.choice([4, 7, 8, 14, 16]))
+            dt = rnd.choice([0, 1])
+            V = 4 if dt == 0 else 8
+            b.tune(b.KNOB_STAGED_DEPTH, rnd.choice([0, 1, 2, 3]))
+            b.tune(b.KNOB_STAGED_MAX_BUF_UNITS, rnd.choice([0, 64, 100, 500]))
+            grid = rnd.choice([3, 5, 148])
+            geo = b.staged_geometry(dt, shape, sm_count=grid)
+            if (shape[1] * shape[2] * shape[3]) % V or shape[2] * shape[3] < V:
+                assert geo is None
+                continue
+            if geo is not None:
+                planned += 1
+                _check_geometry(shape, dt, 0, geo)
+    finally:
+        for k in range(5):
+            b.tune(k, 0)
+    assert planned > 500

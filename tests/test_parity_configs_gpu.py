@@ -1,0 +1,122 @@
+"""Parity on the five synthetic activation sets at their full sizes, in the launch
+configuration the benchmark times (default plan, fused forward + backward), every element
+compared with the CPU oracle: min / max, codes and STE mask bit-exact, y within
+1e-6 * scale (asserted bit-exact as well, which is what the arithmetic delivers)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import granq_oracle as orc
+from paper_2503_18339_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def b():
+    from paper_2503_18339_b200 import binding
+    binding.lib()
+    for k in range(5):
+        binding.tune(k, 0)
+    return binding
+
+
+def to_dev(a):
+    if a.dtype == np.uint16:
+        return torch.from_numpy(a.view(np.int16)).cuda().view(torch.bfloat16)
+    return torch.from_numpy(a).cuda()
+
+
+def to_np(t):
+    if t.dtype == torch.bfloat16:
+        return t.view(torch.int16).cpu().numpy().view(np.uint16)
+    return t.cpu().numpy()
+
+
+def same_bits(a, c):
+    v = np.uint16 if a.dtype == np.uint16 else np.uint32
+    return np.array_equal(np.ascontiguousarray(a).view(v), np.ascontiguousarray(c).view(v))
+
+
+def widen64(a):
+    return (wl.bf16_bits_to_f32(a) if a.dtype == np.uint16 else a).astype(np.float64)
+
+
+def check(b, x, gy, bits, mode, with_codes, expect_staged=True):
+    dt = b.F32 if x.dtype == np.float32 else b.BF16
+    plan, _ = b.fused_plan(dt, x.shape, group=mode, with_backward=gy is not None)
+    if expect_staged:
+        assert plan == b.PLAN_STAGED, "the benchmarked plan for this tensor is the staged one"
+    ref = orc.fused(x, bits, gy=gy, group_mode=mode, want_codes=with_codes)
+    got = b.granq_fakequant_fused(to_dev(x), bits, gy=None if gy is None else to_dev(gy), group=mode,
+                                  want_codes=with_codes, want_mask=with_codes, want_params=True)
+    assert b.workspace_status(got.workspace) == b.OK
+    assert same_bits(to_np(got.lo), ref.lo) and same_bits(to_np(got.hi), ref.hi)
+    assert same_bits(to_np(got.s), ref.s) and same_bits(to_np(got.z), ref.z)
+    y = to_np(got.y)
+    n, c = x.shape[0], x.shape[1]
+    s_of = ref.s.astype(np.float64)
+    tol = 1e-6 * (s_of.reshape(1, c, 1, 1) if mode == orc.GROUP_CHANNEL else s_of.reshape(n, c, 1, 1))
+    assert np.all(np.abs(widen64(y) - widen64(ref.y)) <= tol)
+    assert same_bits(y, ref.y)
+    if with_codes:
+        assert np.array_equal(to_np(got.codes), ref.codes)
+    if gy is not None:
+        assert same_bits(to_np(got.gx), ref.gx)
+        if with_codes:
+            assert np.array_equal(to_np(got.mask), ref.mask)
+    return ref
+
+
+def distinct(specs):
+    seen, out = set(), []
+    for s in specs:
+        if s.shape not in seen:
+            seen.add(s.shape)
+            out.append(s)
+    return out
+
+
+def test_config1_resnet20_first_layer(b):
+    spec = wl.config_tensors(1)[0]
+    x, gy = wl.make_activation(spec), wl.make_upstream_grad(spec)
+    ref = check(b, x, gy, 3, orc.GROUP_CHANNEL, True)
+    assert (ref.lo == 0).all() and (ref.z == 0).all()          # post-ReLU: every channel starts at 0
+    check(b, x, gy, 3, orc.GROUP_SAMPLE_CHANNEL, True)
+
+
+@pytest.mark.parametrize("spec", distinct(wl.config_tensors(2)), ids=lambda s: s.name)
+def test_config2_resnet20_cifar_set(b, spec):
+    x, gy = wl.make_activation(spec), wl.make_upstream_grad(spec)
+    dead = np.flatnonzero(wl.channel_sigma(spec) == 0)
+    for bits in spec.bits:
+        ref = check(b, x, gy, bits, orc.GROUP_CHANNEL, True)
+        assert (ref.codes[:, dead] == 0).all() and (ref.y[:, dead] == 0).all()
+    check(b, x, gy, 3, orc.GROUP_SAMPLE_CHANNEL, True)
+
+
+@pytest.mark.parametrize("spec", wl.config_tensors(3) + wl.config_tensors(4), ids=lambda s: s.name)
+def test_config3_4_imagenet_shaped(b, spec):
+    x, gy = wl.make_activation(spec), wl.make_upstream_grad(spec)
+    check(b, x, gy, spec.bits[0], orc.GROUP_CHANNEL, True)
+    check(b, x, gy, spec.bits[1], orc.GROUP_CHANNEL, False)     # exactly what the benchmark launches
+    if spec.numel <= 30_000_000:
+        check(b, x, gy, spec.bits[0], orc.GROUP_SAMPLE_CHANNEL, True)
+
+
+CFG5_BITS = {   # (fused bits, forward-only bits) per tensor and dtype: bits 2..8 all appear both ways
+    (0, "f32"): (2, 8), (0, "bf16"): (3, 7), (1, "f32"): (4, 6), (1, "bf16"): (5, 2),
+    (2, "f32"): (6, 3), (2, "bf16"): (7, 4), (3, "f32"): (8, 5), (3, "bf16"): (2, 8),
+}
+
+
+@pytest.mark.parametrize("spec", wl.config_tensors(5), ids=lambda s: s.name)
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_config5_bandwidth_sweep(b, spec, dtype):
+    x, gy = wl.make_activation(spec), wl.make_upstream_grad(spec)
+    if dtype == "bf16":
+        x, gy = wl.to_bf16_bits(x), wl.to_bf16_bits(gy)
+    fused_bits, fwd_bits = CFG5_BITS[(spec.index, dtype)]
+    ref = check(b, x, gy, fused_bits, orc.GROUP_CHANNEL, True)
+    assert (ref.z != 0).any()                                     # signed data: the zero-point path is live
+    check(b, x, None, fwd_bits, orc.GROUP_CHANNEL, False)
