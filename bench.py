@@ -1,0 +1,378 @@
+#!/usr/bin/env python
+"""Benchmark of the GranQ fake-quantization hot path on B200.
+
+One step = fused forward + backward fake-quantization (range -> scale / zero-point ->
+quantize / clamp / dequantize -> STE backward, one library call per tensor) of every tensor
+of the ResNet-18 and MobileNetV2 ImageNet-shaped activation sets (12 fp32 tensors, batch
+128) at both of their bit-widths (4 and 5): 24 calls, 914 M elements, 14.6 GB of
+algorithmic traffic (16 B per element: read x, read gy, write y, write gx).
+
+Prints ONE JSON line.  `value` is algorithmic GB/s with all tensors resident in HBM;
+`e2e` is the same metric through the host-buffer entry point (pinned host memory, copies
+inside the timed region); `roofline` relates the dominant kernel to the measured HBM copy
+bandwidth; `cpu_baseline` is the CPU oracle timed on a bounded sample of the same workload.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import hashlib
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2503_18339_b200 import workloads as wl  # noqa: E402
+
+METRIC = "fake-quant fwd+bwd GB/s (algorithmic bytes: 16 B/element fp32)"
+UNIT = "GB/s"
+WORKLOAD = ("configs 3+4: ResNet-18 + MobileNetV2 ImageNet-shaped activations, batch 128, fp32, "
+            "12 tensors x b in {4,5}, fused fwd+bwd, channel groups over (n,h,w)")
+BYTES_PER_ELEM = 16
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+CPU_SAMPLE = "cfg3.1-3.4 ([128,64,56,56] [128,128,28,28] [128,256,14,14] [128,512,7,7]), b=4 and b=5, fused fwd+bwd"
+
+
+def workload_specs():
+    return wl.config_tensors(3) + wl.config_tensors(4)
+
+
+def measured_peak():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as fh:
+            return float(json.load(fh)["hbm_gbs"]), "measured (MEASURED_PEAKS.json hbm_gbs)"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
+
+
+def kernel_source_hash() -> str:
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_2503_18339_b200", "csrc")
+    for name in sorted(os.listdir(csrc)):
+        with open(os.path.join(csrc, name), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def recorded_traffic():
+    """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None
+    when there is none or the kernel sources have changed since it was taken."""
+    path = os.path.join(ROOT, "profiles", "staged_kernel_traffic.json")
+    try:
+        with open(path) as fh:
+            rec = json.load(fh)
+        if rec.get("kernel_source_hash") != kernel_source_hash():
+            return None
+        return rec
+    except Exception:
+        return None
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [c.strip() for c in line.split(",")]))
+
+    def stop(self, t0: float, t1: float):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        rows = [r for (t, r) in self.rows if t0 <= t <= t1 + 0.2 and len(r) >= 7] or \
+               [r for (_, r) in self.rows if len(r) >= 7]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        sm = [float(r[0]) for r in rows]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[3 + i].lower().startswith("active") for r in rows)]
+        return {"sm_mhz": statistics.median(sm), "sm_max_mhz": float(rows[0][1]), "reasons": reasons,
+                "samples": len(rows), "power_w_max": max(float(r[2]) for r in rows)}
+
+
+def time_oracle(specs_bits):
+    """Seconds the CPU oracle needs for fused fwd+bwd on the given (spec, bits) list; elements processed."""
+    from oracle import granq_oracle as orc
+    orc.lib()
+    elems, secs = 0, 0.0
+    cache = {}
+    for spec, bits in specs_bits:
+        if spec.name not in cache:
+            cache[spec.name] = (wl.make_activation(spec), wl.make_upstream_grad(spec))
+        x, gy = cache[spec.name]
+        t = time.perf_counter()
+        orc.fused(x, bits, gy=gy, want_codes=False)
+        secs += time.perf_counter() - t
+        elems += spec.numel
+    return secs, elems
+
+
+def cpu_sample():
+    specs = wl.config_tensors(3)[1:]
+    return [(s, b) for s in specs for b in s.bits]
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: each step is the bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    sample = cpu_sample()
+    for _ in range(min(args.warmup, 1)):
+        time_oracle(sample[:1])
+    total_s, total_e = 0.0, 0
+    for _ in range(args.steps):
+        s, e = time_oracle(sample)
+        total_s += s
+        total_e += e
+    value = total_e * BYTES_PER_ELEM / total_s / 1e9
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total_s / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "step": "bounded sample: " + CPU_SAMPLE},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": CPU_SAMPLE},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "elements_per_s": total_e / total_s,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--table", action="store_true", help="also print a per-tensor table to stderr")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        if args.steps > 3:
+            args.steps = 3          # each step is ~10 s of CPU work
+        run_reference(args)
+        return
+
+    import torch
+    import torch.distributed as dist
+    from paper_2503_18339_b200 import binding as b
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    b.lib()
+    warmup = max(args.warmup, 3)
+
+    specs = workload_specs()
+    # ---- host (pinned) inputs and outputs; every rank has its own batch (weak scaling, no exchange) ----
+    host = []
+    for s in specs:
+        xs = torch.empty(s.shape, dtype=torch.float32).pin_memory()
+        gs = torch.empty(s.shape, dtype=torch.float32).pin_memory()
+        wl.make_activation(s, out=xs.numpy(), block_offset=1000 * rank)
+        wl.make_upstream_grad(s, out=gs.numpy(), block_offset=1000 * rank)
+        host.append((xs, gs))
+    dev = []
+    for s, (xs, gs) in zip(specs, host):
+        x = xs.cuda(non_blocking=True)
+        gy = gs.cuda(non_blocking=True)
+        out = b.FakeQuantOut(y=torch.empty_like(x), gx=torch.empty_like(x),
+                             lo=torch.empty(s.shape[1], device="cuda"), hi=torch.empty(s.shape[1], device="cuda"),
+                             workspace=b.make_workspace(x))
+        dev.append((x, gy, out))
+    torch.cuda.synchronize()
+    calls = [(i, bits) for i, s in enumerate(specs) for bits in s.bits]
+    elems_per_step = sum(specs[i].numel for i, _ in calls)
+    bytes_per_step = elems_per_step * BYTES_PER_ELEM
+    plans = [b.fused_plan(b.F32, specs[i].shape) for i, _ in calls]
+    launches_per_step = sum(n for _, n in plans)
+    stream = torch.cuda.current_stream()
+
+    def step(events=None):
+        for ci, (i, bits) in enumerate(calls):
+            x, gy, out = dev[i]
+            if events is not None:
+                events[ci][0].record(stream)
+            b.granq_fakequant_fused(x, bits, gy=gy, out=out, stream=stream)
+            if events is not None:
+                events[ci][1].record(stream)
+
+    for _ in range(warmup):
+        step()
+    torch.cuda.synchronize()
+    for _, _, out in dev:
+        assert b.workspace_status(out.workspace) == b.OK
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region: K steps, device time, max over ranks ----
+    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in calls]
+          for _ in range(args.steps)]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sampler = ClockSampler(local)
+    sampler.start()
+    time.sleep(0.25)
+    barrier()
+    t0 = time.time()
+    e0.record(stream)
+    for k in range(args.steps):
+        step(ev[k])
+    e1.record(stream)
+    barrier()
+    t1 = time.time()
+    total_ms = e0.elapsed_time(e1)
+    # keep the GPU under the same load a little longer so the clock sampler sees it
+    if t1 - t0 < 0.6:
+        tend = time.time() + 0.6
+        while time.time() < tend:
+            step()
+        torch.cuda.synchronize()
+        t1 = time.time()
+    clocks = sampler.stop(t0, t1)
+    if world > 1:
+        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        total_ms = float(t.item())
+    ms_per_step = total_ms / args.steps
+    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
+
+    # ---- per-call device times inside the timed region -> roofline of the dominant kernel ----
+    per_call_ms = [statistics.mean(ev[k][ci][0].elapsed_time(ev[k][ci][1]) for k in range(args.steps))
+                   for ci in range(len(calls))]
+    dominant = [ci for ci, (i, _) in enumerate(calls) if (specs[i].shape[2] * specs[i].shape[3]) % 4 == 0
+                and plans[ci][0] == b.PLAN_STAGED]
+    dom_bytes = sum(specs[calls[ci][0]].numel for ci in dominant) * BYTES_PER_ELEM
+    dom_ms = sum(per_call_ms[ci] for ci in dominant)
+    peak, peak_src = measured_peak()
+    achieved = dom_bytes / (dom_ms * 1e-3) / 1e9 if dominant else None
+    rec = recorded_traffic()
+    roofline = {
+        "bound": "hbm", "kernel": "staged_kernel<float, fwd+bwd, aligned planes>",
+        "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
+        "peak_source": peak_src, "frac_of_nominal_8TBs": (achieved / NOMINAL_HBM_GBS) if achieved else None,
+        "launches_per_step": len(dominant),
+        "avg_launch_ms": dom_ms / max(1, len(dominant)),
+        "avg_algorithmic_bytes_per_launch": dom_bytes / max(1, len(dominant)),
+        "traffic": (rec["dram_bytes_per_launch_scaled_to_avg_launch"] if rec else None),
+        "note": "achieved = algorithmic bytes of the launches / their CUDA-event time (memset node included)",
+    }
+    per_tensor = []
+    for ci, (i, bits) in enumerate(calls):
+        gbs = specs[i].numel * BYTES_PER_ELEM / (per_call_ms[ci] * 1e-3) / 1e9
+        per_tensor.append({"tensor": specs[i].name, "bits": bits, "us": round(per_call_ms[ci] * 1e3, 2),
+                           "GBps": round(gbs, 1), "frac_measured": round(gbs / peak, 3),
+                           "frac_8TBs": round(gbs / NOMINAL_HBM_GBS, 3), "plan": plans[ci][0]})
+
+    # ---- end to end through the host-buffer entry point (pinned memory, copies timed) ----
+    e2e = None
+    if args.e2e_steps > 0:
+        big = max(specs, key=lambda s: s.numel)
+        arena = torch.empty(b.host_arena_bytes(b.F32, big.shape), dtype=torch.uint8, device="cuda")
+        yh = torch.empty(big.shape, dtype=torch.float32).pin_memory()
+        gxh = torch.empty(big.shape, dtype=torch.float32).pin_memory()
+        cmax = max(s.shape[1] for s in specs)
+        loh, hih = torch.empty(cmax).pin_memory(), torch.empty(cmax).pin_memory()
+
+        def e2e_step():
+            for i, bits in calls:
+                xs, gs = host[i]
+                n, c = specs[i].numel, specs[i].shape[1]
+                b.granq_fakequant_fused_host(xs, bits, gs, yh.view(-1)[:n].view(specs[i].shape),
+                                             gxh.view(-1)[:n].view(specs[i].shape), loh[:c], hih[:c], arena,
+                                             stream=stream)
+        e2e_step()
+        barrier()
+        a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a0.record(stream)
+        for _ in range(args.e2e_steps):
+            e2e_step()
+        a1.record(stream)
+        barrier()
+        e_ms = a0.elapsed_time(a1)
+        if world > 1:
+            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e_ms = float(t.item())
+        e2e = {"value": world * bytes_per_step / (e_ms / args.e2e_steps * 1e-3) / 1e9, "unit": UNIT,
+               "h2d_bytes_per_step": elems_per_step * 8, "d2h_bytes_per_step": elems_per_step * 8 +
+               sum(specs[i].shape[1] * 8 for i, _ in calls),
+               "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
+               "api": "granq_fakequant_fused_host (pinned host buffers)"}
+
+    # ---- the CPU oracle on a bounded sample, rank 0 at N = 1 only ----
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        s, e = time_oracle(cpu_sample())
+        cpu = {"value": e * BYTES_PER_ELEM / s / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "sample": CPU_SAMPLE, "seconds": round(s, 2), "elements_per_s": e / s,
+               "host_cores_available": os.cpu_count()}
+
+    if rank == 0:
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": warmup,
+            "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "f32", "data": "synthetic",
+            "config": {"workload": WORKLOAD, "elements_per_step_per_gpu": elems_per_step,
+                       "calls_per_step": len(calls), "l2": "inputs larger than L2 (7.3 GB working set per step)",
+                       "group_mode": "channel", "parallelism": f"replicas x{world} (independent batches, no exchange)"},
+            "elements_per_s": world * elems_per_step / (ms_per_step * 1e-3),
+            "frac_of_measured_hbm": value / world / peak, "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
+            "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "e2e": e2e, "roofline": roofline,
+            "cpu_baseline": cpu, "per_tensor": per_tensor,
+        }
+        print(json.dumps(line))
+        if args.table:
+            for r in per_tensor:
+                print(f"{r['tensor']:28s} b={r['bits']} {r['us']:9.1f} us {r['GBps']:8.1f} GB/s "
+                      f"{100 * r['frac_measured']:5.1f}% of measured {100 * r['frac_8TBs']:5.1f}% of 8 TB/s",
+                      file=sys.stderr)
+    if world > 1:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

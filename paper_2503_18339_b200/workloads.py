@@ -90,11 +90,11 @@ def channel_sigma(spec: TensorSpec) -> np.ndarray:
     return sigma
 
 
-def _fill_block(spec: TensorSpec, sigma: np.ndarray, out: np.ndarray, b: int) -> None:
+def _fill_block(spec: TensorSpec, sigma: np.ndarray, out: np.ndarray, b: int, block_offset: int = 0) -> None:
     n0 = b * _BLOCK
     n1 = min(n0 + _BLOCK, spec.shape[0])
     shp = (n1 - n0,) + tuple(spec.shape[1:])
-    g = _rng(spec.seed, _STREAM_X, b)
+    g = _rng(spec.seed, _STREAM_X, b + block_offset)
     v = g.standard_normal(shp, dtype=np.float32)
     if spec.dist == "student_t3":
         q = np.square(g.standard_normal(shp, dtype=np.float32))
@@ -121,16 +121,19 @@ def _parallel_blocks(n: int, fn, threads: int) -> None:
             list(ex.map(fn, range(nb)))
 
 
-def make_activation(spec: TensorSpec, out: np.ndarray | None = None, threads: int = 8) -> np.ndarray:
-    """float32 NCHW activation tensor of the spec (finite, no -0)."""
+def make_activation(spec: TensorSpec, out: np.ndarray | None = None, threads: int = 8,
+                    block_offset: int = 0) -> np.ndarray:
+    """float32 NCHW activation tensor of the spec (finite, no -0).  `block_offset` shifts the
+    random streams, giving another batch of the same law (one per data-parallel replica)."""
     if out is None:
         out = np.empty(spec.shape, np.float32)
     sigma = channel_sigma(spec)
-    _parallel_blocks(spec.shape[0], lambda b: _fill_block(spec, sigma, out, b), threads)
+    _parallel_blocks(spec.shape[0], lambda b: _fill_block(spec, sigma, out, b, block_offset), threads)
     return out
 
 
-def make_upstream_grad(spec: TensorSpec, out: np.ndarray | None = None, threads: int = 8) -> np.ndarray:
+def make_upstream_grad(spec: TensorSpec, out: np.ndarray | None = None, threads: int = 8,
+                       block_offset: int = 0) -> np.ndarray:
     """float32 upstream gradient ~ N(0, 1) of the same shape."""
     if out is None:
         out = np.empty(spec.shape, np.float32)
@@ -138,7 +141,7 @@ def make_upstream_grad(spec: TensorSpec, out: np.ndarray | None = None, threads:
     def fill(b):
         n0 = b * _BLOCK
         n1 = min(n0 + _BLOCK, spec.shape[0])
-        out[n0:n1] = _rng(spec.seed, _STREAM_GY, b).standard_normal((n1 - n0,) + tuple(spec.shape[1:]),
+        out[n0:n1] = _rng(spec.seed, _STREAM_GY, b + block_offset).standard_normal((n1 - n0,) + tuple(spec.shape[1:]),
                                                                     dtype=np.float32)
     _parallel_blocks(spec.shape[0], fill, threads)
     return out
