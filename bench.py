@@ -184,6 +184,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="also print a per-tensor table to stderr")
+    ap.add_argument("--only", default="", help="profiling aid: keep only workload tensors whose name contains this")
     args = ap.parse_args()
     if args.impl == "reference":
         if args.steps > 3:
@@ -204,7 +205,7 @@ def main():
     b.lib()
     warmup = max(args.warmup, 3)
 
-    specs = workload_specs()
+    specs = [s for s in workload_specs() if args.only in s.name]
     # ---- host (pinned) inputs and outputs; every rank has its own batch (weak scaling, no exchange) ----
     host = []
     for s in specs:
