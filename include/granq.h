@@ -185,6 +185,17 @@ int granq_staged_geometry(int dtype, const int64_t dims[4], int channel_axis, in
                           int smem_bytes, int64_t out[8]);
 
 /*
+ * Device self-test (no counterpart in the paper).  The staged kernel divides by the
+ * per-group scale with a product and two exact-residual corrections from the correctly
+ * rounded reciprocal; this runs `pairs` generated (x, s) pairs, hard cases included,
+ * through that sequence and through IEEE division and counts the pairs whose bits differ
+ * (expected: 0).  `device_mismatches` is one 64-bit counter in DEVICE memory, written by
+ * the call; read it after the stream has passed.
+ */
+int granq_selftest_division(uint64_t pairs, uint64_t seed, unsigned long long* device_mismatches,
+                            void* cuda_stream);
+
+/*
  * Planner overrides for tests and tuning (no counterpart in the paper).  Process-wide and
  * not thread-safe; value 0 restores the automatic choice.  They change how the staged plan
  * cuts a tensor into waves and chunks, never its results.

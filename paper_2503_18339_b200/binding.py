@@ -27,7 +27,7 @@ EXPORTS = [
     "granq_status_string", "granq_num_groups", "granq_workspace_bytes", "granq_range",
     "granq_fakequant_fwd", "granq_fakequant_bwd", "granq_fakequant_fused", "granq_workspace_status",
     "granq_host_arena_bytes", "granq_fakequant_fused_host", "granq_fused_plan", "granq_staged_geometry",
-    "granq_tune",
+    "granq_tune", "granq_selftest_division",
 ]
 
 
@@ -77,6 +77,8 @@ def lib() -> ctypes.CDLL:
         L.granq_fused_plan.argtypes = [ci, i64p, ci, ci, ci, u32, ctypes.POINTER(ci)]
         L.granq_staged_geometry.restype = ci
         L.granq_staged_geometry.argtypes = [ci, i64p, ci, ci, ci, ci, i64p]
+        L.granq_selftest_division.restype = ci
+        L.granq_selftest_division.argtypes = [ctypes.c_uint64, ctypes.c_uint64, vp, vp]
         L.granq_tune.restype = ci
         L.granq_tune.argtypes = [ci, ci]
         _lib = L
@@ -271,6 +273,14 @@ def granq_fakequant_fused(x: torch.Tensor, bits: int, gy: torch.Tensor = None, c
         _dev(o.codes, "codes"), _dev(o.mask if gy is not None else None, "mask"), _dev(o.s, "s"), _dev(o.z, "z"),
         _dev(o.workspace, "workspace"), o.workspace.numel(), flags, _stream(stream)), "granq_fakequant_fused")
     return o
+
+
+def selftest_division(pairs: int, seed: int = 0, stream=None) -> int:
+    """Pairs (out of `pairs` generated ones) on which the kernel's division differs from IEEE division."""
+    counter = torch.zeros(1, dtype=torch.int64, device="cuda")
+    _check(lib().granq_selftest_division(pairs, seed, _dev(counter, "counter"), _stream(stream)),
+           "granq_selftest_division")
+    return int(counter.item())
 
 
 def workspace_status(workspace: torch.Tensor, stream=None) -> int:

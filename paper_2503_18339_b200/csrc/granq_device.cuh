@@ -44,21 +44,45 @@ __device__ __forceinline__ QParam make_qparam(float lo, float hi, float qmax) {
     return p;
 }
 
-// Rounds u = x / s + z to the nearest integer (ties to even) and clamps it to [0, qmax].
-// The value is first clamped to [-1, qmax + 1]: rounding is monotone and the bounds are
-// integers, so this changes neither the clamped code nor whether the clamp was active, and
-// it makes the add/subtract of 1.5 * 2^23 an exact round-half-to-even (|u| < 2^22) that
-// never yields -0.
-__device__ __forceinline__ float quant_one(float x, QParam p, float qmax, float& y, bool& inside) {
+// Given t = x / s: rounds u = t + z to the nearest integer (ties to even) and clamps it to
+// [0, qmax].  The value is first clamped to [-1, qmax + 1]: rounding is monotone and the
+// bounds are integers, so this changes neither the clamped code nor whether the clamp was
+// active, and it makes the add/subtract of 1.5 * 2^23 an exact round-half-to-even
+// (|u| < 2^22) that never yields -0.
+__device__ __forceinline__ float quant_from_quotient(float t, float s, float z, float qmax, float& y, bool& inside) {
     const float kMagic = 12582912.0f;  // 1.5 * 2^23
-    float t = __fdiv_rn(x, p.s);
-    float u = __fadd_rn(t, p.z);
+    float u = __fadd_rn(t, z);
     float uc = fminf(fmaxf(u, -1.0f), __fadd_rn(qmax, 1.0f));
     float r = __fsub_rn(__fadd_rn(uc, kMagic), kMagic);
     float q = fminf(fmaxf(r, 0.0f), qmax);
     inside = (r == q);
-    y = __fmul_rn(p.s, __fsub_rn(q, p.z));
+    y = __fmul_rn(s, __fsub_rn(q, z));
     return q;
+}
+
+__device__ __forceinline__ float quant_one(float x, QParam p, float qmax, float& y, bool& inside) {
+    return quant_from_quotient(__fdiv_rn(x, p.s), p.s, p.z, qmax, y, inside);
+}
+
+// Correctly rounded x / s from the correctly rounded reciprocal rcp = RN(1 / s): a product
+// and two residual corrections, each residual x - q * s being exact in one fused
+// multiply-add.  After the first correction q is a faithful rounding of x / s; a further
+// correction of a faithful quotient with a correctly rounded reciprocal gives RN(x / s)
+// (Markstein's division theorem), provided nothing over- or underflows on the way.
+// div_is_safe() states the range for which that holds; groups outside it use __fdiv_rn.
+__device__ __forceinline__ float div_by_scale(float x, float s, float rcp) {
+    float q = __fmul_rn(x, rcp);
+    float e = __fmaf_rn(-q, s, x);
+    q = __fmaf_rn(e, rcp, q);
+    e = __fmaf_rn(-q, s, x);
+    return __fmaf_rn(e, rcp, q);
+}
+// s and every |x| of the group within [2^-60, 2^60] (x may also be tiny or zero: a quotient
+// below 2^-120 cannot move u = x / s + z across a rounding boundary).
+__device__ __forceinline__ bool div_is_safe(float s, float lo, float hi) {
+    const float kBig = 1152921504606846976.0f;       // 2^60
+    const float kSmall = 8.67361737988403547e-19f;   // 2^-60
+    return s >= kSmall && s <= kBig && fmaxf(fabsf(lo), fabsf(hi)) <= kBig;
 }
 
 // ---------------------------------------------------------------------------------------

@@ -23,9 +23,11 @@ namespace granq {
 namespace {
 
 constexpr int kStagedThreads = 512;
-constexpr int kStagedUnroll = 4;
+constexpr int kStagedWarps = kStagedThreads / 32;
+constexpr uint32_t kRowUnits = 128;          // units one warp handles per step: 4 per lane
 constexpr uint32_t kMaxDepth = 3;
-constexpr uint32_t kTabMax = 2048;           // channel groups per wave (size of the (s, z) table)
+constexpr uint32_t kMaxChunks = 64;          // chunks of one wave per CTA
+constexpr uint32_t kTabMax = 2048;           // channel groups per wave (size of the parameter table)
 constexpr uint32_t kSmemHeader = 128;        // mbarriers
 constexpr uint32_t kMbarTries = 1u << 22;    // bounded wait on a bulk-copy barrier
 constexpr uint32_t kSpinLimit = 1u << 24;    // bounded wait on a wave counter (x ~64 ns)
@@ -37,6 +39,14 @@ struct WaveShape {
     uint32_t cps;        // chunks per slab
     uint32_t nchunks;    // outer * cps
     FastDiv div_cps;
+};
+
+// One chunk of a wave as staged by this CTA.
+struct ChunkDesc {
+    uint32_t gu0;    // global 16-byte unit index of its first unit
+    uint32_t su0;    // unit offset inside the wave's slab (gives the channel)
+    uint32_t len;    // units
+    uint32_t pad;
 };
 
 struct StagedArgs {
@@ -60,10 +70,11 @@ struct StagedArgs {
     uint32_t cw;             // channels per regular wave
     uint32_t wave_units;     // units of one slab of a regular wave (= cw * inner / V)
     uint32_t cu;             // units per chunk
+    uint32_t rpc;            // rows (of kRowUnits units) per chunk
     uint32_t nwaves, depth, buf_units, tab_entries;
     uint32_t spin_limit, mbar_tries, expected;
     WaveShape shape[2];      // regular wave, last wave
-    FastDiv div_cu;
+    FastDiv div_rpc;
     FastDiv div_plane;       // units per plane (aligned planes) or elements per plane
 };
 
@@ -109,7 +120,7 @@ __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
 // ---- chunk bookkeeping ---------------------------------------------------------------------------
 struct WaveCtx {
     uint32_t c0;           // first channel
-    uint64_t base_units;   // unit offset of the wave's first channel inside a slab
+    uint32_t base_units;   // unit offset of the wave's first channel inside a slab
     const WaveShape* sh;
     uint32_t nk;           // chunks of this CTA
 };
@@ -117,31 +128,53 @@ struct WaveCtx {
 __device__ __forceinline__ WaveCtx wave_ctx(const StagedArgs& a, uint32_t w) {
     WaveCtx c;
     c.c0 = w * a.cw;
-    c.base_units = (uint64_t)w * a.wave_units;
+    c.base_units = w * a.wave_units;
     c.sh = &a.shape[(w + 1 == a.nwaves) ? 1 : 0];
     c.nk = (blockIdx.x < c.sh->nchunks) ? (c.sh->nchunks - blockIdx.x + gridDim.x - 1) / gridDim.x : 0u;
     return c;
 }
 
-// chunk k of this CTA -> (slab, first unit inside the wave's slab, length in units)
-__device__ __forceinline__ void chunk_of(const StagedArgs& a, const WaveCtx& c, uint32_t k, uint32_t& slab,
-                                         uint32_t& su0, uint32_t& len) {
-    uint32_t j = blockIdx.x + k * gridDim.x, ci;
+// chunk k of this CTA
+__device__ __forceinline__ ChunkDesc chunk_of(const StagedArgs& a, const WaveCtx& c, uint32_t k) {
+    uint32_t j = blockIdx.x + k * gridDim.x, slab, ci;
     c.sh->div_cps.divmod(j, slab, ci);
-    su0 = ci * a.cu;
-    len = min(a.cu, c.sh->units - su0);
+    ChunkDesc d;
+    d.su0 = ci * a.cu;
+    d.len = min(a.cu, c.sh->units - d.su0);
+    d.gu0 = slab * a.slab_units + c.base_units + d.su0;
+    d.pad = 0;
+    return d;
 }
 
-template <typename T, int MODE, bool ALIGNED>
+// per-lane min / max of the floats of one pack
+template <typename T>
+__device__ __forceinline__ void pack_minmax(const Pack<T>& p, int first, int last, float& mn, float& mx) {
+#pragma unroll
+    for (int i = 0; i < Pack<T>::V; ++i) {
+        if (i >= first && i < last) {
+            float v = p.get(i);
+            mn = fminf(mn, v);
+            mx = fmaxf(mx, v);
+        }
+    }
+}
+
+// EXTRAS: the optional per-element codes / mask outputs are compiled in
+template <typename T, int MODE, bool ALIGNED, bool EXTRAS>
 __global__ void __launch_bounds__(kStagedThreads, 1) staged_kernel(const StagedArgs a) {
     constexpr int V = Pack<T>::V;
-    constexpr bool kFwd = (MODE & MODE_FWD) != 0, kBwd = (MODE & MODE_BWD) != 0;
+    constexpr bool kBwd = (MODE & MODE_BWD) != 0;
     extern __shared__ __align__(128) unsigned char smem[];
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem);                       // [depth]
-    QParam* tab = reinterpret_cast<QParam*>(smem + kSmemHeader);              // [tab_entries]
-    uint4* bufs = reinterpret_cast<uint4*>(smem + kSmemHeader + a.tab_entries * sizeof(QParam));
-    const uint32_t tid = threadIdx.x;
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem);                                    // [depth]
+    ChunkDesc* descs = reinterpret_cast<ChunkDesc*>(smem + kSmemHeader);                   // [kMaxDepth][kMaxChunks]
+    float2* tab_sz = reinterpret_cast<float2*>(smem + kSmemHeader + kMaxDepth * kMaxChunks * sizeof(ChunkDesc));
+    float* tab_r = reinterpret_cast<float*>(tab_sz + a.tab_entries);                       // reciprocal or 0
+    uint4* bufs = reinterpret_cast<uint4*>(tab_r + a.tab_entries);
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint4* xg = reinterpret_cast<const uint4*>(a.x);
+    const uint4* gyg = reinterpret_cast<const uint4*>(a.gy);
+    uint4* yg = reinterpret_cast<uint4*>(a.y);
+    uint4* gxg = reinterpret_cast<uint4*>(a.gx);
 
     if (tid == 0) {
         for (uint32_t d = 0; d < a.depth; ++d) mbar_init(&bars[d], 1);
@@ -156,27 +189,27 @@ __global__ void __launch_bounds__(kStagedThreads, 1) staged_kernel(const StagedA
 
     // ---- issue the bulk loads of wave w into its buffer (warp 0, one chunk per lane and round) ----
     auto issue = [&](uint32_t w) {
-        if (tid < 32) {
+        if (warp == 0) {
             const WaveCtx c = wave_ctx(a, w);
-            uint64_t* bar = &bars[w % a.depth];
-            uint4* buf = bufs + (size_t)(w % a.depth) * a.buf_units;
+            const uint32_t b = w % a.depth;
+            uint64_t* bar = &bars[b];
+            uint4* buf = bufs + (size_t)b * a.buf_units;
+            ChunkDesc* dsc = descs + b * kMaxChunks;
             uint32_t total = 0;
-            for (uint32_t k = tid; k < c.nk; k += 32) {
-                uint32_t slab, su0, len;
-                chunk_of(a, c, k, slab, su0, len);
-                total += len;
+            for (uint32_t k = lane; k < c.nk; k += 32) {
+                const ChunkDesc d = chunk_of(a, c, k);
+                dsc[k] = d;
+                total += d.len;
             }
             total = __reduce_add_sync(kFullMask, total);
-            if (tid == 0) {
+            if (lane == 0) {
                 asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
                 mbar_expect_tx(bar, total * 16u);
             }
             __syncwarp();
-            for (uint32_t k = tid; k < c.nk; k += 32) {
-                uint32_t slab, su0, len;
-                chunk_of(a, c, k, slab, su0, len);
-                const uint4* src = xg + ((uint64_t)slab * a.slab_units + c.base_units + su0);
-                bulk_load(buf + (size_t)k * a.cu, src, len * 16u, bar);
+            for (uint32_t k = lane; k < c.nk; k += 32) {
+                const ChunkDesc d = dsc[k];
+                bulk_load(buf + (size_t)k * a.cu, xg + d.gu0, d.len * 16u, bar);
             }
         }
     };
@@ -184,56 +217,63 @@ __global__ void __launch_bounds__(kStagedThreads, 1) staged_kernel(const StagedA
     // ---- phase 1: staged data -> min/max keys of the wave's groups; then arrive ----
     auto reduce_wave = [&](uint32_t w) -> bool {
         const WaveCtx c = wave_ctx(a, w);
-        const uint4* buf = bufs + (size_t)(w % a.depth) * a.buf_units;
-        bool landed = mbar_wait_bounded(&bars[w % a.depth], (w / a.depth) & 1u, a.mbar_tries);
+        const uint32_t b = w % a.depth;
+        const uint4* buf = bufs + (size_t)b * a.buf_units;
+        const ChunkDesc* dsc = descs + b * kMaxChunks;
+        bool landed = mbar_wait_bounded(&bars[b], (w / a.depth) & 1u, a.mbar_tries);
         if (!__syncthreads_and(landed)) return false;
         WarpRun run{kNoGroup, 0u, 0u}, run2{kNoGroup, 0u, 0u};
-        const uint32_t total = c.nk * a.cu;
-        for (uint32_t f0 = 0; f0 < total; f0 += kStagedThreads) {
-            const uint32_t f = f0 + tid;
-            uint32_t k, uo, slab, su0 = 0, len = 0;
-            a.div_cu.divmod(f, k, uo);
-            bool valid = f < total;
-            if (valid) {
-                chunk_of(a, c, k, slab, su0, len);
-                valid = uo < len;
+        const uint32_t rows = c.nk * a.rpc;
+        for (uint32_t row = warp; row < rows; row += kStagedWarps) {
+            const uint32_t k = a.div_rpc.div(row), rr = row - k * a.rpc;
+            const ChunkDesc d = dsc[k];
+            const uint32_t r0 = rr * kRowUnits;
+            if (r0 >= d.len) continue;
+            const uint4* src = buf + (size_t)k * a.cu;
+            Pack<T> p[4];
+            bool v[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t uo = r0 + j * 32 + lane;
+                v[j] = uo < d.len;
+                if (v[j]) p[j].raw = src[uo];
             }
-            uint32_t g1 = kNoGroup, mn1 = 0, mx1 = 0, g2 = kNoGroup, mn2 = 0, mx2 = 0;
-            bool valid2 = false;
-            if (valid) {
-                Pack<T> p;
-                p.raw = buf[f];
-                const uint32_t su = su0 + uo;
-                if constexpr (ALIGNED) {
-                    g1 = c.c0 + a.div_plane.div(su);
+            if constexpr (ALIGNED) {
+                float mn[4], mx[4];
 #pragma unroll
-                    for (int i = 0; i < V; ++i) {
-                        uint32_t e = enc(p.get(i));
-                        mn1 = max(mn1, ~e);
-                        mx1 = max(mx1, e);
-                    }
+                for (int j = 0; j < 4; ++j) {
+                    mn[j] = INFINITY;
+                    mx[j] = -INFINITY;
+                    if (v[j]) pack_minmax(p[j], 0, V, mn[j], mx[j]);
+                }
+                const uint32_t ch_first = a.div_plane.div(d.su0 + r0);
+                const uint32_t ch_last = a.div_plane.div(d.su0 + min(r0 + kRowUnits, d.len) - 1);
+                if (ch_first == ch_last) {       // the whole row lies in one channel
+                    const float m0 = fminf(fminf(mn[0], mn[1]), fminf(mn[2], mn[3]));
+                    const float m1 = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                    run_add(run, v[0], c.c0 + ch_first, ~enc(m0), enc(m1), a.kmin, a.kmax);
                 } else {
-                    uint32_t pl, rem;
-                    a.div_plane.divmod(su * V, pl, rem);
-                    g1 = c.c0 + pl;
-                    const uint32_t n1 = min((uint32_t)V, a.inner - rem);   // elements that belong to g1
-                    valid2 = n1 < (uint32_t)V;
-                    g2 = valid2 ? g1 + 1 : kNoGroup;
 #pragma unroll
-                    for (int i = 0; i < V; ++i) {
-                        uint32_t e = enc(p.get(i));
-                        if ((uint32_t)i < n1) {
-                            mn1 = max(mn1, ~e);
-                            mx1 = max(mx1, e);
-                        } else {
-                            mn2 = max(mn2, ~e);
-                            mx2 = max(mx2, e);
-                        }
+                    for (int j = 0; j < 4; ++j) {
+                        const uint32_t g = c.c0 + a.div_plane.div(d.su0 + r0 + j * 32 + lane);
+                        run_add(run, v[j], g, ~enc(mn[j]), enc(mx[j]), a.kmin, a.kmax);
                     }
                 }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t pl = 0, rem = 0;
+                    a.div_plane.divmod((d.su0 + r0 + j * 32 + lane) * V, pl, rem);
+                    const int n1 = (int)min((uint32_t)V, a.inner - rem);      // elements of the first channel
+                    float mn1 = INFINITY, mx1 = -INFINITY, mn2 = INFINITY, mx2 = -INFINITY;
+                    if (v[j]) {
+                        pack_minmax(p[j], 0, n1, mn1, mx1);
+                        pack_minmax(p[j], n1, V, mn2, mx2);
+                    }
+                    run_add(run, v[j], c.c0 + pl, ~enc(mn1), enc(mx1), a.kmin, a.kmax);
+                    run_add(run2, v[j] && n1 < V, c.c0 + pl + 1, ~enc(mn2), enc(mx2), a.kmin, a.kmax);
+                }
             }
-            run_add(run, valid, g1, mn1, mx1, a.kmin, a.kmax);
-            if constexpr (!ALIGNED) run_add(run2, valid2, g2, mn2, mx2, a.kmin, a.kmax);
         }
         run_flush(run, a.kmin, a.kmax);
         if constexpr (!ALIGNED) run_flush(run2, a.kmin, a.kmax);
@@ -246,7 +286,7 @@ __global__ void __launch_bounds__(kStagedThreads, 1) staged_kernel(const StagedA
         return true;
     };
 
-    // ---- wait until every CTA has published wave w, then build the (s, z) table ----
+    // ---- wait until every CTA has published wave w, then build the parameter table ----
     auto params_of_wave = [&](uint32_t w) -> bool {
         bool done = true;
         if (tid == 0) {
@@ -267,7 +307,8 @@ __global__ void __launch_bounds__(kStagedThreads, 1) staged_kernel(const StagedA
             float lo, hi;
             keys_to_range(__ldcg(a.kmin + g), __ldcg(a.kmax + g), lo, hi);
             const QParam p = make_qparam(lo, hi, a.qmax);
-            tab[t] = p;
+            tab_sz[t] = make_float2(p.s, p.z);
+            tab_r[t] = div_is_safe(p.s, lo, hi) ? __frcp_rn(p.s) : 0.0f;
             if (writer) {
                 a.lo[g] = lo;
                 a.hi[g] = hi;
@@ -282,74 +323,93 @@ __global__ void __launch_bounds__(kStagedThreads, 1) staged_kernel(const StagedA
     // ---- phase 2: quantize the wave from shared memory ----
     auto quantize_wave = [&](uint32_t w) {
         const WaveCtx c = wave_ctx(a, w);
-        const uint4* buf = bufs + (size_t)(w % a.depth) * a.buf_units;
-        const uint32_t total = c.nk * a.cu;
-        for (uint32_t f0 = 0; f0 < total; f0 += kStagedThreads * kStagedUnroll) {
-            uint32_t f[kStagedUnroll], su[kStagedUnroll];
-            uint64_t gu[kStagedUnroll];   // global unit index
-            bool valid[kStagedUnroll];
-            Pack<T> pg[kStagedUnroll];
+        const uint32_t b = w % a.depth;
+        const uint4* buf = bufs + (size_t)b * a.buf_units;
+        const ChunkDesc* dsc = descs + b * kMaxChunks;
+        const uint32_t rows = c.nk * a.rpc;
+        const float qmax = a.qmax;
+        for (uint32_t row = warp; row < rows; row += kStagedWarps) {
+            const uint32_t k = a.div_rpc.div(row), rr = row - k * a.rpc;
+            const ChunkDesc d = dsc[k];
+            const uint32_t r0 = rr * kRowUnits;
+            if (r0 >= d.len) continue;
+            const uint4* src = buf + (size_t)k * a.cu;
+            Pack<T> pg[4];
+            bool v[4];
 #pragma unroll
-            for (int j = 0; j < kStagedUnroll; ++j) {
-                f[j] = f0 + j * kStagedThreads + tid;
-                uint32_t k, uo, slab, su0, len;
-                a.div_cu.divmod(f[j], k, uo);
-                valid[j] = f[j] < total;
-                su[j] = 0;
-                gu[j] = 0;
-                if (valid[j]) {
-                    chunk_of(a, c, k, slab, su0, len);
-                    valid[j] = uo < len;
-                    su[j] = su0 + uo;
-                    gu[j] = (uint64_t)slab * a.slab_units + c.base_units + su[j];
-                    if constexpr (kBwd) {
-                        if (valid[j]) pg[j].raw = ld_stream_16(reinterpret_cast<const uint4*>(a.gy) + gu[j]);
-                    }
+            for (int j = 0; j < 4; ++j) {
+                const uint32_t uo = r0 + j * 32 + lane;
+                v[j] = uo < d.len;
+                if constexpr (kBwd) {
+                    if (v[j]) pg[j].raw = ld_stream_16(gyg + d.gu0 + uo);
                 }
             }
 #pragma unroll
-            for (int j = 0; j < kStagedUnroll; ++j) {
-                if (!valid[j]) continue;
+            for (int j = 0; j < 4; ++j) {
+                if (!v[j]) continue;
+                const uint32_t uo = r0 + j * 32 + lane;
                 Pack<T> px, py, pgx;
-                px.raw = buf[f[j]];
-                QParam p1, p2;
-                uint32_t n1 = V;
+                px.raw = src[uo];
+                float2 sz1, sz2;
+                float r1, r2;
+                int n1 = V;
                 if constexpr (ALIGNED) {
-                    p1 = tab[a.div_plane.div(su[j])];
-                    p2 = p1;
+                    const uint32_t ci = a.div_plane.div(d.su0 + uo);
+                    sz1 = tab_sz[ci];
+                    r1 = tab_r[ci];
+                    sz2 = sz1;
+                    r2 = r1;
                 } else {
                     uint32_t pl, rem;
-                    a.div_plane.divmod(su[j] * V, pl, rem);
-                    n1 = min((uint32_t)V, a.inner - rem);
-                    p1 = tab[pl];
-                    p2 = tab[min(pl + 1, c.sh->channels - 1)];
+                    a.div_plane.divmod((d.su0 + uo) * V, pl, rem);
+                    n1 = (int)min((uint32_t)V, a.inner - rem);
+                    const uint32_t pl2 = min(pl + 1, c.sh->channels - 1);
+                    sz1 = tab_sz[pl];
+                    r1 = tab_r[pl];
+                    sz2 = tab_sz[pl2];
+                    r2 = tab_r[pl2];
                 }
                 uint32_t cb[V / 4] = {}, mb[V / 4] = {};
-#pragma unroll
-                for (int i = 0; i < V; ++i) {
-                    const QParam p = (ALIGNED || (uint32_t)i < n1) ? p1 : p2;
+                const bool fast = (r1 != 0.0f) && (r2 != 0.0f);
+                auto element = [&](int i, float t, float s, float z) {
                     float yv;
                     bool in;
-                    float code = quant_one(px.get(i), p, a.qmax, yv, in);
+                    const float code = quant_from_quotient(t, s, z, qmax, yv, in);
                     py.set(i, yv);
-                    cb[i / 4] |= (uint32_t)code << (8 * (i % 4));
-                    mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
                     if constexpr (kBwd) pgx.set(i, in ? pg[j].get(i) : 0.0f);
+                    if constexpr (EXTRAS) {
+                        cb[i / 4] |= (uint32_t)code << (8 * (i % 4));
+                        mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
+                    }
+                };
+                if (fast) {
+#pragma unroll
+                    for (int i = 0; i < V; ++i) {
+                        const bool first = ALIGNED || i < n1;
+                        const float s = first ? sz1.x : sz2.x, z = first ? sz1.y : sz2.y, r = first ? r1 : r2;
+                        element(i, div_by_scale(px.get(i), s, r), s, z);
+                    }
+                } else {
+#pragma unroll
+                    for (int i = 0; i < V; ++i) {
+                        const bool first = ALIGNED || i < n1;
+                        const float s = first ? sz1.x : sz2.x, z = first ? sz1.y : sz2.y;
+                        element(i, __fdiv_rn(px.get(i), s), s, z);
+                    }
                 }
-                if constexpr (kFwd) {
-                    st_stream_16(reinterpret_cast<uint4*>(a.y) + gu[j], py.raw);
+                const uint32_t gu = d.gu0 + uo;
+                st_stream_16(yg + gu, py.raw);
+                if constexpr (kBwd) st_stream_16(gxg + gu, pgx.raw);
+                if constexpr (EXTRAS) {
                     if (a.codes) {
 #pragma unroll
                         for (int i = 0; i < V / 4; ++i)
-                            reinterpret_cast<uint32_t*>(a.codes)[gu[j] * (V / 4) + i] = cb[i];
+                            reinterpret_cast<uint32_t*>(a.codes)[(size_t)gu * (V / 4) + i] = cb[i];
                     }
-                }
-                if constexpr (kBwd) {
-                    st_stream_16(reinterpret_cast<uint4*>(a.gx) + gu[j], pgx.raw);
-                    if (a.mask) {
+                    if (kBwd && a.mask) {
 #pragma unroll
                         for (int i = 0; i < V / 4; ++i)
-                            reinterpret_cast<uint32_t*>(a.mask)[gu[j] * (V / 4) + i] = mb[i];
+                            reinterpret_cast<uint32_t*>(a.mask)[(size_t)gu * (V / 4) + i] = mb[i];
                     }
                 }
             }
@@ -403,9 +463,9 @@ inline uint32_t gcd_u32(uint32_t a, uint32_t b) {
 
 bool aligned16(const void* p) { return p == nullptr || ((uintptr_t)p & 15) == 0; }
 
-template <typename T, int MODE, bool ALIGNED>
+template <typename T, int MODE, bool ALIGNED, bool EXTRAS>
 cudaError_t launch_t(const StagedPlan& plan, StagedArgs& args, cudaStream_t st) {
-    auto kern = staged_kernel<T, MODE, ALIGNED>;
+    auto kern = staged_kernel<T, MODE, ALIGNED, EXTRAS>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
     if (e != cudaSuccess) return e;
     void* params[] = {(void*)&args};
@@ -413,11 +473,18 @@ cudaError_t launch_t(const StagedPlan& plan, StagedArgs& args, cudaStream_t st) 
                                        plan.smem_bytes, st);
 }
 
+template <typename T, int MODE>
+cudaError_t launch_mode(const StagedPlan& plan, StagedArgs& args, bool aligned, bool extras, cudaStream_t st) {
+    if (aligned)
+        return extras ? launch_t<T, MODE, true, true>(plan, args, st) : launch_t<T, MODE, true, false>(plan, args, st);
+    return extras ? launch_t<T, MODE, false, true>(plan, args, st) : launch_t<T, MODE, false, false>(plan, args, st);
+}
+
 template <typename T>
 cudaError_t launch_dtype(const StagedPlan& plan, StagedArgs& args, int mode, bool aligned, cudaStream_t st) {
-    if (mode == MODE_FWD)
-        return aligned ? launch_t<T, MODE_FWD, true>(plan, args, st) : launch_t<T, MODE_FWD, false>(plan, args, st);
-    return aligned ? launch_t<T, MODE_BOTH, true>(plan, args, st) : launch_t<T, MODE_BOTH, false>(plan, args, st);
+    const bool extras = args.codes != nullptr || args.mask != nullptr;
+    if (mode == MODE_FWD) return launch_mode<T, MODE_FWD>(plan, args, aligned, extras, st);
+    return launch_mode<T, MODE_BOTH>(plan, args, aligned, extras, st);
 }
 
 struct DeviceInfo {
@@ -444,7 +511,8 @@ StagedPlan plan_staged(int dtype, const Geom& g, const QuantIO& io, int device, 
 }
 
 // Chooses the wave / chunk geometry.  Cost model: a wave takes as long as its busiest CTA,
-// i.e. (chunks per CTA) x (units per chunk + a per-copy overhead), plus a fixed per-wave overhead.
+// i.e. (chunks per CTA) x (units per chunk rounded up to whole warp rows + a per-copy overhead), plus a
+// fixed per-wave overhead.
 StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_count, int smem_optin,
                           const StagedTuning& tune) {
     StagedPlan best{};
@@ -461,7 +529,7 @@ StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_co
     const uint32_t grid = (uint32_t)((tune.grid > 0 && tune.grid < sm_count) ? tune.grid : sm_count);
     const uint32_t tab_entries = ((std::min(C, kTabMax) + 15u) / 16u) * 16u;
     const uint32_t smem_total = (uint32_t)smem_optin;
-    const uint32_t fixed = kSmemHeader + tab_entries * (uint32_t)sizeof(QParam);
+    const uint32_t fixed = kSmemHeader + kMaxDepth * kMaxChunks * (uint32_t)sizeof(ChunkDesc) + tab_entries * 12u;
     if (smem_total <= fixed + 4096) return best;
     const uint32_t units_total = (smem_total - fixed) / 16u;
     const uint64_t plane_units_x_q = (uint64_t)q * inner / V;   // units of q channels in one slab
@@ -497,7 +565,7 @@ StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_co
             const uint64_t wu64 = (uint64_t)cw * inner / V, lu64 = (uint64_t)c_last * inner / V;
             if (wu64 >= (1ull << 30)) continue;
             const uint32_t wave_units = (uint32_t)wu64, last_units = (uint32_t)lu64;
-            for (uint32_t nk = 1; nk <= 64; ++nk) {
+            for (uint32_t nk = 1; nk <= kMaxChunks; ++nk) {
                 uint64_t cps = ((uint64_t)grid * nk) / O;
                 if (cps == 0) continue;
                 cps = std::min<uint64_t>(cps, wave_units);
@@ -508,9 +576,12 @@ StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_co
                 const uint32_t cps_l = (last_units + cu - 1) / cu;
                 const uint64_t nk_l = ((uint64_t)O * cps_l + grid - 1) / grid;
                 if (nk_r * cu > buf_units || nk_l * cu > buf_units) continue;
+                if (nk_r > kMaxChunks || nk_l > kMaxChunks) continue;
                 if ((uint64_t)O * cps_r >= (1ull << 30)) continue;
-                double cost = (double)(nwaves - 1) * (double)nk_r * (cu + chunk_overhead) +
-                              (double)nk_l * (cu + chunk_overhead) +
+                // a warp works through a chunk in rows of kRowUnits units
+                const double row_units = (double)((cu + kRowUnits - 1) / kRowUnits) * kRowUnits;
+                double cost = (double)(nwaves - 1) * (double)nk_r * (row_units + chunk_overhead) +
+                              (double)nk_l * (row_units + chunk_overhead) +
                               wave_overhead * nwaves * (depth == 2 ? 2.0 : 1.0);
                 any = true;
                 if (cost < best_cost) {
@@ -558,6 +629,8 @@ cudaError_t launch_staged(const StagedPlan& plan, const QuantIO& io, int mode, i
     a.cw = plan.cw;
     a.wave_units = (uint32_t)((uint64_t)plan.cw * inner / V);
     a.cu = plan.cu;
+    a.rpc = (plan.cu + kRowUnits - 1) / kRowUnits;
+    a.div_rpc = make_fastdiv(a.rpc);
     a.nwaves = plan.nwaves;
     a.depth = (uint32_t)plan.depth;
     a.buf_units = plan.buf_units;
@@ -575,7 +648,6 @@ cudaError_t launch_staged(const StagedPlan& plan, const QuantIO& io, int mode, i
         s.nchunks = O * s.cps;
         s.div_cps = make_fastdiv(s.cps);
     }
-    a.div_cu = make_fastdiv(plan.cu);
     const bool aligned = (inner % V) == 0;
     a.div_plane = make_fastdiv(aligned ? inner / V : inner);
     if (dtype == 0) return launch_dtype<float>(plan, a, mode, aligned, st);

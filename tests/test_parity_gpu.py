@@ -325,6 +325,12 @@ def test_bounded_wait_reports_timeout_and_context_survives(b, knobs):
     assert_parity(got, ref, shape, 1, orc.GROUP_CHANNEL, backward=True)
 
 
+# ---- 6b. the staged kernel's division is IEEE division ---------------------------------------------------------
+def test_reciprocal_division_matches_ieee_division(b):
+    for seed in range(4):
+        assert b.selftest_division(1 << 30, seed) == 0
+
+
 # ---- 7. host-buffer entry point --------------------------------------------------------------------------------------
 def test_fused_host_entry_point(b):
     shape = (8, 16, 14, 14)
