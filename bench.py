@@ -184,6 +184,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=2)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="also print a per-tensor table to stderr")
+    ap.add_argument("--tune", default="", help="planner overrides for experiments, e.g. depth=3,max_buf_units=4000")
     ap.add_argument("--only", default="", help="profiling aid: keep only workload tensors whose name contains this")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -203,6 +204,11 @@ def main():
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     b.lib()
+    knob_ids = {"depth": b.KNOB_STAGED_DEPTH, "max_buf_units": b.KNOB_STAGED_MAX_BUF_UNITS,
+                "grid": b.KNOB_STAGED_GRID, "ctas_per_sm": b.KNOB_STAGED_CTAS_PER_SM}
+    for item in filter(None, args.tune.split(",")):
+        name, val = item.split("=")
+        b.tune(knob_ids[name], int(val))
     warmup = max(args.warmup, 3)
 
     specs = [s for s in workload_specs() if args.only in s.name]

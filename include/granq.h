@@ -205,9 +205,10 @@ enum granq_knob {
     GRANQ_KNOB_STAGED_MAX_BUF_UNITS = 1,  /* cap on 16-byte units per buffer (forces small waves)  */
     GRANQ_KNOB_STAGED_GRID = 2,           /* cap on the number of CTAs                             */
     GRANQ_KNOB_SPIN_LIMIT = 3,            /* iteration limit of the wait on a wave's arrival count */
-    GRANQ_KNOB_TEST_EXTRA_ARRIVALS = 4    /* test hook: a wave waits for this many arrivals more
+    GRANQ_KNOB_TEST_EXTRA_ARRIVALS = 4,   /* test hook: a wave waits for this many arrivals more
                                              than the grid provides, so the bounded wait runs out
                                              and the call ends with GRANQ_ERR_TIMEOUT              */
+    GRANQ_KNOB_STAGED_CTAS_PER_SM = 5     /* CTAs that share one SM (1, 2 or 4)                    */
 };
 int granq_tune(int knob, int value);
 

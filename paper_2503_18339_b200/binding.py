@@ -20,7 +20,9 @@ F32, BF16 = 0, 1
 GROUP_CHANNEL, GROUP_SAMPLE_CHANNEL, GROUP_TENSOR = 0, 1, 2
 FLAG_FORCE_TWO_PASS, FLAG_FORCE_NAIVE, FLAG_FORCE_STAGED = 1, 2, 4
 PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED = 0, 1, 2
-KNOB_STAGED_DEPTH, KNOB_STAGED_MAX_BUF_UNITS, KNOB_STAGED_GRID, KNOB_SPIN_LIMIT, KNOB_TEST_EXTRA_ARRIVALS = range(5)
+(KNOB_STAGED_DEPTH, KNOB_STAGED_MAX_BUF_UNITS, KNOB_STAGED_GRID, KNOB_SPIN_LIMIT, KNOB_TEST_EXTRA_ARRIVALS,
+ KNOB_STAGED_CTAS_PER_SM) = range(6)
+N_KNOBS = 6
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 
 EXPORTS = [

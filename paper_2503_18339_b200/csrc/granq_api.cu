@@ -10,7 +10,7 @@ namespace {
 
 constexpr int64_t kMaxElements = 1ll << 40;
 
-StagedTuning g_tune = {0, 0, 0, 0, 0};
+StagedTuning g_tune = {0, 0, 0, 0, 0, 0};
 
 bool make_geom(const int64_t dims[4], int axis, int group, Geom& g, int64_t& G) {
     if (!dims || axis < 0 || axis > 3 || group < 0 || group > 2) return false;
@@ -299,6 +299,7 @@ int granq_tune(int knob, int value) {
         case GRANQ_KNOB_STAGED_GRID: g_tune.grid = value; return GRANQ_OK;
         case GRANQ_KNOB_SPIN_LIMIT: g_tune.spin_limit = value; return GRANQ_OK;
         case GRANQ_KNOB_TEST_EXTRA_ARRIVALS: g_tune.extra_arrivals = value; return GRANQ_OK;
+        case GRANQ_KNOB_STAGED_CTAS_PER_SM: g_tune.ctas_per_sm = value; return GRANQ_OK;
         default: return GRANQ_ERR_INVALID_ARG;
     }
 }

@@ -22,9 +22,9 @@ namespace granq {
 
 namespace {
 
-constexpr int kStagedThreads = 512;
-constexpr int kStagedWarps = kStagedThreads / 32;
+constexpr int kThreadsPerSm = 512;           // split over the CTAs that share an SM
 constexpr uint32_t kRowUnits = 128;          // units one warp handles per step: 4 per lane
+constexpr uint32_t kDefaultCtasPerSm = 2;
 constexpr uint32_t kMaxDepth = 3;
 constexpr uint32_t kMaxChunks = 64;          // chunks of one wave per CTA
 constexpr uint32_t kTabMax = 2048;           // channel groups per wave (size of the parameter table)
@@ -160,8 +160,9 @@ __device__ __forceinline__ void pack_minmax(const Pack<T>& p, int first, int las
 }
 
 // EXTRAS: the optional per-element codes / mask outputs are compiled in
-template <typename T, int MODE, bool ALIGNED, bool EXTRAS>
-__global__ void __launch_bounds__(kStagedThreads, 1) staged_kernel(const StagedArgs a) {
+template <typename T, int MODE, bool ALIGNED, bool EXTRAS, int NT>
+__global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const StagedArgs a) {
+    constexpr int kStagedThreads = NT, kStagedWarps = NT / 32;
     constexpr int V = Pack<T>::V;
     constexpr bool kBwd = (MODE & MODE_BWD) != 0;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -277,7 +278,6 @@ __global__ void __launch_bounds__(kStagedThreads, 1) staged_kernel(const StagedA
         }
         run_flush(run, a.kmin, a.kmax);
         if constexpr (!ALIGNED) run_flush(run2, a.kmin, a.kmax);
-        __threadfence();
         __syncthreads();
         if (tid == 0) {
             __threadfence();
@@ -463,14 +463,21 @@ inline uint32_t gcd_u32(uint32_t a, uint32_t b) {
 
 bool aligned16(const void* p) { return p == nullptr || ((uintptr_t)p & 15) == 0; }
 
-template <typename T, int MODE, bool ALIGNED, bool EXTRAS>
-cudaError_t launch_t(const StagedPlan& plan, StagedArgs& args, cudaStream_t st) {
-    auto kern = staged_kernel<T, MODE, ALIGNED, EXTRAS>;
+template <typename T, int MODE, bool ALIGNED, bool EXTRAS, int NT>
+cudaError_t launch_nt(const StagedPlan& plan, StagedArgs& args, cudaStream_t st) {
+    auto kern = staged_kernel<T, MODE, ALIGNED, EXTRAS, NT>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
     if (e != cudaSuccess) return e;
     void* params[] = {(void*)&args};
     return cudaLaunchCooperativeKernel((const void*)kern, dim3(plan.grid), dim3(plan.threads), params,
                                        plan.smem_bytes, st);
+}
+
+template <typename T, int MODE, bool ALIGNED, bool EXTRAS>
+cudaError_t launch_t(const StagedPlan& plan, StagedArgs& args, cudaStream_t st) {
+    if (plan.threads == 512) return launch_nt<T, MODE, ALIGNED, EXTRAS, 512>(plan, args, st);
+    if (plan.threads == 256) return launch_nt<T, MODE, ALIGNED, EXTRAS, 256>(plan, args, st);
+    return launch_nt<T, MODE, ALIGNED, EXTRAS, 128>(plan, args, st);
 }
 
 template <typename T, int MODE>
@@ -526,9 +533,14 @@ StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_co
 
     const uint32_t inner = (uint32_t)g.inner, C = (uint32_t)g.C, O = (uint32_t)g.outer;
     const uint32_t q = V / gcd_u32(inner, V);          // waves hold multiples of q channels (16-byte slabs)
-    const uint32_t grid = (uint32_t)((tune.grid > 0 && tune.grid < sm_count) ? tune.grid : sm_count);
+    const uint32_t cps_sm = (tune.ctas_per_sm == 1 || tune.ctas_per_sm == 2 || tune.ctas_per_sm == 4)
+                                ? (uint32_t)tune.ctas_per_sm : kDefaultCtasPerSm;
+    const uint32_t full_grid = (uint32_t)sm_count * cps_sm;
+    const uint32_t grid = (tune.grid > 0 && (uint32_t)tune.grid < full_grid) ? (uint32_t)tune.grid : full_grid;
     const uint32_t tab_entries = ((std::min(C, kTabMax) + 15u) / 16u) * 16u;
-    const uint32_t smem_total = (uint32_t)smem_optin;
+    // an SM holds 1 KB more than one CTA may ask for, and reserves 1 KB per resident CTA
+    const uint32_t smem_total = cps_sm == 1 ? (uint32_t)smem_optin
+                                            : (((uint32_t)smem_optin + 1024u) / cps_sm - 1024u) & ~127u;
     const uint32_t fixed = kSmemHeader + kMaxDepth * kMaxChunks * (uint32_t)sizeof(ChunkDesc) + tab_entries * 12u;
     if (smem_total <= fixed + 4096) return best;
     const uint32_t units_total = (smem_total - fixed) / 16u;
@@ -588,7 +600,7 @@ StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_co
                     best_cost = cost;
                     best.ok = true;
                     best.grid = (int)grid;
-                    best.threads = kStagedThreads;
+                    best.threads = kThreadsPerSm / (int)cps_sm;
                     best.depth = (int)std::min(depth, nwaves);
                     best.buf_units = buf_units;
                     best.smem_bytes = fixed + depth * buf_units * 16u;

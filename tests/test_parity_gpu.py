@@ -23,7 +23,7 @@ def b():
     from paper_2503_18339_b200 import binding
     binding.lib()
     yield binding
-    for k in range(5):
+    for k in range(6):
         binding.tune(k, 0)
 
 
@@ -37,7 +37,7 @@ def knobs(b):
         for k, v in kw.items():
             b.tune(names[k], v)
     yield set_
-    for k in range(5):
+    for k in range(6):
         b.tune(k, 0)
 
 
