@@ -5,15 +5,21 @@
 // (contiguous runs inside one slab), dealt round-robin to the CTAs, and each CTA pulls its
 // chunks into shared memory with bulk asynchronous copies (TMA, no multicast) that complete
 // on an mbarrier.  Phase 1 of a wave reduces the staged data to per-group min/max keys
-// (Eq. 4) and publishes them with atomics; a per-wave arrival counter tells when every CTA
-// has done so.  Phase 2 turns the keys into (s, z) (Eq. 5) and quantizes the wave from
-// shared memory (Eq. 1, clamp, Eq. 6) while streaming gy in and y / gx out (STE).  With
-// `depth` buffers per CTA the loads of wave w + depth are in flight, and phase 1 of wave
-// w + depth - 1 has already been published, while wave w is quantized, so neither the load
-// latency nor the grid-wide wait is exposed.
+// (Eq. 4): warps combine in shared memory and the last warp of the CTA publishes the
+// CTA's keys with global atomics and bumps the wave's arrival counter.  Phase 2 waits for
+// that counter to reach the grid size, turns the keys into (s, z) (Eq. 5) and quantizes the
+// wave from shared memory (Eq. 1, clamp, Eq. 6) while streaming gy in and y / gx out (STE).
 //
-// Every wait is bounded: when one runs out the CTA records GRANQ_ERR_TIMEOUT in the
-// workspace status word, waits (bounded again) for its own copies in flight and returns.
+// There is no CTA-wide barrier in the steady state.  Every warp runs the same program
+//     phase 1 of waves 0 .. depth-2;  then for each wave w:  phase 2 of w, phase 1 of w+depth-1
+// over its own rows (128 units, 4 per lane), and the warps meet only through counters: the
+// last warp to finish phase 2 of a wave re-fills that wave's buffer with wave w + depth.
+// With depth 3 the loads of two waves are in flight and a wave's arrival counter has had a
+// whole phase 2 to fill up before anybody waits on it.
+//
+// Every wait is bounded: when one runs out the warp records GRANQ_ERR_TIMEOUT in the
+// workspace status word and raises the CTA's abort flag; all warps then leave their loops,
+// the CTA waits (bounded again) for its own copies in flight and returns.
 #include "granq_internal.h"
 
 #include <algorithm>
@@ -23,12 +29,13 @@ namespace granq {
 namespace {
 
 constexpr int kThreadsPerSm = 512;           // split over the CTAs that share an SM
+constexpr uint32_t kDefaultCtasPerSm = 1;
 constexpr uint32_t kRowUnits = 128;          // units one warp handles per step: 4 per lane
-constexpr uint32_t kDefaultCtasPerSm = 2;
 constexpr uint32_t kMaxDepth = 3;
 constexpr uint32_t kMaxChunks = 64;          // chunks of one wave per CTA
-constexpr uint32_t kTabMax = 2048;           // channel groups per wave (size of the parameter table)
-constexpr uint32_t kSmemHeader = 128;        // mbarriers
+constexpr uint32_t kTabMax = 2048;           // channel groups per wave
+constexpr uint32_t kSmemBars = 128;          // mbarriers
+constexpr uint32_t kSmemCtl = 128;           // control words
 constexpr uint32_t kMbarTries = 1u << 22;    // bounded wait on a bulk-copy barrier
 constexpr uint32_t kSpinLimit = 1u << 24;    // bounded wait on a wave counter (x ~64 ns)
 constexpr uint32_t kStatusTimeout = 5;       // GRANQ_ERR_TIMEOUT
@@ -47,6 +54,14 @@ struct ChunkDesc {
     uint32_t su0;    // unit offset inside the wave's slab (gives the channel)
     uint32_t len;    // units
     uint32_t pad;
+};
+
+// control words in shared memory
+struct Control {
+    uint32_t p1_done[2];          // warps that finished phase 1 of the wave with this parity
+    uint32_t p2_done[kMaxDepth];  // warps that finished phase 2 on this buffer
+    uint32_t issued;              // waves whose loads have been issued
+    uint32_t abort;               // a bounded wait ran out somewhere in this CTA
 };
 
 struct StagedArgs {
@@ -99,11 +114,6 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
         : "memory");
     return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait_bounded(uint64_t* bar, uint32_t parity, uint32_t tries) {
-    for (uint32_t i = 0; i < tries; ++i)
-        if (mbar_try_wait(bar, parity)) return true;
-    return false;
-}
 // global -> shared bulk copy; src, dst 16-byte aligned, bytes a multiple of 16
 __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint32_t bytes, uint64_t* bar) {
     asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
@@ -114,6 +124,11 @@ __device__ __forceinline__ void bulk_load(void* dst_smem, const void* src, uint3
 __device__ __forceinline__ uint32_t ld_acquire(const uint32_t* p) {
     uint32_t v;
     asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ uint32_t ld_volatile_shared(const uint32_t* p) {
+    uint32_t v;
+    asm volatile("ld.volatile.shared.u32 %0, [%1];" : "=r"(v) : "r"(smem_u32(p)) : "memory");
     return v;
 }
 
@@ -146,7 +161,7 @@ __device__ __forceinline__ ChunkDesc chunk_of(const StagedArgs& a, const WaveCtx
     return d;
 }
 
-// per-lane min / max of the floats of one pack
+// per-lane min / max of elements [first, last) of one pack
 template <typename T>
 __device__ __forceinline__ void pack_minmax(const Pack<T>& p, int first, int last, float& mn, float& mx) {
 #pragma unroll
@@ -159,73 +174,111 @@ __device__ __forceinline__ void pack_minmax(const Pack<T>& p, int first, int las
     }
 }
 
+// scale, zero-point and reciprocal (0 = use IEEE division) of one group from its published keys
+struct GroupParam {
+    float s, z, r;
+};
+__device__ __forceinline__ GroupParam group_param(const StagedArgs& a, uint32_t g, float& lo, float& hi) {
+    keys_to_range(__ldcg(a.kmin + g), __ldcg(a.kmax + g), lo, hi);
+    const QParam p = make_qparam(lo, hi, a.qmax);
+    GroupParam gp;
+    gp.s = p.s;
+    gp.z = p.z;
+    gp.r = div_is_safe(p.s, lo, hi) ? __frcp_rn(p.s) : 0.0f;
+    return gp;
+}
+
 // EXTRAS: the optional per-element codes / mask outputs are compiled in
 template <typename T, int MODE, bool ALIGNED, bool EXTRAS, int NT>
 __global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const StagedArgs a) {
-    constexpr int kStagedThreads = NT, kStagedWarps = NT / 32;
+    constexpr uint32_t kWarps = NT / 32;
     constexpr int V = Pack<T>::V;
     constexpr bool kBwd = (MODE & MODE_BWD) != 0;
     extern __shared__ __align__(128) unsigned char smem[];
-    uint64_t* bars = reinterpret_cast<uint64_t*>(smem);                                    // [depth]
-    ChunkDesc* descs = reinterpret_cast<ChunkDesc*>(smem + kSmemHeader);                   // [kMaxDepth][kMaxChunks]
-    float2* tab_sz = reinterpret_cast<float2*>(smem + kSmemHeader + kMaxDepth * kMaxChunks * sizeof(ChunkDesc));
-    float* tab_r = reinterpret_cast<float*>(tab_sz + a.tab_entries);                       // reciprocal or 0
-    uint4* bufs = reinterpret_cast<uint4*>(tab_r + a.tab_entries);
+    uint64_t* bars = reinterpret_cast<uint64_t*>(smem);                                        // [depth]
+    Control* ctl = reinterpret_cast<Control*>(smem + kSmemBars);
+    ChunkDesc* descs = reinterpret_cast<ChunkDesc*>(smem + kSmemBars + kSmemCtl);             // [kMaxDepth][kMaxChunks]
+    uint32_t* s_keys = reinterpret_cast<uint32_t*>(descs + kMaxDepth * kMaxChunks);           // [2][2][tab_entries]
+    uint4* bufs = reinterpret_cast<uint4*>(s_keys + 4 * a.tab_entries);
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint4* xg = reinterpret_cast<const uint4*>(a.x);
     const uint4* gyg = reinterpret_cast<const uint4*>(a.gy);
     uint4* yg = reinterpret_cast<uint4*>(a.y);
     uint4* gxg = reinterpret_cast<uint4*>(a.gx);
+    const uint32_t W = a.nwaves, D = a.depth;
 
     if (tid == 0) {
-        for (uint32_t d = 0; d < a.depth; ++d) mbar_init(&bars[d], 1);
+        for (uint32_t d = 0; d < D; ++d) mbar_init(&bars[d], 1);
+        *ctl = Control{};
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
+    for (uint32_t i = tid; i < 4 * a.tab_entries; i += NT) s_keys[i] = 0;
     __syncthreads();
 
-    uint32_t issued = 0;   // waves whose loads have been issued
-    uint32_t reduced = 0;  // waves whose phase 1 is done
-    bool ok = true;
+    bool alive = true;   // warp-uniform: no bounded wait has run out so far
 
-    // ---- issue the bulk loads of wave w into its buffer (warp 0, one chunk per lane and round) ----
+    auto give_up = [&]() {
+        if (lane == 0) {
+            atomicExch(a.status, kStatusTimeout);
+            atomicExch(&ctl->abort, 1u);
+        }
+        alive = false;
+    };
+
+    // ---- issue the bulk loads of wave w into its buffer (one warp; one chunk per lane and round) ----
     auto issue = [&](uint32_t w) {
-        if (warp == 0) {
-            const WaveCtx c = wave_ctx(a, w);
-            const uint32_t b = w % a.depth;
-            uint64_t* bar = &bars[b];
-            uint4* buf = bufs + (size_t)b * a.buf_units;
-            ChunkDesc* dsc = descs + b * kMaxChunks;
-            uint32_t total = 0;
-            for (uint32_t k = lane; k < c.nk; k += 32) {
-                const ChunkDesc d = chunk_of(a, c, k);
-                dsc[k] = d;
-                total += d.len;
-            }
-            total = __reduce_add_sync(kFullMask, total);
-            if (lane == 0) {
-                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-                mbar_expect_tx(bar, total * 16u);
-            }
-            __syncwarp();
-            for (uint32_t k = lane; k < c.nk; k += 32) {
-                const ChunkDesc d = dsc[k];
-                bulk_load(buf + (size_t)k * a.cu, xg + d.gu0, d.len * 16u, bar);
-            }
+        const WaveCtx c = wave_ctx(a, w);
+        const uint32_t b = w % D;
+        uint64_t* bar = &bars[b];
+        uint4* buf = bufs + (size_t)b * a.buf_units;
+        ChunkDesc* dsc = descs + b * kMaxChunks;
+        uint32_t total = 0;
+        for (uint32_t k = lane; k < c.nk; k += 32) {
+            const ChunkDesc d = chunk_of(a, c, k);
+            dsc[k] = d;
+            total += d.len;
+        }
+        total = __reduce_add_sync(kFullMask, total);
+        __syncwarp();
+        if (lane == 0) {
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            mbar_expect_tx(bar, total * 16u);      // release: the descriptors are visible to whoever sees the phase
+            atomicAdd(&ctl->issued, 1u);
+        }
+        __syncwarp();
+        for (uint32_t k = lane; k < c.nk; k += 32) {
+            const ChunkDesc d = dsc[k];
+            bulk_load(buf + (size_t)k * a.cu, xg + d.gu0, d.len * 16u, bar);
         }
     };
 
-    // ---- phase 1: staged data -> min/max keys of the wave's groups; then arrive ----
-    auto reduce_wave = [&](uint32_t w) -> bool {
+    // ---- wait (bounded) until the loads of wave w have landed in its buffer ----
+    auto wait_loaded = [&](uint32_t w) -> bool {
+        uint64_t* bar = &bars[w % D];
+        const uint32_t parity = (w / D) & 1u;
+        for (uint32_t i = 0; i < a.mbar_tries; ++i) {
+            if (mbar_try_wait(bar, parity)) return true;
+            if ((i & 63u) == 63u && ld_volatile_shared(&ctl->abort)) return false;
+        }
+        return false;
+    };
+
+    // ---- phase 1: this warp's rows of wave w -> min/max keys; the CTA's last warp publishes ----
+    auto reduce_wave = [&](uint32_t w) {
         const WaveCtx c = wave_ctx(a, w);
-        const uint32_t b = w % a.depth;
+        const uint32_t b = w % D, par = w & 1u;
         const uint4* buf = bufs + (size_t)b * a.buf_units;
         const ChunkDesc* dsc = descs + b * kMaxChunks;
-        bool landed = mbar_wait_bounded(&bars[b], (w / a.depth) & 1u, a.mbar_tries);
-        if (!__syncthreads_and(landed)) return false;
+        uint32_t* kmn = s_keys + (2 * par) * a.tab_entries;
+        uint32_t* kmx = kmn + a.tab_entries;
+        if (!__all_sync(kFullMask, wait_loaded(w))) {
+            give_up();
+            return;
+        }
         WarpRun run{kNoGroup, 0u, 0u}, run2{kNoGroup, 0u, 0u};
         const uint32_t rows = c.nk * a.rpc;
-        for (uint32_t row = warp; row < rows; row += kStagedWarps) {
+        for (uint32_t row = warp; row < rows; row += kWarps) {
             const uint32_t k = a.div_rpc.div(row), rr = row - k * a.rpc;
             const ChunkDesc d = dsc[k];
             const uint32_t r0 = rr * kRowUnits;
@@ -252,12 +305,12 @@ __global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const St
                 if (ch_first == ch_last) {       // the whole row lies in one channel
                     const float m0 = fminf(fminf(mn[0], mn[1]), fminf(mn[2], mn[3]));
                     const float m1 = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                    run_add(run, v[0], c.c0 + ch_first, ~enc(m0), enc(m1), a.kmin, a.kmax);
+                    run_add(run, v[0], ch_first, ~enc(m0), enc(m1), kmn, kmx);
                 } else {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint32_t g = c.c0 + a.div_plane.div(d.su0 + r0 + j * 32 + lane);
-                        run_add(run, v[j], g, ~enc(mn[j]), enc(mx[j]), a.kmin, a.kmax);
+                        const uint32_t g = a.div_plane.div(d.su0 + r0 + j * 32 + lane);
+                        run_add(run, v[j], g, ~enc(mn[j]), enc(mx[j]), kmn, kmx);
                     }
                 }
             } else {
@@ -271,64 +324,76 @@ __global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const St
                         pack_minmax(p[j], 0, n1, mn1, mx1);
                         pack_minmax(p[j], n1, V, mn2, mx2);
                     }
-                    run_add(run, v[j], c.c0 + pl, ~enc(mn1), enc(mx1), a.kmin, a.kmax);
-                    run_add(run2, v[j] && n1 < V, c.c0 + pl + 1, ~enc(mn2), enc(mx2), a.kmin, a.kmax);
+                    run_add(run, v[j], pl, ~enc(mn1), enc(mx1), kmn, kmx);
+                    run_add(run2, v[j] && n1 < V, pl + 1, ~enc(mn2), enc(mx2), kmn, kmx);
                 }
             }
         }
-        run_flush(run, a.kmin, a.kmax);
-        if constexpr (!ALIGNED) run_flush(run2, a.kmin, a.kmax);
-        __syncthreads();
-        if (tid == 0) {
-            __threadfence();
-            atomicAdd(a.counters + w, 1u);
+        run_flush(run, kmn, kmx);               // shared-memory atomics on the wave-local group index
+        if constexpr (!ALIGNED) run_flush(run2, kmn, kmx);
+        __syncwarp();
+        uint32_t prev = 0;
+        if (lane == 0) {
+            __threadfence_block();
+            prev = atomicAdd(&ctl->p1_done[par], 1u);
         }
-        return true;
+        prev = __shfl_sync(kFullMask, prev, 0);
+        if (prev == kWarps - 1) {
+            // last warp of the CTA: publish the groups this CTA touched, then arrive on the wave counter
+            __threadfence_block();
+            for (uint32_t t = lane; t < c.sh->channels; t += 32) {
+                const uint32_t k1 = atomicExch(kmn + t, 0u), k2 = atomicExch(kmx + t, 0u);
+                if (k1 | k2) {
+                    atomicMax(a.kmin + c.c0 + t, k1);
+                    atomicMax(a.kmax + c.c0 + t, k2);
+                }
+            }
+            __syncwarp();
+            if (lane == 0) {
+                atomicExch(&ctl->p1_done[par], 0u);
+                __threadfence();
+                atomicAdd(a.counters + w, 1u);
+            }
+        }
     };
 
-    // ---- wait until every CTA has published wave w, then build the parameter table ----
-    auto params_of_wave = [&](uint32_t w) -> bool {
-        bool done = true;
-        if (tid == 0) {
-            done = false;
+    // ---- phase 2: this warp's rows of wave w, quantized from shared memory ----
+    auto quantize_wave = [&](uint32_t w) {
+        const WaveCtx c = wave_ctx(a, w);
+        const uint32_t b = w % D;
+        const uint4* buf = bufs + (size_t)b * a.buf_units;
+        const ChunkDesc* dsc = descs + b * kMaxChunks;
+        const float qmax = a.qmax;
+        // every CTA must have published wave w
+        bool ready = true;
+        if (lane == 0) {
+            ready = false;
             for (uint32_t i = 0; i < a.spin_limit; ++i) {
                 if (ld_acquire(a.counters + w) >= a.expected) {
-                    done = true;
+                    ready = true;
                     break;
                 }
+                if (ld_volatile_shared(&ctl->abort)) break;
                 __nanosleep(64);
             }
         }
-        if (!__syncthreads_and(done)) return false;
-        const WaveCtx c = wave_ctx(a, w);
-        const bool writer = (w % gridDim.x) == blockIdx.x;
-        for (uint32_t t = tid; t < c.sh->channels; t += kStagedThreads) {
-            const uint32_t g = c.c0 + t;
-            float lo, hi;
-            keys_to_range(__ldcg(a.kmin + g), __ldcg(a.kmax + g), lo, hi);
-            const QParam p = make_qparam(lo, hi, a.qmax);
-            tab_sz[t] = make_float2(p.s, p.z);
-            tab_r[t] = div_is_safe(p.s, lo, hi) ? __frcp_rn(p.s) : 0.0f;
-            if (writer) {
-                a.lo[g] = lo;
-                a.hi[g] = hi;
-                if (a.s_out) a.s_out[g] = p.s;
-                if (a.z_out) a.z_out[g] = p.z;
+        ready = __all_sync(kFullMask, ready) && __all_sync(kFullMask, wait_loaded(w));
+        if (!ready) {
+            give_up();
+            return;
+        }
+        if (warp == 0 && (w % gridDim.x) == blockIdx.x) {       // one warp in the grid reports the wave's groups
+            for (uint32_t t = lane; t < c.sh->channels; t += 32) {
+                float lo, hi;
+                const GroupParam gp = group_param(a, c.c0 + t, lo, hi);
+                a.lo[c.c0 + t] = lo;
+                a.hi[c.c0 + t] = hi;
+                if (a.s_out) a.s_out[c.c0 + t] = gp.s;
+                if (a.z_out) a.z_out[c.c0 + t] = gp.z;
             }
         }
-        __syncthreads();
-        return true;
-    };
-
-    // ---- phase 2: quantize the wave from shared memory ----
-    auto quantize_wave = [&](uint32_t w) {
-        const WaveCtx c = wave_ctx(a, w);
-        const uint32_t b = w % a.depth;
-        const uint4* buf = bufs + (size_t)b * a.buf_units;
-        const ChunkDesc* dsc = descs + b * kMaxChunks;
         const uint32_t rows = c.nk * a.rpc;
-        const float qmax = a.qmax;
-        for (uint32_t row = warp; row < rows; row += kStagedWarps) {
+        for (uint32_t row = warp; row < rows; row += kWarps) {
             const uint32_t k = a.div_rpc.div(row), rr = row - k * a.rpc;
             const ChunkDesc d = dsc[k];
             const uint32_t r0 = rr * kRowUnits;
@@ -344,33 +409,53 @@ __global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const St
                     if (v[j]) pg[j].raw = ld_stream_16(gyg + d.gu0 + uo);
                 }
             }
+            // parameters of the channels this row touches: lane l holds channel ch_first + l
+            const uint32_t last_u = d.su0 + min(r0 + kRowUnits, d.len) - 1;
+            const uint32_t ch_first = ALIGNED ? a.div_plane.div(d.su0 + r0) : a.div_plane.div((d.su0 + r0) * V);
+            const uint32_t ch_last = ALIGNED ? a.div_plane.div(last_u) : a.div_plane.div(last_u * V + (V - 1));
+            const uint32_t nch = ch_last - ch_first + 1;
+            const bool shared_params = nch <= 32;
+            GroupParam mine{1.0f, 0.0f, 0.0f};
+            if (shared_params && lane < nch) {
+                float lo, hi;
+                mine = group_param(a, c.c0 + ch_first + lane, lo, hi);
+            }
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                if (!v[j]) continue;
                 const uint32_t uo = r0 + j * 32 + lane;
-                Pack<T> px, py, pgx;
-                px.raw = src[uo];
-                float2 sz1, sz2;
-                float r1, r2;
+                uint32_t ci1 = 0, ci2 = 0;
                 int n1 = V;
                 if constexpr (ALIGNED) {
-                    const uint32_t ci = a.div_plane.div(d.su0 + uo);
-                    sz1 = tab_sz[ci];
-                    r1 = tab_r[ci];
-                    sz2 = sz1;
-                    r2 = r1;
+                    ci1 = a.div_plane.div(d.su0 + (v[j] ? uo : r0));
+                    ci2 = ci1;
                 } else {
-                    uint32_t pl, rem;
-                    a.div_plane.divmod((d.su0 + uo) * V, pl, rem);
+                    uint32_t rem;
+                    a.div_plane.divmod((d.su0 + (v[j] ? uo : r0)) * V, ci1, rem);
                     n1 = (int)min((uint32_t)V, a.inner - rem);
-                    const uint32_t pl2 = min(pl + 1, c.sh->channels - 1);
-                    sz1 = tab_sz[pl];
-                    r1 = tab_r[pl];
-                    sz2 = tab_sz[pl2];
-                    r2 = tab_r[pl2];
+                    ci2 = min(ci1 + 1, c.sh->channels - 1);
                 }
+                GroupParam g1, g2;
+                if (shared_params) {
+                    const uint32_t i1 = ci1 - ch_first, i2 = min(ci2 - ch_first, nch - 1);
+                    g1.s = __shfl_sync(kFullMask, mine.s, i1);
+                    g1.z = __shfl_sync(kFullMask, mine.z, i1);
+                    g1.r = __shfl_sync(kFullMask, mine.r, i1);
+                    if constexpr (ALIGNED) {
+                        g2 = g1;
+                    } else {
+                        g2.s = __shfl_sync(kFullMask, mine.s, i2);
+                        g2.z = __shfl_sync(kFullMask, mine.z, i2);
+                        g2.r = __shfl_sync(kFullMask, mine.r, i2);
+                    }
+                } else {
+                    float lo, hi;
+                    g1 = group_param(a, c.c0 + ci1, lo, hi);
+                    g2 = ALIGNED ? g1 : group_param(a, c.c0 + ci2, lo, hi);
+                }
+                if (!v[j]) continue;
+                Pack<T> px, py, pgx;
+                px.raw = src[uo];
                 uint32_t cb[V / 4] = {}, mb[V / 4] = {};
-                const bool fast = (r1 != 0.0f) && (r2 != 0.0f);
                 auto element = [&](int i, float t, float s, float z) {
                     float yv;
                     bool in;
@@ -382,18 +467,18 @@ __global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const St
                         mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
                     }
                 };
-                if (fast) {
+                if ((g1.r != 0.0f) && (g2.r != 0.0f)) {
 #pragma unroll
                     for (int i = 0; i < V; ++i) {
                         const bool first = ALIGNED || i < n1;
-                        const float s = first ? sz1.x : sz2.x, z = first ? sz1.y : sz2.y, r = first ? r1 : r2;
+                        const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z, r = first ? g1.r : g2.r;
                         element(i, div_by_scale(px.get(i), s, r), s, z);
                     }
                 } else {
 #pragma unroll
                     for (int i = 0; i < V; ++i) {
                         const bool first = ALIGNED || i < n1;
-                        const float s = first ? sz1.x : sz2.x, z = first ? sz1.y : sz2.y;
+                        const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z;
                         element(i, __fdiv_rn(px.get(i), s), s, z);
                     }
                 }
@@ -414,41 +499,43 @@ __global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const St
                 }
             }
         }
+        // the last warp to leave the buffer re-fills it with wave w + depth
+        __syncwarp();
+        uint32_t prev = 0;
+        if (lane == 0) {
+            __threadfence_block();
+            prev = atomicAdd(&ctl->p2_done[b], 1u);
+        }
+        prev = __shfl_sync(kFullMask, prev, 0);
+        if (prev == kWarps - 1) {
+            if (lane == 0) atomicExch(&ctl->p2_done[b], 0u);
+            __syncwarp();
+            if (w + D < W) issue(w + D);
+        }
     };
 
-    // ---- the pipeline ----
-    const uint32_t W = a.nwaves, D = a.depth;
-    for (; issued < min(D, W); ++issued) issue(issued);
-    if (D > 1) {
-        const uint32_t npre = min(D - 1, W);
-        while (ok && reduced < npre) {
-            ok = reduce_wave(reduced);
-            if (ok) ++reduced;
+    // ---- the per-warp program ----
+    if (warp == 0)
+        for (uint32_t w = 0; w < min(D, W); ++w) issue(w);
+    if (D == 1) {
+        reduce_wave(0);
+        if (alive) quantize_wave(0);
+    } else {
+        for (uint32_t w = 0; alive && w < min(D - 1, W); ++w) reduce_wave(w);
+        for (uint32_t w = 0; alive && w < W; ++w) {
+            quantize_wave(w);
+            if (alive && w + D - 1 < W) reduce_wave(w + D - 1);
         }
     }
-    for (uint32_t w = 0; ok && w < W; ++w) {
-        if (D == 1) {
-            ok = reduce_wave(w);
-            if (!ok) break;
-            reduced = w + 1;
+    __syncthreads();
+    if (ld_volatile_shared(&ctl->abort)) {
+        // let this CTA's outstanding copies land before its shared memory is given away
+        const uint32_t n = ld_volatile_shared(&ctl->issued);
+        for (uint32_t w = (n > D ? n - D : 0); w < n; ++w) {
+            uint64_t* bar = &bars[w % D];
+            for (uint32_t i = 0; i < kMbarTries; ++i)
+                if (mbar_try_wait(bar, (w / D) & 1u)) break;
         }
-        ok = params_of_wave(w);
-        if (!ok) break;
-        quantize_wave(w);
-        if (issued < W) {
-            __syncthreads();          // every thread is done reading the buffer that is refilled
-            issue(issued);
-            ++issued;
-        }
-        if (D > 1 && reduced < W) {
-            ok = reduce_wave(reduced);
-            if (ok) ++reduced;
-        }
-    }
-    if (!ok) {
-        // a bounded wait ran out: flag it, then let this CTA's outstanding copies land before leaving
-        if (tid == 0) atomicExch(a.status, kStatusTimeout);
-        for (uint32_t w = reduced; w < issued; ++w) mbar_wait_bounded(&bars[w % D], (w / D) & 1u, kMbarTries);
     }
 }
 
@@ -510,6 +597,11 @@ DeviceInfo device_info(int device) {
     return d;
 }
 
+uint32_t table_entries(uint32_t cw) { return ((cw + 15u) / 16u) * 16u; }
+uint32_t fixed_smem(uint32_t cw) {
+    return kSmemBars + kSmemCtl + kMaxDepth * kMaxChunks * (uint32_t)sizeof(ChunkDesc) + 16u * table_entries(cw);
+}
+
 }  // namespace
 
 StagedPlan plan_staged(int dtype, const Geom& g, const QuantIO& io, int device, const StagedTuning& tune) {
@@ -537,13 +629,9 @@ StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_co
                                 ? (uint32_t)tune.ctas_per_sm : kDefaultCtasPerSm;
     const uint32_t full_grid = (uint32_t)sm_count * cps_sm;
     const uint32_t grid = (tune.grid > 0 && (uint32_t)tune.grid < full_grid) ? (uint32_t)tune.grid : full_grid;
-    const uint32_t tab_entries = ((std::min(C, kTabMax) + 15u) / 16u) * 16u;
     // an SM holds 1 KB more than one CTA may ask for, and reserves 1 KB per resident CTA
     const uint32_t smem_total = cps_sm == 1 ? (uint32_t)smem_optin
                                             : (((uint32_t)smem_optin + 1024u) / cps_sm - 1024u) & ~127u;
-    const uint32_t fixed = kSmemHeader + kMaxDepth * kMaxChunks * (uint32_t)sizeof(ChunkDesc) + tab_entries * 12u;
-    if (smem_total <= fixed + 4096) return best;
-    const uint32_t units_total = (smem_total - fixed) / 16u;
     const uint64_t plane_units_x_q = (uint64_t)q * inner / V;   // units of q channels in one slab
     const uint32_t mult_total = C / q;                           // C is a multiple of q (slabs are whole packs)
 
@@ -552,24 +640,20 @@ StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_co
     const double chunk_overhead = 32.0;   // units-equivalent of issuing one bulk copy
     for (uint32_t depth = 1; depth <= kMaxDepth; ++depth) {
         if (tune.depth > 0 && (int)depth != tune.depth) continue;
-        uint32_t buf_units = units_total / depth;
-        if (tune.max_buf_units > 0) buf_units = std::min<uint32_t>(buf_units, (uint32_t)tune.max_buf_units);
-        // largest wave (in multiples of q channels) whose data fits the grid's buffers
-        uint64_t cap_units = (uint64_t)grid * buf_units;
-        uint64_t max_mult = cap_units / ((uint64_t)O * plane_units_x_q);
-        max_mult = std::min<uint64_t>(max_mult, kTabMax / q);
-        if (max_mult == 0) continue;
-        if (depth == 1 && max_mult < mult_total) continue;        // depth 1 only for a single wave
-        if (depth > 1 && max_mult >= mult_total && best.ok && tune.depth == 0) continue;
-        const uint32_t waves_min = (uint32_t)((mult_total + max_mult - 1) / max_mult);
-        // candidate wave sizes: from the largest that fits downwards, until four of them
-        // have produced a feasible chunking (imbalance can make the largest ones infeasible)
+        if (depth > 1 && best.ok && best.nwaves == 1 && tune.depth == 0) continue;   // a single wave needs no pipeline
+        // candidate wave sizes from the largest downwards, until four of them have produced a
+        // feasible chunking (imbalance between CTAs can make the largest ones infeasible)
         uint32_t feasible = 0, tried = 0, prev_cw = 0;
-        for (uint32_t nw = waves_min; nw <= mult_total && feasible < 4 && tried < 256; ++nw) {
-            if (depth == 1 && nw != 1) break;
+        for (uint32_t nw = 1; nw <= mult_total && feasible < 4 && tried < 256; ++nw) {
+            if (depth == 1 && nw != 1) break;                    // depth 1 only for a single wave
             const uint32_t cw = ((mult_total + nw - 1) / nw) * q;
             if (cw > kTabMax || cw == prev_cw) continue;
             prev_cw = cw;
+            const uint32_t fixed = fixed_smem(cw);
+            if (smem_total <= fixed + 2048) continue;
+            uint32_t buf_units = (smem_total - fixed) / 16u / depth;
+            if (tune.max_buf_units > 0) buf_units = std::min<uint32_t>(buf_units, (uint32_t)tune.max_buf_units);
+            if ((uint64_t)grid * buf_units < (uint64_t)O * (cw / q) * plane_units_x_q) continue;   // cannot fit
             ++tried;
             bool any = false;
             const uint32_t nwaves = (C + cw - 1) / cw;
@@ -649,7 +733,7 @@ cudaError_t launch_staged(const StagedPlan& plan, const QuantIO& io, int mode, i
     a.spin_limit = tune.spin_limit > 0 ? (uint32_t)tune.spin_limit : kSpinLimit;
     a.mbar_tries = kMbarTries;
     a.expected = (uint32_t)plan.grid + (uint32_t)(tune.extra_arrivals > 0 ? tune.extra_arrivals : 0);
-    a.tab_entries = ((std::min(C, kTabMax) + 15u) / 16u) * 16u;
+    a.tab_entries = table_entries(plan.cw);
     const uint32_t c_last = C - (plan.nwaves - 1) * plan.cw;
     const uint32_t ch[2] = {plan.nwaves > 1 ? plan.cw : c_last, c_last};
     for (int i = 0; i < 2; ++i) {
