@@ -208,7 +208,7 @@ enum granq_knob {
     GRANQ_KNOB_TEST_EXTRA_ARRIVALS = 4,   /* test hook: a wave waits for this many arrivals more
                                              than the grid provides, so the bounded wait runs out
                                              and the call ends with GRANQ_ERR_TIMEOUT              */
-    GRANQ_KNOB_STAGED_CTAS_PER_SM = 5     /* CTAs that share one SM (1, 2 or 4)                    */
+    GRANQ_KNOB_STAGED_CTAS_PER_SM = 5     /* CTAs that share one SM (1 or 2)                       */
 };
 int granq_tune(int knob, int value);
 

@@ -89,7 +89,7 @@ struct StagedTuning {
     int grid;             // cap on the number of CTAs
     int spin_limit;       // iteration limit of the wait on a wave's arrival count
     int extra_arrivals;   // test hook: arrivals a wave waits for beyond the grid size (never come)
-    int ctas_per_sm;      // CTAs sharing one SM (1, 2 or 4); they split its threads and shared memory
+    int ctas_per_sm;      // CTAs sharing one SM (1 or 2); they split its threads and shared memory
 };
 StagedPlan plan_staged(int dtype, const Geom& g, const QuantIO& io, int device, const StagedTuning& tune);
 StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_count, int smem_optin,

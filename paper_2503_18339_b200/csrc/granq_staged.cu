@@ -10,12 +10,13 @@
 // that counter to reach the grid size, turns the keys into (s, z) (Eq. 5) and quantizes the
 // wave from shared memory (Eq. 1, clamp, Eq. 6) while streaming gy in and y / gx out (STE).
 //
-// There is no CTA-wide barrier in the steady state.  Every warp runs the same program
-//     phase 1 of waves 0 .. depth-2;  then for each wave w:  phase 2 of w, phase 1 of w+depth-1
-// over its own rows (128 units, 4 per lane), and the warps meet only through counters: the
-// last warp to finish phase 2 of a wave re-fills that wave's buffer with wave w + depth.
-// With depth 3 the loads of two waves are in flight and a wave's arrival counter has had a
-// whole phase 2 to fill up before anybody waits on it.
+// The warps of a CTA are specialised and there is no CTA-wide barrier in the steady state.
+// A few reducer warps run phase 1 wave after wave, as far ahead as loaded buffers allow;
+// the other (quantizer) warps run phase 2 wave after wave over rows of 128 units (4 per
+// lane), fetching the gy packs of their next row before doing the arithmetic of the current
+// one.  The last quantizer warp to finish a wave re-fills that wave's buffer with wave
+// w + depth.  With depth >= 2 a wave's arrival counter has filled up long before the
+// quantizers reach it, so neither the loads nor the grid-wide wait are exposed.
 //
 // Every wait is bounded: when one runs out the warp records GRANQ_ERR_TIMEOUT in the
 // workspace status word and raises the CTA's abort flag; all warps then leave their loops,
@@ -31,6 +32,8 @@ namespace {
 constexpr int kThreadsPerSm = 512;           // split over the CTAs that share an SM
 constexpr uint32_t kDefaultCtasPerSm = 1;
 constexpr uint32_t kRowUnits = 128;          // units one warp handles per step: 4 per lane
+constexpr uint32_t kReduceWarpsAligned = 2;  // warps of a CTA that run phase 1 (planes of whole packs)
+constexpr uint32_t kReduceWarpsRagged = 4;   // ... when packs straddle channels (more work per unit)
 constexpr uint32_t kMaxDepth = 3;
 constexpr uint32_t kMaxChunks = 64;          // chunks of one wave per CTA
 constexpr uint32_t kTabMax = 2048;           // channel groups per wave
@@ -58,8 +61,7 @@ struct ChunkDesc {
 
 // control words in shared memory
 struct Control {
-    uint32_t p1_done[2];          // warps that finished phase 1 of the wave with this parity
-    uint32_t p2_done[kMaxDepth];  // warps that finished phase 2 on this buffer
+    uint32_t p2_done[kMaxDepth];  // quantizer warps that finished phase 2 on this buffer
     uint32_t issued;              // waves whose loads have been issued
     uint32_t abort;               // a bounded wait ran out somewhere in this CTA
 };
@@ -188,10 +190,16 @@ __device__ __forceinline__ GroupParam group_param(const StagedArgs& a, uint32_t 
     return gp;
 }
 
+__device__ __forceinline__ void named_barrier(uint32_t id, uint32_t threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(threads) : "memory");
+}
+
 // EXTRAS: the optional per-element codes / mask outputs are compiled in
 template <typename T, int MODE, bool ALIGNED, bool EXTRAS, int NT>
 __global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const StagedArgs a) {
     constexpr uint32_t kWarps = NT / 32;
+    constexpr uint32_t kRWarps = ALIGNED ? kReduceWarpsAligned : kReduceWarpsRagged;   // reducer warps
+    constexpr uint32_t kQWarps = kWarps - kRWarps;                                     // quantizer warps
     constexpr int V = Pack<T>::V;
     constexpr bool kBwd = (MODE & MODE_BWD) != 0;
     extern __shared__ __align__(128) unsigned char smem[];
@@ -216,14 +224,11 @@ __global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const St
     for (uint32_t i = tid; i < 4 * a.tab_entries; i += NT) s_keys[i] = 0;
     __syncthreads();
 
-    bool alive = true;   // warp-uniform: no bounded wait has run out so far
-
     auto give_up = [&]() {
         if (lane == 0) {
             atomicExch(a.status, kStatusTimeout);
             atomicExch(&ctl->abort, 1u);
         }
-        alive = false;
     };
 
     // ---- issue the bulk loads of wave w into its buffer (one warp; one chunk per lane and round) ----
@@ -264,267 +269,276 @@ __global__ void __launch_bounds__(NT, kThreadsPerSm / NT) staged_kernel(const St
         return false;
     };
 
-    // ---- phase 1: this warp's rows of wave w -> min/max keys; the CTA's last warp publishes ----
-    auto reduce_wave = [&](uint32_t w) {
-        const WaveCtx c = wave_ctx(a, w);
-        const uint32_t b = w % D, par = w & 1u;
-        const uint4* buf = bufs + (size_t)b * a.buf_units;
-        const ChunkDesc* dsc = descs + b * kMaxChunks;
-        uint32_t* kmn = s_keys + (2 * par) * a.tab_entries;
-        uint32_t* kmx = kmn + a.tab_entries;
-        if (!__all_sync(kFullMask, wait_loaded(w))) {
-            give_up();
-            return;
-        }
-        WarpRun run{kNoGroup, 0u, 0u}, run2{kNoGroup, 0u, 0u};
-        const uint32_t rows = c.nk * a.rpc;
-        for (uint32_t row = warp; row < rows; row += kWarps) {
-            const uint32_t k = a.div_rpc.div(row), rr = row - k * a.rpc;
-            const ChunkDesc d = dsc[k];
-            const uint32_t r0 = rr * kRowUnits;
-            if (r0 >= d.len) continue;
-            const uint4* src = buf + (size_t)k * a.cu;
-            Pack<T> p[4];
-            bool v[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t uo = r0 + j * 32 + lane;
-                v[j] = uo < d.len;
-                if (v[j]) p[j].raw = src[uo];
-            }
-            if constexpr (ALIGNED) {
-                float mn[4], mx[4];
+    if (warp == 0)
+        for (uint32_t w = 0; w < min(D, W); ++w) issue(w);
+
+    if (warp < kRWarps) {
+        // =========================== reducer warps: phase 1 of every wave ===========================
+        for (uint32_t w = 0; w < W; ++w) {
+            const WaveCtx c = wave_ctx(a, w);
+            const uint32_t b = w % D, par = w & 1u;
+            const uint4* buf = bufs + (size_t)b * a.buf_units;
+            const ChunkDesc* dsc = descs + b * kMaxChunks;
+            uint32_t* kmn = s_keys + (2 * par) * a.tab_entries;
+            uint32_t* kmx = kmn + a.tab_entries;
+            const bool landed = __all_sync(kFullMask, wait_loaded(w));
+            if (!landed) give_up();
+            WarpRun run{kNoGroup, 0u, 0u}, run2{kNoGroup, 0u, 0u};
+            const uint32_t rows = landed ? c.nk * a.rpc : 0u;
+            for (uint32_t row = warp; row < rows; row += kRWarps) {
+                const uint32_t k = a.div_rpc.div(row), rr = row - k * a.rpc;
+                const ChunkDesc d = dsc[k];
+                const uint32_t r0 = rr * kRowUnits;
+                if (r0 >= d.len) continue;
+                const uint4* src = buf + (size_t)k * a.cu;
+                Pack<T> p[4];
+                bool v[4];
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    mn[j] = INFINITY;
-                    mx[j] = -INFINITY;
-                    if (v[j]) pack_minmax(p[j], 0, V, mn[j], mx[j]);
+                    const uint32_t uo = r0 + j * 32 + lane;
+                    v[j] = uo < d.len;
+                    if (v[j]) p[j].raw = src[uo];
                 }
-                const uint32_t ch_first = a.div_plane.div(d.su0 + r0);
-                const uint32_t ch_last = a.div_plane.div(d.su0 + min(r0 + kRowUnits, d.len) - 1);
-                if (ch_first == ch_last) {       // the whole row lies in one channel
-                    const float m0 = fminf(fminf(mn[0], mn[1]), fminf(mn[2], mn[3]));
-                    const float m1 = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-                    run_add(run, v[0], ch_first, ~enc(m0), enc(m1), kmn, kmx);
+                if constexpr (ALIGNED) {
+                    float mn[4], mx[4];
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        mn[j] = INFINITY;
+                        mx[j] = -INFINITY;
+                        if (v[j]) pack_minmax(p[j], 0, V, mn[j], mx[j]);
+                    }
+                    const uint32_t ch_first = a.div_plane.div(d.su0 + r0);
+                    const uint32_t ch_last = a.div_plane.div(d.su0 + min(r0 + kRowUnits, d.len) - 1);
+                    if (ch_first == ch_last) {       // the whole row lies in one channel
+                        const float m0 = fminf(fminf(mn[0], mn[1]), fminf(mn[2], mn[3]));
+                        const float m1 = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                        run_add(run, v[0], ch_first, ~enc(m0), enc(m1), kmn, kmx);
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t g = a.div_plane.div(d.su0 + r0 + j * 32 + lane);
+                            run_add(run, v[j], g, ~enc(mn[j]), enc(mx[j]), kmn, kmx);
+                        }
+                    }
                 } else {
 #pragma unroll
                     for (int j = 0; j < 4; ++j) {
-                        const uint32_t g = a.div_plane.div(d.su0 + r0 + j * 32 + lane);
-                        run_add(run, v[j], g, ~enc(mn[j]), enc(mx[j]), kmn, kmx);
+                        uint32_t pl = 0, rem = 0;
+                        a.div_plane.divmod((d.su0 + r0 + j * 32 + lane) * V, pl, rem);
+                        const int n1 = (int)min((uint32_t)V, a.inner - rem);      // elements of the first channel
+                        float mn1 = INFINITY, mx1 = -INFINITY, mn2 = INFINITY, mx2 = -INFINITY;
+                        if (v[j]) {
+                            pack_minmax(p[j], 0, n1, mn1, mx1);
+                            pack_minmax(p[j], n1, V, mn2, mx2);
+                        }
+                        run_add(run, v[j], pl, ~enc(mn1), enc(mx1), kmn, kmx);
+                        run_add(run2, v[j] && n1 < V, pl + 1, ~enc(mn2), enc(mx2), kmn, kmx);
                     }
                 }
-            } else {
+            }
+            run_flush(run, kmn, kmx);               // shared-memory atomics on the wave-local group index
+            if constexpr (!ALIGNED) run_flush(run2, kmn, kmx);
+            // all reducer warps meet; warp 0 then publishes the groups this CTA touched and arrives
+            named_barrier(1, kRWarps * 32);
+            const bool aborting = ld_volatile_shared(&ctl->abort) != 0;
+            if (warp == 0 && !aborting) {
+                for (uint32_t t = lane; t < c.sh->channels; t += 32) {
+                    const uint32_t k1 = atomicExch(kmn + t, 0u), k2 = atomicExch(kmx + t, 0u);
+                    if (k1 | k2) {
+                        atomicMax(a.kmin + c.c0 + t, k1);
+                        atomicMax(a.kmax + c.c0 + t, k2);
+                    }
+                }
+                __syncwarp();
+                if (lane == 0) {
+                    __threadfence();
+                    atomicAdd(a.counters + w, 1u);
+                }
+            }
+            if (aborting) break;     // uniform across the reducer warps: the flag was read after their barrier
+        }
+    } else {
+        // =========================== quantizer warps: phase 2 of every wave ===========================
+        const uint32_t qwarp = warp - kRWarps;
+        const float qmax = a.qmax;
+        for (uint32_t w = 0; w < W; ++w) {
+            const WaveCtx c = wave_ctx(a, w);
+            const uint32_t b = w % D;
+            const uint4* buf = bufs + (size_t)b * a.buf_units;
+            const ChunkDesc* dsc = descs + b * kMaxChunks;
+            // every CTA must have published wave w
+            bool ready = true;
+            if (lane == 0) {
+                ready = false;
+                for (uint32_t i = 0; i < a.spin_limit; ++i) {
+                    if (ld_acquire(a.counters + w) >= a.expected) {
+                        ready = true;
+                        break;
+                    }
+                    if (ld_volatile_shared(&ctl->abort)) break;
+                    __nanosleep(64);
+                }
+            }
+            ready = __all_sync(kFullMask, ready) && __all_sync(kFullMask, wait_loaded(w));
+            if (!ready) {
+                give_up();
+                break;
+            }
+            if (qwarp == 0 && (w % gridDim.x) == blockIdx.x) {       // one warp in the grid reports the wave's groups
+                for (uint32_t t = lane; t < c.sh->channels; t += 32) {
+                    float lo, hi;
+                    const GroupParam gp = group_param(a, c.c0 + t, lo, hi);
+                    a.lo[c.c0 + t] = lo;
+                    a.hi[c.c0 + t] = hi;
+                    if (a.s_out) a.s_out[c.c0 + t] = gp.s;
+                    if (a.z_out) a.z_out[c.c0 + t] = gp.z;
+                }
+            }
+            const uint32_t rows = c.nk * a.rpc;
+
+            // a row: where it is, and its gy packs (fetched one row ahead of the arithmetic)
+            struct Row {
+                ChunkDesc d;
+                uint32_t k, r0;
+                bool any;
+            };
+            auto fetch = [&](uint32_t row, Row& r, Pack<T> (&pg)[4]) {
+                r.any = row < rows;
+                if (!r.any) return;
+                r.k = a.div_rpc.div(row);
+                r.d = dsc[r.k];
+                r.r0 = (row - r.k * a.rpc) * kRowUnits;
+                r.any = r.r0 < r.d.len;
+                if constexpr (kBwd) {
+                    if (r.any) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            const uint32_t uo = r.r0 + j * 32 + lane;
+                            if (uo < r.d.len) pg[j].raw = ld_stream_16(gyg + r.d.gu0 + uo);
+                        }
+                    }
+                }
+            };
+            auto compute = [&](const Row& r, const Pack<T> (&pg)[4]) {
+                if (!r.any) return;
+                const ChunkDesc d = r.d;
+                const uint32_t r0 = r.r0;
+                const uint4* src = buf + (size_t)r.k * a.cu;
+                // parameters of the channels this row touches: lane l holds channel ch_first + l
+                const uint32_t last_u = d.su0 + min(r0 + kRowUnits, d.len) - 1;
+                const uint32_t ch_first = ALIGNED ? a.div_plane.div(d.su0 + r0) : a.div_plane.div((d.su0 + r0) * V);
+                const uint32_t ch_last = ALIGNED ? a.div_plane.div(last_u) : a.div_plane.div(last_u * V + (V - 1));
+                const uint32_t nch = ch_last - ch_first + 1;
+                const bool shared_params = nch <= 32;
+                GroupParam mine{1.0f, 0.0f, 0.0f};
+                if (shared_params && lane < nch) {
+                    float lo, hi;
+                    mine = group_param(a, c.c0 + ch_first + lane, lo, hi);
+                }
 #pragma unroll
                 for (int j = 0; j < 4; ++j) {
-                    uint32_t pl = 0, rem = 0;
-                    a.div_plane.divmod((d.su0 + r0 + j * 32 + lane) * V, pl, rem);
-                    const int n1 = (int)min((uint32_t)V, a.inner - rem);      // elements of the first channel
-                    float mn1 = INFINITY, mx1 = -INFINITY, mn2 = INFINITY, mx2 = -INFINITY;
-                    if (v[j]) {
-                        pack_minmax(p[j], 0, n1, mn1, mx1);
-                        pack_minmax(p[j], n1, V, mn2, mx2);
-                    }
-                    run_add(run, v[j], pl, ~enc(mn1), enc(mx1), kmn, kmx);
-                    run_add(run2, v[j] && n1 < V, pl + 1, ~enc(mn2), enc(mx2), kmn, kmx);
-                }
-            }
-        }
-        run_flush(run, kmn, kmx);               // shared-memory atomics on the wave-local group index
-        if constexpr (!ALIGNED) run_flush(run2, kmn, kmx);
-        __syncwarp();
-        uint32_t prev = 0;
-        if (lane == 0) {
-            __threadfence_block();
-            prev = atomicAdd(&ctl->p1_done[par], 1u);
-        }
-        prev = __shfl_sync(kFullMask, prev, 0);
-        if (prev == kWarps - 1) {
-            // last warp of the CTA: publish the groups this CTA touched, then arrive on the wave counter
-            __threadfence_block();
-            for (uint32_t t = lane; t < c.sh->channels; t += 32) {
-                const uint32_t k1 = atomicExch(kmn + t, 0u), k2 = atomicExch(kmx + t, 0u);
-                if (k1 | k2) {
-                    atomicMax(a.kmin + c.c0 + t, k1);
-                    atomicMax(a.kmax + c.c0 + t, k2);
-                }
-            }
-            __syncwarp();
-            if (lane == 0) {
-                atomicExch(&ctl->p1_done[par], 0u);
-                __threadfence();
-                atomicAdd(a.counters + w, 1u);
-            }
-        }
-    };
-
-    // ---- phase 2: this warp's rows of wave w, quantized from shared memory ----
-    auto quantize_wave = [&](uint32_t w) {
-        const WaveCtx c = wave_ctx(a, w);
-        const uint32_t b = w % D;
-        const uint4* buf = bufs + (size_t)b * a.buf_units;
-        const ChunkDesc* dsc = descs + b * kMaxChunks;
-        const float qmax = a.qmax;
-        // every CTA must have published wave w
-        bool ready = true;
-        if (lane == 0) {
-            ready = false;
-            for (uint32_t i = 0; i < a.spin_limit; ++i) {
-                if (ld_acquire(a.counters + w) >= a.expected) {
-                    ready = true;
-                    break;
-                }
-                if (ld_volatile_shared(&ctl->abort)) break;
-                __nanosleep(64);
-            }
-        }
-        ready = __all_sync(kFullMask, ready) && __all_sync(kFullMask, wait_loaded(w));
-        if (!ready) {
-            give_up();
-            return;
-        }
-        if (warp == 0 && (w % gridDim.x) == blockIdx.x) {       // one warp in the grid reports the wave's groups
-            for (uint32_t t = lane; t < c.sh->channels; t += 32) {
-                float lo, hi;
-                const GroupParam gp = group_param(a, c.c0 + t, lo, hi);
-                a.lo[c.c0 + t] = lo;
-                a.hi[c.c0 + t] = hi;
-                if (a.s_out) a.s_out[c.c0 + t] = gp.s;
-                if (a.z_out) a.z_out[c.c0 + t] = gp.z;
-            }
-        }
-        const uint32_t rows = c.nk * a.rpc;
-        for (uint32_t row = warp; row < rows; row += kWarps) {
-            const uint32_t k = a.div_rpc.div(row), rr = row - k * a.rpc;
-            const ChunkDesc d = dsc[k];
-            const uint32_t r0 = rr * kRowUnits;
-            if (r0 >= d.len) continue;
-            const uint4* src = buf + (size_t)k * a.cu;
-            Pack<T> pg[4];
-            bool v[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t uo = r0 + j * 32 + lane;
-                v[j] = uo < d.len;
-                if constexpr (kBwd) {
-                    if (v[j]) pg[j].raw = ld_stream_16(gyg + d.gu0 + uo);
-                }
-            }
-            // parameters of the channels this row touches: lane l holds channel ch_first + l
-            const uint32_t last_u = d.su0 + min(r0 + kRowUnits, d.len) - 1;
-            const uint32_t ch_first = ALIGNED ? a.div_plane.div(d.su0 + r0) : a.div_plane.div((d.su0 + r0) * V);
-            const uint32_t ch_last = ALIGNED ? a.div_plane.div(last_u) : a.div_plane.div(last_u * V + (V - 1));
-            const uint32_t nch = ch_last - ch_first + 1;
-            const bool shared_params = nch <= 32;
-            GroupParam mine{1.0f, 0.0f, 0.0f};
-            if (shared_params && lane < nch) {
-                float lo, hi;
-                mine = group_param(a, c.c0 + ch_first + lane, lo, hi);
-            }
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-                const uint32_t uo = r0 + j * 32 + lane;
-                uint32_t ci1 = 0, ci2 = 0;
-                int n1 = V;
-                if constexpr (ALIGNED) {
-                    ci1 = a.div_plane.div(d.su0 + (v[j] ? uo : r0));
-                    ci2 = ci1;
-                } else {
-                    uint32_t rem;
-                    a.div_plane.divmod((d.su0 + (v[j] ? uo : r0)) * V, ci1, rem);
-                    n1 = (int)min((uint32_t)V, a.inner - rem);
-                    ci2 = min(ci1 + 1, c.sh->channels - 1);
-                }
-                GroupParam g1, g2;
-                if (shared_params) {
-                    const uint32_t i1 = ci1 - ch_first, i2 = min(ci2 - ch_first, nch - 1);
-                    g1.s = __shfl_sync(kFullMask, mine.s, i1);
-                    g1.z = __shfl_sync(kFullMask, mine.z, i1);
-                    g1.r = __shfl_sync(kFullMask, mine.r, i1);
+                    const uint32_t uo = r0 + j * 32 + lane;
+                    const bool valid = uo < d.len;
+                    uint32_t ci1 = 0, ci2 = 0;
+                    int n1 = V;
                     if constexpr (ALIGNED) {
-                        g2 = g1;
+                        ci1 = a.div_plane.div(d.su0 + (valid ? uo : r0));
+                        ci2 = ci1;
                     } else {
-                        g2.s = __shfl_sync(kFullMask, mine.s, i2);
-                        g2.z = __shfl_sync(kFullMask, mine.z, i2);
-                        g2.r = __shfl_sync(kFullMask, mine.r, i2);
+                        uint32_t rem;
+                        a.div_plane.divmod((d.su0 + (valid ? uo : r0)) * V, ci1, rem);
+                        n1 = (int)min((uint32_t)V, a.inner - rem);
+                        ci2 = min(ci1 + 1, c.sh->channels - 1);
                     }
-                } else {
-                    float lo, hi;
-                    g1 = group_param(a, c.c0 + ci1, lo, hi);
-                    g2 = ALIGNED ? g1 : group_param(a, c.c0 + ci2, lo, hi);
-                }
-                if (!v[j]) continue;
-                Pack<T> px, py, pgx;
-                px.raw = src[uo];
-                uint32_t cb[V / 4] = {}, mb[V / 4] = {};
-                auto element = [&](int i, float t, float s, float z) {
-                    float yv;
-                    bool in;
-                    const float code = quant_from_quotient(t, s, z, qmax, yv, in);
-                    py.set(i, yv);
-                    if constexpr (kBwd) pgx.set(i, in ? pg[j].get(i) : 0.0f);
+                    GroupParam g1, g2;
+                    if (shared_params) {
+                        const uint32_t i1 = ci1 - ch_first, i2 = min(ci2 - ch_first, nch - 1);
+                        g1.s = __shfl_sync(kFullMask, mine.s, i1);
+                        g1.z = __shfl_sync(kFullMask, mine.z, i1);
+                        g1.r = __shfl_sync(kFullMask, mine.r, i1);
+                        if constexpr (ALIGNED) {
+                            g2 = g1;
+                        } else {
+                            g2.s = __shfl_sync(kFullMask, mine.s, i2);
+                            g2.z = __shfl_sync(kFullMask, mine.z, i2);
+                            g2.r = __shfl_sync(kFullMask, mine.r, i2);
+                        }
+                    } else {
+                        float lo, hi;
+                        g1 = group_param(a, c.c0 + ci1, lo, hi);
+                        g2 = ALIGNED ? g1 : group_param(a, c.c0 + ci2, lo, hi);
+                    }
+                    if (!valid) continue;
+                    Pack<T> px, py, pgx;
+                    px.raw = src[uo];
+                    uint32_t cb[V / 4] = {}, mb[V / 4] = {};
+                    auto element = [&](int i, float t, float s, float z) {
+                        float yv;
+                        bool in;
+                        const float code = quant_from_quotient(t, s, z, qmax, yv, in);
+                        py.set(i, yv);
+                        if constexpr (kBwd) pgx.set(i, in ? pg[j].get(i) : 0.0f);
+                        if constexpr (EXTRAS) {
+                            cb[i / 4] |= (uint32_t)code << (8 * (i % 4));
+                            mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
+                        }
+                    };
+                    if ((g1.r != 0.0f) && (g2.r != 0.0f)) {
+#pragma unroll
+                        for (int i = 0; i < V; ++i) {
+                            const bool first = ALIGNED || i < n1;
+                            const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z, rc = first ? g1.r : g2.r;
+                            element(i, div_by_scale(px.get(i), s, rc), s, z);
+                        }
+                    } else {
+#pragma unroll
+                        for (int i = 0; i < V; ++i) {
+                            const bool first = ALIGNED || i < n1;
+                            const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z;
+                            element(i, __fdiv_rn(px.get(i), s), s, z);
+                        }
+                    }
+                    const uint32_t gu = d.gu0 + uo;
+                    st_stream_16(yg + gu, py.raw);
+                    if constexpr (kBwd) st_stream_16(gxg + gu, pgx.raw);
                     if constexpr (EXTRAS) {
-                        cb[i / 4] |= (uint32_t)code << (8 * (i % 4));
-                        mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
-                    }
-                };
-                if ((g1.r != 0.0f) && (g2.r != 0.0f)) {
+                        if (a.codes) {
 #pragma unroll
-                    for (int i = 0; i < V; ++i) {
-                        const bool first = ALIGNED || i < n1;
-                        const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z, r = first ? g1.r : g2.r;
-                        element(i, div_by_scale(px.get(i), s, r), s, z);
-                    }
-                } else {
+                            for (int i = 0; i < V / 4; ++i)
+                                reinterpret_cast<uint32_t*>(a.codes)[(size_t)gu * (V / 4) + i] = cb[i];
+                        }
+                        if (kBwd && a.mask) {
 #pragma unroll
-                    for (int i = 0; i < V; ++i) {
-                        const bool first = ALIGNED || i < n1;
-                        const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z;
-                        element(i, __fdiv_rn(px.get(i), s), s, z);
+                            for (int i = 0; i < V / 4; ++i)
+                                reinterpret_cast<uint32_t*>(a.mask)[(size_t)gu * (V / 4) + i] = mb[i];
+                        }
                     }
                 }
-                const uint32_t gu = d.gu0 + uo;
-                st_stream_16(yg + gu, py.raw);
-                if constexpr (kBwd) st_stream_16(gxg + gu, pgx.raw);
-                if constexpr (EXTRAS) {
-                    if (a.codes) {
-#pragma unroll
-                        for (int i = 0; i < V / 4; ++i)
-                            reinterpret_cast<uint32_t*>(a.codes)[(size_t)gu * (V / 4) + i] = cb[i];
-                    }
-                    if (kBwd && a.mask) {
-#pragma unroll
-                        for (int i = 0; i < V / 4; ++i)
-                            reinterpret_cast<uint32_t*>(a.mask)[(size_t)gu * (V / 4) + i] = mb[i];
-                    }
-                }
-            }
-        }
-        // the last warp to leave the buffer re-fills it with wave w + depth
-        __syncwarp();
-        uint32_t prev = 0;
-        if (lane == 0) {
-            __threadfence_block();
-            prev = atomicAdd(&ctl->p2_done[b], 1u);
-        }
-        prev = __shfl_sync(kFullMask, prev, 0);
-        if (prev == kWarps - 1) {
-            if (lane == 0) atomicExch(&ctl->p2_done[b], 0u);
-            __syncwarp();
-            if (w + D < W) issue(w + D);
-        }
-    };
+            };
 
-    // ---- the per-warp program ----
-    if (warp == 0)
-        for (uint32_t w = 0; w < min(D, W); ++w) issue(w);
-    if (D == 1) {
-        reduce_wave(0);
-        if (alive) quantize_wave(0);
-    } else {
-        for (uint32_t w = 0; alive && w < min(D - 1, W); ++w) reduce_wave(w);
-        for (uint32_t w = 0; alive && w < W; ++w) {
-            quantize_wave(w);
-            if (alive && w + D - 1 < W) reduce_wave(w + D - 1);
+            Row ra, rb;
+            Pack<T> pa[4], pb[4];
+            fetch(qwarp, ra, pa);
+            for (uint32_t row = qwarp; row < rows; row += 2 * kQWarps) {
+                fetch(row + kQWarps, rb, pb);
+                compute(ra, pa);
+                fetch(row + 2 * kQWarps, ra, pa);
+                compute(rb, pb);
+            }
+
+            // the last quantizer warp to leave the buffer re-fills it with wave w + depth
+            __syncwarp();
+            uint32_t prev = 0;
+            if (lane == 0) {
+                __threadfence_block();
+                prev = atomicAdd(&ctl->p2_done[b], 1u);
+            }
+            prev = __shfl_sync(kFullMask, prev, 0);
+            if (prev == kQWarps - 1) {
+                if (lane == 0) atomicExch(&ctl->p2_done[b], 0u);
+                __syncwarp();
+                if (w + D < W) issue(w + D);
+            }
         }
     }
     __syncthreads();
@@ -563,8 +577,7 @@ cudaError_t launch_nt(const StagedPlan& plan, StagedArgs& args, cudaStream_t st)
 template <typename T, int MODE, bool ALIGNED, bool EXTRAS>
 cudaError_t launch_t(const StagedPlan& plan, StagedArgs& args, cudaStream_t st) {
     if (plan.threads == 512) return launch_nt<T, MODE, ALIGNED, EXTRAS, 512>(plan, args, st);
-    if (plan.threads == 256) return launch_nt<T, MODE, ALIGNED, EXTRAS, 256>(plan, args, st);
-    return launch_nt<T, MODE, ALIGNED, EXTRAS, 128>(plan, args, st);
+    return launch_nt<T, MODE, ALIGNED, EXTRAS, 256>(plan, args, st);
 }
 
 template <typename T, int MODE>
@@ -625,8 +638,8 @@ StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_co
 
     const uint32_t inner = (uint32_t)g.inner, C = (uint32_t)g.C, O = (uint32_t)g.outer;
     const uint32_t q = V / gcd_u32(inner, V);          // waves hold multiples of q channels (16-byte slabs)
-    const uint32_t cps_sm = (tune.ctas_per_sm == 1 || tune.ctas_per_sm == 2 || tune.ctas_per_sm == 4)
-                                ? (uint32_t)tune.ctas_per_sm : kDefaultCtasPerSm;
+    const uint32_t cps_sm = (tune.ctas_per_sm == 1 || tune.ctas_per_sm == 2) ? (uint32_t)tune.ctas_per_sm
+                                                                             : kDefaultCtasPerSm;
     const uint32_t full_grid = (uint32_t)sm_count * cps_sm;
     const uint32_t grid = (tune.grid > 0 && (uint32_t)tune.grid < full_grid) ? (uint32_t)tune.grid : full_grid;
     // an SM holds 1 KB more than one CTA may ask for, and reserves 1 KB per resident CTA
