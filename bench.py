@@ -185,6 +185,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="also print a per-tensor table to stderr")
     ap.add_argument("--tune", default="", help="planner overrides for experiments, e.g. depth=3,max_buf_units=4000")
+    ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged"],
+                    help="force an execution plan of the fused entry point (experiments)")
     ap.add_argument("--only", default="", help="profiling aid: keep only workload tensors whose name contains this")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -210,6 +212,8 @@ def main():
         name, val = item.split("=")
         b.tune(knob_ids[name], int(val))
     warmup = max(args.warmup, 3)
+    flags = {"auto": 0, "two_pass": b.FLAG_FORCE_TWO_PASS, "naive": b.FLAG_FORCE_NAIVE,
+             "staged": b.FLAG_FORCE_STAGED}[args.plan]
 
     specs = [s for s in workload_specs() if args.only in s.name]
     # ---- host (pinned) inputs and outputs; every rank has its own batch (weak scaling, no exchange) ----
@@ -232,7 +236,7 @@ def main():
     calls = [(i, bits) for i, s in enumerate(specs) for bits in s.bits]
     elems_per_step = sum(specs[i].numel for i, _ in calls)
     bytes_per_step = elems_per_step * BYTES_PER_ELEM
-    plans = [b.fused_plan(b.F32, specs[i].shape) for i, _ in calls]
+    plans = [b.fused_plan(b.F32, specs[i].shape, flags=flags) for i, _ in calls]
     launches_per_step = sum(n for _, n in plans)
     stream = torch.cuda.current_stream()
 
@@ -241,7 +245,7 @@ def main():
             x, gy, out = dev[i]
             if events is not None:
                 events[ci][0].record(stream)
-            b.granq_fakequant_fused(x, bits, gy=gy, out=out, stream=stream)
+            b.granq_fakequant_fused(x, bits, gy=gy, out=out, flags=flags, stream=stream)
             if events is not None:
                 events[ci][1].record(stream)
 

@@ -224,4 +224,102 @@ __device__ __forceinline__ void run_add(WarpRun& r, bool valid, uint32_t g, uint
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Per-group parameters from the published min / max keys, and the arithmetic of one pack.
+// ---------------------------------------------------------------------------------------
+struct GroupParam {
+    float s, z, r;   // scale, zero-point, RN(1 / s) or 0 when the group must use IEEE division
+};
+
+__device__ __forceinline__ GroupParam group_param_from_keys(const uint32_t* kmin, const uint32_t* kmax, uint32_t g,
+                                                            float qmax, float& lo, float& hi) {
+    keys_to_range(__ldcg(kmin + g), __ldcg(kmax + g), lo, hi);
+    const QParam p = make_qparam(lo, hi, qmax);
+    GroupParam gp;
+    gp.s = p.s;
+    gp.z = p.z;
+    gp.r = div_is_safe(p.s, lo, hi) ? __frcp_rn(p.s) : 0.0f;
+    return gp;
+}
+
+// Quantize one pack: elements [0, n1) belong to the group with parameters g1, the rest to
+// g2 (n1 = V when the pack lies in one group).  EXTRAS also packs the codes and the mask
+// (one byte per element).
+template <typename T, bool BWD, bool SPLIT, bool EXTRAS>
+__device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& pg, const GroupParam& g1,
+                                              const GroupParam& g2, int n1, float qmax, Pack<T>& py, Pack<T>& pgx,
+                                              uint32_t (&cb)[Pack<T>::V / 4], uint32_t (&mb)[Pack<T>::V / 4]) {
+    constexpr int V = Pack<T>::V;
+#pragma unroll
+    for (int i = 0; i < V / 4; ++i) {
+        cb[i] = 0;
+        mb[i] = 0;
+    }
+    auto element = [&](int i, float t, float s, float z) {
+        float yv;
+        bool in;
+        const float code = quant_from_quotient(t, s, z, qmax, yv, in);
+        py.set(i, yv);
+        if constexpr (BWD) pgx.set(i, in ? pg.get(i) : 0.0f);
+        if constexpr (EXTRAS) {
+            cb[i / 4] |= (uint32_t)code << (8 * (i % 4));
+            mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
+        }
+    };
+    const bool fast = SPLIT ? (g1.r != 0.0f && g2.r != 0.0f) : (g1.r != 0.0f);
+    if (fast) {
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const bool first = !SPLIT || i < n1;
+            const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z, rc = first ? g1.r : g2.r;
+            element(i, div_by_scale(px.get(i), s, rc), s, z);
+        }
+    } else {
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const bool first = !SPLIT || i < n1;
+            const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z;
+            element(i, __fdiv_rn(px.get(i), s), s, z);
+        }
+    }
+}
+
+// per-lane min / max of elements [first, last) of one pack
+template <typename T>
+__device__ __forceinline__ void pack_minmax(const Pack<T>& p, int first, int last, float& mn, float& mx) {
+#pragma unroll
+    for (int i = 0; i < Pack<T>::V; ++i) {
+        if (i >= first && i < last) {
+            float v = p.get(i);
+            mn = fminf(mn, v);
+            mx = fmaxf(mx, v);
+        }
+    }
+}
+
+// 128-bit global accesses with an L2 eviction policy (createpolicy.fractional.L2::evict_*)
+__device__ __forceinline__ uint64_t l2_policy_evict_last() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_last.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
+__device__ __forceinline__ uint4 ld_hint_16(const void* p, uint64_t policy) {
+    uint4 v;
+    asm volatile("ld.global.L1::no_allocate.L2::cache_hint.v4.u32 {%0,%1,%2,%3}, [%4], %5;"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+                 : "l"(p), "l"(policy)
+                 : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_hint_16(void* p, uint4 v, uint64_t policy) {
+    asm volatile("st.global.L2::cache_hint.v4.u32 [%0], {%1,%2,%3,%4}, %5;" ::"l"(p), "r"(v.x), "r"(v.y), "r"(v.z),
+                 "r"(v.w), "l"(policy)
+                 : "memory");
+}
+
 }  // namespace granq

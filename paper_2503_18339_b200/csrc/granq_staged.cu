@@ -163,31 +163,9 @@ __device__ __forceinline__ ChunkDesc chunk_of(const StagedArgs& a, const WaveCtx
     return d;
 }
 
-// per-lane min / max of elements [first, last) of one pack
-template <typename T>
-__device__ __forceinline__ void pack_minmax(const Pack<T>& p, int first, int last, float& mn, float& mx) {
-#pragma unroll
-    for (int i = 0; i < Pack<T>::V; ++i) {
-        if (i >= first && i < last) {
-            float v = p.get(i);
-            mn = fminf(mn, v);
-            mx = fmaxf(mx, v);
-        }
-    }
-}
-
-// scale, zero-point and reciprocal (0 = use IEEE division) of one group from its published keys
-struct GroupParam {
-    float s, z, r;
-};
+// scale, zero-point and reciprocal of one group from its published keys
 __device__ __forceinline__ GroupParam group_param(const StagedArgs& a, uint32_t g, float& lo, float& hi) {
-    keys_to_range(__ldcg(a.kmin + g), __ldcg(a.kmax + g), lo, hi);
-    const QParam p = make_qparam(lo, hi, a.qmax);
-    GroupParam gp;
-    gp.s = p.s;
-    gp.z = p.z;
-    gp.r = div_is_safe(p.s, lo, hi) ? __frcp_rn(p.s) : 0.0f;
-    return gp;
+    return group_param_from_keys(a.kmin, a.kmax, g, a.qmax, lo, hi);
 }
 
 __device__ __forceinline__ void named_barrier(uint32_t id, uint32_t threads) {
