@@ -185,7 +185,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="also print a per-tensor table to stderr")
     ap.add_argument("--tune", default="", help="planner overrides for experiments, e.g. depth=3,max_buf_units=4000")
-    ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged"],
+    ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged", "l2wave"],
                     help="force an execution plan of the fused entry point (experiments)")
     ap.add_argument("--only", default="", help="profiling aid: keep only workload tensors whose name contains this")
     args = ap.parse_args()
@@ -207,13 +207,14 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     b.lib()
     knob_ids = {"depth": b.KNOB_STAGED_DEPTH, "max_buf_units": b.KNOB_STAGED_MAX_BUF_UNITS,
-                "grid": b.KNOB_STAGED_GRID, "ctas_per_sm": b.KNOB_STAGED_CTAS_PER_SM}
+                "grid": b.KNOB_STAGED_GRID, "ctas_per_sm": b.KNOB_STAGED_CTAS_PER_SM,
+                "l2_wave_kb": b.KNOB_L2_WAVE_KB, "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM}
     for item in filter(None, args.tune.split(",")):
         name, val = item.split("=")
         b.tune(knob_ids[name], int(val))
     warmup = max(args.warmup, 3)
     flags = {"auto": 0, "two_pass": b.FLAG_FORCE_TWO_PASS, "naive": b.FLAG_FORCE_NAIVE,
-             "staged": b.FLAG_FORCE_STAGED}[args.plan]
+             "staged": b.FLAG_FORCE_STAGED, "l2wave": b.FLAG_FORCE_L2WAVE}[args.plan]
 
     specs = [s for s in workload_specs() if args.only in s.name]
     # ---- host (pinned) inputs and outputs; every rank has its own batch (weak scaling, no exchange) ----

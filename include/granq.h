@@ -80,7 +80,8 @@ enum granq_flags {
     GRANQ_FLAG_FORCE_TWO_PASS = 1u,  /* fused: range launch + quantize launch (x is read twice)      */
     GRANQ_FLAG_FORCE_NAIVE = 2u,     /* fused: host loop over channels, three launches per channel -
                                         the "conventional" scalar-loop scheme of Section 5.3.2       */
-    GRANQ_FLAG_FORCE_STAGED = 4u     /* fused: on-chip-staged persistent kernel or GRANQ_ERR_UNSUPPORTED */
+    GRANQ_FLAG_FORCE_STAGED = 4u,    /* fused: on-chip-staged persistent kernel or GRANQ_ERR_UNSUPPORTED */
+    GRANQ_FLAG_FORCE_L2WAVE = 8u     /* fused: L2-resident-wave persistent kernel or GRANQ_ERR_UNSUPPORTED */
 };
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -168,7 +169,8 @@ int granq_fakequant_fused_host(const void* x_host, const void* gy_host_opt, int 
 
 /*
  * Plan that granq_fakequant_fused() would take for this geometry and flags on the current
- * device: 0 = two-pass, 1 = naive per-channel loop, 2 = on-chip staged; negative = -status.
+ * device: 0 = two-pass, 1 = naive per-channel loop, 2 = on-chip staged, 3 = L2-resident waves;
+ * negative = -status.
  * `launches_out` (HOST, may be NULL) receives the number of kernel launches of that plan.
  */
 int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,
@@ -208,7 +210,10 @@ enum granq_knob {
     GRANQ_KNOB_TEST_EXTRA_ARRIVALS = 4,   /* test hook: a wave waits for this many arrivals more
                                              than the grid provides, so the bounded wait runs out
                                              and the call ends with GRANQ_ERR_TIMEOUT              */
-    GRANQ_KNOB_STAGED_CTAS_PER_SM = 5     /* CTAs that share one SM (1 or 2)                       */
+    GRANQ_KNOB_STAGED_CTAS_PER_SM = 5,    /* CTAs that share one SM (1 or 2)                       */
+    GRANQ_KNOB_L2_WAVE_KB = 6,            /* L2-wave plan: x bytes of one wave, in KiB             */
+    GRANQ_KNOB_L2_UPL = 7,                /* L2-wave plan: 16-byte units per lane and step (2, 4)  */
+    GRANQ_KNOB_L2_CTAS_PER_SM = 8         /* L2-wave plan: cap on resident CTAs per SM             */
 };
 int granq_tune(int knob, int value);
 

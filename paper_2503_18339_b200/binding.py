@@ -18,11 +18,11 @@ LIB_PATH = os.path.join(_HERE, "libgranq.so")
 
 F32, BF16 = 0, 1
 GROUP_CHANNEL, GROUP_SAMPLE_CHANNEL, GROUP_TENSOR = 0, 1, 2
-FLAG_FORCE_TWO_PASS, FLAG_FORCE_NAIVE, FLAG_FORCE_STAGED = 1, 2, 4
-PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED = 0, 1, 2
+FLAG_FORCE_TWO_PASS, FLAG_FORCE_NAIVE, FLAG_FORCE_STAGED, FLAG_FORCE_L2WAVE = 1, 2, 4, 8
+PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED, PLAN_L2WAVE = 0, 1, 2, 3
 (KNOB_STAGED_DEPTH, KNOB_STAGED_MAX_BUF_UNITS, KNOB_STAGED_GRID, KNOB_SPIN_LIMIT, KNOB_TEST_EXTRA_ARRIVALS,
- KNOB_STAGED_CTAS_PER_SM) = range(6)
-N_KNOBS = 6
+ KNOB_STAGED_CTAS_PER_SM, KNOB_L2_WAVE_KB, KNOB_L2_UPL, KNOB_L2_CTAS_PER_SM) = range(9)
+N_KNOBS = 9
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 
 EXPORTS = [

@@ -10,7 +10,7 @@ namespace {
 
 constexpr int64_t kMaxElements = 1ll << 40;
 
-StagedTuning g_tune = {0, 0, 0, 0, 0, 0};
+StagedTuning g_tune = {0, 0, 0, 0, 0, 0, 0, 0, 0};
 
 bool make_geom(const int64_t dims[4], int axis, int group, Geom& g, int64_t& G) {
     if (!dims || axis < 0 || axis > 3 || group < 0 || group > 2) return false;
@@ -55,12 +55,19 @@ int check_workspace(const void* ws, size_t bytes, int64_t G) {
 
 int cuda_status(cudaError_t e) { return e == cudaSuccess ? GRANQ_OK : GRANQ_ERR_CUDA; }
 
-enum { PLAN_TWO_PASS = 0, PLAN_NAIVE = 1, PLAN_STAGED = 2 };
+enum { PLAN_TWO_PASS = 0, PLAN_NAIVE = 1, PLAN_STAGED = 2, PLAN_L2WAVE = 3 };
 
 // plan of the fused entry point; `plan_out` is filled when the staged plan is taken
-int choose_plan(int dtype, const Geom& g, const QuantIO& io, uint32_t flags, StagedPlan* plan_out) {
+int choose_plan(int dtype, const Geom& g, const QuantIO& io, uint32_t flags, StagedPlan* plan_out,
+                L2Plan* l2_out) {
     if (flags & GRANQ_FLAG_FORCE_NAIVE) return PLAN_NAIVE;
     if (flags & GRANQ_FLAG_FORCE_TWO_PASS) return PLAN_TWO_PASS;
+    if (flags & GRANQ_FLAG_FORCE_L2WAVE) {
+        L2Plan lp = plan_l2wave(dtype, g, io, g_tune);
+        if (!lp.ok) return -GRANQ_ERR_UNSUPPORTED;
+        if (l2_out) *l2_out = lp;
+        return PLAN_L2WAVE;
+    }
     int dev = 0;
     if (cudaGetDevice(&dev) != cudaSuccess) return -GRANQ_ERR_CUDA;
     StagedPlan p = plan_staged(dtype, g, io, dev, g_tune);
@@ -179,7 +186,8 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
     const int mode = gy_opt ? MODE_BOTH : MODE_FWD;
     QuantIO io{x, gy_opt, y, gx_opt, codes_opt, mask_opt};
     StagedPlan sp{};
-    const int plan = choose_plan(dtype, g, io, flags, &sp);
+    L2Plan lp{};
+    const int plan = choose_plan(dtype, g, io, flags, &sp, &lp);
     if (plan < 0) return -plan;
 
     Workspace ws = carve_workspace(workspace, G);
@@ -187,6 +195,8 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
     if (e != cudaSuccess) return GRANQ_ERR_CUDA;
     if (plan == PLAN_STAGED) {
         e = launch_staged(sp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
+    } else if (plan == PLAN_L2WAVE) {
+        e = launch_l2wave(lp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
     } else if (plan == PLAN_NAIVE) {
         e = launch_naive(io, mode, dtype, g, bits, ws.kmin, ws.kmax, min_out, max_out, st, nullptr);
         if (e == cudaSuccess && (scale_opt || zp_opt))
@@ -270,9 +280,9 @@ int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int gro
     if (!dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G)) return -GRANQ_ERR_INVALID_ARG;
     (void)with_backward;
     QuantIO io{};   // null pointers: alignment is assumed
-    const int plan = choose_plan(dtype, g, io, flags, nullptr);
+    const int plan = choose_plan(dtype, g, io, flags, nullptr, nullptr);
     if (launches_out) {
-        if (plan == PLAN_STAGED) *launches_out = 1;
+        if (plan == PLAN_STAGED || plan == PLAN_L2WAVE) *launches_out = 1;
         else if (plan == PLAN_NAIVE) *launches_out = (int)(3 * g.C);
         else if (plan == PLAN_TWO_PASS) *launches_out = 3;
     }
@@ -300,6 +310,9 @@ int granq_tune(int knob, int value) {
         case GRANQ_KNOB_SPIN_LIMIT: g_tune.spin_limit = value; return GRANQ_OK;
         case GRANQ_KNOB_TEST_EXTRA_ARRIVALS: g_tune.extra_arrivals = value; return GRANQ_OK;
         case GRANQ_KNOB_STAGED_CTAS_PER_SM: g_tune.ctas_per_sm = value; return GRANQ_OK;
+        case GRANQ_KNOB_L2_WAVE_KB: g_tune.l2_wave_kb = value; return GRANQ_OK;
+        case GRANQ_KNOB_L2_UPL: g_tune.l2_upl = value; return GRANQ_OK;
+        case GRANQ_KNOB_L2_CTAS_PER_SM: g_tune.l2_ctas_per_sm = value; return GRANQ_OK;
         default: return GRANQ_ERR_INVALID_ARG;
     }
 }

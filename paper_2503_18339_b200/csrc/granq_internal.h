@@ -90,11 +90,27 @@ struct StagedTuning {
     int spin_limit;       // iteration limit of the wait on a wave's arrival count
     int extra_arrivals;   // test hook: arrivals a wave waits for beyond the grid size (never come)
     int ctas_per_sm;      // CTAs sharing one SM (1 or 2); they split its threads and shared memory
+    int l2_wave_kb;       // L2-wave plan: target x bytes of one wave, in KiB
+    int l2_upl;           // L2-wave plan: 16-byte units per lane and step (2 or 4)
+    int l2_ctas_per_sm;   // L2-wave plan: cap on resident CTAs per SM
 };
 StagedPlan plan_staged(int dtype, const Geom& g, const QuantIO& io, int device, const StagedTuning& tune);
 StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_count, int smem_optin,
                           const StagedTuning& tune);
 cudaError_t launch_staged(const StagedPlan& plan, const QuantIO& io, int mode, int dtype, const Geom& g, int bits,
+                          const Workspace& ws, float* lo, float* hi, float* s_opt, float* z_opt,
+                          const StagedTuning& tune, cudaStream_t st);
+
+// ---- L2-resident-wave persistent kernel ---------------------------------------------------
+struct L2Plan {
+    bool ok;
+    int upl;                 // 16-byte units per lane and step
+    uint32_t smem_bytes;     // dynamic shared memory per CTA
+    uint32_t cw;             // channels per wave
+    uint32_t nwaves;
+};
+L2Plan plan_l2wave(int dtype, const Geom& g, const QuantIO& io, const StagedTuning& tune);
+cudaError_t launch_l2wave(const L2Plan& plan, const QuantIO& io, int mode, int dtype, const Geom& g, int bits,
                           const Workspace& ws, float* lo, float* hi, float* s_opt, float* z_opt,
                           const StagedTuning& tune, cudaStream_t st);
 

@@ -154,6 +154,6 @@ def test_staged_plan_under_forced_small_buffers(lib):
                 planned += 1
                 _check_geometry(shape, dt, 0, geo)
     finally:
-        for k in range(6):
+        for k in range(9):
             b.tune(k, 0)
     assert planned > 500

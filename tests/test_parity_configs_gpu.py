@@ -16,7 +16,7 @@ pytestmark = pytest.mark.gpu
 def b():
     from paper_2503_18339_b200 import binding
     binding.lib()
-    for k in range(6):
+    for k in range(9):
         binding.tune(k, 0)
     return binding
 

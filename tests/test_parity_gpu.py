@@ -23,7 +23,7 @@ def b():
     from paper_2503_18339_b200 import binding
     binding.lib()
     yield binding
-    for k in range(6):
+    for k in range(9):
         binding.tune(k, 0)
 
 
@@ -33,11 +33,12 @@ def knobs(b):
     def set_(**kw):
         names = {"depth": b.KNOB_STAGED_DEPTH, "max_buf_units": b.KNOB_STAGED_MAX_BUF_UNITS,
                  "grid": b.KNOB_STAGED_GRID, "spin_limit": b.KNOB_SPIN_LIMIT,
-                 "extra_arrivals": b.KNOB_TEST_EXTRA_ARRIVALS}
+                 "extra_arrivals": b.KNOB_TEST_EXTRA_ARRIVALS, "l2_wave_kb": b.KNOB_L2_WAVE_KB,
+                 "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM}
         for k, v in kw.items():
             b.tune(names[k], v)
     yield set_
-    for k in range(6):
+    for k in range(9):
         b.tune(k, 0)
 
 
@@ -136,11 +137,15 @@ def test_fused_small_all_plans(b, shape, mode, dtype):
     bits = 2 + (sum(shape) + mode) % 7
     x, gy = make_case(shape, seed=sum(shape) * 7 + mode, dtype=dtype, relu=(shape[0] % 2 == 0))
     ref = orc.fused(x, bits, gy=gy, group_mode=mode)
-    for flags in (0, b.FLAG_FORCE_TWO_PASS, b.FLAG_FORCE_NAIVE):
+    for flags in (0, b.FLAG_FORCE_TWO_PASS, b.FLAG_FORCE_NAIVE, b.FLAG_FORCE_L2WAVE):
         if flags == b.FLAG_FORCE_NAIVE and b.num_groups(shape, 1, mode) > 300:
             continue
-        got = b.granq_fakequant_fused(to_dev(x), bits, gy=to_dev(gy), group=mode, want_codes=True,
-                                      want_mask=True, want_params=True, flags=flags)
+        try:
+            got = b.granq_fakequant_fused(to_dev(x), bits, gy=to_dev(gy), group=mode, want_codes=True,
+                                          want_mask=True, want_params=True, flags=flags)
+        except b.GranqError as err:      # the L2-wave plan does not take every geometry
+            assert flags == b.FLAG_FORCE_L2WAVE and err.status == b.ERR_UNSUPPORTED
+            continue
         assert b.workspace_status(got.workspace) == b.OK
         assert_parity(got, ref, shape, 1, mode, backward=True)
     # forward only
@@ -189,6 +194,41 @@ def test_staged_multiwave(b, knobs, shape, depth, dtype):
                                       want_params=True, flags=b.FLAG_FORCE_STAGED)
         assert b.workspace_status(got.workspace) == b.OK
         assert_parity(got, ref, shape, 1, orc.GROUP_CHANNEL, backward=True)
+
+
+@pytest.mark.parametrize("shape", [(4, 16, 14, 14), (3, 8, 7, 7), (6, 12, 32, 32), (2, 40, 56, 56), (5, 24, 7, 7)],
+                         ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("upl", [2, 4])
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_l2wave_multiwave(b, knobs, shape, upl, dtype):
+    """The L2-resident-wave plan cut into many small waves (a few channels each)."""
+    if dtype == "bf16" and (shape[1] * shape[2] * shape[3]) % 8 != 0:
+        pytest.skip("slab not a whole number of 16-byte packs")
+    x, gy = make_case(shape, seed=sum(shape) + upl, dtype=dtype)
+    bits = 2 + upl
+    ref = orc.fused(x, bits, gy=gy)
+    ref_f = orc.fused(x, bits)
+    for wave_kb, cap in ((1, 1), (8, 0), (0, 0)):
+        knobs(l2_wave_kb=wave_kb, l2_upl=upl, l2_ctas_per_sm=cap)
+        got = b.granq_fakequant_fused(to_dev(x), bits, gy=to_dev(gy), want_codes=True, want_mask=True,
+                                      want_params=True, flags=b.FLAG_FORCE_L2WAVE)
+        assert b.workspace_status(got.workspace) == b.OK
+        assert_parity(got, ref, shape, 1, orc.GROUP_CHANNEL, backward=True)
+        got = b.granq_fakequant_fused(to_dev(x), bits, flags=b.FLAG_FORCE_L2WAVE)      # forward only, no extras
+        assert_parity(got, ref_f, shape, 1, orc.GROUP_CHANNEL, backward=False)
+
+
+def test_l2wave_bounded_wait_reports_timeout(b, knobs):
+    shape = (4, 16, 14, 14)
+    x, gy = make_case(shape, seed=2)
+    knobs(extra_arrivals=1, spin_limit=2000)
+    got = b.granq_fakequant_fused(to_dev(x), 4, gy=to_dev(gy), flags=b.FLAG_FORCE_L2WAVE)
+    assert b.workspace_status(got.workspace) == b.ERR_TIMEOUT
+    knobs(extra_arrivals=0, spin_limit=0)
+    got = b.granq_fakequant_fused(to_dev(x), 4, gy=to_dev(gy), want_codes=True, want_mask=True, want_params=True,
+                                  flags=b.FLAG_FORCE_L2WAVE)
+    assert b.workspace_status(got.workspace) == b.OK
+    assert_parity(got, orc.fused(x, 4, gy=gy), shape, 1, orc.GROUP_CHANNEL, backward=True)
 
 
 def test_staged_geometry_really_has_many_waves(b, knobs):
