@@ -197,6 +197,8 @@ __global__ void __launch_bounds__(kLThreads) l2wave_kernel(const LArgs a) {
                 if (a.z_out) a.z_out[c0 + t] = gp.z;
             }
         }
+        GroupParam mine{1.0f, 0.0f, 0.0f};
+        uint32_t have_first = kNoGroup, have_nch = 0;
         for (uint32_t tile = blockIdx.x; tile < sh.ntiles; tile += gridDim.x) {
             uint32_t slab, ti;
             sh.div_tps.divmod(tile, slab, ti);
@@ -213,48 +215,63 @@ __global__ void __launch_bounds__(kLThreads) l2wave_kernel(const LArgs a) {
                 }
             }
             // parameters of the channels this row touches: lane l holds channel ch_first + l
+            // (kept from the previous row when the channel range has not changed)
             const uint32_t last_u = min(r0 + kRow, sh.units) - 1;
             const uint32_t ch_first = ALIGNED ? a.div_plane.div(r0) : a.div_plane.div(r0 * V);
             const uint32_t ch_last = ALIGNED ? a.div_plane.div(last_u) : a.div_plane.div(last_u * V + (V - 1));
             const uint32_t nch = ch_last - ch_first + 1;
             const bool shared_params = nch <= 32;
-            GroupParam mine{1.0f, 0.0f, 0.0f};
-            if (shared_params && lane < nch) {
-                float lo, hi;
-                mine = group_param_from_keys(a.kmin, a.kmax, c0 + ch_first + lane, qmax, lo, hi);
+            if (shared_params && (ch_first != have_first || nch != have_nch)) {
+                have_first = ch_first;
+                have_nch = nch;
+                if (lane < nch) {
+                    float lo, hi;
+                    mine = group_param_from_keys(a.kmin, a.kmax, c0 + ch_first + lane, qmax, lo, hi);
+                }
+            }
+            GroupParam row_g{1.0f, 0.0f, 0.0f};
+            if (nch == 1) {                      // the whole row lies in one channel
+                row_g.s = __shfl_sync(kFullMask, mine.s, 0);
+                row_g.z = __shfl_sync(kFullMask, mine.z, 0);
+                row_g.r = __shfl_sync(kFullMask, mine.r, 0);
             }
 #pragma unroll
             for (int j = 0; j < UPL; ++j) {
                 const uint32_t uo = r0 + j * 32 + lane;
                 const bool valid = uo < sh.units;
-                uint32_t ci1 = 0, ci2 = 0;
                 int n1 = V;
-                if constexpr (ALIGNED) {
-                    ci1 = a.div_plane.div(valid ? uo : r0);
-                    ci2 = ci1;
-                } else {
-                    uint32_t rem;
-                    a.div_plane.divmod((valid ? uo : r0) * V, ci1, rem);
-                    n1 = (int)min((uint32_t)V, a.inner - rem);
-                    ci2 = min(ci1 + 1, sh.channels - 1);
-                }
                 GroupParam g1, g2;
-                if (shared_params) {
-                    const uint32_t i1 = ci1 - ch_first, i2 = min(ci2 - ch_first, nch - 1);
-                    g1.s = __shfl_sync(kFullMask, mine.s, i1);
-                    g1.z = __shfl_sync(kFullMask, mine.z, i1);
-                    g1.r = __shfl_sync(kFullMask, mine.r, i1);
-                    if constexpr (ALIGNED) {
-                        g2 = g1;
-                    } else {
-                        g2.s = __shfl_sync(kFullMask, mine.s, i2);
-                        g2.z = __shfl_sync(kFullMask, mine.z, i2);
-                        g2.r = __shfl_sync(kFullMask, mine.r, i2);
-                    }
+                if (nch == 1) {
+                    g1 = row_g;
+                    g2 = row_g;
                 } else {
-                    float lo, hi;
-                    g1 = group_param_from_keys(a.kmin, a.kmax, c0 + ci1, qmax, lo, hi);
-                    g2 = ALIGNED ? g1 : group_param_from_keys(a.kmin, a.kmax, c0 + ci2, qmax, lo, hi);
+                    uint32_t ci1 = 0, ci2 = 0;
+                    if constexpr (ALIGNED) {
+                        ci1 = a.div_plane.div(valid ? uo : r0);
+                        ci2 = ci1;
+                    } else {
+                        uint32_t rem;
+                        a.div_plane.divmod((valid ? uo : r0) * V, ci1, rem);
+                        n1 = (int)min((uint32_t)V, a.inner - rem);
+                        ci2 = min(ci1 + 1, sh.channels - 1);
+                    }
+                    if (shared_params) {
+                        const uint32_t i1 = ci1 - ch_first, i2 = min(ci2 - ch_first, nch - 1);
+                        g1.s = __shfl_sync(kFullMask, mine.s, i1);
+                        g1.z = __shfl_sync(kFullMask, mine.z, i1);
+                        g1.r = __shfl_sync(kFullMask, mine.r, i1);
+                        if constexpr (ALIGNED) {
+                            g2 = g1;
+                        } else {
+                            g2.s = __shfl_sync(kFullMask, mine.s, i2);
+                            g2.z = __shfl_sync(kFullMask, mine.z, i2);
+                            g2.r = __shfl_sync(kFullMask, mine.r, i2);
+                        }
+                    } else {
+                        float lo, hi;
+                        g1 = group_param_from_keys(a.kmin, a.kmax, c0 + ci1, qmax, lo, hi);
+                        g2 = ALIGNED ? g1 : group_param_from_keys(a.kmin, a.kmax, c0 + ci2, qmax, lo, hi);
+                    }
                 }
                 if (!valid) continue;
                 Pack<T> py, pgx;
