@@ -69,7 +69,7 @@ def kernel_source_hash() -> str:
 def recorded_traffic():
     """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None
     when there is none or the kernel sources have changed since it was taken."""
-    path = os.path.join(ROOT, "profiles", "staged_kernel_traffic.json")
+    path = os.path.join(ROOT, "profiles", "l2wave_kernel_traffic.json")
     try:
         with open(path) as fh:
             rec = json.load(fh)
@@ -296,14 +296,14 @@ def main():
     per_call_ms = [statistics.mean(ev[k][ci][0].elapsed_time(ev[k][ci][1]) for k in range(args.steps))
                    for ci in range(len(calls))]
     dominant = [ci for ci, (i, _) in enumerate(calls) if (specs[i].shape[2] * specs[i].shape[3]) % 4 == 0
-                and plans[ci][0] == b.PLAN_STAGED]
+                and plans[ci][0] == b.PLAN_L2WAVE]
     dom_bytes = sum(specs[calls[ci][0]].numel for ci in dominant) * BYTES_PER_ELEM
     dom_ms = sum(per_call_ms[ci] for ci in dominant)
     peak, peak_src = measured_peak()
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9 if dominant else None
     rec = recorded_traffic()
     roofline = {
-        "bound": "hbm", "kernel": "staged_kernel<float, fwd+bwd, aligned planes>",
+        "bound": "hbm", "kernel": "l2wave_kernel<float, fwd+bwd, aligned planes>",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
         "peak_source": peak_src, "frac_of_nominal_8TBs": (achieved / NOMINAL_HBM_GBS) if achieved else None,
         "launches_per_step": len(dominant),

@@ -45,7 +45,7 @@
  * (null required pointer, bits outside 1..8, non-positive dim, more than 2^40 elements,
  * bad enum, workspace too small or misaligned) are detected on the host before anything
  * is launched and leave all outputs untouched.  CUDA launch errors are returned as
- * GRANQ_ERR_CUDA.  The on-chip-staged plan of granq_fakequant_fused() contains bounded
+ * GRANQ_ERR_CUDA.  The persistent plans of granq_fakequant_fused() contain bounded
  * device-side waits; should one run out (it cannot unless the GPU is preempted for
  * seconds) the kernel stops, outputs are unspecified, and granq_workspace_status()
  * reports GRANQ_ERR_TIMEOUT.
@@ -129,7 +129,8 @@ int granq_fakequant_bwd(const void* gy, const void* x, int dtype, const int64_t 
 /*
  * The whole path in one call (Algorithm 1, range step through pre-scale step, plus the
  * backward): range of x itself -> scale / zero-point -> y, and gx when gy_opt is given.
- * Where a channel group fits in the GPU's shared memory the tensor is read from HBM once.
+ * The default plan processes the tensor in waves of channel groups that stay in the L2 cache
+ * between the range pass and the quantize pass, so x is read from HBM (about) once.
  *   x                 in   E elements          gy_opt   in   E elements or NULL (forward only)
  *   y                 out  E elements          gx_opt   out  E elements (required iff gy_opt)
  *   min_out, max_out  out  G floats each (required)
@@ -142,7 +143,7 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
                           void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream);
 
 /*
- * Status word the staged plan leaves in the workspace.  Synchronises `cuda_stream`, then
+ * Status word the persistent plans leave in the workspace.  Synchronises `cuda_stream`, then
  * returns GRANQ_OK, GRANQ_ERR_TIMEOUT (a bounded device-side wait ran out), or
  * GRANQ_ERR_CUDA.  `workspace` is the pointer given to the preceding call.
  */

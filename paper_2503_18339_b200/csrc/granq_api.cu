@@ -68,14 +68,21 @@ int choose_plan(int dtype, const Geom& g, const QuantIO& io, uint32_t flags, Sta
         if (l2_out) *l2_out = lp;
         return PLAN_L2WAVE;
     }
-    int dev = 0;
-    if (cudaGetDevice(&dev) != cudaSuccess) return -GRANQ_ERR_CUDA;
-    StagedPlan p = plan_staged(dtype, g, io, dev, g_tune);
-    if (p.ok) {
+    if (flags & GRANQ_FLAG_FORCE_STAGED) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) return -GRANQ_ERR_CUDA;
+        StagedPlan p = plan_staged(dtype, g, io, dev, g_tune);
+        if (!p.ok) return -GRANQ_ERR_UNSUPPORTED;
         if (plan_out) *plan_out = p;
         return PLAN_STAGED;
     }
-    if (flags & GRANQ_FLAG_FORCE_STAGED) return -GRANQ_ERR_UNSUPPORTED;
+    // default: the L2-resident-wave kernel wherever the geometry qualifies (it has measured
+    // faster than the shared-memory-staged kernel on every workload tensor)
+    L2Plan lp = plan_l2wave(dtype, g, io, g_tune);
+    if (lp.ok) {
+        if (l2_out) *l2_out = lp;
+        return PLAN_L2WAVE;
+    }
     return PLAN_TWO_PASS;
 }
 

@@ -1,8 +1,8 @@
 // L2-resident-wave GranQ kernel: one persistent cooperative launch with many resident warps
 // and no shared-memory staging.
 //
-// The tensor is processed in waves of whole channel groups, sized so that the x bytes of
-// two waves fit in the L2 cache.  A wave is cut into tiles (contiguous runs inside one
+// The tensor is processed in waves of whole channel groups, sized (64 MB of x by default)
+// so that a wave's x stays in the L2 cache between its two phases.  A wave is cut into tiles (contiguous runs inside one
 // slab) dealt round-robin to the CTAs; the same CTA handles a tile in both phases.
 //   phase 1 (Eq. 4): read the tile's x with an evict-last L2 policy, reduce to per-group
 //                    min/max keys (warp runs -> shared memory -> one global atomic per group
@@ -372,7 +372,7 @@ L2Plan plan_l2wave(int dtype, const Geom& g, const QuantIO& io, const StagedTuni
     if ((g.C * g.inner) % V != 0 || g.E / V >= (1ll << 31)) return p;
     const uint32_t inner = (uint32_t)g.inner, C = (uint32_t)g.C;
     const uint32_t q = V / l_gcd(inner, V);
-    const uint64_t target = (tune.l2_wave_kb > 0 ? (uint64_t)tune.l2_wave_kb : 24ull * 1024) * 1024;
+    const uint64_t target = (tune.l2_wave_kb > 0 ? (uint64_t)tune.l2_wave_kb : 64ull * 1024) * 1024;
     const uint64_t group_bytes = (uint64_t)g.outer * inner * (16 / V);           // x bytes of one channel group
     const uint32_t mult_total = C / q;
     uint64_t max_mult = target / (group_bytes * q);
@@ -382,7 +382,8 @@ L2Plan plan_l2wave(int dtype, const Geom& g, const QuantIO& io, const StagedTuni
     p.cw = ((mult_total + nw - 1) / nw) * q;
     p.nwaves = (C + p.cw - 1) / p.cw;
     if ((uint64_t)p.cw * inner / V >= (1ull << 30)) return p;
-    p.upl = (tune.l2_upl == 4) ? 4 : 2;
+    // long planes: rows of 128 units lie in one channel and amortise the row set-up; short planes: 64
+    p.upl = tune.l2_upl == 4 ? 4 : (tune.l2_upl == 2 ? 2 : ((inner / V) >= 512 ? 4 : 2));
     p.smem_bytes = 8u * (((p.cw + 15u) / 16u) * 16u);
     p.ok = true;
     return p;
