@@ -69,7 +69,7 @@ def kernel_source_hash() -> str:
 def recorded_traffic():
     """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None
     when there is none or the kernel sources have changed since it was taken."""
-    path = os.path.join(ROOT, "profiles", "l2wave_kernel_traffic.json")
+    path = os.path.join(ROOT, "profiles", "l2wave_kernel_traffic.txt")
     try:
         with open(path) as fh:
             rec = json.load(fh)
