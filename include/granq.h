@@ -104,6 +104,28 @@ int granq_range(const void* x, int dtype, const int64_t dims[4], int channel_axi
                 void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream);
 
 /*
+ * granq_range() without a workspace (the paper has no counterpart: this exists for callers,
+ * not for the method).  Some callers cannot allocate device memory where they need the range:
+ * code running inside a framework's allocator callback or out-of-memory handler, a plugin that
+ * is handed nothing but its input and output buffers, a latency-critical loop that must stay
+ * out of the driver's allocator.  For them the min/max scratch is an array inside the library
+ * itself, so the call allocates and frees nothing (no cudaMalloc / cudaFree, no allocating
+ * library routine).
+ *   - Limit: at most GRANQ_NOALLOC_MAX_GROUPS groups; more gives GRANQ_ERR_UNSUPPORTED and
+ *     nothing is launched.  The array (256 KB) is resident on every GPU that loads the library,
+ *     until the process exits.
+ *   - The first call on a device looks up the array's device address (with that device
+ *     current); make that first call before starting any stream capture.
+ *   - Every call uses the same array: calls that overlap on the GPU (two streams, two host
+ *     threads) race with each other.  Calls issued on one stream are safe; the array is
+ *     cleared at the start of each call.
+ * Arguments and results are those of granq_range() (x, min_out, max_out in DEVICE memory).
+ */
+#define GRANQ_NOALLOC_MAX_GROUPS 32768
+int granq_range_noalloc(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                        float* min_out, float* max_out, void* cuda_stream);
+
+/*
  * Eq. 1 + clamp + Eq. 6 with a range supplied by the caller (for instance one measured on
  * another batch): y = s * (clamp(round(x / s + z)) - z), with s, z from Eq. 2 / Eq. 5.
  *   min_in, max_in  in   G floats each

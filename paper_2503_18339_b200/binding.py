@@ -29,8 +29,9 @@ EXPORTS = [
     "granq_status_string", "granq_num_groups", "granq_workspace_bytes", "granq_range",
     "granq_fakequant_fwd", "granq_fakequant_bwd", "granq_fakequant_fused", "granq_workspace_status",
     "granq_host_arena_bytes", "granq_fakequant_fused_host", "granq_fused_plan", "granq_staged_geometry",
-    "granq_tune", "granq_selftest_division",
+    "granq_tune", "granq_selftest_division", "granq_range_noalloc",
 ]
+NOALLOC_MAX_GROUPS = 32768
 
 
 class GranqError(RuntimeError):
@@ -81,6 +82,8 @@ def lib() -> ctypes.CDLL:
         L.granq_staged_geometry.argtypes = [ci, i64p, ci, ci, ci, ci, i64p]
         L.granq_selftest_division.restype = ci
         L.granq_selftest_division.argtypes = [ctypes.c_uint64, ctypes.c_uint64, vp, vp]
+        L.granq_range_noalloc.restype = ci
+        L.granq_range_noalloc.argtypes = [vp, ci, i64p, ci, ci, vp, vp, vp]
         L.granq_tune.restype = ci
         L.granq_tune.argtypes = [ci, ci]
         _lib = L
@@ -200,6 +203,14 @@ def granq_range(x: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANN
                              _dev(hi, "hi"), _dev(ws, "workspace"), ws.numel(), flags, _stream(stream)),
            "granq_range")
     return lo, hi
+
+
+def granq_range_noalloc(x: torch.Tensor, lo: torch.Tensor, hi: torch.Tensor, channel_axis: int = 1,
+                        group: int = GROUP_CHANNEL, stream=None) -> None:
+    """Per-group (lo, hi) of x into caller-provided tensors, using the library's built-in scratch:
+    for callers that cannot allocate device memory at this point (nothing is allocated here either)."""
+    _check(lib().granq_range_noalloc(_dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, _dev(lo, "lo"),
+                                     _dev(hi, "hi"), _stream(stream)), "granq_range_noalloc")
 
 
 def granq_fakequant_fwd(x: torch.Tensor, bits: int, lo: torch.Tensor, hi: torch.Tensor, channel_axis: int = 1,
