@@ -7,8 +7,9 @@
 //   phase 1 (Eq. 4): read the tile's x with an evict-last L2 policy, reduce to per-group
 //                    min/max keys (warp runs -> shared memory -> one global atomic per group
 //                    and CTA), then bump the wave's arrival counter;
-//   phase 2 (Eq. 5, 1, 6, STE): once the counter shows every CTA has arrived, read x again
-//                    (an L2 hit), stream gy in and y / gx out with evict-first policies.
+//   phase 2 (Eq. 5, 1, 6, STE): once the counter shows every CTA has arrived, turn the wave's keys
+//                    into a shared-memory table of (s, z, 1/s), read x again (an L2 hit),
+//                    stream gy in and y / gx out with evict-first policies.
 // Each CTA runs  P1(0);  then for every wave w:  P1(w+1), wait(w), P2(w)  - so a wave's
 // counter has had a whole phase to fill up before anybody waits on it.
 //
@@ -70,14 +71,16 @@ __device__ __forceinline__ uint32_t l_ld_acquire(const uint32_t* p) {
 
 // UPL = 16-byte units per lane and step; a warp handles rows of 32 * UPL consecutive units
 template <typename T, int MODE, bool ALIGNED, bool EXTRAS, int UPL>
-__global__ void __launch_bounds__(kLThreads) l2wave_kernel(const LArgs a) {
+__global__ void __launch_bounds__(kLThreads, UPL == 2 ? 4 : 3) l2wave_kernel(const LArgs a) {
     constexpr int V = Pack<T>::V;
     constexpr bool kBwd = (MODE & MODE_BWD) != 0;
     constexpr uint32_t kRow = 32 * UPL, kTile = kLWarps * kRow;
-    extern __shared__ uint32_t s_keys[];                       // [2][tab]: min keys, max keys
+    extern __shared__ uint32_t s_keys[];                       // [2][tab] min / max keys, then the wave's parameters
     const uint32_t tab = ((a.cw + 15u) / 16u) * 16u;
     uint32_t* s_kmn = s_keys;
     uint32_t* s_kmx = s_keys + tab;
+    float2* s_sz = reinterpret_cast<float2*>(s_keys + 2 * tab);   // [tab] (scale, zero-point)
+    float* s_rcp = reinterpret_cast<float*>(s_sz + tab);          // [tab] RN(1 / scale), or 0 = use IEEE division
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint4* xg = reinterpret_cast<const uint4*>(a.x);
     const uint4* gyg = reinterpret_cast<const uint4*>(a.gy);
@@ -187,18 +190,21 @@ __global__ void __launch_bounds__(kLThreads) l2wave_kernel(const LArgs a) {
         const LShape& sh = a.shape[(w + 1 == W) ? 1 : 0];
         const uint32_t c0 = w * a.cw, base = w * a.wave_units;
         const float qmax = a.qmax;
-        if (warp == 0 && (w % gridDim.x) == blockIdx.x) {       // one warp in the grid reports the wave's groups
-            for (uint32_t t = lane; t < sh.channels; t += 32) {
-                float lo, hi;
-                const GroupParam gp = group_param_from_keys(a.kmin, a.kmax, c0 + t, qmax, lo, hi);
+        // the wave's parameters (Eq. 5), once per CTA; one CTA in the grid also reports them
+        const bool writer = (w % gridDim.x) == blockIdx.x;
+        for (uint32_t t = tid; t < sh.channels; t += kLThreads) {
+            float lo, hi;
+            const GroupParam gp = group_param_from_keys(a.kmin, a.kmax, c0 + t, qmax, lo, hi);
+            s_sz[t] = make_float2(gp.s, gp.z);
+            s_rcp[t] = gp.r;
+            if (writer) {
                 a.lo[c0 + t] = lo;
                 a.hi[c0 + t] = hi;
                 if (a.s_out) a.s_out[c0 + t] = gp.s;
                 if (a.z_out) a.z_out[c0 + t] = gp.z;
             }
         }
-        GroupParam mine{1.0f, 0.0f, 0.0f};
-        uint32_t have_first = kNoGroup, have_nch = 0;
+        __syncthreads();
         for (uint32_t tile = blockIdx.x; tile < sh.ntiles; tile += gridDim.x) {
             uint32_t slab, ti;
             sh.div_tps.divmod(tile, slab, ti);
@@ -214,63 +220,46 @@ __global__ void __launch_bounds__(kLThreads) l2wave_kernel(const LArgs a) {
                     if constexpr (kBwd) pg[j].raw = ld_hint_16(gyg + gbase + uo, drop);
                 }
             }
-            // parameters of the channels this row touches: lane l holds channel ch_first + l
-            // (kept from the previous row when the channel range has not changed)
+            // a row that lies in one channel looks its parameters up once
             const uint32_t last_u = min(r0 + kRow, sh.units) - 1;
             const uint32_t ch_first = ALIGNED ? a.div_plane.div(r0) : a.div_plane.div(r0 * V);
             const uint32_t ch_last = ALIGNED ? a.div_plane.div(last_u) : a.div_plane.div(last_u * V + (V - 1));
-            const uint32_t nch = ch_last - ch_first + 1;
-            const bool shared_params = nch <= 32;
-            if (shared_params && (ch_first != have_first || nch != have_nch)) {
-                have_first = ch_first;
-                have_nch = nch;
-                if (lane < nch) {
-                    float lo, hi;
-                    mine = group_param_from_keys(a.kmin, a.kmax, c0 + ch_first + lane, qmax, lo, hi);
-                }
-            }
-            GroupParam row_g{1.0f, 0.0f, 0.0f};
-            if (nch == 1) {                      // the whole row lies in one channel
-                row_g.s = __shfl_sync(kFullMask, mine.s, 0);
-                row_g.z = __shfl_sync(kFullMask, mine.z, 0);
-                row_g.r = __shfl_sync(kFullMask, mine.r, 0);
+            const bool one_channel = ch_first == ch_last;
+            GroupParam row_g;
+            {
+                const float2 sz = s_sz[ch_first];
+                row_g.s = sz.x;
+                row_g.z = sz.y;
+                row_g.r = s_rcp[ch_first];
             }
 #pragma unroll
             for (int j = 0; j < UPL; ++j) {
                 const uint32_t uo = r0 + j * 32 + lane;
                 const bool valid = uo < sh.units;
                 int n1 = V;
-                GroupParam g1, g2;
-                if (nch == 1) {
-                    g1 = row_g;
-                    g2 = row_g;
-                } else {
-                    uint32_t ci1 = 0, ci2 = 0;
+                GroupParam g1 = row_g, g2 = row_g;
+                if (!one_channel && valid) {
+                    uint32_t ci1, ci2;
                     if constexpr (ALIGNED) {
-                        ci1 = a.div_plane.div(valid ? uo : r0);
+                        ci1 = a.div_plane.div(uo);
                         ci2 = ci1;
                     } else {
                         uint32_t rem;
-                        a.div_plane.divmod((valid ? uo : r0) * V, ci1, rem);
+                        a.div_plane.divmod(uo * V, ci1, rem);
                         n1 = (int)min((uint32_t)V, a.inner - rem);
                         ci2 = min(ci1 + 1, sh.channels - 1);
                     }
-                    if (shared_params) {
-                        const uint32_t i1 = ci1 - ch_first, i2 = min(ci2 - ch_first, nch - 1);
-                        g1.s = __shfl_sync(kFullMask, mine.s, i1);
-                        g1.z = __shfl_sync(kFullMask, mine.z, i1);
-                        g1.r = __shfl_sync(kFullMask, mine.r, i1);
-                        if constexpr (ALIGNED) {
-                            g2 = g1;
-                        } else {
-                            g2.s = __shfl_sync(kFullMask, mine.s, i2);
-                            g2.z = __shfl_sync(kFullMask, mine.z, i2);
-                            g2.r = __shfl_sync(kFullMask, mine.r, i2);
-                        }
+                    const float2 sz1 = s_sz[ci1];
+                    g1.s = sz1.x;
+                    g1.z = sz1.y;
+                    g1.r = s_rcp[ci1];
+                    if constexpr (ALIGNED) {
+                        g2 = g1;
                     } else {
-                        float lo, hi;
-                        g1 = group_param_from_keys(a.kmin, a.kmax, c0 + ci1, qmax, lo, hi);
-                        g2 = ALIGNED ? g1 : group_param_from_keys(a.kmin, a.kmax, c0 + ci2, qmax, lo, hi);
+                        const float2 sz2 = s_sz[ci2];
+                        g2.s = sz2.x;
+                        g2.z = sz2.y;
+                        g2.r = s_rcp[ci2];
                     }
                 }
                 if (!valid) continue;
@@ -384,7 +373,7 @@ L2Plan plan_l2wave(int dtype, const Geom& g, const QuantIO& io, const StagedTuni
     if ((uint64_t)p.cw * inner / V >= (1ull << 30)) return p;
     // long planes: rows of 128 units lie in one channel and amortise the row set-up; short planes: 64
     p.upl = tune.l2_upl == 4 ? 4 : (tune.l2_upl == 2 ? 2 : ((inner / V) >= 512 ? 4 : 2));
-    p.smem_bytes = 8u * (((p.cw + 15u) / 16u) * 16u);
+    p.smem_bytes = 20u * (((p.cw + 15u) / 16u) * 16u);     // keys (8 B) and parameters (12 B) per group
     p.ok = true;
     return p;
 }
