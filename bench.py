@@ -365,9 +365,13 @@ def main():
         arrays = {sp.name: (xs.numpy(), gs.numpy()) for sp, (xs, gs) in zip(specs, host)}
         sample = [(specs[i], bits) for i, bits in calls if specs[i].numel <= 60_000_000]
         s, e = time_oracle(sample, arrays)
+        repeats = max(1, min(8, int(10.0 / max(s, 1e-3))))        # about 10 s of CPU work in all
+        for _ in range(repeats - 1):
+            s2, e2 = time_oracle(sample, arrays)
+            s, e = s + s2, e + e2
         cpu = {"value": e * BYTES_PER_ELEM / s / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
-               "sample": "every workload tensor of at most 60 M elements, b=4 and b=5 (%d calls, %d M elements)"
-                         % (len(sample), e // 1_000_000), "seconds": round(s, 2), "elements_per_s": e / s,
+               "sample": "every workload tensor of at most 60 M elements, b=4 and b=5 (%d calls), %d times over: %d M elements"
+                         % (len(sample), repeats, e // 1_000_000), "seconds": round(s, 2), "elements_per_s": e / s,
                "host_cores_available": os.cpu_count()}
 
     if rank == 0:
