@@ -127,6 +127,22 @@ class ClockSampler:
                 "samples": len(rows), "power_w_max": max(float(r[2]) for r in rows)}
 
 
+def max_over_ranks(ms: float, device: str = "cuda") -> float:
+    """The slowest rank's device time (every rank gets it); the identity when not distributed."""
+    import torch
+    import torch.distributed as dist
+    if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size() == 1:
+        return float(ms)
+    t = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_gbs(bytes_per_step_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Aggregate algorithmic GB/s of `world` replicas that each process one step in ms_per_step."""
+    return world * bytes_per_step_per_rank / (ms_per_step * 1e-3) / 1e9
+
+
 def time_oracle(specs_bits, arrays=None):
     """Seconds the CPU oracle needs for fused fwd+bwd on the given (spec, bits) list; elements processed.
     `arrays` maps spec.name -> (x, gy) numpy arrays already generated."""
@@ -286,12 +302,9 @@ def main():
         torch.cuda.synchronize()
         t1 = time.time()
     clocks = sampler.stop(t0, t1)
-    if world > 1:
-        t = torch.tensor([total_ms], device="cuda", dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        total_ms = float(t.item())
+    total_ms = max_over_ranks(total_ms)
     ms_per_step = total_ms / args.steps
-    value = world * bytes_per_step / (ms_per_step * 1e-3) / 1e9
+    value = whole_job_gbs(bytes_per_step, world, ms_per_step)
 
     # ---- per-call device times inside the timed region -> roofline of the dominant kernel ----
     per_call_ms = [statistics.mean(ev[k][ci][0].elapsed_time(ev[k][ci][1]) for k in range(args.steps))
@@ -349,11 +362,8 @@ def main():
         a1.record(stream)
         barrier()
         e_ms = a0.elapsed_time(a1)
-        if world > 1:
-            t = torch.tensor([e_ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e_ms = float(t.item())
-        e2e = {"value": world * bytes_per_step / (e_ms / args.e2e_steps * 1e-3) / 1e9, "unit": UNIT,
+        e_ms = max_over_ranks(e_ms)
+        e2e = {"value": whole_job_gbs(bytes_per_step, world, e_ms / args.e2e_steps), "unit": UNIT,
                "h2d_bytes_per_step": elems_per_step * 8, "d2h_bytes_per_step": elems_per_step * 8 +
                sum(specs[i].shape[1] * 8 for i, _ in calls),
                "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
