@@ -204,6 +204,8 @@ def main():
     ap.add_argument("--tune", default="", help="planner overrides for experiments, e.g. depth=3,max_buf_units=4000")
     ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged", "l2wave"],
                     help="force an execution plan of the fused entry point (experiments)")
+    ap.add_argument("--op", default="fused", choices=["fused", "range", "fwd", "bwd"],
+                    help="time another entry point instead of the fused one (experiments; bytes/element 4, 8, 12)")
     ap.add_argument("--only", default="", help="profiling aid: keep only workload tensors whose name contains this")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -258,12 +260,23 @@ def main():
     launches_per_step = sum(n for _, n in plans)
     stream = torch.cuda.current_stream()
 
+    global BYTES_PER_ELEM
+    BYTES_PER_ELEM = {"fused": 16, "range": 4, "fwd": 8, "bwd": 12}[args.op]
+    bytes_per_step = elems_per_step * BYTES_PER_ELEM
+
     def step(events=None):
         for ci, (i, bits) in enumerate(calls):
             x, gy, out = dev[i]
             if events is not None:
                 events[ci][0].record(stream)
-            b.granq_fakequant_fused(x, bits, gy=gy, out=out, flags=flags, stream=stream)
+            if args.op == "fused":
+                b.granq_fakequant_fused(x, bits, gy=gy, out=out, flags=flags, stream=stream)
+            elif args.op == "range":
+                b.granq_range(x, lo=out.lo, hi=out.hi, workspace=out.workspace, stream=stream)
+            elif args.op == "fwd":
+                b.granq_fakequant_fwd(x, bits, out.lo, out.hi, y=out.y, stream=stream)
+            else:
+                b.granq_fakequant_bwd(gy, x, bits, out.lo, out.hi, gx=out.gx, stream=stream)
             if events is not None:
                 events[ci][1].record(stream)
 

@@ -93,12 +93,10 @@ __global__ void __launch_bounds__(kThreads) range_flat_kernel(const T* __restric
                     } else {
                         Pack<T> p;
                         p.raw = *reinterpret_cast<const uint4*>(x + e0 + k[j]);
-#pragma unroll
-                        for (int i = 0; i < V; ++i) {
-                            uint32_t e = enc(p.get(i));
-                            mn[j] = max(mn[j], ~e);
-                            mx[j] = max(mx[j], e);
-                        }
+                        float lo = INFINITY, hi = -INFINITY;
+                        pack_minmax(p, 0, V, lo, hi);
+                        mn[j] = ~enc(lo);
+                        mx[j] = enc(hi);
                     }
                 }
             }
@@ -138,12 +136,9 @@ __global__ void params_kernel(const float* __restrict__ lo, const float* __restr
     if (z_opt) z_opt[i] = p.z;
 }
 
-__device__ __forceinline__ uint32_t pack4(const uint8_t* b) {
-    return (uint32_t)b[0] | ((uint32_t)b[1] << 8) | ((uint32_t)b[2] << 16) | ((uint32_t)b[3] << 24);
-}
-
 // ---- Eq. 1, clamp, Eq. 6, STE: elementwise pass with a given per-group range ----------------------
-template <typename T, int V, int MODE>
+// EXTRAS: the optional codes / mask outputs are compiled in
+template <typename T, int V, int MODE, bool EXTRAS>
 __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restrict__ x, const T* __restrict__ gy,
                                                               T* __restrict__ y, T* __restrict__ gx,
                                                               uint8_t* __restrict__ codes,
@@ -151,7 +146,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                                                               const float* __restrict__ lo,
                                                               const float* __restrict__ hi) {
     __shared__ TileBase s_base;
-    __shared__ QParam s_tab[kTableMax];
+    __shared__ float s_tab_s[kTableMax], s_tab_z[kTableMax], s_tab_r[kTableMax];
     constexpr bool kFwd = (MODE & MODE_FWD) != 0, kBwd = (MODE & MODE_BWD) != 0;
     for (int64_t tile = blockIdx.x; tile < g.ntiles; tile += gridDim.x) {
         const int64_t e0 = tile * (int64_t)kTile;
@@ -165,7 +160,10 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
         if (tabled) {
             for (uint32_t q = threadIdx.x; q < nplanes; q += kThreads) {
                 uint32_t grp = group_at(g, base, q);
-                s_tab[q] = make_qparam(__fadd_rn(lo[grp], 0.0f), __fadd_rn(hi[grp], 0.0f), qmax);
+                const QParam qp = make_qparam(__fadd_rn(lo[grp], 0.0f), __fadd_rn(hi[grp], 0.0f), qmax);
+                s_tab_s[q] = qp.s;
+                s_tab_z[q] = qp.z;
+                s_tab_r[q] = div_is_safe(qp.s, 0.0f, 0.0f) ? __frcp_rn(qp.s) : 0.0f;
             }
             __syncthreads();
         }
@@ -191,8 +189,11 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                 if (k[j] >= ne) continue;
                 const uint32_t q = plane_offset(g, base, k[j]);
                 QParam p;
+                float rcp = 0.0f;            // reciprocal of the scale when the short division applies
                 if (tabled) {
-                    p = s_tab[q];
+                    p.s = s_tab_s[q];
+                    p.z = s_tab_z[q];
+                    rcp = s_tab_r[q];
                 } else {
                     uint32_t grp = group_at(g, base, q);
                     p = make_qparam(__fadd_rn(lo[grp], 0.0f), __fadd_rn(hi[grp], 0.0f), qmax);
@@ -212,29 +213,29 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                     }
                 } else {
                     Pack<T> py, pgx;
-                    uint8_t cb[V], mb[V];
+                    uint32_t cb[V / 4 > 0 ? V / 4 : 1], mb[V / 4 > 0 ? V / 4 : 1];
+                    // x may lie outside the given range: the short division needs |x| <= 2^60
+                    float amax = 0.0f;
 #pragma unroll
-                    for (int i = 0; i < V; ++i) {
-                        float yv;
-                        bool in;
-                        float code = quant_one(px[j].get(i), p, qmax, yv, in);
-                        py.set(i, yv);
-                        cb[i] = (uint8_t)code;
-                        mb[i] = in ? 1 : 0;
-                        if constexpr (kBwd) pgx.set(i, in ? pg[j].get(i) : 0.0f);
-                    }
+                    for (int i = 0; i < V; ++i) amax = fmaxf(amax, fabsf(px[j].get(i)));
+                    GroupParam gp{p.s, p.z, (amax <= 1152921504606846976.0f) ? rcp : 0.0f};
+                    quantize_pack<T, kBwd, false, EXTRAS>(px[j], pg[j], gp, gp, V, qmax, py, pgx, cb, mb);
                     if constexpr (kFwd) {
                         st_stream_16(y + e, py.raw);
-                        if (codes) {
+                        if constexpr (EXTRAS) {
+                            if (codes) {
 #pragma unroll
-                            for (int i = 0; i < V; i += 4) *reinterpret_cast<uint32_t*>(codes + e + i) = pack4(cb + i);
+                                for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(codes + e)[i] = cb[i];
+                            }
                         }
                     }
                     if constexpr (kBwd) {
                         st_stream_16(gx + e, pgx.raw);
-                        if (mask) {
+                        if constexpr (EXTRAS) {
+                            if (mask) {
 #pragma unroll
-                            for (int i = 0; i < V; i += 4) *reinterpret_cast<uint32_t*>(mask + e + i) = pack4(mb + i);
+                                for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(mask + e)[i] = mb[i];
+                            }
                         }
                     }
                 }
@@ -326,12 +327,16 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
                ((uintptr_t)io.codes % 4 == 0) && ((uintptr_t)io.mask % 4 == 0);
     int grid = flat_grid(f);
     float qmax = (float)((1 << bits) - 1);
-    if (vec)
-        quant_flat_kernel<T, VF, MODE><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                  (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
+    const bool extras = io.codes != nullptr || io.mask != nullptr;
+    if (vec && extras)
+        quant_flat_kernel<T, VF, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
+                                                                        (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
+    else if (vec)
+        quant_flat_kernel<T, VF, MODE, false><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
+                                                                         (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
     else
-        quant_flat_kernel<T, 1, MODE><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                 (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
+        quant_flat_kernel<T, 1, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
+                                                                       (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
     return cudaGetLastError();
 }
 
