@@ -260,9 +260,11 @@ def main():
     launches_per_step = sum(n for _, n in plans)
     stream = torch.cuda.current_stream()
 
-    global BYTES_PER_ELEM
-    BYTES_PER_ELEM = {"fused": 16, "range": 4, "fwd": 8, "bwd": 12}[args.op]
-    bytes_per_step = elems_per_step * BYTES_PER_ELEM
+    bpe = {"fused": 16, "range": 4, "fwd": 8, "bwd": 12}[args.op]
+    bytes_per_step = elems_per_step * bpe
+    if args.op != "fused":          # the stand-alone entry points need a range: take each tensor's own
+        for x, gy, out in dev:
+            b.granq_fakequant_fused(x, 4, gy=gy, out=out, stream=stream)
 
     def step(events=None):
         for ci, (i, bits) in enumerate(calls):
@@ -325,7 +327,7 @@ def main():
     # dominant kernel: the L2-wave instantiation for long planes (>= 512 packs per plane, 4 packs per lane)
     dominant = [ci for ci, (i, _) in enumerate(calls) if (specs[i].shape[2] * specs[i].shape[3]) % 4 == 0
                 and specs[i].shape[2] * specs[i].shape[3] // 4 >= 512 and plans[ci][0] == b.PLAN_L2WAVE]
-    dom_bytes = sum(specs[calls[ci][0]].numel for ci in dominant) * BYTES_PER_ELEM
+    dom_bytes = sum(specs[calls[ci][0]].numel for ci in dominant) * bpe
     dom_ms = sum(per_call_ms[ci] for ci in dominant)
     peak, peak_src = measured_peak()
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9 if dominant else None
@@ -344,7 +346,7 @@ def main():
     }
     per_tensor = []
     for ci, (i, bits) in enumerate(calls):
-        gbs = specs[i].numel * BYTES_PER_ELEM / (per_call_ms[ci] * 1e-3) / 1e9
+        gbs = specs[i].numel * bpe / (per_call_ms[ci] * 1e-3) / 1e9
         per_tensor.append({"tensor": specs[i].name, "bits": bits, "us": round(per_call_ms[ci] * 1e3, 2),
                            "GBps": round(gbs, 1), "frac_measured": round(gbs / peak, 3),
                            "frac_8TBs": round(gbs / NOMINAL_HBM_GBS, 3), "plan": plans[ci][0]})
