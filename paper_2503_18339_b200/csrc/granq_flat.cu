@@ -111,6 +111,89 @@ __global__ void __launch_bounds__(kThreads) range_flat_kernel(const T* __restric
     run_flush(run, kmin, kmax);
 }
 
+// ---- Eq. 4: range, vector path -----------------------------------------------------------------
+// Planes made of whole 16-byte packs, fewer than 2^31 packs: a warp takes rows of 128 consecutive
+// packs (two rows in flight), a row that lies in one plane costs one run update, and the CTA
+// combines its warps' keys in shared memory before touching the global keys.
+constexpr uint32_t kRangeSmemGroups = 1024;
+
+template <typename T>
+__global__ void __launch_bounds__(kThreads) range_rows_kernel(const uint4* __restrict__ x, uint32_t n_units,
+                                                              FastDiv div_plane, FastDiv div_C,
+                                                              uint32_t groups, uint32_t* __restrict__ kmin,
+                                                              uint32_t* __restrict__ kmax) {
+    constexpr int V = Pack<T>::V;
+    __shared__ uint32_t s_kmn[kRangeSmemGroups], s_kmx[kRangeSmemGroups];
+    const bool combine = groups <= kRangeSmemGroups;       // else: straight to the global keys
+    if (combine) {
+        for (uint32_t i = threadIdx.x; i < groups; i += kThreads) {
+            s_kmn[i] = 0;
+            s_kmx[i] = 0;
+        }
+        __syncthreads();
+    }
+    uint32_t* dmn = combine ? s_kmn : kmin;
+    uint32_t* dmx = combine ? s_kmx : kmax;
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t nwarps = gridDim.x * (kThreads / 32), gw = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
+    const uint32_t nrows = (n_units + 127u) / 128u;
+    WarpRun run{kNoGroup, 0u, 0u};
+    auto fetch = [&](uint32_t row, Pack<T> (&p)[4]) {
+        if (row >= nrows) return;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const uint32_t u = row * 128u + j * 32 + lane;
+            if (u < n_units) p[j].raw = ld_stream_16(x + u);
+        }
+    };
+    auto reduce = [&](uint32_t row, const Pack<T> (&p)[4]) {
+        if (row >= nrows) return;
+        const uint32_t r0 = row * 128u;
+        float mn[4], mx[4];
+        bool v[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            v[j] = r0 + j * 32 + lane < n_units;
+            mn[j] = INFINITY;
+            mx[j] = -INFINITY;
+            if (v[j]) pack_minmax(p[j], 0, V, mn[j], mx[j]);
+        }
+        const uint32_t pl_first = div_plane.div(r0), pl_last = div_plane.div(min(r0 + 128u, n_units) - 1);
+        if (pl_first == pl_last) {
+            uint32_t q, g;
+            div_C.divmod(pl_first, q, g);
+            const float m0 = fminf(fminf(mn[0], mn[1]), fminf(mn[2], mn[3]));
+            const float m1 = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+            run_add(run, v[0], g, ~enc(m0), enc(m1), dmn, dmx);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint32_t q, g;
+                div_C.divmod(div_plane.div(v[j] ? r0 + j * 32 + lane : r0), q, g);
+                run_add(run, v[j], g, ~enc(mn[j]), enc(mx[j]), dmn, dmx);
+            }
+        }
+    };
+    for (uint32_t row = gw; row < nrows; row += 2 * nwarps) {
+        Pack<T> pa[4], pb[4];
+        fetch(row, pa);
+        fetch(row + nwarps, pb);
+        reduce(row, pa);
+        reduce(row + nwarps, pb);
+    }
+    run_flush(run, dmn, dmx);
+    if (combine) {
+        __syncthreads();
+        for (uint32_t i = threadIdx.x; i < groups; i += kThreads) {
+            const uint32_t k1 = s_kmn[i], k2 = s_kmx[i];
+            if (k1 | k2) {
+                atomicMax(kmin + i, k1);
+                atomicMax(kmax + i, k2);
+            }
+        }
+    }
+}
+
 __global__ void finalize_range_kernel(const uint32_t* __restrict__ kmin, const uint32_t* __restrict__ kmax,
                                       int64_t G, float* __restrict__ lo, float* __restrict__ hi, int bits,
                                       float* __restrict__ s_opt, float* __restrict__ z_opt) {
@@ -311,7 +394,13 @@ cudaError_t range_flat_t(const void* x, const Geom& g, uint32_t* kmin, uint32_t*
     constexpr int VF = Pack<T>::V;
     bool vec = aligned16(x) && (g.inner % VF == 0);
     int grid = flat_grid(f);
-    if (vec)
+    if (vec && g.E / VF < (1ll << 31) && g.C < (1ll << 30) && g.inner / VF < (1ll << 30)) {
+        const uint32_t n_units = (uint32_t)(g.E / VF);
+        int64_t rows = ((int64_t)n_units + 127) / 128, ctas = (rows + 2 * (kThreads / 32) - 1) / (2 * (kThreads / 32));
+        int rgrid = (int)(ctas < grid / 2 ? ctas : grid / 2);      // 4 resident CTAs per SM at 64 registers
+        range_rows_kernel<T><<<rgrid, kThreads, 0, st>>>((const uint4*)x, n_units, make_fastdiv((uint32_t)(g.inner / VF)),
+                                                         make_fastdiv((uint32_t)g.C), (uint32_t)g.C, kmin, kmax);
+    } else if (vec)
         range_flat_kernel<T, VF><<<grid, kThreads, 0, st>>>((const T*)x, f, kmin, kmax);
     else
         range_flat_kernel<T, 1><<<grid, kThreads, 0, st>>>((const T*)x, f, kmin, kmax);
