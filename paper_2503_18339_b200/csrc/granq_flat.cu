@@ -388,6 +388,13 @@ int flat_grid(const FlatGeom& f) {
     return (int)(f.ntiles < cap ? f.ntiles : cap);
 }
 
+int range_rows_ctas() {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    return sms * 4;
+}
+
 template <typename T>
 cudaError_t range_flat_t(const void* x, const Geom& g, uint32_t* kmin, uint32_t* kmax, cudaStream_t st) {
     FlatGeom f = make_flat(g);
@@ -397,7 +404,8 @@ cudaError_t range_flat_t(const void* x, const Geom& g, uint32_t* kmin, uint32_t*
     if (vec && g.E / VF < (1ll << 31) && g.C < (1ll << 30) && g.inner / VF < (1ll << 30)) {
         const uint32_t n_units = (uint32_t)(g.E / VF);
         int64_t rows = ((int64_t)n_units + 127) / 128, ctas = (rows + 2 * (kThreads / 32) - 1) / (2 * (kThreads / 32));
-        int rgrid = (int)(ctas < grid / 2 ? ctas : grid / 2);      // 4 resident CTAs per SM at 64 registers
+        const int64_t cap = (int64_t)range_rows_ctas();                 // 4 resident CTAs per SM at 64 registers
+        int rgrid = (int)(ctas < cap ? ctas : cap);
         range_rows_kernel<T><<<rgrid, kThreads, 0, st>>>((const uint4*)x, n_units, make_fastdiv((uint32_t)(g.inner / VF)),
                                                          make_fastdiv((uint32_t)g.C), (uint32_t)g.C, kmin, kmax);
     } else if (vec)
