@@ -117,9 +117,11 @@ __global__ void __launch_bounds__(kThreads) range_flat_kernel(const T* __restric
 // combines its warps' keys in shared memory before touching the global keys.
 constexpr uint32_t kRangeSmemGroups = 1024;
 
-template <typename T>
+// ALIGNED: planes are whole packs (div_plane divides pack indices); otherwise a pack may straddle two
+// planes (div_plane divides element indices, `inner` >= V elements per plane).
+template <typename T, bool ALIGNED>
 __global__ void __launch_bounds__(kThreads) range_rows_kernel(const uint4* __restrict__ x, uint32_t n_units,
-                                                              FastDiv div_plane, FastDiv div_C,
+                                                              uint32_t inner, FastDiv div_plane, FastDiv div_C,
                                                               uint32_t groups, uint32_t* __restrict__ kmin,
                                                               uint32_t* __restrict__ kmax) {
     constexpr int V = Pack<T>::V;
@@ -137,7 +139,7 @@ __global__ void __launch_bounds__(kThreads) range_rows_kernel(const uint4* __res
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t nwarps = gridDim.x * (kThreads / 32), gw = blockIdx.x * (kThreads / 32) + (threadIdx.x >> 5);
     const uint32_t nrows = (n_units + 127u) / 128u;
-    WarpRun run{kNoGroup, 0u, 0u};
+    WarpRun run{kNoGroup, 0u, 0u}, run2{kNoGroup, 0u, 0u};
     auto fetch = [&](uint32_t row, Pack<T> (&p)[4]) {
         if (row >= nrows) return;
 #pragma unroll
@@ -149,28 +151,47 @@ __global__ void __launch_bounds__(kThreads) range_rows_kernel(const uint4* __res
     auto reduce = [&](uint32_t row, const Pack<T> (&p)[4]) {
         if (row >= nrows) return;
         const uint32_t r0 = row * 128u;
-        float mn[4], mx[4];
         bool v[4];
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            v[j] = r0 + j * 32 + lane < n_units;
-            mn[j] = INFINITY;
-            mx[j] = -INFINITY;
-            if (v[j]) pack_minmax(p[j], 0, V, mn[j], mx[j]);
-        }
-        const uint32_t pl_first = div_plane.div(r0), pl_last = div_plane.div(min(r0 + 128u, n_units) - 1);
-        if (pl_first == pl_last) {
-            uint32_t q, g;
-            div_C.divmod(pl_first, q, g);
-            const float m0 = fminf(fminf(mn[0], mn[1]), fminf(mn[2], mn[3]));
-            const float m1 = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
-            run_add(run, v[0], g, ~enc(m0), enc(m1), dmn, dmx);
+        for (int j = 0; j < 4; ++j) v[j] = r0 + j * 32 + lane < n_units;
+        if constexpr (ALIGNED) {
+            float mn[4], mx[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                mn[j] = INFINITY;
+                mx[j] = -INFINITY;
+                if (v[j]) pack_minmax(p[j], 0, V, mn[j], mx[j]);
+            }
+            const uint32_t pl_first = div_plane.div(r0), pl_last = div_plane.div(min(r0 + 128u, n_units) - 1);
+            if (pl_first == pl_last) {
+                uint32_t q, g;
+                div_C.divmod(pl_first, q, g);
+                const float m0 = fminf(fminf(mn[0], mn[1]), fminf(mn[2], mn[3]));
+                const float m1 = fmaxf(fmaxf(mx[0], mx[1]), fmaxf(mx[2], mx[3]));
+                run_add(run, v[0], g, ~enc(m0), enc(m1), dmn, dmx);
+            } else {
+#pragma unroll
+                for (int j = 0; j < 4; ++j) {
+                    uint32_t q, g;
+                    div_C.divmod(div_plane.div(v[j] ? r0 + j * 32 + lane : r0), q, g);
+                    run_add(run, v[j], g, ~enc(mn[j]), enc(mx[j]), dmn, dmx);
+                }
+            }
         } else {
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                uint32_t q, g;
-                div_C.divmod(div_plane.div(v[j] ? r0 + j * 32 + lane : r0), q, g);
-                run_add(run, v[j], g, ~enc(mn[j]), enc(mx[j]), dmn, dmx);
+                uint32_t pl, rem, q, g1, g2;
+                div_plane.divmod((v[j] ? r0 + j * 32 + lane : r0) * V, pl, rem);
+                const int n1 = (int)min((uint32_t)V, inner - rem);          // elements of the first plane
+                div_C.divmod(pl, q, g1);
+                div_C.divmod(pl + 1, q, g2);
+                float mn1 = INFINITY, mx1 = -INFINITY, mn2 = INFINITY, mx2 = -INFINITY;
+                if (v[j]) {
+                    pack_minmax(p[j], 0, n1, mn1, mx1);
+                    pack_minmax(p[j], n1, V, mn2, mx2);
+                }
+                run_add(run, v[j], g1, ~enc(mn1), enc(mx1), dmn, dmx);
+                run_add(run2, v[j] && n1 < V, g2, ~enc(mn2), enc(mx2), dmn, dmx);
             }
         }
     };
@@ -182,6 +203,7 @@ __global__ void __launch_bounds__(kThreads) range_rows_kernel(const uint4* __res
         reduce(row + nwarps, pb);
     }
     run_flush(run, dmn, dmx);
+    if constexpr (!ALIGNED) run_flush(run2, dmn, dmx);
     if (combine) {
         __syncthreads();
         for (uint32_t i = threadIdx.x; i < groups; i += kThreads) {
@@ -401,13 +423,21 @@ cudaError_t range_flat_t(const void* x, const Geom& g, uint32_t* kmin, uint32_t*
     constexpr int VF = Pack<T>::V;
     bool vec = aligned16(x) && (g.inner % VF == 0);
     int grid = flat_grid(f);
-    if (vec && g.E / VF < (1ll << 31) && g.C < (1ll << 30) && g.inner / VF < (1ll << 30)) {
+    const bool rows_ok = aligned16(x) && g.E % VF == 0 && g.inner >= VF && g.E < (1ll << 31) &&
+                         g.C < (1ll << 30) && g.inner < (1ll << 30);
+    if (rows_ok) {
         const uint32_t n_units = (uint32_t)(g.E / VF);
         int64_t rows = ((int64_t)n_units + 127) / 128, ctas = (rows + 2 * (kThreads / 32) - 1) / (2 * (kThreads / 32));
         const int64_t cap = (int64_t)range_rows_ctas();                 // 4 resident CTAs per SM at 64 registers
         int rgrid = (int)(ctas < cap ? ctas : cap);
-        range_rows_kernel<T><<<rgrid, kThreads, 0, st>>>((const uint4*)x, n_units, make_fastdiv((uint32_t)(g.inner / VF)),
-                                                         make_fastdiv((uint32_t)g.C), (uint32_t)g.C, kmin, kmax);
+        if (vec)
+            range_rows_kernel<T, true><<<rgrid, kThreads, 0, st>>>((const uint4*)x, n_units, (uint32_t)g.inner,
+                                                                   make_fastdiv((uint32_t)(g.inner / VF)),
+                                                                   make_fastdiv((uint32_t)g.C), (uint32_t)g.C, kmin, kmax);
+        else
+            range_rows_kernel<T, false><<<rgrid, kThreads, 0, st>>>((const uint4*)x, n_units, (uint32_t)g.inner,
+                                                                    make_fastdiv((uint32_t)g.inner),
+                                                                    make_fastdiv((uint32_t)g.C), (uint32_t)g.C, kmin, kmax);
     } else if (vec)
         range_flat_kernel<T, VF><<<grid, kThreads, 0, st>>>((const T*)x, f, kmin, kmax);
     else
