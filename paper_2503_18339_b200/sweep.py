@@ -1,0 +1,81 @@
+"""Bandwidth sweep of the fused entry point over one synthetic activation set.
+
+    python -m paper_2503_18339_b200.sweep --config 5            # ResNet-50 shapes, fp32 + bf16, b = 2..8
+
+Per tensor, element type, bit-width and mode (forward only / forward + backward) it prints the
+CUDA-event time of one call (median of `--iters`, after warm-up, an L2-sized scratch write between
+calls), the algorithmic GB/s (fp32: 8 / 16 B per element, bf16: 4 / 8) and its fraction of the
+measured copy bandwidth.  Inputs come from `workloads.py`; bf16 inputs are the round-to-nearest-even
+of the fp32 sample.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+
+import torch
+
+from . import binding as b
+from . import workloads as wl
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _peak() -> float:
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            return float(json.load(fh)["hbm_gbs"])
+    except Exception:
+        return 6650.0
+
+
+def main() -> None:
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--config", type=int, default=5)
+    ap.add_argument("--iters", type=int, default=5)
+    ap.add_argument("--bits", default="", help="comma list; default: the config's own")
+    ap.add_argument("--dtypes", default="", help="comma list of f32,bf16; default: the config's own")
+    args = ap.parse_args()
+    b.lib()
+    peak = _peak()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    seen = set()
+    print("tensor dtype bits mode us GB/s frac_of_measured")
+    for spec in wl.config_tensors(args.config):
+        if spec.shape in seen:
+            continue
+        seen.add(spec.shape)
+        x32 = torch.from_numpy(wl.make_activation(spec)).cuda()
+        g32 = torch.from_numpy(wl.make_upstream_grad(spec)).cuda()
+        for dt in (args.dtypes.split(",") if args.dtypes else spec.dtypes):
+            x = x32 if dt == "f32" else x32.to(torch.bfloat16)
+            gy = g32 if dt == "f32" else g32.to(torch.bfloat16)
+            out = b.FakeQuantOut(y=torch.empty_like(x), gx=torch.empty_like(x))
+            esize = x.element_size()
+            for bits in ([int(v) for v in args.bits.split(",")] if args.bits else spec.bits):
+                for mode in ("fwd", "fwd+bwd"):
+                    g = gy if mode == "fwd+bwd" else None
+                    for _ in range(2):
+                        b.granq_fakequant_fused(x, bits, gy=g, out=out)
+                    times = []
+                    for _ in range(args.iters):
+                        flush.fill_(1)
+                        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        e0.record()
+                        b.granq_fakequant_fused(x, bits, gy=g, out=out)
+                        e1.record()
+                        torch.cuda.synchronize()
+                        times.append(e0.elapsed_time(e1) * 1e3)
+                    assert b.workspace_status(out.workspace) == b.OK
+                    us = statistics.median(times)
+                    nbytes = x.numel() * esize * (4 if g is not None else 2)
+                    gbs = nbytes / us / 1e3
+                    print(f"{spec.name} {dt} {bits} {mode} {us:.1f} {gbs:.0f} {gbs / peak:.3f}", flush=True)
+            del x, gy, out
+        del x32, g32
+
+
+if __name__ == "__main__":
+    main()
