@@ -92,12 +92,19 @@ __global__ void __launch_bounds__(kLThreads, UPL == 2 ? 4 : 3) l2wave_kernel(con
     for (uint32_t i = tid; i < 2 * tab; i += kLThreads) s_keys[i] = 0;
     __syncthreads();
 
+    // Tiles are dealt round-robin over the CTAs and the deal carries on from wave to wave, so the
+    // CTAs that get one tile more differ from wave to wave; both phases of a wave use the same deal.
+    auto first_tile = [&](uint32_t w) -> uint32_t {
+        const uint32_t dealt = (uint32_t)(((uint64_t)w * a.shape[0].ntiles) % gridDim.x);
+        return (blockIdx.x + gridDim.x - dealt) % gridDim.x;
+    };
+
     // ---- phase 1: this CTA's tiles of wave w -> min / max keys, then arrive ----
     auto phase1 = [&](uint32_t w) {
         const LShape& sh = a.shape[(w + 1 == W) ? 1 : 0];
         const uint32_t c0 = w * a.cw, base = w * a.wave_units;
         WarpRun run{kNoGroup, 0u, 0u}, run2{kNoGroup, 0u, 0u};
-        for (uint32_t tile = blockIdx.x; tile < sh.ntiles; tile += gridDim.x) {
+        for (uint32_t tile = first_tile(w); tile < sh.ntiles; tile += gridDim.x) {
             uint32_t slab, ti;
             sh.div_tps.divmod(tile, slab, ti);
             const uint32_t r0 = ti * kTile + warp * kRow;
@@ -205,7 +212,7 @@ __global__ void __launch_bounds__(kLThreads, UPL == 2 ? 4 : 3) l2wave_kernel(con
             }
         }
         __syncthreads();
-        for (uint32_t tile = blockIdx.x; tile < sh.ntiles; tile += gridDim.x) {
+        for (uint32_t tile = first_tile(w); tile < sh.ntiles; tile += gridDim.x) {
             uint32_t slab, ti;
             sh.div_tps.divmod(tile, slab, ti);
             const uint32_t r0 = ti * kTile + warp * kRow;
