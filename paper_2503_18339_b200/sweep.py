@@ -37,14 +37,21 @@ def main() -> None:
     ap.add_argument("--iters", type=int, default=5)
     ap.add_argument("--bits", default="", help="comma list; default: the config's own")
     ap.add_argument("--dtypes", default="", help="comma list of f32,bf16; default: the config's own")
+    ap.add_argument("--modes", default="fwd,fwd+bwd")
+    ap.add_argument("--only", default="", help="keep tensors whose name contains this")
+    ap.add_argument("--tune", default="", help="planner knobs, e.g. l2_wave_kb=32768,l2_upl=2")
     args = ap.parse_args()
     b.lib()
+    knobs = {"l2_wave_kb": b.KNOB_L2_WAVE_KB, "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM}
+    for item in filter(None, args.tune.split(",")):
+        name, val = item.split("=")
+        b.tune(knobs[name], int(val))
     peak = _peak()
     flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
     seen = set()
     print("tensor dtype bits mode us GB/s frac_of_measured")
     for spec in wl.config_tensors(args.config):
-        if spec.shape in seen:
+        if spec.shape in seen or args.only not in spec.name:
             continue
         seen.add(spec.shape)
         x32 = torch.from_numpy(wl.make_activation(spec)).cuda()
@@ -55,7 +62,7 @@ def main() -> None:
             out = b.FakeQuantOut(y=torch.empty_like(x), gx=torch.empty_like(x))
             esize = x.element_size()
             for bits in ([int(v) for v in args.bits.split(",")] if args.bits else spec.bits):
-                for mode in ("fwd", "fwd+bwd"):
+                for mode in args.modes.split(","):
                     g = gy if mode == "fwd+bwd" else None
                     for _ in range(2):
                         b.granq_fakequant_fused(x, bits, gy=g, out=out)

@@ -347,6 +347,31 @@ def test_non_default_stream(b):
     assert_parity(got, ref, shape, 1, orc.GROUP_CHANNEL, backward=True)
 
 
+def test_more_than_2_to_the_31_elements(b):
+    """Index arithmetic beyond 32 bits: a bf16 tensor of 2^31 + 2^21 elements through the range,
+    forward and fused entry points, every element compared with the oracle."""
+    shape = (2, 4, 16384, 16400)
+    n = int(np.prod(shape, dtype=np.int64))
+    assert n > 2 ** 31
+    rng = np.random.default_rng(31)
+    # bf16 bit patterns of finite values in about [-4, 4): sign + exponent 120..128 + 7 mantissa bits
+    xb = (rng.integers(120, 129, n, dtype=np.uint16) << 7) | rng.integers(0, 128, n, dtype=np.uint16)
+    xb |= rng.integers(0, 2, n, dtype=np.uint16) << 15
+    xb = xb.reshape(shape)
+    xd = to_dev(xb)
+    lo_ref, hi_ref = orc.range_(xb)
+    lo, hi = b.granq_range(xd)
+    assert same_bits(to_np(lo), lo_ref) and same_bits(to_np(hi), hi_ref)
+    ref = orc.fakequant(xb, 4, lo_ref, hi_ref)
+    fw = b.granq_fakequant_fwd(xd, 4, lo, hi, want_codes=True)
+    assert np.array_equal(to_np(fw.codes), ref.codes) and same_bits(to_np(fw.y), ref.y)
+    del fw
+    got = b.granq_fakequant_fused(xd, 4, want_codes=True)
+    assert b.workspace_status(got.workspace) == b.OK
+    assert same_bits(to_np(got.lo), lo_ref) and same_bits(to_np(got.hi), hi_ref)
+    assert np.array_equal(to_np(got.codes), ref.codes) and same_bits(to_np(got.y), ref.y)
+
+
 # ---- 6. the bounded device-side wait gives up cleanly ------------------------------------------------------------
 def test_bounded_wait_reports_timeout_and_context_survives(b, knobs):
     """A wave is told to wait for one arrival more than the grid can provide, with a short
