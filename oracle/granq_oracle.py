@@ -46,7 +46,9 @@ _lib = None
 def lib() -> ctypes.CDLL:
     global _lib
     if _lib is None:
-        L = ctypes.CDLL(build())
+        # GRANQ_ORACLE_LIB_OVERRIDE: a deliberately broken build, used by the test that checks that the
+        # pins notice planted mistakes
+        L = ctypes.CDLL(os.environ.get("GRANQ_ORACLE_LIB_OVERRIDE") or build())
         vp, i64p, fp, u8p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.c_void_p, ctypes.c_void_p
         ci = ctypes.c_int
         L.granq_oracle_num_groups.restype = ctypes.c_int64

@@ -1,0 +1,43 @@
+"""The pins must notice plausible mistakes.  Each case plants one mistake in a copy of the oracle's
+C source (on the CPU, nothing here touches a GPU), builds it, and runs the pin tests against it in
+a subprocess: they have to fail."""
+import os
+import subprocess
+import sys
+
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+SRC = os.path.join(ROOT, "oracle", "granq_oracle.c")
+
+MUTATIONS = {
+    "wrong_sign_of_zero_point_in_eq1": ("float u = t + zk;", "float u = t - zk;"),
+    "ties_away_from_zero": ("float r = rintf(u);", "float r = floorf(u + 0.5f);"),
+    "scale_divided_by_2_pow_b": ("float s = (hi - lo) / qmax;", "float s = (hi - lo) / (qmax + 1.0f);"),
+    "no_upper_clamp": ("if (q > qmax) q = qmax;", ""),
+    "mask_excludes_code_zero": ("int inside = (r >= 0.0f) && (r <= qmax);", "int inside = (r > 0.0f) && (r <= qmax);"),
+    "dequantize_without_zero_point": ("float yv = sk * d;", "float yv = sk * q;"),
+    "zero_point_from_plus_lo": ("float z = rintf((-lo) / s);", "float z = rintf(lo / s);"),
+    "max_taken_as_min": ("if (v > hi[k]) hi[k] = v;", "if (v < hi[k]) hi[k] = v;"),
+    "sample_channel_groups_collapsed": ("return o * g->C + c;", "return c;"),
+    "bf16_ties_away": ("u += 0x7FFFu + lsb;", "u += 0x8000u;"),
+    "no_degenerate_floor": ("if (!(s >= 1e-8f)) s = 1e-8f;", "if (!(s > 0.0f)) s = 1.0f;"),
+    "gradient_not_masked": ("inside ? gv : 0.0f", "gv"),
+}
+
+
+@pytest.mark.parametrize("name", sorted(MUTATIONS))
+def test_pins_catch_planted_mistake(name, tmp_path):
+    old, new = MUTATIONS[name]
+    text = open(SRC).read()
+    assert text.count(old) == 1, f"mutation target not found exactly once: {old!r}"
+    src = tmp_path / "granq_oracle.c"
+    src.write_text(text.replace(old, new))
+    (tmp_path / "granq_oracle.h").write_text(open(os.path.join(ROOT, "oracle", "granq_oracle.h")).read())
+    lib = tmp_path / "libmutant.so"
+    subprocess.check_call(["gcc", "-O2", "-std=c11", "-ffp-contract=off", "-fno-fast-math", "-shared", "-fPIC",
+                           "-o", str(lib), str(src), "-lm"])
+    env = dict(os.environ, GRANQ_ORACLE_LIB_OVERRIDE=str(lib))
+    r = subprocess.run([sys.executable, "-m", "pytest", os.path.join(ROOT, "tests", "test_oracle_pins.py"), "-x", "-q",
+                        "-p", "no:cacheprovider"], env=env, cwd=ROOT, capture_output=True, text=True)
+    assert r.returncode != 0, f"the pins did not notice: {name}\n{r.stdout[-800:]}"
