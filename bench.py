@@ -202,10 +202,13 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="also print a per-tensor table to stderr")
     ap.add_argument("--tune", default="", help="planner overrides for experiments, e.g. depth=3,max_buf_units=4000")
-    ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged", "l2wave"],
+    ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged", "l2wave", "colwalk"],
                     help="force an execution plan of the fused entry point (experiments)")
     ap.add_argument("--op", default="fused", choices=["fused", "range", "fwd", "bwd"],
                     help="time another entry point instead of the fused one (experiments; bytes/element 4, 8, 12)")
+    ap.add_argument("--clear-workspace", action="store_true",
+                    help="let every call clear its workspace (one more memset node per call) instead of "
+                         "passing GRANQ_FLAG_WORKSPACE_ZEROED")
     ap.add_argument("--only", default="", help="profiling aid: keep only workload tensors whose name contains this")
     args = ap.parse_args()
     if args.impl == "reference":
@@ -227,13 +230,18 @@ def main():
     b.lib()
     knob_ids = {"depth": b.KNOB_STAGED_DEPTH, "max_buf_units": b.KNOB_STAGED_MAX_BUF_UNITS,
                 "grid": b.KNOB_STAGED_GRID, "ctas_per_sm": b.KNOB_STAGED_CTAS_PER_SM,
-                "l2_wave_kb": b.KNOB_L2_WAVE_KB, "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM}
+                "l2_wave_kb": b.KNOB_L2_WAVE_KB, "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM,
+                "l2_lag": b.KNOB_L2_LAG}
     for item in filter(None, args.tune.split(",")):
         name, val = item.split("=")
         b.tune(knob_ids[name], int(val))
     warmup = max(args.warmup, 3)
     flags = {"auto": 0, "two_pass": b.FLAG_FORCE_TWO_PASS, "naive": b.FLAG_FORCE_NAIVE,
-             "staged": b.FLAG_FORCE_STAGED, "l2wave": b.FLAG_FORCE_L2WAVE}[args.plan]
+             "staged": b.FLAG_FORCE_STAGED, "l2wave": b.FLAG_FORCE_L2WAVE,
+             "colwalk": b.FLAG_FORCE_COLWALK}[args.plan]
+    plan_flags = flags
+    if not args.clear_workspace:      # the workspaces are cleared once below and every call leaves them clear
+        flags |= b.FLAG_WORKSPACE_ZEROED
 
     specs = [s for s in workload_specs() if args.only in s.name]
     # ---- host (pinned) inputs and outputs; every rank has its own batch (weak scaling, no exchange) ----
@@ -250,13 +258,13 @@ def main():
         gy = gs.cuda(non_blocking=True)
         out = b.FakeQuantOut(y=torch.empty_like(x), gx=torch.empty_like(x),
                              lo=torch.empty(s.shape[1], device="cuda"), hi=torch.empty(s.shape[1], device="cuda"),
-                             workspace=b.make_workspace(x))
+                             workspace=b.make_workspace(x, zeroed=True))
         dev.append((x, gy, out))
     torch.cuda.synchronize()
     calls = [(i, bits) for i, s in enumerate(specs) for bits in s.bits]
     elems_per_step = sum(specs[i].numel for i, _ in calls)
     bytes_per_step = elems_per_step * BYTES_PER_ELEM
-    plans = [b.fused_plan(b.F32, specs[i].shape, flags=flags) for i, _ in calls]
+    plans = [b.fused_plan(b.F32, specs[i].shape, flags=plan_flags) for i, _ in calls]
     launches_per_step = sum(n for _, n in plans)
     stream = torch.cuda.current_stream()
 
@@ -406,7 +414,9 @@ def main():
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": WORKLOAD, "elements_per_step_per_gpu": elems_per_step,
                        "calls_per_step": len(calls), "l2": "inputs larger than L2 (7.3 GB working set per step)",
-                       "group_mode": "channel", "parallelism": f"replicas x{world} (independent batches, no exchange)"},
+                       "group_mode": "channel",
+                       "workspace": ("cleared by every call" if args.clear_workspace else
+                                     "cleared once at allocation, GRANQ_FLAG_WORKSPACE_ZEROED on every call"), "parallelism": f"replicas x{world} (independent batches, no exchange)"},
             "elements_per_s": world * elems_per_step / (ms_per_step * 1e-3),
             "frac_of_measured_hbm": value / world / peak, "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "e2e": e2e, "roofline": roofline,

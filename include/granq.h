@@ -33,7 +33,8 @@
  * memory owned by the caller, valid until the stream has passed the call.  The library
  * never allocates or frees device memory and keeps no results between calls; scratch comes
  * from the caller's `workspace` (at least granq_workspace_bytes(), 256-byte aligned,
- * contents irrelevant on entry, overwritten by the call).  Outputs must not overlap
+ * contents irrelevant on entry unless GRANQ_FLAG_WORKSPACE_ZEROED says otherwise, overwritten by
+ * the call).  Outputs must not overlap
  * inputs.  Inputs must be finite (NaN / Inf give unspecified results, never a fault).
  *
  * Execution.  All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*;
@@ -81,7 +82,13 @@ enum granq_flags {
     GRANQ_FLAG_FORCE_NAIVE = 2u,     /* fused: host loop over channels, three launches per channel -
                                         the "conventional" scalar-loop scheme of Section 5.3.2       */
     GRANQ_FLAG_FORCE_STAGED = 4u,    /* fused: on-chip-staged persistent kernel or GRANQ_ERR_UNSUPPORTED */
-    GRANQ_FLAG_FORCE_L2WAVE = 8u     /* fused: L2-resident-wave persistent kernel or GRANQ_ERR_UNSUPPORTED */
+    GRANQ_FLAG_FORCE_L2WAVE = 8u,    /* fused: L2-resident-wave persistent kernel or GRANQ_ERR_UNSUPPORTED */
+    GRANQ_FLAG_FORCE_COLWALK = 16u,  /* fused: column-walk persistent kernel or GRANQ_ERR_UNSUPPORTED     */
+    GRANQ_FLAG_WORKSPACE_ZEROED = 32u /* fused: the caller guarantees that the whole workspace is zero on
+                                        entry (cleared after allocation, or left by an earlier call with
+                                        this flag that ended with status GRANQ_OK); the call then skips
+                                        its own clearing step and leaves the workspace zero again on
+                                        success.  After GRANQ_ERR_TIMEOUT clear it before the next use. */
 };
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -192,8 +199,8 @@ int granq_fakequant_fused_host(const void* x_host, const void* gy_host_opt, int 
 
 /*
  * Plan that granq_fakequant_fused() would take for this geometry and flags on the current
- * device: 0 = two-pass, 1 = naive per-channel loop, 2 = on-chip staged, 3 = L2-resident waves;
- * negative = -status.
+ * device: 0 = two-pass, 1 = naive per-channel loop, 2 = on-chip staged, 3 = L2-resident waves,
+ * 4 = column walk; negative = -status.
  * `launches_out` (HOST, may be NULL) receives the number of kernel launches of that plan.
  */
 int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,
@@ -236,7 +243,8 @@ enum granq_knob {
     GRANQ_KNOB_STAGED_CTAS_PER_SM = 5,    /* CTAs that share one SM (1 or 2)                       */
     GRANQ_KNOB_L2_WAVE_KB = 6,            /* L2-wave plan: x bytes of one wave, in KiB             */
     GRANQ_KNOB_L2_UPL = 7,                /* L2-wave plan: 16-byte units per lane and step (2, 4)  */
-    GRANQ_KNOB_L2_CTAS_PER_SM = 8         /* L2-wave plan: cap on resident CTAs per SM             */
+    GRANQ_KNOB_L2_CTAS_PER_SM = 8,        /* L2-wave / column-walk plans: cap on resident CTAs per SM */
+    GRANQ_KNOB_L2_LAG = 9                 /* column-walk plan: waves the range phase runs ahead (1..3) */
 };
 int granq_tune(int knob, int value);
 

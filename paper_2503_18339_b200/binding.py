@@ -18,11 +18,12 @@ LIB_PATH = os.path.join(_HERE, "libgranq.so")
 
 F32, BF16 = 0, 1
 GROUP_CHANNEL, GROUP_SAMPLE_CHANNEL, GROUP_TENSOR = 0, 1, 2
-FLAG_FORCE_TWO_PASS, FLAG_FORCE_NAIVE, FLAG_FORCE_STAGED, FLAG_FORCE_L2WAVE = 1, 2, 4, 8
-PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED, PLAN_L2WAVE = 0, 1, 2, 3
+FLAG_FORCE_TWO_PASS, FLAG_FORCE_NAIVE, FLAG_FORCE_STAGED, FLAG_FORCE_L2WAVE, FLAG_FORCE_COLWALK = 1, 2, 4, 8, 16
+FLAG_WORKSPACE_ZEROED = 32
+PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED, PLAN_L2WAVE, PLAN_COLWALK = 0, 1, 2, 3, 4
 (KNOB_STAGED_DEPTH, KNOB_STAGED_MAX_BUF_UNITS, KNOB_STAGED_GRID, KNOB_SPIN_LIMIT, KNOB_TEST_EXTRA_ARRIVALS,
- KNOB_STAGED_CTAS_PER_SM, KNOB_L2_WAVE_KB, KNOB_L2_UPL, KNOB_L2_CTAS_PER_SM) = range(9)
-N_KNOBS = 9
+ KNOB_STAGED_CTAS_PER_SM, KNOB_L2_WAVE_KB, KNOB_L2_UPL, KNOB_L2_CTAS_PER_SM, KNOB_L2_LAG) = range(10)
+N_KNOBS = 10
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 
 EXPORTS = [
@@ -148,9 +149,12 @@ def workspace_bytes(dtype: int, shape, channel_axis: int = 1, group: int = GROUP
     return int(lib().granq_workspace_bytes(dtype, _dims(shape), channel_axis, group))
 
 
-def make_workspace(x: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL) -> torch.Tensor:
+def make_workspace(x: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL,
+                   zeroed: bool = False) -> torch.Tensor:
+    """Scratch for the entry points that take a workspace; `zeroed` clears it, as calls made with
+    FLAG_WORKSPACE_ZEROED expect of a workspace they see for the first time."""
     n = workspace_bytes(_dtype(x), x.shape, channel_axis, group)
-    return torch.empty(n, dtype=torch.uint8, device=x.device)
+    return (torch.zeros if zeroed else torch.empty)(n, dtype=torch.uint8, device=x.device)
 
 
 def tune(knob: int, value: int) -> None:

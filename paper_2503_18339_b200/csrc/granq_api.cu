@@ -10,7 +10,7 @@ namespace {
 
 constexpr int64_t kMaxElements = 1ll << 40;
 
-StagedTuning g_tune = {0, 0, 0, 0, 0, 0, 0, 0, 0};
+StagedTuning g_tune = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
 
 bool make_geom(const int64_t dims[4], int axis, int group, Geom& g, int64_t& G) {
     if (!dims || axis < 0 || axis > 3 || group < 0 || group > 2) return false;
@@ -55,13 +55,19 @@ int check_workspace(const void* ws, size_t bytes, int64_t G) {
 
 int cuda_status(cudaError_t e) { return e == cudaSuccess ? GRANQ_OK : GRANQ_ERR_CUDA; }
 
-enum { PLAN_TWO_PASS = 0, PLAN_NAIVE = 1, PLAN_STAGED = 2, PLAN_L2WAVE = 3 };
+enum { PLAN_TWO_PASS = 0, PLAN_NAIVE = 1, PLAN_STAGED = 2, PLAN_L2WAVE = 3, PLAN_COLWALK = 4 };
 
 // plan of the fused entry point; `plan_out` is filled when the staged plan is taken
 int choose_plan(int dtype, const Geom& g, const QuantIO& io, uint32_t flags, StagedPlan* plan_out,
-                L2Plan* l2_out) {
+                L2Plan* l2_out, ColPlan* col_out) {
     if (flags & GRANQ_FLAG_FORCE_NAIVE) return PLAN_NAIVE;
     if (flags & GRANQ_FLAG_FORCE_TWO_PASS) return PLAN_TWO_PASS;
+    if (flags & GRANQ_FLAG_FORCE_COLWALK) {
+        ColPlan cp = plan_colwalk(dtype, g, io, g_tune);
+        if (!cp.ok) return -GRANQ_ERR_UNSUPPORTED;
+        if (col_out) *col_out = cp;
+        return PLAN_COLWALK;
+    }
     if (flags & GRANQ_FLAG_FORCE_L2WAVE) {
         L2Plan lp = plan_l2wave(dtype, g, io, g_tune);
         if (!lp.ok) return -GRANQ_ERR_UNSUPPORTED;
@@ -76,8 +82,13 @@ int choose_plan(int dtype, const Geom& g, const QuantIO& io, uint32_t flags, Sta
         if (plan_out) *plan_out = p;
         return PLAN_STAGED;
     }
-    // default: the L2-resident-wave kernel wherever the geometry qualifies (it has measured
-    // faster than the shared-memory-staged kernel on every workload tensor)
+    // default: the column-walk kernel where there are slabs to walk, else the L2-resident-wave
+    // kernel (both have measured faster than the shared-memory-staged kernel on every workload tensor)
+    ColPlan cp = plan_colwalk(dtype, g, io, g_tune);
+    if (cp.ok) {
+        if (col_out) *col_out = cp;
+        return PLAN_COLWALK;
+    }
     L2Plan lp = plan_l2wave(dtype, g, io, g_tune);
     if (lp.ok) {
         if (l2_out) *l2_out = lp;
@@ -194,16 +205,24 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
     QuantIO io{x, gy_opt, y, gx_opt, codes_opt, mask_opt};
     StagedPlan sp{};
     L2Plan lp{};
-    const int plan = choose_plan(dtype, g, io, flags, &sp, &lp);
+    ColPlan cp{};
+    const int plan = choose_plan(dtype, g, io, flags, &sp, &lp, &cp);
     if (plan < 0) return -plan;
 
     Workspace ws = carve_workspace(workspace, G);
-    cudaError_t e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
+    // The column-walk kernel leaves a zeroed workspace zeroed; with the caller's word that it is
+    // zero on entry nothing has to be cleared.  The other plans clear before and, to keep that
+    // word true for the next call, after.
+    const bool zeroed = (flags & GRANQ_FLAG_WORKSPACE_ZEROED) != 0;
+    cudaError_t e = cudaSuccess;
+    if (!(zeroed && plan == PLAN_COLWALK)) e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
     if (e != cudaSuccess) return GRANQ_ERR_CUDA;
     if (plan == PLAN_STAGED) {
         e = launch_staged(sp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
     } else if (plan == PLAN_L2WAVE) {
         e = launch_l2wave(lp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
+    } else if (plan == PLAN_COLWALK) {
+        e = launch_colwalk(cp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
     } else if (plan == PLAN_NAIVE) {
         e = launch_naive(io, mode, dtype, g, bits, ws.kmin, ws.kmax, min_out, max_out, st, nullptr);
         if (e == cudaSuccess && (scale_opt || zp_opt))
@@ -214,6 +233,8 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
             e = launch_finalize_range(ws.kmin, ws.kmax, G, min_out, max_out, bits, scale_opt, zp_opt, st);
         if (e == cudaSuccess) e = launch_quant_flat(io, mode, dtype, g, bits, min_out, max_out, st);
     }
+    if (e == cudaSuccess && zeroed && plan != PLAN_COLWALK)
+        e = cudaMemsetAsync((char*)workspace + sizeof(uint32_t), 0, ws.clear_bytes - sizeof(uint32_t), st);
     return cuda_status(e);
 }
 
@@ -287,9 +308,9 @@ int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int gro
     if (!dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G)) return -GRANQ_ERR_INVALID_ARG;
     (void)with_backward;
     QuantIO io{};   // null pointers: alignment is assumed
-    const int plan = choose_plan(dtype, g, io, flags, nullptr, nullptr);
+    const int plan = choose_plan(dtype, g, io, flags, nullptr, nullptr, nullptr);
     if (launches_out) {
-        if (plan == PLAN_STAGED || plan == PLAN_L2WAVE) *launches_out = 1;
+        if (plan == PLAN_STAGED || plan == PLAN_L2WAVE || plan == PLAN_COLWALK) *launches_out = 1;
         else if (plan == PLAN_NAIVE) *launches_out = (int)(3 * g.C);
         else if (plan == PLAN_TWO_PASS) *launches_out = 3;
     }
@@ -320,6 +341,7 @@ int granq_tune(int knob, int value) {
         case GRANQ_KNOB_L2_WAVE_KB: g_tune.l2_wave_kb = value; return GRANQ_OK;
         case GRANQ_KNOB_L2_UPL: g_tune.l2_upl = value; return GRANQ_OK;
         case GRANQ_KNOB_L2_CTAS_PER_SM: g_tune.l2_ctas_per_sm = value; return GRANQ_OK;
+        case GRANQ_KNOB_L2_LAG: g_tune.l2_lag = value; return GRANQ_OK;
         default: return GRANQ_ERR_INVALID_ARG;
     }
 }

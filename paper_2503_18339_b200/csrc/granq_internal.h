@@ -92,7 +92,8 @@ struct StagedTuning {
     int ctas_per_sm;      // CTAs sharing one SM (1 or 2); they split its threads and shared memory
     int l2_wave_kb;       // L2-wave plan: target x bytes of one wave, in KiB
     int l2_upl;           // L2-wave plan: 16-byte units per lane and step (2 or 4)
-    int l2_ctas_per_sm;   // L2-wave plan: cap on resident CTAs per SM
+    int l2_ctas_per_sm;   // L2-wave and column-walk plans: cap on resident CTAs per SM
+    int l2_lag;           // column-walk plan: waves of phase 1 running ahead of phase 2 (1..3)
 };
 StagedPlan plan_staged(int dtype, const Geom& g, const QuantIO& io, int device, const StagedTuning& tune);
 StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_count, int smem_optin,
@@ -113,5 +114,17 @@ L2Plan plan_l2wave(int dtype, const Geom& g, const QuantIO& io, const StagedTuni
 cudaError_t launch_l2wave(const L2Plan& plan, const QuantIO& io, int mode, int dtype, const Geom& g, int bits,
                           const Workspace& ws, float* lo, float* hi, float* s_opt, float* z_opt,
                           const StagedTuning& tune, cudaStream_t st);
+
+// ---- column-walk persistent kernel (L2-resident waves, one unit column per thread) ----------
+struct ColPlan {
+    bool ok;
+    uint32_t cw;             // channels per wave
+    uint32_t nwaves;
+    uint32_t lag;            // waves of phase 1 running ahead of phase 2
+};
+ColPlan plan_colwalk(int dtype, const Geom& g, const QuantIO& io, const StagedTuning& tune);
+cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int dtype, const Geom& g, int bits,
+                           const Workspace& ws, float* lo, float* hi, float* s_opt, float* z_opt,
+                           const StagedTuning& tune, cudaStream_t st);
 
 }  // namespace granq

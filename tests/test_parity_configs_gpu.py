@@ -46,7 +46,8 @@ def check(b, x, gy, bits, mode, with_codes, expect_staged=True):
     dt = b.F32 if x.dtype == np.float32 else b.BF16
     plan, _ = b.fused_plan(dt, x.shape, group=mode, with_backward=gy is not None)
     if expect_staged:
-        assert plan == b.PLAN_L2WAVE, "the benchmarked plan for this tensor is the L2-resident-wave kernel"
+        want = b.PLAN_COLWALK if mode == orc.GROUP_CHANNEL else b.PLAN_L2WAVE
+        assert plan == want, "the benchmarked plan: column walk over the batch, L2-resident waves for per-sample groups"
     ref = orc.fused(x, bits, gy=gy, group_mode=mode, want_codes=with_codes)
     got = b.granq_fakequant_fused(to_dev(x), bits, gy=None if gy is None else to_dev(gy), group=mode,
                                   want_codes=with_codes, want_mask=with_codes, want_params=True)

@@ -23,7 +23,7 @@ def b():
     from paper_2503_18339_b200 import binding
     binding.lib()
     yield binding
-    for k in range(9):
+    for k in range(binding.N_KNOBS):
         binding.tune(k, 0)
 
 
@@ -34,11 +34,11 @@ def knobs(b):
         names = {"depth": b.KNOB_STAGED_DEPTH, "max_buf_units": b.KNOB_STAGED_MAX_BUF_UNITS,
                  "grid": b.KNOB_STAGED_GRID, "spin_limit": b.KNOB_SPIN_LIMIT,
                  "extra_arrivals": b.KNOB_TEST_EXTRA_ARRIVALS, "l2_wave_kb": b.KNOB_L2_WAVE_KB,
-                 "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM}
+                 "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM, "l2_lag": b.KNOB_L2_LAG}
         for k, v in kw.items():
             b.tune(names[k], v)
     yield set_
-    for k in range(9):
+    for k in range(b.N_KNOBS):
         b.tune(k, 0)
 
 
@@ -137,14 +137,14 @@ def test_fused_small_all_plans(b, shape, mode, dtype):
     bits = 2 + (sum(shape) + mode) % 7
     x, gy = make_case(shape, seed=sum(shape) * 7 + mode, dtype=dtype, relu=(shape[0] % 2 == 0))
     ref = orc.fused(x, bits, gy=gy, group_mode=mode)
-    for flags in (0, b.FLAG_FORCE_TWO_PASS, b.FLAG_FORCE_NAIVE, b.FLAG_FORCE_L2WAVE):
+    for flags in (0, b.FLAG_FORCE_TWO_PASS, b.FLAG_FORCE_NAIVE, b.FLAG_FORCE_L2WAVE, b.FLAG_FORCE_COLWALK):
         if flags == b.FLAG_FORCE_NAIVE and b.num_groups(shape, 1, mode) > 300:
             continue
         try:
             got = b.granq_fakequant_fused(to_dev(x), bits, gy=to_dev(gy), group=mode, want_codes=True,
                                           want_mask=True, want_params=True, flags=flags)
-        except b.GranqError as err:      # the L2-wave plan does not take every geometry
-            assert flags == b.FLAG_FORCE_L2WAVE and err.status == b.ERR_UNSUPPORTED
+        except b.GranqError as err:      # the persistent plans do not take every geometry
+            assert flags in (b.FLAG_FORCE_L2WAVE, b.FLAG_FORCE_COLWALK) and err.status == b.ERR_UNSUPPORTED
             continue
         assert b.workspace_status(got.workspace) == b.OK
         assert_parity(got, ref, shape, 1, mode, backward=True)
@@ -227,6 +227,72 @@ def test_l2wave_bounded_wait_reports_timeout(b, knobs):
     knobs(extra_arrivals=0, spin_limit=0)
     got = b.granq_fakequant_fused(to_dev(x), 4, gy=to_dev(gy), want_codes=True, want_mask=True, want_params=True,
                                   flags=b.FLAG_FORCE_L2WAVE)
+    assert b.workspace_status(got.workspace) == b.OK
+    assert_parity(got, orc.fused(x, 4, gy=gy), shape, 1, orc.GROUP_CHANNEL, backward=True)
+
+
+@pytest.mark.parametrize("shape", [(8, 16, 14, 14), (9, 8, 7, 7), (16, 12, 32, 32), (8, 40, 56, 56), (13, 24, 7, 7),
+                                   (300, 8, 5, 5), (8, 3, 4, 4), (40, 72, 3, 3)],
+                         ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_colwalk_multiwave(b, knobs, shape, dtype):
+    """The column-walk plan cut into many small waves, every lag, few and many CTAs."""
+    if dtype == "bf16" and ((shape[1] * shape[2] * shape[3]) % 8 != 0 or shape[2] * shape[3] < 8):
+        pytest.skip("slab not a whole number of 16-byte packs, or planes shorter than a pack")
+    x, gy = make_case(shape, seed=sum(shape) + 3, dtype=dtype)
+    bits = 2 + sum(shape) % 7
+    ref = orc.fused(x, bits, gy=gy)
+    ref_f = orc.fused(x, bits)
+    for wave_kb, cap, lag in ((1, 1, 1), (1, 0, 2), (8, 0, 3), (0, 0, 0)):
+        knobs(l2_wave_kb=wave_kb, l2_ctas_per_sm=cap, l2_lag=lag)
+        assert b.fused_plan(b.BF16 if dtype == "bf16" else b.F32, shape, flags=b.FLAG_FORCE_COLWALK)[0] == b.PLAN_COLWALK
+        got = b.granq_fakequant_fused(to_dev(x), bits, gy=to_dev(gy), want_codes=True, want_mask=True,
+                                      want_params=True, flags=b.FLAG_FORCE_COLWALK)
+        assert b.workspace_status(got.workspace) == b.OK
+        assert_parity(got, ref, shape, 1, orc.GROUP_CHANNEL, backward=True)
+        got = b.granq_fakequant_fused(to_dev(x), bits, flags=b.FLAG_FORCE_COLWALK)      # forward only, no extras
+        assert_parity(got, ref_f, shape, 1, orc.GROUP_CHANNEL, backward=False)
+
+
+def test_colwalk_needs_slabs_to_walk(b):
+    """Too few slabs (or the sample-channel / tensor views, which have one): left to the other plans."""
+    with pytest.raises(b.GranqError) as err:
+        b.granq_fakequant_fused(to_dev(make_case((2, 8, 8, 8), seed=1)[0]), 4, flags=b.FLAG_FORCE_COLWALK)
+    assert err.value.status == b.ERR_UNSUPPORTED
+    assert b.fused_plan(b.F32, (2, 8, 8, 8))[0] == b.PLAN_L2WAVE
+    assert b.fused_plan(b.F32, (64, 8, 8, 8))[0] == b.PLAN_COLWALK
+    assert b.fused_plan(b.F32, (64, 8, 8, 8), group=b.GROUP_SAMPLE_CHANNEL)[0] == b.PLAN_L2WAVE
+
+
+def test_colwalk_workspace_stays_zeroed(b, knobs):
+    """FLAG_WORKSPACE_ZEROED: a cleared workspace serves call after call without being cleared again,
+    also when plans, shapes sharing the workspace size, bit-widths and wave cuts alternate."""
+    shape = (16, 24, 14, 14)
+    x, gy = make_case(shape, seed=11)
+    x2, gy2 = make_case(shape, seed=12)
+    ws = b.make_workspace(to_dev(x), zeroed=True)
+    for k, (xx, gg, bits, extra, wave_kb) in enumerate([(x, gy, 4, 0, 0), (x2, gy2, 3, 0, 1), (x, None, 5, 0, 4),
+                                                        (x2, gy2, 6, b.FLAG_FORCE_TWO_PASS, 0),
+                                                        (x, gy, 2, b.FLAG_FORCE_L2WAVE, 0), (x2, gy2, 8, 0, 2)]):
+        knobs(l2_wave_kb=wave_kb)
+        out = b.FakeQuantOut(workspace=ws)
+        got = b.granq_fakequant_fused(to_dev(xx), bits, gy=None if gg is None else to_dev(gg), out=out,
+                                      want_codes=True, want_mask=True, want_params=True,
+                                      flags=b.FLAG_WORKSPACE_ZEROED | extra)
+        assert b.workspace_status(ws) == b.OK
+        assert_parity(got, orc.fused(xx, bits, gy=gg), shape, 1, orc.GROUP_CHANNEL, backward=gg is not None)
+        assert int(ws.view(torch.int32).abs().sum().item()) == 0, f"call {k} left the workspace dirty"
+
+
+def test_colwalk_bounded_wait_reports_timeout(b, knobs):
+    shape = (8, 16, 14, 14)
+    x, gy = make_case(shape, seed=2)
+    knobs(extra_arrivals=1, spin_limit=2000)
+    got = b.granq_fakequant_fused(to_dev(x), 4, gy=to_dev(gy), flags=b.FLAG_FORCE_COLWALK)
+    assert b.workspace_status(got.workspace) == b.ERR_TIMEOUT
+    knobs(extra_arrivals=0, spin_limit=0)
+    got = b.granq_fakequant_fused(to_dev(x), 4, gy=to_dev(gy), want_codes=True, want_mask=True, want_params=True,
+                                  flags=b.FLAG_FORCE_COLWALK)
     assert b.workspace_status(got.workspace) == b.OK
     assert_parity(got, orc.fused(x, 4, gy=gy), shape, 1, orc.GROUP_CHANNEL, backward=True)
 
