@@ -57,10 +57,14 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
+DOMINANT_KERNEL_SOURCES = ("granq_colwalk.cu", "granq_device.cuh", "granq_internal.h")
+
+
 def kernel_source_hash() -> str:
+    """Hash of the files the dominant kernel is compiled from."""
     h = hashlib.sha256()
     csrc = os.path.join(ROOT, "paper_2503_18339_b200", "csrc")
-    for name in sorted(os.listdir(csrc)):
+    for name in DOMINANT_KERNEL_SOURCES:
         with open(os.path.join(csrc, name), "rb") as fh:
             h.update(fh.read())
     return h.hexdigest()[:16]
@@ -69,7 +73,7 @@ def kernel_source_hash() -> str:
 def recorded_traffic():
     """DRAM bytes per launch of the dominant kernel from the committed ncu summary, or None
     when there is none or the kernel sources have changed since it was taken."""
-    path = os.path.join(ROOT, "profiles", "l2wave_kernel_traffic.txt")
+    path = os.path.join(ROOT, "profiles", "colwalk_kernel_traffic.txt")
     try:
         with open(path) as fh:
             rec = json.load(fh)
@@ -332,16 +336,16 @@ def main():
     # ---- per-call device times inside the timed region -> roofline of the dominant kernel ----
     per_call_ms = [statistics.mean(ev[k][ci][0].elapsed_time(ev[k][ci][1]) for k in range(args.steps))
                    for ci in range(len(calls))]
-    # dominant kernel: the L2-wave instantiation for long planes (>= 512 packs per plane, 4 packs per lane)
+    # dominant kernel: the column-walk instantiation for planes that are whole 16-byte packs (all but the 7x7 ones)
     dominant = [ci for ci, (i, _) in enumerate(calls) if (specs[i].shape[2] * specs[i].shape[3]) % 4 == 0
-                and specs[i].shape[2] * specs[i].shape[3] // 4 >= 512 and plans[ci][0] == b.PLAN_L2WAVE]
+                and plans[ci][0] == b.PLAN_COLWALK]
     dom_bytes = sum(specs[calls[ci][0]].numel for ci in dominant) * bpe
     dom_ms = sum(per_call_ms[ci] for ci in dominant)
     peak, peak_src = measured_peak()
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9 if dominant else None
     rec = recorded_traffic()
     roofline = {
-        "bound": "hbm", "kernel": "l2wave_kernel<float, fwd+bwd, aligned planes, 4 packs per lane>",
+        "bound": "hbm", "kernel": "colwalk_kernel<float, fwd+bwd, aligned planes>",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": (achieved / peak) if achieved else None,
         "peak_source": peak_src, "frac_of_nominal_8TBs": (achieved / NOMINAL_HBM_GBS) if achieved else None,
         "launches_per_step": len(dominant),
@@ -350,7 +354,7 @@ def main():
         "traffic": (rec["dram_bytes_per_algorithmic_byte"] * dom_bytes / max(1, len(dominant)) if rec else None),
         "traffic_source": (rec["source"] if rec else None),
         "share_of_step_time": dom_ms / sum(per_call_ms),
-        "note": "achieved = algorithmic bytes of the launches / their CUDA-event time (memset node included)",
+        "note": "achieved = algorithmic bytes of the launches / their CUDA-event time (launch gaps included)",
     }
     per_tensor = []
     for ci, (i, bits) in enumerate(calls):
