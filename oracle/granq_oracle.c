@@ -159,3 +159,27 @@ int granq_oracle_fused(const void* x, const void* gy, int dtype, const int64_t d
     return granq_oracle_fakequant(x, gy, dtype, dims, channel_axis, group_mode, bits,
                                   lo, hi, y, gx, codes, mask, s, z);
 }
+
+/* ---- mask-carrying split of forward and backward (Section 2.1: the STE needs only the mask) ---- */
+
+/* Bit e % 8 of byte e / 8 (least significant bit first) is mask[e] != 0; the unused high bits
+ * of a last partial byte are 0. */
+int granq_oracle_pack_mask(const uint8_t* mask, int64_t E, uint8_t* packed) {
+    if (!mask || !packed || E < 0) return -1;
+    for (int64_t b = 0; b < (E + 7) / 8; ++b) packed[b] = 0;
+    for (int64_t e = 0; e < E; ++e)
+        if (mask[e]) packed[e / 8] = (uint8_t)(packed[e / 8] | (1u << (e % 8)));
+    return 0;
+}
+
+/* STE backward from the packed mask alone: gx[e] = gy[e] where bit e is set, else +0. */
+int granq_oracle_bwd_packed(const void* gy, const uint8_t* packed, int dtype, int64_t E, void* gx) {
+    if (!gy || !packed || !gx || E < 0) return -1;
+    for (int64_t e = 0; e < E; ++e) {
+        int bit = (packed[e / 8] >> (e % 8)) & 1;
+        float gv = load_elem(gy, dtype, e);
+        store_elem(gx, dtype, e, bit ? gv : 0.0f);
+    }
+    return 0;
+}
+

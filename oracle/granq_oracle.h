@@ -66,6 +66,14 @@ int granq_oracle_fused(const void* x, const void* gy, int dtype, const int64_t d
                        void* y, void* gx, float* lo, float* hi,
                        uint8_t* codes, uint8_t* mask, float* s, float* z);
 
+/* Mask-carrying split of forward and backward (Section 2.1: the straight-through estimator
+ * needs nothing of the forward pass but the mask).  The forward pass stores its STE mask
+ * at one bit per element: bit e % 8 (least significant first) of byte e / 8, ceil(E / 8)
+ * bytes, unused high bits of the last byte 0.  The backward pass then reads gy and the
+ * packed mask instead of gy and x. */
+int granq_oracle_pack_mask(const uint8_t* mask, int64_t E, uint8_t* packed);
+int granq_oracle_bwd_packed(const void* gy, const uint8_t* packed, int dtype, int64_t E, void* gx);
+
 #ifdef __cplusplus
 }
 #endif

@@ -61,6 +61,10 @@ def lib() -> ctypes.CDLL:
         L.granq_oracle_fakequant.argtypes = [vp, vp, ci, i64p, ci, ci, ci, fp, fp, vp, vp, u8p, u8p, fp, fp]
         L.granq_oracle_fused.restype = ci
         L.granq_oracle_fused.argtypes = [vp, vp, ci, i64p, ci, ci, ci, vp, vp, fp, fp, u8p, u8p, fp, fp]
+        L.granq_oracle_pack_mask.restype = ci
+        L.granq_oracle_pack_mask.argtypes = [u8p, ctypes.c_int64, u8p]
+        L.granq_oracle_bwd_packed.restype = ci
+        L.granq_oracle_bwd_packed.argtypes = [vp, u8p, ci, ctypes.c_int64, vp]
         _lib = L
     return _lib
 
@@ -174,3 +178,25 @@ def fused(x: np.ndarray, bits: int, gy: Optional[np.ndarray] = None, channel_axi
                                     _p(y), _p(gx), _p(lo), _p(hi), _p(codes), _p(mask), _p(s), _p(z)),
            "granq_oracle_fused")
     return FakeQuantResult(y, gx, lo, hi, s, z, codes, mask)
+
+
+def pack_mask(mask: np.ndarray) -> np.ndarray:
+    """One bit per element, least significant bit first, ceil(E / 8) bytes (Section 2.1: all the
+    backward pass needs of the forward pass)."""
+    mask = np.ascontiguousarray(mask, np.uint8)
+    packed = np.empty((mask.size + 7) // 8, np.uint8)
+    _check(lib().granq_oracle_pack_mask(_p(mask), mask.size, _p(packed)), "granq_oracle_pack_mask")
+    return packed
+
+
+def bwd_packed(gy: np.ndarray, packed: np.ndarray) -> np.ndarray:
+    """STE backward from the packed mask alone: gx = gy where the bit is set, else +0."""
+    gy = np.ascontiguousarray(gy)
+    packed = np.ascontiguousarray(packed, np.uint8)
+    if packed.size != (gy.size + 7) // 8:
+        raise ValueError("packed mask must hold ceil(E / 8) bytes")
+    gx = np.empty_like(gy)
+    _check(lib().granq_oracle_bwd_packed(_p(gy), _p(packed), _dtype_of(gy), gy.size, _p(gx)),
+           "granq_oracle_bwd_packed")
+    return gx
+

@@ -23,6 +23,11 @@ MUTATIONS = {
     "bf16_ties_away": ("u += 0x7FFFu + lsb;", "u += 0x8000u;"),
     "no_degenerate_floor": ("if (!(s >= 1e-8f)) s = 1e-8f;", "if (!(s > 0.0f)) s = 1.0f;"),
     "gradient_not_masked": ("inside ? gv : 0.0f", "gv"),
+    "packed_mask_most_significant_bit_first": ("(1u << (e % 8))", "(0x80u >> (e % 8))"),
+    "packed_backward_reads_bits_in_reverse": ("(packed[e / 8] >> (e % 8)) & 1", "(packed[e / 8] >> (7 - e % 8)) & 1"),
+    "packed_backward_ignores_mask": ("bit ? gv : 0.0f", "gv"),
+    "packed_mask_last_byte_not_cleared": ("for (int64_t b = 0; b < (E + 7) / 8; ++b) packed[b] = 0;",
+                                          "for (int64_t b = 0; b < E / 8; ++b) packed[b] = 0;"),
 }
 
 

@@ -372,3 +372,56 @@ def test_bf16_backward_passes_bits_through():
     # ranges are the exact widened extremes
     wide = (xb.astype(np.uint32) << 16).view(np.float32)
     assert np.array_equal(res.lo, wide.min(axis=(0, 2, 3))) and np.array_equal(res.hi, wide.max(axis=(0, 2, 3)))
+
+
+# --------------------------------------------------------------------------------------
+# 9. mask-carrying split of forward and backward (Section 2.1): the packed 1-bit mask
+# --------------------------------------------------------------------------------------
+def test_packed_mask_hand_case():
+    """The stale-range hand case: mask [0,0,1,0,1,1,1,0 | 1], least significant bit first ->
+    byte 0 = 4 + 16 + 32 + 64 = 0x74, byte 1 = 0x01; the backward keeps gy at elements 2, 4, 5, 6, 8."""
+    case = next(c for c in HAND if c["name"] == "H6_stale_range")
+    x = f32(case["x"]).reshape(case["shape"])
+    res = orc.fakequant(x, case["bits"], f32(case["lo"]), f32(case["hi"]))
+    packed = orc.pack_mask(res.mask)
+    assert packed.tolist() == [0x74, 0x01]
+    gy = f32([10, 20, 30, 40, 50, 60, 70, 80, 90]).reshape(case["shape"])
+    assert orc.bwd_packed(gy, packed).ravel().tolist() == [0, 0, 30, 0, 50, 60, 70, 0, 90]
+
+
+@pytest.mark.parametrize("n", [0, 1, 7, 8, 9, 15, 16, 17, 63, 64, 65, 1000, 4099])
+def test_packed_mask_matches_numpy_bit_packing(n):
+    rng = np.random.default_rng(n)
+    m = (rng.random(n) < 0.7).astype(np.uint8)
+    packed = np.full((n + 7) // 8, 0xFF, np.uint8)          # pre-filled: the last partial byte must come out clean
+    packed[:] = orc.pack_mask(m)
+    assert np.array_equal(packed, np.packbits(m, bitorder="little"))
+    assert np.array_equal(np.unpackbits(packed, bitorder="little")[:n], m)
+    assert int(sum(bin(b).count("1") for b in packed.tolist())) == int(m.sum())
+    # any non-zero byte counts as set
+    assert np.array_equal(orc.pack_mask(m * 200), packed)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_backward_from_packed_mask_equals_backward_from_x(dtype):
+    """With the forward pass's own mask the split backward is the STE backward of the fused path,
+    for a range that clips on both sides; and gx is bitwise gy or +0."""
+    rng = np.random.default_rng(5)
+    shape = (3, 5, 7, 7)                                       # 735 elements: a last partial byte
+    x = rng.standard_normal(shape).astype(np.float32)
+    gy = rng.standard_normal(shape).astype(np.float32)
+    gy[0, 0, 0, :3] = [-0.0, 0.0, -1.5]
+    if dtype == "bf16":
+        x = (x.view(np.uint32) >> 16).astype(np.uint16)
+        gy = (gy.view(np.uint32) >> 16).astype(np.uint16)
+    lo = np.full(5, -0.5, np.float32)
+    hi = np.full(5, 0.8, np.float32)
+    ref = orc.fakequant(x, 3, lo, hi, gy=gy)
+    assert 0 < ref.mask.sum() < ref.mask.size
+    packed = orc.pack_mask(ref.mask)
+    gx = orc.bwd_packed(gy, packed)
+    u = np.uint16 if dtype == "bf16" else np.uint32
+    assert np.array_equal(gx.view(u), ref.gx.view(u))
+    bits = np.unpackbits(packed, bitorder="little")[:x.size].reshape(shape).astype(bool)
+    assert np.array_equal(gx.view(u), np.where(bits, gy.view(u), u(0)))
+
