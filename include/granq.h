@@ -172,6 +172,44 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
                           void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream);
 
 /*
+ * Mask-carrying split of forward and backward (Section 2.1: the straight-through estimator
+ * needs nothing of the forward pass but where the clamp was inactive).  In training the
+ * upstream gradient does not exist yet when the forward pass runs, so the forward pass
+ * stores its mask at ONE BIT per element and the backward pass reads gy and that mask
+ * instead of gy and x: 8.125 instead of 12 bytes per fp32 element.
+ *
+ * Packed mask layout: bit e % 32 of the 32-bit word e / 32 (on this little-endian target the
+ * same as bit e % 8 of byte e / 8) is 1 iff 0 <= round(x_e / s + z) <= 2^b - 1.  The buffer
+ * holds granq_packmask_bytes() = 4 * ceil(E / 32) bytes, 4-byte aligned, DEVICE memory; bits
+ * beyond element E - 1 are written as 0.
+ */
+size_t granq_packmask_bytes(const int64_t dims[4]);
+
+/* Eq. 1 + clamp + Eq. 6 with a supplied range, as granq_fakequant_fwd(), also writing the packed mask.
+ *   x in E elements;  y out E elements;  packed_mask out;  scale_opt, zp_opt G floats or NULL */
+int granq_fakequant_fwd_packmask(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                                 int bits, const float* min_in, const float* max_in, void* y,
+                                 uint32_t* packed_mask, float* scale_opt, float* zp_opt, uint32_t flags,
+                                 void* cuda_stream);
+
+/* STE backward from the packed mask alone: gx_e = gy_e where bit e is set, else +0.  Needs neither x
+ * nor the range, hence no channel axis or grouping.
+ *   gy in E elements;  packed_mask in;  gx out E elements (must not overlap gy) */
+int granq_fakequant_bwd_packmask(const void* gy, const uint32_t* packed_mask, int dtype, const int64_t dims[4],
+                                 void* gx, uint32_t flags, void* cuda_stream);
+
+/* The forward half of the whole path in one call (Algorithm 1, range step through pre-scale step):
+ * range of x itself -> scale / zero-point -> y and the packed mask.  Takes the column-walk plan
+ * when slabs and waves are whole mask words, else a range pass followed by an elementwise pass
+ * (GRANQ_FLAG_FORCE_TWO_PASS / GRANQ_FLAG_FORCE_COLWALK select one; GRANQ_FLAG_WORKSPACE_ZEROED
+ * as for granq_fakequant_fused()).
+ *   min_out, max_out out G floats each (required);  scale_opt, zp_opt G floats or NULL */
+int granq_fakequant_fused_fwd_packmask(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                                       int bits, void* y, uint32_t* packed_mask, float* min_out, float* max_out,
+                                       float* scale_opt, float* zp_opt, void* workspace, size_t workspace_bytes,
+                                       uint32_t flags, void* cuda_stream);
+
+/*
  * Status word the persistent plans leave in the workspace.  Synchronises `cuda_stream`, then
  * returns GRANQ_OK, GRANQ_ERR_TIMEOUT (a bounded device-side wait ran out), or
  * GRANQ_ERR_CUDA.  `workspace` is the pointer given to the preceding call.

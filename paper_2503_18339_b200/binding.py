@@ -30,7 +30,8 @@ EXPORTS = [
     "granq_status_string", "granq_num_groups", "granq_workspace_bytes", "granq_range",
     "granq_fakequant_fwd", "granq_fakequant_bwd", "granq_fakequant_fused", "granq_workspace_status",
     "granq_host_arena_bytes", "granq_fakequant_fused_host", "granq_fused_plan", "granq_staged_geometry",
-    "granq_tune", "granq_selftest_division", "granq_range_noalloc",
+    "granq_tune", "granq_selftest_division", "granq_range_noalloc", "granq_packmask_bytes",
+    "granq_fakequant_fwd_packmask", "granq_fakequant_bwd_packmask", "granq_fakequant_fused_fwd_packmask",
 ]
 NOALLOC_MAX_GROUPS = 32768
 
@@ -87,6 +88,15 @@ def lib() -> ctypes.CDLL:
         L.granq_range_noalloc.argtypes = [vp, ci, i64p, ci, ci, vp, vp, vp]
         L.granq_tune.restype = ci
         L.granq_tune.argtypes = [ci, ci]
+        L.granq_packmask_bytes.restype = sz
+        L.granq_packmask_bytes.argtypes = [i64p]
+        L.granq_fakequant_fwd_packmask.restype = ci
+        L.granq_fakequant_fwd_packmask.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, u32, vp]
+        L.granq_fakequant_bwd_packmask.restype = ci
+        L.granq_fakequant_bwd_packmask.argtypes = [vp, vp, ci, i64p, vp, u32, vp]
+        L.granq_fakequant_fused_fwd_packmask.restype = ci
+        L.granq_fakequant_fused_fwd_packmask.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, sz,
+                                                         u32, vp]
         _lib = L
     return _lib
 
@@ -194,6 +204,7 @@ class FakeQuantOut:
     codes: Optional[torch.Tensor] = None
     mask: Optional[torch.Tensor] = None
     workspace: Optional[torch.Tensor] = None
+    packed_mask: Optional[torch.Tensor] = None      # int32 words, one bit per element
 
 
 def granq_range(x: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL, lo: torch.Tensor = None,
@@ -289,6 +300,74 @@ def granq_fakequant_fused(x: torch.Tensor, bits: int, gy: torch.Tensor = None, c
         _dev(o.y, "y"), _dev(o.gx if gy is not None else None, "gx"), _dev(o.lo, "lo"), _dev(o.hi, "hi"),
         _dev(o.codes, "codes"), _dev(o.mask if gy is not None else None, "mask"), _dev(o.s, "s"), _dev(o.z, "z"),
         _dev(o.workspace, "workspace"), o.workspace.numel(), flags, _stream(stream)), "granq_fakequant_fused")
+    return o
+
+
+def packmask_bytes(shape) -> int:
+    return int(lib().granq_packmask_bytes(_dims(shape)))
+
+
+def make_packed_mask(x: torch.Tensor) -> torch.Tensor:
+    """Buffer for the STE mask of x at one bit per element (int32 words)."""
+    return torch.empty(packmask_bytes(x.shape) // 4, dtype=torch.int32, device=x.device)
+
+
+def granq_fakequant_fwd_packmask(x: torch.Tensor, bits: int, lo: torch.Tensor, hi: torch.Tensor,
+                                 channel_axis: int = 1, group: int = GROUP_CHANNEL, y: torch.Tensor = None,
+                                 packed_mask: torch.Tensor = None, want_params: bool = False, flags: int = 0,
+                                 stream=None) -> FakeQuantOut:
+    """Forward with a given range that also stores the STE mask at one bit per element (Section 2.1)."""
+    G = num_groups(x.shape, channel_axis, group)
+    o = FakeQuantOut(lo=lo, hi=hi)
+    o.y = torch.empty_like(x) if y is None else y
+    o.packed_mask = make_packed_mask(x) if packed_mask is None else packed_mask
+    if want_params:
+        o.s = torch.empty(G, dtype=torch.float32, device=x.device)
+        o.z = torch.empty(G, dtype=torch.float32, device=x.device)
+    _check(lib().granq_fakequant_fwd_packmask(_dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, bits,
+                                              _dev(lo, "lo"), _dev(hi, "hi"), _dev(o.y, "y"),
+                                              _dev(o.packed_mask, "packed_mask"), _dev(o.s, "s"), _dev(o.z, "z"),
+                                              flags, _stream(stream)), "granq_fakequant_fwd_packmask")
+    return o
+
+
+def granq_fakequant_bwd_packmask(gy: torch.Tensor, packed_mask: torch.Tensor, gx: torch.Tensor = None,
+                                 flags: int = 0, stream=None) -> torch.Tensor:
+    """STE backward from the packed mask alone: gx = gy where the bit is set, else 0."""
+    if packed_mask.numel() * packed_mask.element_size() < packmask_bytes(gy.shape):
+        raise ValueError("packed mask too small for gy")
+    gx = torch.empty_like(gy) if gx is None else gx
+    _check(lib().granq_fakequant_bwd_packmask(_dev(gy, "gy"), _dev(packed_mask, "packed_mask"), _dtype(gy),
+                                              _dims(gy.shape), _dev(gx, "gx"), flags, _stream(stream)),
+           "granq_fakequant_bwd_packmask")
+    return gx
+
+
+def granq_fakequant_fused_fwd_packmask(x: torch.Tensor, bits: int, channel_axis: int = 1,
+                                       group: int = GROUP_CHANNEL, out: FakeQuantOut = None,
+                                       want_params: bool = False, flags: int = 0, stream=None) -> FakeQuantOut:
+    """Range of x itself -> scale / zero-point -> y and the packed STE mask, in one call."""
+    G = num_groups(x.shape, channel_axis, group)
+    o = out if out is not None else FakeQuantOut()
+    dev = x.device
+    if o.y is None:
+        o.y = torch.empty_like(x)
+    if o.packed_mask is None:
+        o.packed_mask = make_packed_mask(x)
+    if o.lo is None:
+        o.lo = torch.empty(G, dtype=torch.float32, device=dev)
+    if o.hi is None:
+        o.hi = torch.empty(G, dtype=torch.float32, device=dev)
+    if want_params and o.s is None:
+        o.s = torch.empty(G, dtype=torch.float32, device=dev)
+        o.z = torch.empty(G, dtype=torch.float32, device=dev)
+    if o.workspace is None:
+        o.workspace = make_workspace(x, channel_axis, group)
+    _check(lib().granq_fakequant_fused_fwd_packmask(
+        _dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, bits, _dev(o.y, "y"),
+        _dev(o.packed_mask, "packed_mask"), _dev(o.lo, "lo"), _dev(o.hi, "hi"), _dev(o.s, "s"), _dev(o.z, "z"),
+        _dev(o.workspace, "workspace"), o.workspace.numel(), flags, _stream(stream)),
+        "granq_fakequant_fused_fwd_packmask")
     return o
 
 

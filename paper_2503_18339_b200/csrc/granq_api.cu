@@ -238,6 +238,86 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
     return cuda_status(e);
 }
 
+size_t granq_packmask_bytes(const int64_t dims[4]) {
+    Geom g;
+    int64_t G;
+    if (!make_geom(dims, 1, GRANQ_GROUP_TENSOR, g, G)) return 0;
+    return (size_t)((g.E + 31) / 32) * 4;
+}
+
+int granq_fakequant_fwd_packmask(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                                 int bits, const float* min_in, const float* max_in, void* y,
+                                 uint32_t* packed_mask, float* scale_opt, float* zp_opt, uint32_t flags,
+                                 void* cuda_stream) {
+    (void)flags;
+    Geom g;
+    int64_t G;
+    if (!x || !y || !packed_mask || !min_in || !max_in || bits < 1 || bits > 8 || !dtype_ok(dtype) ||
+        !make_geom(dims, channel_axis, group, g, G) || ((uintptr_t)packed_mask & 3))
+        return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
+    const size_t nb = (size_t)g.E * elt_size(dtype), mb = (size_t)((g.E + 31) / 32) * 4;
+    if (overlaps(x, nb, y, nb) || overlaps(x, nb, packed_mask, mb) || overlaps(y, nb, packed_mask, mb))
+        return GRANQ_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    QuantIO io{x, nullptr, y, nullptr, nullptr, nullptr, packed_mask};
+    cudaError_t e = launch_quant_flat(io, MODE_FWD, dtype, g, bits, min_in, max_in, st);
+    if (e == cudaSuccess && (scale_opt || zp_opt)) e = launch_params(min_in, max_in, G, bits, scale_opt, zp_opt, st);
+    return cuda_status(e);
+}
+
+int granq_fakequant_bwd_packmask(const void* gy, const uint32_t* packed_mask, int dtype, const int64_t dims[4],
+                                 void* gx, uint32_t flags, void* cuda_stream) {
+    (void)flags;
+    Geom g;
+    int64_t G;
+    if (!gy || !gx || !packed_mask || !dtype_ok(dtype) || !make_geom(dims, 1, GRANQ_GROUP_TENSOR, g, G) ||
+        ((uintptr_t)packed_mask & 3))
+        return GRANQ_ERR_INVALID_ARG;
+    const size_t nb = (size_t)g.E * elt_size(dtype), mb = (size_t)((g.E + 31) / 32) * 4;
+    if (overlaps(gy, nb, gx, nb) || overlaps(packed_mask, mb, gx, nb)) return GRANQ_ERR_INVALID_ARG;
+    return cuda_status(launch_bwd_packmask(gy, packed_mask, gx, dtype, g.E, (cudaStream_t)cuda_stream));
+}
+
+int granq_fakequant_fused_fwd_packmask(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                                       int bits, void* y, uint32_t* packed_mask, float* min_out, float* max_out,
+                                       float* scale_opt, float* zp_opt, void* workspace, size_t workspace_bytes,
+                                       uint32_t flags, void* cuda_stream) {
+    Geom g;
+    int64_t G;
+    if (!x || !y || !packed_mask || !min_out || !max_out || bits < 1 || bits > 8 || !dtype_ok(dtype) ||
+        !make_geom(dims, channel_axis, group, g, G) || ((uintptr_t)packed_mask & 3))
+        return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
+    const size_t nb = (size_t)g.E * elt_size(dtype), mb = (size_t)((g.E + 31) / 32) * 4;
+    if (overlaps(x, nb, y, nb) || overlaps(x, nb, packed_mask, mb) || overlaps(y, nb, packed_mask, mb))
+        return GRANQ_ERR_INVALID_ARG;
+    if (int rc = check_workspace(workspace, workspace_bytes, G)) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    QuantIO io{x, nullptr, y, nullptr, nullptr, nullptr, packed_mask};
+    // the column-walk kernel where the geometry allows whole mask words per wave, else range pass + flat pass
+    ColPlan cp{};
+    const bool two_pass = (flags & GRANQ_FLAG_FORCE_TWO_PASS) != 0;
+    if (!two_pass) cp = plan_colwalk(dtype, g, io, g_tune);
+    if ((flags & GRANQ_FLAG_FORCE_COLWALK) && !cp.ok) return GRANQ_ERR_UNSUPPORTED;
+    Workspace ws = carve_workspace(workspace, G);
+    const bool zeroed = (flags & GRANQ_FLAG_WORKSPACE_ZEROED) != 0;
+    cudaError_t e = cudaSuccess;
+    if (!(zeroed && cp.ok)) e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
+    if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+    if (cp.ok) {
+        e = launch_colwalk(cp, io, MODE_FWD, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
+    } else {
+        e = launch_range_flat(x, dtype, g, ws.kmin, ws.kmax, st);
+        if (e == cudaSuccess)
+            e = launch_finalize_range(ws.kmin, ws.kmax, G, min_out, max_out, bits, scale_opt, zp_opt, st);
+        if (e == cudaSuccess) e = launch_quant_flat(io, MODE_FWD, dtype, g, bits, min_out, max_out, st);
+        if (e == cudaSuccess && zeroed)
+            e = cudaMemsetAsync((char*)workspace + sizeof(uint32_t), 0, ws.clear_bytes - sizeof(uint32_t), st);
+    }
+    return cuda_status(e);
+}
+
 int granq_workspace_status(const void* workspace, void* cuda_stream) {
     if (!workspace) return GRANQ_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;

@@ -49,6 +49,7 @@ struct CArgs {
     void* gx;
     uint8_t* codes;
     uint8_t* mask;
+    uint32_t* pmask;       // mask at one bit per element, or null
     uint32_t* status;
     uint32_t* kmin;
     uint32_t* kmax;
@@ -313,6 +314,19 @@ __global__ void __launch_bounds__(kCThreads, 4) colwalk_kernel(const CArgs a) {
 #pragma unroll
                         for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.mask)[at * (V / 4) + i] = mb[i];
                     }
+                    if (a.pmask) {
+                        // 32 / V neighbouring lanes own the 32 elements of one mask word; the planner has made
+                        // every slab and wave a whole number of words, so such a group of lanes is here together
+                        constexpr uint32_t kLanes = 32 / V;
+                        const uint32_t members = ((1u << kLanes) - 1u) << (lane & ~(kLanes - 1));
+                        uint32_t bits = 0;
+#pragma unroll
+                        for (int i = 0; i < V; ++i) bits |= ((mb[i / 4] >> (8 * (i % 4))) & 1u) << i;
+                        uint32_t wv = bits << (V * (lane & (kLanes - 1)));
+#pragma unroll
+                        for (uint32_t d = 1; d < kLanes; d <<= 1) wv |= __shfl_xor_sync(members, wv, d);
+                        if ((lane & (kLanes - 1)) == 0) a.pmask[(at * V) >> 5] = wv;
+                    }
                 }
             };
             uint32_t n = it.n0;
@@ -459,7 +473,9 @@ ColPlan plan_colwalk(int dtype, const Geom& g, const QuantIO& io, const StagedTu
     if (g.inner < (int64_t)V || g.inner >= (1ll << 28) || g.C >= (1ll << 28)) return p;
     if ((g.C * g.inner) % V != 0 || g.E / V >= (1ll << 31)) return p;
     const uint32_t inner = (uint32_t)g.inner, C = (uint32_t)g.C;
-    const uint32_t q = V / c_gcd(inner, V);
+    // waves are whole 16-byte units; with a packed mask also whole 32-element mask words
+    if (io.pmask && (((uintptr_t)io.pmask & 3) || (g.C * g.inner) % 32 != 0)) return p;
+    const uint32_t q = io.pmask ? 32 / c_gcd(inner, 32) : V / c_gcd(inner, V);
     const uint64_t target = (tune.l2_wave_kb > 0 ? (uint64_t)tune.l2_wave_kb : 32ull * 1024) * 1024;
     const uint64_t group_bytes = (uint64_t)g.outer * inner * (16 / V);           // x bytes of one channel group
     const uint32_t mult_total = C / q;
@@ -509,6 +525,7 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
     a.gx = io.gx;
     a.codes = io.codes;
     a.mask = io.mask;
+    a.pmask = io.pmask;
     a.status = ws.status;
     a.kmin = ws.kmin;
     a.kmax = ws.kmax;
@@ -540,7 +557,7 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
     }
     const bool aligned = (inner % V) == 0;
     a.div_plane = make_fastdiv(aligned ? inner / V : inner);
-    const bool extras = io.codes != nullptr || io.mask != nullptr;
+    const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr;
     const int cap = tune.l2_ctas_per_sm;
     if (dtype == 0) {
         if (mode == MODE_FWD) return c_launch_mode<float, MODE_FWD>(a, aligned, extras, sms, cap, st);

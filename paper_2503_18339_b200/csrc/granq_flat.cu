@@ -242,12 +242,15 @@ __global__ void params_kernel(const float* __restrict__ lo, const float* __restr
 }
 
 // ---- Eq. 1, clamp, Eq. 6, STE: elementwise pass with a given per-group range ----------------------
-// EXTRAS: the optional codes / mask outputs are compiled in
+// EXTRAS: the optional codes / mask / packed-mask outputs are compiled in.  The packed mask holds
+// one bit per element (bit e % 32 of word e / 32): a warp's lanes own consecutive elements or packs
+// starting at a multiple of 32 elements, so whole words are assembled with warp shuffles.
 template <typename T, int V, int MODE, bool EXTRAS>
 __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restrict__ x, const T* __restrict__ gy,
                                                               T* __restrict__ y, T* __restrict__ gx,
                                                               uint8_t* __restrict__ codes,
-                                                              uint8_t* __restrict__ mask, FlatGeom g, float qmax,
+                                                              uint8_t* __restrict__ mask,
+                                                              uint32_t* __restrict__ pmask, FlatGeom g, float qmax,
                                                               const float* __restrict__ lo,
                                                               const float* __restrict__ hi) {
     __shared__ TileBase s_base;
@@ -291,7 +294,9 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
             }
 #pragma unroll
             for (int j = 0; j < kUnroll; ++j) {
-                if (k[j] >= ne) continue;
+                const bool valid = k[j] < ne;
+                uint32_t inside_bits = 0;            // bit i: the clamp was inactive for this thread's element i
+                if (valid) {
                 const uint32_t q = plane_offset(g, base, k[j]);
                 QParam p;
                 float rcp = 0.0f;            // reciprocal of the scale when the short division applies
@@ -308,6 +313,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                     float yv;
                     bool in;
                     float code = quant_one(sx[j], p, qmax, yv, in);
+                    inside_bits = in ? 1u : 0u;
                     if constexpr (kFwd) {
                         store_scalar(y + e, yv);
                         if (codes) codes[e] = (uint8_t)code;
@@ -325,6 +331,10 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                     for (int i = 0; i < V; ++i) amax = fmaxf(amax, fabsf(px[j].get(i)));
                     GroupParam gp{p.s, p.z, (amax <= 1152921504606846976.0f) ? rcp : 0.0f};
                     quantize_pack<T, kBwd, false, EXTRAS>(px[j], pg[j], gp, gp, V, qmax, py, pgx, cb, mb);
+                    if constexpr (EXTRAS) {
+#pragma unroll
+                        for (int i = 0; i < V; ++i) inside_bits |= ((mb[i / 4] >> (8 * (i % 4))) & 1u) << i;
+                    }
                     if constexpr (kFwd) {
                         st_stream_16(y + e, py.raw);
                         if constexpr (EXTRAS) {
@@ -341,6 +351,23 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
 #pragma unroll
                                 for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(mask + e)[i] = mb[i];
                             }
+                        }
+                    }
+                }
+                }
+                if constexpr (EXTRAS && kFwd) {
+                    if (pmask) {          // every lane of the warp is here: assemble whole 32-bit words
+                        const uint32_t lane = threadIdx.x & 31;
+                        const int64_t word = (e0 + k[j]) >> 5;
+                        if constexpr (V == 1) {
+                            const uint32_t w = __ballot_sync(kFullMask, inside_bits != 0);
+                            if (lane == 0 && valid) pmask[word] = w;
+                        } else {
+                            constexpr uint32_t kLanes = 32 / V;             // lanes that share one word
+                            uint32_t w = inside_bits << (V * (lane & (kLanes - 1)));
+#pragma unroll
+                            for (uint32_t d = 1; d < kLanes; d <<= 1) w |= __shfl_xor_sync(kFullMask, w, d);
+                            if ((lane & (kLanes - 1)) == 0 && valid) pmask[word] = w;
                         }
                     }
                 }
@@ -400,6 +427,44 @@ __global__ void __launch_bounds__(kThreads) naive_quant_kernel(const T* __restri
     }
 }
 
+// ---- STE backward from the packed mask alone (Section 2.1): gx = gy where the element's bit is set ----
+// V = elements per thread and step: a 16-byte pack when E and the pointers allow it, else 1.
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads) bwd_packmask_kernel(const T* __restrict__ gy,
+                                                                const uint32_t* __restrict__ pmask,
+                                                                T* __restrict__ gx, int64_t E) {
+    const int64_t nunits = E / V;
+    const int64_t stride = (int64_t)gridDim.x * kThreads * kUnroll;
+    for (int64_t u0 = (int64_t)blockIdx.x * kThreads * kUnroll; u0 < nunits; u0 += stride) {
+        int64_t e[kUnroll];
+        Pack<T> pg[kUnroll];
+        float sg[kUnroll];
+        uint32_t w[kUnroll];
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) {
+            e[j] = (u0 + j * kThreads + threadIdx.x) * V;
+            if (e[j] < E) {
+                if constexpr (V == 1) sg[j] = load_scalar(gy + e[j]);
+                else pg[j].raw = ld_stream_16(gy + e[j]);
+                w[j] = __ldg(pmask + (e[j] >> 5));
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < kUnroll; ++j) {
+            if (e[j] >= E) continue;
+            const uint32_t bits = w[j] >> (uint32_t)(e[j] & 31);
+            if constexpr (V == 1) {
+                store_scalar(gx + e[j], (bits & 1u) ? sg[j] : 0.0f);
+            } else {
+                Pack<T> out;
+#pragma unroll
+                for (int i = 0; i < V; ++i) out.set(i, ((bits >> i) & 1u) ? pg[j].get(i) : 0.0f);
+                st_stream_16(gx + e[j], out.raw);
+            }
+        }
+    }
+}
+
 bool aligned16(const void* p) { return p == nullptr || ((uintptr_t)p & 15) == 0; }
 
 int flat_grid(const FlatGeom& f) {
@@ -454,16 +519,16 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
                ((uintptr_t)io.codes % 4 == 0) && ((uintptr_t)io.mask % 4 == 0);
     int grid = flat_grid(f);
     float qmax = (float)((1 << bits) - 1);
-    const bool extras = io.codes != nullptr || io.mask != nullptr;
+    const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr;
     if (vec && extras)
         quant_flat_kernel<T, VF, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                        (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
+                                                                        (T*)io.gx, io.codes, io.mask, io.pmask, f, qmax, lo, hi);
     else if (vec)
         quant_flat_kernel<T, VF, MODE, false><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                         (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
+                                                                         (T*)io.gx, io.codes, io.mask, io.pmask, f, qmax, lo, hi);
     else
         quant_flat_kernel<T, 1, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                       (T*)io.gx, io.codes, io.mask, f, qmax, lo, hi);
+                                                                       (T*)io.gx, io.codes, io.mask, io.pmask, f, qmax, lo, hi);
     return cudaGetLastError();
 }
 
@@ -528,6 +593,32 @@ cudaError_t launch_naive(const QuantIO& io, int mode, int dtype, const Geom& g, 
     }
     if (mode == MODE_FWD) return naive_t<__nv_bfloat16, MODE_FWD>(io, g, bits, kmin, kmax, lo, hi, st, launches);
     return naive_t<__nv_bfloat16, MODE_BOTH>(io, g, bits, kmin, kmax, lo, hi, st, launches);
+}
+
+cudaError_t launch_bwd_packmask(const void* gy, const uint32_t* pmask, void* gx, int dtype, int64_t E,
+                                cudaStream_t st) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int VF = dtype == 0 ? 4 : 8;
+    const bool vec = aligned16(gy) && aligned16(gx) && (E % VF == 0);
+    const int64_t units = vec ? E / VF : E;
+    const int64_t per_cta = (int64_t)kThreads * kUnroll;
+    int64_t ctas = (units + per_cta - 1) / per_cta;
+    const int64_t cap = (int64_t)sms * 16;
+    const int grid = (int)(ctas < 1 ? 1 : (ctas < cap ? ctas : cap));
+    if (dtype == 0) {
+        if (vec) bwd_packmask_kernel<float, 4><<<grid, kThreads, 0, st>>>((const float*)gy, pmask, (float*)gx, E);
+        else bwd_packmask_kernel<float, 1><<<grid, kThreads, 0, st>>>((const float*)gy, pmask, (float*)gx, E);
+    } else {
+        if (vec)
+            bwd_packmask_kernel<__nv_bfloat16, 8><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)gy, pmask,
+                                                                             (__nv_bfloat16*)gx, E);
+        else
+            bwd_packmask_kernel<__nv_bfloat16, 1><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)gy, pmask,
+                                                                             (__nv_bfloat16*)gx, E);
+    }
+    return cudaGetLastError();
 }
 
 }  // namespace granq

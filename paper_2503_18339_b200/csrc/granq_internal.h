@@ -53,6 +53,7 @@ struct QuantIO {
     void* gx;         // MODE_BWD / MODE_BOTH
     uint8_t* codes;   // optional
     uint8_t* mask;    // optional
+    uint32_t* pmask;  // optional: the mask at one bit per element (forward plans that support it)
 };
 
 // ---- generic ("flat") kernels: any geometry, any alignment --------------------------------
@@ -68,6 +69,9 @@ cudaError_t launch_params(const float* lo, const float* hi, int64_t G, int bits,
 // elementwise quantize / backward with a per-group range in lo / hi
 cudaError_t launch_quant_flat(const QuantIO& io, int mode, int dtype, const Geom& g, int bits, const float* lo,
                               const float* hi, cudaStream_t st);
+// STE backward from the mask at one bit per element (bit e % 32 of word e / 32)
+cudaError_t launch_bwd_packmask(const void* gy, const uint32_t* pmask, void* gx, int dtype, int64_t E,
+                                cudaStream_t st);
 // the "conventional" scheme: a host loop over groups with three launches each
 cudaError_t launch_naive(const QuantIO& io, int mode, int dtype, const Geom& g, int bits, uint32_t* kmin,
                          uint32_t* kmax, float* lo, float* hi, cudaStream_t st, int* launches);
