@@ -208,8 +208,10 @@ def main():
     ap.add_argument("--tune", default="", help="planner overrides for experiments, e.g. depth=3,max_buf_units=4000")
     ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged", "l2wave", "colwalk"],
                     help="force an execution plan of the fused entry point (experiments)")
-    ap.add_argument("--op", default="fused", choices=["fused", "range", "fwd", "bwd"],
-                    help="time another entry point instead of the fused one (experiments; bytes/element 4, 8, 12)")
+    ap.add_argument("--op", default="fused", choices=["fused", "range", "fwd", "bwd", "fused_fwd_packmask",
+                                                      "bwd_packmask"],
+                    help="time another entry point instead of the fused one (bytes/element 4, 8, 12; 8.125 for the "
+                         "two halves of the mask-carrying split)")
     ap.add_argument("--clear-workspace", action="store_true",
                     help="let every call clear its workspace (one more memset node per call) instead of "
                          "passing GRANQ_FLAG_WORKSPACE_ZEROED")
@@ -272,11 +274,16 @@ def main():
     launches_per_step = sum(n for _, n in plans)
     stream = torch.cuda.current_stream()
 
-    bpe = {"fused": 16, "range": 4, "fwd": 8, "bwd": 12}[args.op]
-    bytes_per_step = elems_per_step * bpe
+    bpe = {"fused": 16, "range": 4, "fwd": 8, "bwd": 12, "fused_fwd_packmask": 8.125, "bwd_packmask": 8.125}[args.op]
+    bytes_per_step = int(elems_per_step * bpe)
+    if args.op.endswith("packmask"):
+        for x, gy, out in dev:
+            out.packed_mask = b.make_packed_mask(x)
     if args.op != "fused":          # the stand-alone entry points need a range: take each tensor's own
         for x, gy, out in dev:
             b.granq_fakequant_fused(x, 4, gy=gy, out=out, stream=stream)
+            if args.op == "bwd_packmask":
+                b.granq_fakequant_fused_fwd_packmask(x, 4, out=out, stream=stream)
 
     def step(events=None):
         for ci, (i, bits) in enumerate(calls):
@@ -289,6 +296,10 @@ def main():
                 b.granq_range(x, lo=out.lo, hi=out.hi, workspace=out.workspace, stream=stream)
             elif args.op == "fwd":
                 b.granq_fakequant_fwd(x, bits, out.lo, out.hi, y=out.y, stream=stream)
+            elif args.op == "fused_fwd_packmask":
+                b.granq_fakequant_fused_fwd_packmask(x, bits, out=out, flags=flags, stream=stream)
+            elif args.op == "bwd_packmask":
+                b.granq_fakequant_bwd_packmask(gy, out.packed_mask, gx=out.gx, stream=stream)
             else:
                 b.granq_fakequant_bwd(gy, x, bits, out.lo, out.hi, gx=out.gx, stream=stream)
             if events is not None:

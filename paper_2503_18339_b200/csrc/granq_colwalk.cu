@@ -548,6 +548,7 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
     a.expected = (uint32_t)(tune.extra_arrivals > 0 ? tune.extra_arrivals : 0);   // + grid, added at launch
     const uint32_t c_last = C - (plan.nwaves - 1) * plan.cw;
     const uint32_t ch[2] = {plan.nwaves > 1 ? plan.cw : c_last, c_last};
+    const bool aligned = (inner % V) == 0;
     for (int i = 0; i < 2; ++i) {
         CShape& s = a.shape[i];
         s.channels = ch[i];
@@ -555,7 +556,6 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
         s.ncol = (s.units + kCThreads - 1) / kCThreads;
         s.div_ncol = make_fastdiv(s.ncol);
     }
-    const bool aligned = (inner % V) == 0;
     a.div_plane = make_fastdiv(aligned ? inner / V : inner);
     const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr;
     const int cap = tune.l2_ctas_per_sm;

@@ -243,7 +243,7 @@ def test_colwalk_multiwave(b, knobs, shape, dtype):
     bits = 2 + sum(shape) % 7
     ref = orc.fused(x, bits, gy=gy)
     ref_f = orc.fused(x, bits)
-    for wave_kb, cap, lag in ((1, 1, 1), (1, 0, 2), (8, 0, 3), (0, 0, 0)):
+    for wave_kb, cap, lag in ((1, 1, 1), (1, 0, 2), (8, 0, 3), (0, 0, 0), (2, 2, 1)):
         knobs(l2_wave_kb=wave_kb, l2_ctas_per_sm=cap, l2_lag=lag)
         assert b.fused_plan(b.BF16 if dtype == "bf16" else b.F32, shape, flags=b.FLAG_FORCE_COLWALK)[0] == b.PLAN_COLWALK
         got = b.granq_fakequant_fused(to_dev(x), bits, gy=to_dev(gy), want_codes=True, want_mask=True,
