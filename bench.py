@@ -377,35 +377,58 @@ def main():
     # ---- end to end through the host-buffer entry point (pinned memory, copies timed) ----
     e2e = None
     if args.e2e_steps > 0:
+        # Two streams, each with its own arena and host result buffers: while one call's results go
+        # down to the host the next call's inputs go up (PCIe is full duplex).
         big = max(specs, key=lambda s: s.numel)
-        arena = torch.empty(b.host_arena_bytes(b.F32, big.shape), dtype=torch.uint8, device="cuda")
-        yh = torch.empty(big.shape, dtype=torch.float32).pin_memory()
-        gxh = torch.empty(big.shape, dtype=torch.float32).pin_memory()
         cmax = max(s.shape[1] for s in specs)
-        loh, hih = torch.empty(cmax).pin_memory(), torch.empty(cmax).pin_memory()
+        lanes = []
+        for _ in range(2):
+            lanes.append({
+                "stream": torch.cuda.Stream(),
+                "arena": torch.empty(b.host_arena_bytes(b.F32, big.shape), dtype=torch.uint8, device="cuda"),
+                "y": torch.empty(big.shape, dtype=torch.float32).pin_memory(),
+                "gx": torch.empty(big.shape, dtype=torch.float32).pin_memory(),
+                "lo": torch.empty(cmax).pin_memory(), "hi": torch.empty(cmax).pin_memory(), "last": None})
 
         def e2e_step():
-            for i, bits in calls:
+            for k, (i, bits) in enumerate(calls):
+                ln = lanes[k % 2]
                 xs, gs = host[i]
                 n, c = specs[i].numel, specs[i].shape[1]
-                b.granq_fakequant_fused_host(xs, bits, gs, yh.view(-1)[:n].view(specs[i].shape),
-                                             gxh.view(-1)[:n].view(specs[i].shape), loh[:c], hih[:c], arena,
-                                             stream=stream)
+                b.granq_fakequant_fused_host(xs, bits, gs, ln["y"].view(-1)[:n].view(specs[i].shape),
+                                             ln["gx"].view(-1)[:n].view(specs[i].shape), ln["lo"][:c], ln["hi"][:c],
+                                             ln["arena"], flags=b.FLAG_HOST_ASYNC, stream=ln["stream"])
+                ln["last"] = specs[i].shape
+
+        def e2e_fence(check):
+            for ln in lanes:
+                stream.wait_stream(ln["stream"])
+                if check:
+                    assert b.host_arena_status(b.F32, ln["last"], ln["arena"], stream=ln["stream"]) == b.OK
+
+        for ln in lanes:
+            ln["stream"].wait_stream(stream)
         e2e_step()
+        e2e_fence(True)
         barrier()
         a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         a0.record(stream)
+        for ln in lanes:
+            ln["stream"].wait_stream(stream)
         for _ in range(args.e2e_steps):
             e2e_step()
+        e2e_fence(False)
         a1.record(stream)
         barrier()
+        e2e_fence(True)
         e_ms = a0.elapsed_time(a1)
         e_ms = max_over_ranks(e_ms)
         e2e = {"value": whole_job_gbs(bytes_per_step, world, e_ms / args.e2e_steps), "unit": UNIT,
                "h2d_bytes_per_step": elems_per_step * 8, "d2h_bytes_per_step": elems_per_step * 8 +
                sum(specs[i].shape[1] * 8 for i, _ in calls),
                "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
-               "api": "granq_fakequant_fused_host (pinned host buffers)"}
+               "api": "granq_fakequant_fused_host (pinned host buffers; calls alternate between two streams and arenas, "
+                      "so one call's downloads overlap the next call's uploads)"}
 
     # ---- the CPU oracle on a bounded sample, rank 0 at N = 1 only ----
     cpu = None

@@ -84,11 +84,15 @@ enum granq_flags {
     GRANQ_FLAG_FORCE_STAGED = 4u,    /* fused: on-chip-staged persistent kernel or GRANQ_ERR_UNSUPPORTED */
     GRANQ_FLAG_FORCE_L2WAVE = 8u,    /* fused: L2-resident-wave persistent kernel or GRANQ_ERR_UNSUPPORTED */
     GRANQ_FLAG_FORCE_COLWALK = 16u,  /* fused: column-walk persistent kernel or GRANQ_ERR_UNSUPPORTED     */
-    GRANQ_FLAG_WORKSPACE_ZEROED = 32u /* fused: the caller guarantees that the whole workspace is zero on
+    GRANQ_FLAG_WORKSPACE_ZEROED = 32u, /* fused: the caller guarantees that the whole workspace is zero on
                                         entry (cleared after allocation, or left by an earlier call with
                                         this flag that ended with status GRANQ_OK); the call then skips
                                         its own clearing step and leaves the workspace zero again on
                                         success.  After GRANQ_ERR_TIMEOUT clear it before the next use. */
+    GRANQ_FLAG_HOST_ASYNC = 64u       /* granq_fakequant_fused_host(): enqueue only, do not wait for the stream
+                                        (host outputs are valid once the stream has passed the call; ask
+                                        granq_host_arena_status() then).  Lets calls on two streams with two
+                                        arenas overlap one call's uploads with the other's downloads.       */
 };
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -234,6 +238,11 @@ int granq_fakequant_fused_host(const void* x_host, const void* gy_host_opt, int 
                                void* y_host, void* gx_host_opt, float* min_host, float* max_host,
                                float* scale_host_opt, float* zp_host_opt,
                                void* device_arena, size_t arena_bytes, uint32_t flags, void* cuda_stream);
+
+/* For calls made with GRANQ_FLAG_HOST_ASYNC: synchronises `cuda_stream`, then reports the status word of
+ * the workspace inside `device_arena` (same geometry arguments as the call), as granq_workspace_status(). */
+int granq_host_arena_status(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,
+                            const void* device_arena, void* cuda_stream);
 
 /*
  * Plan that granq_fakequant_fused() would take for this geometry and flags on the current

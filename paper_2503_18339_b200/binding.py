@@ -20,6 +20,7 @@ F32, BF16 = 0, 1
 GROUP_CHANNEL, GROUP_SAMPLE_CHANNEL, GROUP_TENSOR = 0, 1, 2
 FLAG_FORCE_TWO_PASS, FLAG_FORCE_NAIVE, FLAG_FORCE_STAGED, FLAG_FORCE_L2WAVE, FLAG_FORCE_COLWALK = 1, 2, 4, 8, 16
 FLAG_WORKSPACE_ZEROED = 32
+FLAG_HOST_ASYNC = 64
 PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED, PLAN_L2WAVE, PLAN_COLWALK = 0, 1, 2, 3, 4
 (KNOB_STAGED_DEPTH, KNOB_STAGED_MAX_BUF_UNITS, KNOB_STAGED_GRID, KNOB_SPIN_LIMIT, KNOB_TEST_EXTRA_ARRIVALS,
  KNOB_STAGED_CTAS_PER_SM, KNOB_L2_WAVE_KB, KNOB_L2_UPL, KNOB_L2_CTAS_PER_SM, KNOB_L2_LAG) = range(10)
@@ -32,6 +33,7 @@ EXPORTS = [
     "granq_host_arena_bytes", "granq_fakequant_fused_host", "granq_fused_plan", "granq_staged_geometry",
     "granq_tune", "granq_selftest_division", "granq_range_noalloc", "granq_packmask_bytes",
     "granq_fakequant_fwd_packmask", "granq_fakequant_bwd_packmask", "granq_fakequant_fused_fwd_packmask",
+    "granq_host_arena_status",
 ]
 NOALLOC_MAX_GROUPS = 32768
 
@@ -88,6 +90,8 @@ def lib() -> ctypes.CDLL:
         L.granq_range_noalloc.argtypes = [vp, ci, i64p, ci, ci, vp, vp, vp]
         L.granq_tune.restype = ci
         L.granq_tune.argtypes = [ci, ci]
+        L.granq_host_arena_status.restype = ci
+        L.granq_host_arena_status.argtypes = [ci, i64p, ci, ci, ci, vp, vp]
         L.granq_packmask_bytes.restype = sz
         L.granq_packmask_bytes.argtypes = [i64p]
         L.granq_fakequant_fwd_packmask.restype = ci
@@ -394,8 +398,17 @@ def granq_fakequant_fused_host(x: torch.Tensor, bits: int, gy: torch.Tensor, y: 
                                group: int = GROUP_CHANNEL, s: torch.Tensor = None, z: torch.Tensor = None,
                                flags: int = 0, stream=None) -> None:
     """Fused path on HOST tensors (pinned memory recommended); `arena` is device scratch of
-    host_arena_bytes() bytes.  Returns when the host outputs are valid."""
+    host_arena_bytes() bytes.  Returns when the host outputs are valid, or right after enqueuing
+    with FLAG_HOST_ASYNC (then host_arena_status() waits and reports)."""
     _check(lib().granq_fakequant_fused_host(
         _host(x, "x"), _host(gy, "gy"), _dtype(x), _dims(x.shape), channel_axis, group, bits,
         _host(y, "y"), _host(gx, "gx"), _host(lo, "lo"), _host(hi, "hi"), _host(s, "s"), _host(z, "z"),
         _dev(arena, "arena"), arena.numel(), flags, _stream(stream)), "granq_fakequant_fused_host")
+
+
+def host_arena_status(dtype: int, shape, arena: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL,
+                      with_backward: bool = True, stream=None) -> int:
+    """Waits for `stream`, then the status of the last FLAG_HOST_ASYNC call that used `arena`."""
+    return lib().granq_host_arena_status(dtype, _dims(shape), channel_axis, group, int(with_backward),
+                                         _dev(arena, "arena"), _stream(stream))
+

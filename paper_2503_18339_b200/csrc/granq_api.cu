@@ -378,6 +378,17 @@ int granq_fakequant_fused_host(const void* x_host, const void* gy_host_opt, int 
         e = cudaMemcpyAsync(scale_host_opt, ds, (size_t)G * 4, cudaMemcpyDeviceToHost, st);
     if (e == cudaSuccess && zp_host_opt) e = cudaMemcpyAsync(zp_host_opt, dz, (size_t)G * 4, cudaMemcpyDeviceToHost, st);
     if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+    if (flags & GRANQ_FLAG_HOST_ASYNC) return GRANQ_OK;
+    return granq_workspace_status(ws, cuda_stream);
+}
+
+int granq_host_arena_status(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,
+                            const void* device_arena, void* cuda_stream) {
+    Geom g;
+    int64_t G;
+    if (!device_arena || !dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G)) return GRANQ_ERR_INVALID_ARG;
+    const size_t nb = align256((size_t)g.E * elt_size(dtype)), gb = align256((size_t)G * 4);
+    const char* ws = (const char*)device_arena + nb * (with_backward ? 4 : 2) + 4 * gb;
     return granq_workspace_status(ws, cuda_stream);
 }
 
