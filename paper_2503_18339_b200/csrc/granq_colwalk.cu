@@ -23,6 +23,7 @@
 #include "granq_internal.h"
 
 #include <algorithm>
+#include <mutex>
 
 namespace granq {
 
@@ -399,7 +400,8 @@ uint32_t c_pick_chunks(uint32_t ncol, uint32_t outer, uint32_t grid, uint64_t* c
     const uint64_t kItemCost = 3;      // set-up and combine of one item, in slabs walked
     uint64_t best = ~0ull;
     uint32_t best_k = 1;
-    const uint32_t kmax = std::min<uint32_t>(outer, 4096);
+    // more than a few items per CTA and wave only adds per-item cost
+    const uint32_t kmax = std::min<uint32_t>(std::min<uint32_t>(outer, 4096), 4 * (grid / ncol + 1));
     for (uint32_t k = 1; k <= kmax; ++k) {
         const uint64_t items = (uint64_t)ncol * k;
         const uint64_t per_cta = (items + grid - 1) / grid;
@@ -482,14 +484,37 @@ ColPlan plan_colwalk(int dtype, const Geom& g, const QuantIO& io, const StagedTu
     const uint64_t cap = std::max<uint64_t>(1, ((1ull << 30) / inner) / q);       // keeps cw * inner below 2^30
     const uint64_t max_mult = std::max<uint64_t>(1, std::min<uint64_t>(target / (group_bytes * q), cap));
     if ((uint64_t)q * inner >= (1ull << 30)) return p;
-    uint32_t nw = (uint32_t)((mult_total + max_mult - 1) / max_mult);
+    const uint32_t nw = (uint32_t)((mult_total + max_mult - 1) / max_mult);
     p.cw = ((mult_total + nw - 1) / nw) * q;
     if (tune.l2_wave_kb <= 0 && nw > 1) {
         // Several waves: among the wave sizes from half the target up to the target take the one whose
         // work items load the CTAs most evenly (the busiest CTA's walk, summed over the waves).
         const uint32_t grid = c_assumed_grid(tune.l2_ctas_per_sm);
+        // the search is host work on every call: remember the last few answers
+        struct Memo {
+            uint32_t V, inner, C, grid;
+            int64_t outer;
+            uint64_t target;
+            uint32_t cw;
+        };
+        static Memo memo[8] = {};
+        static unsigned memo_next = 0;
+        static std::mutex memo_lock;
+        bool found = false;
+        {
+            std::lock_guard<std::mutex> hold(memo_lock);
+            for (const Memo& e : memo)
+                if (e.cw && e.V == V && e.inner == inner && e.C == C && e.grid == grid && e.outer == g.outer &&
+                    e.target == target) {
+                    p.cw = e.cw;
+                    found = true;
+                    break;
+                }
+        }
         uint64_t best = ~0ull;
-        for (uint64_t m = max_mult; m >= std::max<uint64_t>(1, max_mult / 2); --m) {
+        const uint64_t m_lo = std::max<uint64_t>(1, max_mult / 2);
+        const uint64_t m_step = std::max<uint64_t>(1, (max_mult - m_lo) / 24);       // at most ~25 candidates
+        for (uint64_t m = max_mult; !found && m >= m_lo; m -= std::min(m_step, m - m_lo + 1)) {
             const uint32_t waves = (uint32_t)((mult_total + m - 1) / m);
             const uint32_t m_last = mult_total - (waves - 1) * (uint32_t)m;
             uint64_t c_reg = 0, c_last = 0;
@@ -501,6 +526,10 @@ ColPlan plan_colwalk(int dtype, const Geom& g, const QuantIO& io, const StagedTu
                 best = total;
                 p.cw = (uint32_t)m * q;
             }
+        }
+        if (!found) {
+            std::lock_guard<std::mutex> hold(memo_lock);
+            memo[memo_next++ % 8] = Memo{V, inner, C, grid, g.outer, target, p.cw};
         }
     }
     p.nwaves = (C + p.cw - 1) / p.cw;
