@@ -183,3 +183,36 @@ int granq_oracle_bwd_packed(const void* gy, const uint8_t* packed, int dtype, in
     return 0;
 }
 
+/* ---- distortion statistics of a quantization (Section 4.1, Table 2) ---------------------------- */
+
+/* sums[0] = sum x^2, sums[1] = sum q^2, sums[2] = sum x*q, sums[3] = sum (x - q)^2 over all E
+ * elements, every term and every sum in fp64 (the products of two fp32 values are exact in fp64). */
+int granq_oracle_distortion_sums(const void* x, const void* q, int dtype, int64_t E, double sums[4]) {
+    if (!x || !q || !sums || E < 0) return -1;
+    double sxx = 0.0, sqq = 0.0, sxq = 0.0, sdd = 0.0;
+    for (int64_t e = 0; e < E; ++e) {
+        double xv = (double)load_elem(x, dtype, e);
+        double qv = (double)load_elem(q, dtype, e);
+        double d = xv - qv;
+        sxx += xv * xv;
+        sqq += qv * qv;
+        sxq += xv * qv;
+        sdd += d * d;
+    }
+    sums[0] = sxx;
+    sums[1] = sqq;
+    sums[2] = sxq;
+    sums[3] = sdd;
+    return 0;
+}
+
+/* Table 2's two statistics from the sums: cosine similarity X.Q / (|X| |Q|) and relative error
+ * |X - Q| / |X|; 0 where a denominator is 0. */
+int granq_oracle_distortion(const double sums[4], double* cosine, double* rel_error) {
+    if (!sums || !cosine || !rel_error) return -1;
+    double den = sqrt(sums[0]) * sqrt(sums[1]);
+    *cosine = den > 0.0 ? sums[2] / den : 0.0;
+    *rel_error = sums[0] > 0.0 ? sqrt(sums[3]) / sqrt(sums[0]) : 0.0;
+    return 0;
+}
+

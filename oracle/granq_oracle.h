@@ -74,6 +74,13 @@ int granq_oracle_fused(const void* x, const void* gy, int dtype, const int64_t d
 int granq_oracle_pack_mask(const uint8_t* mask, int64_t E, uint8_t* packed);
 int granq_oracle_bwd_packed(const void* gy, const uint8_t* packed, int dtype, int64_t E, void* gx);
 
+/* Distortion statistics of a quantization, the quantities of Table 2 (Section 4.1): with X the
+ * activations and Q their fake-quantized values, sums = { sum X^2, sum Q^2, sum X*Q, sum (X-Q)^2 }
+ * in fp64, and from them the cosine similarity X.Q / (|X|_2 |Q|_2) and the relative error
+ * |X - Q|_2 / |X|_2 (0 where a denominator vanishes). */
+int granq_oracle_distortion_sums(const void* x, const void* q, int dtype, int64_t E, double sums[4]);
+int granq_oracle_distortion(const double sums[4], double* cosine, double* rel_error);
+
 #ifdef __cplusplus
 }
 #endif

@@ -65,6 +65,10 @@ def lib() -> ctypes.CDLL:
         L.granq_oracle_pack_mask.argtypes = [u8p, ctypes.c_int64, u8p]
         L.granq_oracle_bwd_packed.restype = ci
         L.granq_oracle_bwd_packed.argtypes = [vp, u8p, ci, ctypes.c_int64, vp]
+        L.granq_oracle_distortion_sums.restype = ci
+        L.granq_oracle_distortion_sums.argtypes = [vp, vp, ci, ctypes.c_int64, vp]
+        L.granq_oracle_distortion.restype = ci
+        L.granq_oracle_distortion.argtypes = [vp, vp, vp]
         _lib = L
     return _lib
 
@@ -199,4 +203,25 @@ def bwd_packed(gy: np.ndarray, packed: np.ndarray) -> np.ndarray:
     _check(lib().granq_oracle_bwd_packed(_p(gy), _p(packed), _dtype_of(gy), gy.size, _p(gx)),
            "granq_oracle_bwd_packed")
     return gx
+
+
+def distortion_sums(x: np.ndarray, q: np.ndarray) -> np.ndarray:
+    """[sum x^2, sum q^2, sum x*q, sum (x-q)^2] in fp64 (the raw material of Table 2)."""
+    x = np.ascontiguousarray(x)
+    q = np.ascontiguousarray(q)
+    if x.shape != q.shape or x.dtype != q.dtype:
+        raise ValueError("q must match x")
+    sums = np.empty(4, np.float64)
+    _check(lib().granq_oracle_distortion_sums(_p(x), _p(q), _dtype_of(x), x.size, _p(sums)),
+           "granq_oracle_distortion_sums")
+    return sums
+
+
+def distortion(sums: np.ndarray):
+    """(cosine similarity, relative error) of Table 2 from distortion_sums()."""
+    sums = np.ascontiguousarray(sums, np.float64)
+    c = ctypes.c_double(0.0)
+    r = ctypes.c_double(0.0)
+    _check(lib().granq_oracle_distortion(_p(sums), ctypes.byref(c), ctypes.byref(r)), "granq_oracle_distortion")
+    return c.value, r.value
 

@@ -26,6 +26,9 @@ MUTATIONS = {
     "packed_mask_most_significant_bit_first": ("(1u << (e % 8))", "(0x80u >> (e % 8))"),
     "packed_backward_reads_bits_in_reverse": ("(packed[e / 8] >> (e % 8)) & 1", "(packed[e / 8] >> (7 - e % 8)) & 1"),
     "packed_backward_ignores_mask": ("bit ? gv : 0.0f", "gv"),
+    "distortion_error_not_squared_difference": ("sdd += d * d;", "sdd += d;"),
+    "distortion_cosine_without_norm_of_q": ("double den = sqrt(sums[0]) * sqrt(sums[1]);", "double den = sums[0];"),
+    "distortion_relative_error_not_rooted": ("sqrt(sums[3]) / sqrt(sums[0])", "sums[3] / sums[0]"),
     "packed_mask_last_byte_not_cleared": ("for (int64_t b = 0; b < (E + 7) / 8; ++b) packed[b] = 0;",
                                           "for (int64_t b = 0; b < E / 8; ++b) packed[b] = 0;"),
 }

@@ -425,3 +425,46 @@ def test_backward_from_packed_mask_equals_backward_from_x(dtype):
     bits = np.unpackbits(packed, bitorder="little")[:x.size].reshape(shape).astype(bool)
     assert np.array_equal(gx.view(u), np.where(bits, gy.view(u), u(0)))
 
+
+# --------------------------------------------------------------------------------------
+# 10. distortion statistics (Section 4.1, Table 2): cosine similarity and relative error
+# --------------------------------------------------------------------------------------
+def test_distortion_closed_forms():
+    x = f32([3, 4, 0, 0]).reshape(1, 1, 1, 4)
+    cases = [
+        (x, (1.0, 0.0)),                                            # Q = X
+        (2 * x, (1.0, 1.0)),                                        # Q = 2X: same direction, |X - Q| = |X|
+        (f32([0, 0, 5, 0]).reshape(1, 1, 1, 4), (0.0, math.sqrt(2))),   # orthogonal, |X - Q|^2 = 25 + 25
+        (f32([4, 3, 0, 0]).reshape(1, 1, 1, 4), (24 / 25, math.sqrt(2) / 5)),
+        (-x, (-1.0, 2.0)),
+        (0 * x, (0.0, 1.0)),                                        # |Q| = 0: cosine reported as 0
+    ]
+    for q, (cos, rel) in cases:
+        sums = orc.distortion_sums(x, q)
+        got = orc.distortion(sums)
+        assert got[0] == pytest.approx(cos, abs=1e-15) and got[1] == pytest.approx(rel, abs=1e-15)
+    assert orc.distortion_sums(x, f32([4, 3, 0, 0]).reshape(1, 1, 1, 4)).tolist() == [25.0, 25.0, 24.0, 2.0]
+    assert orc.distortion(np.zeros(4)) == (0.0, 0.0)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_distortion_sums_match_float64_dot_products(dtype):
+    rng = np.random.default_rng(8)
+    x = (rng.standard_normal((3, 5, 7, 7)) * 10).astype(np.float32)
+    if dtype == "bf16":
+        xb = (x.view(np.uint32) >> 16).astype(np.uint16)
+        res = orc.fused(xb, 4)
+        xw = (xb.astype(np.uint32) << 16).view(np.float32).astype(np.float64).ravel()
+        qw = (res.y.astype(np.uint32) << 16).view(np.float32).astype(np.float64).ravel()
+        sums = orc.distortion_sums(xb, res.y)
+    else:
+        res = orc.fused(x, 4)
+        xw, qw = x.astype(np.float64).ravel(), res.y.astype(np.float64).ravel()
+        sums = orc.distortion_sums(x, res.y)
+    want = [math.fsum(xw * xw), math.fsum(qw * qw), math.fsum(xw * qw), math.fsum((xw - qw) ** 2)]
+    assert np.allclose(sums, want, rtol=1e-13, atol=0)
+    cos, rel = orc.distortion(sums)
+    assert cos == pytest.approx(np.dot(xw, qw) / (np.linalg.norm(xw) * np.linalg.norm(qw)), rel=1e-12)
+    assert rel == pytest.approx(np.linalg.norm(xw - qw) / np.linalg.norm(xw), rel=1e-12)
+    assert 0.9 < cos <= 1.0 and 0.0 < rel < 0.2
+
