@@ -214,6 +214,27 @@ int granq_fakequant_fused_fwd_packmask(const void* x, int dtype, const int64_t d
                                        uint32_t flags, void* cuda_stream);
 
 /*
+ * Distortion statistics of a quantization (Section 4.1, Table 2).  With X the activations and Q
+ * their fake-quantized values the table reports the cosine similarity X.Q / (|X|_2 |Q|_2) and the
+ * relative error |X - Q|_2 / |X|_2; both follow from four sums over all elements,
+ *   sums_out = { sum X^2, sum Q^2, sum X*Q, sum (X-Q)^2 }      (4 doubles, DEVICE memory, 8-byte aligned)
+ * which these calls write (they clear them first).  The terms of one 16-byte pack are summed in
+ * fp32, everything else in fp64.
+ *
+ * granq_distortion():            the sums for an existing pair (x, q) of E elements each.
+ * granq_fakequant_fused_stats(): the forward half of the whole path (range of x itself -> scale /
+ *     zero-point -> y) that gathers the sums in the pass that writes y, for any grouping - so the
+ *     layer-wise baseline (GRANQ_GROUP_TENSOR) and the channel-wise method can be compared on the
+ *     same tensor as in Table 2.  Plans and flags as granq_fakequant_fused_fwd_packmask().
+ */
+int granq_distortion(const void* x, const void* q, int dtype, const int64_t dims[4], double* sums_out,
+                     uint32_t flags, void* cuda_stream);
+int granq_fakequant_fused_stats(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                                int bits, void* y, float* min_out, float* max_out, float* scale_opt, float* zp_opt,
+                                double* sums_out, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                void* cuda_stream);
+
+/*
  * Status word the persistent plans leave in the workspace.  Synchronises `cuda_stream`, then
  * returns GRANQ_OK, GRANQ_ERR_TIMEOUT (a bounded device-side wait ran out), or
  * GRANQ_ERR_CUDA.  `workspace` is the pointer given to the preceding call.

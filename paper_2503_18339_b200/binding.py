@@ -33,7 +33,7 @@ EXPORTS = [
     "granq_host_arena_bytes", "granq_fakequant_fused_host", "granq_fused_plan", "granq_staged_geometry",
     "granq_tune", "granq_selftest_division", "granq_range_noalloc", "granq_packmask_bytes",
     "granq_fakequant_fwd_packmask", "granq_fakequant_bwd_packmask", "granq_fakequant_fused_fwd_packmask",
-    "granq_host_arena_status",
+    "granq_host_arena_status", "granq_distortion", "granq_fakequant_fused_stats",
 ]
 NOALLOC_MAX_GROUPS = 32768
 
@@ -92,6 +92,10 @@ def lib() -> ctypes.CDLL:
         L.granq_tune.argtypes = [ci, ci]
         L.granq_host_arena_status.restype = ci
         L.granq_host_arena_status.argtypes = [ci, i64p, ci, ci, ci, vp, vp]
+        L.granq_distortion.restype = ci
+        L.granq_distortion.argtypes = [vp, vp, ci, i64p, vp, u32, vp]
+        L.granq_fakequant_fused_stats.restype = ci
+        L.granq_fakequant_fused_stats.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, sz, u32, vp]
         L.granq_packmask_bytes.restype = sz
         L.granq_packmask_bytes.argtypes = [i64p]
         L.granq_fakequant_fwd_packmask.restype = ci
@@ -209,6 +213,7 @@ class FakeQuantOut:
     mask: Optional[torch.Tensor] = None
     workspace: Optional[torch.Tensor] = None
     packed_mask: Optional[torch.Tensor] = None      # int32 words, one bit per element
+    sums: Optional[torch.Tensor] = None             # 4 doubles: sum x^2, sum q^2, sum x*q, sum (x-q)^2
 
 
 def granq_range(x: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL, lo: torch.Tensor = None,
@@ -372,6 +377,50 @@ def granq_fakequant_fused_fwd_packmask(x: torch.Tensor, bits: int, channel_axis:
         _dev(o.packed_mask, "packed_mask"), _dev(o.lo, "lo"), _dev(o.hi, "hi"), _dev(o.s, "s"), _dev(o.z, "z"),
         _dev(o.workspace, "workspace"), o.workspace.numel(), flags, _stream(stream)),
         "granq_fakequant_fused_fwd_packmask")
+    return o
+
+
+def granq_distortion(x: torch.Tensor, q: torch.Tensor, sums: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """[sum x^2, sum q^2, sum x*q, sum (x-q)^2] as 4 doubles on the device (Table 2's raw material)."""
+    if q.shape != x.shape or q.dtype != x.dtype:
+        raise ValueError("q must match x")
+    sums = torch.empty(4, dtype=torch.float64, device=x.device) if sums is None else sums
+    _check(lib().granq_distortion(_dev(x, "x"), _dev(q, "q"), _dtype(x), _dims(x.shape), _dev(sums, "sums"), 0,
+                                  _stream(stream)), "granq_distortion")
+    return sums
+
+
+def distortion_from_sums(sums):
+    """(cosine similarity, relative error) of Table 2 from the four sums (host arithmetic on 4 numbers)."""
+    sxx, sqq, sxq, sdd = (float(v) for v in sums)
+    den = (sxx ** 0.5) * (sqq ** 0.5)
+    return (sxq / den if den > 0 else 0.0), ((sdd ** 0.5) / (sxx ** 0.5) if sxx > 0 else 0.0)
+
+
+def granq_fakequant_fused_stats(x: torch.Tensor, bits: int, channel_axis: int = 1, group: int = GROUP_CHANNEL,
+                                out: FakeQuantOut = None, want_params: bool = False, flags: int = 0,
+                                stream=None) -> FakeQuantOut:
+    """Range of x itself -> scale / zero-point -> y, gathering Table 2's sums in the same pass."""
+    G = num_groups(x.shape, channel_axis, group)
+    o = out if out is not None else FakeQuantOut()
+    dev = x.device
+    if o.y is None:
+        o.y = torch.empty_like(x)
+    if o.sums is None:
+        o.sums = torch.empty(4, dtype=torch.float64, device=dev)
+    if o.lo is None:
+        o.lo = torch.empty(G, dtype=torch.float32, device=dev)
+    if o.hi is None:
+        o.hi = torch.empty(G, dtype=torch.float32, device=dev)
+    if want_params and o.s is None:
+        o.s = torch.empty(G, dtype=torch.float32, device=dev)
+        o.z = torch.empty(G, dtype=torch.float32, device=dev)
+    if o.workspace is None:
+        o.workspace = make_workspace(x, channel_axis, group)
+    _check(lib().granq_fakequant_fused_stats(
+        _dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, bits, _dev(o.y, "y"), _dev(o.lo, "lo"),
+        _dev(o.hi, "hi"), _dev(o.s, "s"), _dev(o.z, "z"), _dev(o.sums, "sums"), _dev(o.workspace, "workspace"),
+        o.workspace.numel(), flags, _stream(stream)), "granq_fakequant_fused_stats")
     return o
 
 

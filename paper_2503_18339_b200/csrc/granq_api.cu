@@ -318,6 +318,59 @@ int granq_fakequant_fused_fwd_packmask(const void* x, int dtype, const int64_t d
     return cuda_status(e);
 }
 
+int granq_distortion(const void* x, const void* q, int dtype, const int64_t dims[4], double* sums_out,
+                     uint32_t flags, void* cuda_stream) {
+    (void)flags;
+    Geom g;
+    int64_t G;
+    if (!x || !q || !sums_out || !dtype_ok(dtype) || !make_geom(dims, 1, GRANQ_GROUP_TENSOR, g, G) ||
+        ((uintptr_t)sums_out & 7))
+        return GRANQ_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaMemsetAsync(sums_out, 0, 4 * sizeof(double), st);
+    if (e == cudaSuccess) e = launch_distortion(x, q, dtype, g.E, sums_out, st);
+    return cuda_status(e);
+}
+
+int granq_fakequant_fused_stats(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
+                                int bits, void* y, float* min_out, float* max_out, float* scale_opt, float* zp_opt,
+                                double* sums_out, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                void* cuda_stream) {
+    Geom g;
+    int64_t G;
+    if (!x || !y || !sums_out || !min_out || !max_out || bits < 1 || bits > 8 || !dtype_ok(dtype) ||
+        !make_geom(dims, channel_axis, group, g, G) || ((uintptr_t)sums_out & 7))
+        return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
+    const size_t nb = (size_t)g.E * elt_size(dtype);
+    if (overlaps(x, nb, y, nb) || overlaps(x, nb, sums_out, 32) || overlaps(y, nb, sums_out, 32))
+        return GRANQ_ERR_INVALID_ARG;
+    if (int rc = check_workspace(workspace, workspace_bytes, G)) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    QuantIO io{x, nullptr, y, nullptr, nullptr, nullptr, nullptr, sums_out};
+    // the column-walk kernel where there are slabs to walk, else range pass + flat pass (layer-wise and
+    // per-sample groups): the statistics are gathered in the pass that writes y either way
+    ColPlan cp{};
+    if (!(flags & GRANQ_FLAG_FORCE_TWO_PASS)) cp = plan_colwalk(dtype, g, io, g_tune);
+    if ((flags & GRANQ_FLAG_FORCE_COLWALK) && !cp.ok) return GRANQ_ERR_UNSUPPORTED;
+    Workspace ws = carve_workspace(workspace, G);
+    const bool zeroed = (flags & GRANQ_FLAG_WORKSPACE_ZEROED) != 0;
+    cudaError_t e = cudaMemsetAsync(sums_out, 0, 4 * sizeof(double), st);
+    if (e == cudaSuccess && !(zeroed && cp.ok)) e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
+    if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+    if (cp.ok) {
+        e = launch_colwalk(cp, io, MODE_FWD, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
+    } else {
+        e = launch_range_flat(x, dtype, g, ws.kmin, ws.kmax, st);
+        if (e == cudaSuccess)
+            e = launch_finalize_range(ws.kmin, ws.kmax, G, min_out, max_out, bits, scale_opt, zp_opt, st);
+        if (e == cudaSuccess) e = launch_quant_flat(io, MODE_FWD, dtype, g, bits, min_out, max_out, st);
+        if (e == cudaSuccess && zeroed)
+            e = cudaMemsetAsync((char*)workspace + sizeof(uint32_t), 0, ws.clear_bytes - sizeof(uint32_t), st);
+    }
+    return cuda_status(e);
+}
+
 int granq_workspace_status(const void* workspace, void* cuda_stream) {
     if (!workspace) return GRANQ_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;

@@ -51,6 +51,7 @@ struct CArgs {
     uint8_t* codes;
     uint8_t* mask;
     uint32_t* pmask;       // mask at one bit per element, or null
+    double* dist;          // four running sums of Table 2's statistics, or null
     uint32_t* status;
     uint32_t* kmin;
     uint32_t* kmax;
@@ -172,6 +173,8 @@ __global__ void __launch_bounds__(kCThreads, 4) colwalk_kernel(const CArgs a) {
     };
 
     uint32_t p1_items = 0;      // items this CTA has reduced so far (selects the shared-memory buffer)
+    DistAcc dacc;               // Table 2's sums over everything this thread quantizes (EXTRAS only)
+    dacc.reset();
 
     // ---- phase 1: this CTA's items of wave w -> min / max keys, then arrive ----
     auto phase1 = [&](uint32_t w) {
@@ -315,6 +318,7 @@ __global__ void __launch_bounds__(kCThreads, 4) colwalk_kernel(const CArgs a) {
 #pragma unroll
                         for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.mask)[at * (V / 4) + i] = mb[i];
                     }
+                    if (a.dist) dacc.add(px, py);
                     if (a.pmask) {
                         // 32 / V neighbouring lanes own the 32 elements of one mask word; the planner has made
                         // every slab and wave a whole number of words, so such a group of lanes is here together
@@ -365,6 +369,10 @@ __global__ void __launch_bounds__(kCThreads, 4) colwalk_kernel(const CArgs a) {
         if (w + lag < W) phase1(w + lag);
         if (!wait_wave(w)) return;
         phase2(w);
+    }
+
+    if constexpr (EXTRAS) {
+        if (a.dist) dacc.flush(a.dist);
     }
 
     // ---- leave the workspace as it was found: the last CTA to finish clears keys and counters ----
@@ -555,6 +563,7 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
     a.codes = io.codes;
     a.mask = io.mask;
     a.pmask = io.pmask;
+    a.dist = io.dist;
     a.status = ws.status;
     a.kmin = ws.kmin;
     a.kmax = ws.kmax;
@@ -586,7 +595,7 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
         s.div_ncol = make_fastdiv(s.ncol);
     }
     a.div_plane = make_fastdiv(aligned ? inner / V : inner);
-    const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr;
+    const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr || io.dist != nullptr;
     const int cap = tune.l2_ctas_per_sm;
     if (dtype == 0) {
         if (mode == MODE_FWD) return c_launch_mode<float, MODE_FWD>(a, aligned, extras, sms, cap, st);

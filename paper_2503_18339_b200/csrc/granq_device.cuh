@@ -297,6 +297,61 @@ __device__ __forceinline__ void pack_minmax(const Pack<T>& p, int first, int las
     }
 }
 
+// ---------------------------------------------------------------------------------------
+// Distortion statistics of a quantization (Section 4.1, Table 2): sum x^2, sum q^2, sum x*q,
+// sum (x - q)^2.  The terms of one pack are summed in fp32 (fused multiply-adds), everything
+// beyond a pack in fp64, so a sum differs from the exact one by at most a few fp32 roundings
+// of a pack-sized partial sum.
+// ---------------------------------------------------------------------------------------
+__device__ __forceinline__ float as_stored(float v, const float*) { return v; }
+__device__ __forceinline__ float as_stored(float v, const __nv_bfloat16*) {
+    return __bfloat162float(__float2bfloat16_rn(v));
+}
+
+struct DistAcc {
+    double xx, qq, xq, dd;
+    __device__ __forceinline__ void reset() { xx = qq = xq = dd = 0.0; }
+    __device__ __forceinline__ void add_one(float x, float q) {
+        const float d = __fsub_rn(x, q);
+        xx += (double)__fmul_rn(x, x);
+        qq += (double)__fmul_rn(q, q);
+        xq += (double)__fmul_rn(x, q);
+        dd += (double)__fmul_rn(d, d);
+    }
+    template <typename T>
+    __device__ __forceinline__ void add(const Pack<T>& px, const Pack<T>& pq) {
+        float a = 0.0f, b = 0.0f, c = 0.0f, e = 0.0f;
+#pragma unroll
+        for (int i = 0; i < Pack<T>::V; ++i) {
+            const float x = px.get(i), q = pq.get(i), d = __fsub_rn(x, q);
+            a = __fmaf_rn(x, x, a);
+            b = __fmaf_rn(q, q, b);
+            c = __fmaf_rn(x, q, c);
+            e = __fmaf_rn(d, d, e);
+        }
+        xx += (double)a;
+        qq += (double)b;
+        xq += (double)c;
+        dd += (double)e;
+    }
+    // must be called by all 32 lanes of a warp: one atomic per warp and sum
+    __device__ __forceinline__ void flush(double* out) {
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) {
+            xx += __shfl_xor_sync(kFullMask, xx, d);
+            qq += __shfl_xor_sync(kFullMask, qq, d);
+            xq += __shfl_xor_sync(kFullMask, xq, d);
+            dd += __shfl_xor_sync(kFullMask, dd, d);
+        }
+        if ((threadIdx.x & 31) == 0) {
+            atomicAdd(out + 0, xx);
+            atomicAdd(out + 1, qq);
+            atomicAdd(out + 2, xq);
+            atomicAdd(out + 3, dd);
+        }
+    }
+};
+
 // 128-bit global accesses with an L2 eviction policy (createpolicy.fractional.L2::evict_*)
 __device__ __forceinline__ uint64_t l2_policy_evict_last() {
     uint64_t p;

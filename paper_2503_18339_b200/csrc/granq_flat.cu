@@ -250,12 +250,15 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                                                               T* __restrict__ y, T* __restrict__ gx,
                                                               uint8_t* __restrict__ codes,
                                                               uint8_t* __restrict__ mask,
-                                                              uint32_t* __restrict__ pmask, FlatGeom g, float qmax,
+                                                              uint32_t* __restrict__ pmask,
+                                                              double* __restrict__ dist, FlatGeom g, float qmax,
                                                               const float* __restrict__ lo,
                                                               const float* __restrict__ hi) {
     __shared__ TileBase s_base;
     __shared__ float s_tab_s[kTableMax], s_tab_z[kTableMax], s_tab_r[kTableMax];
     constexpr bool kFwd = (MODE & MODE_FWD) != 0, kBwd = (MODE & MODE_BWD) != 0;
+    DistAcc dacc;
+    dacc.reset();
     for (int64_t tile = blockIdx.x; tile < g.ntiles; tile += gridDim.x) {
         const int64_t e0 = tile * (int64_t)kTile;
         const uint32_t ne = (uint32_t)min((int64_t)kTile, g.E - e0);
@@ -315,6 +318,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                     float code = quant_one(sx[j], p, qmax, yv, in);
                     inside_bits = in ? 1u : 0u;
                     if constexpr (kFwd) {
+                        if (dist) dacc.add_one(sx[j], as_stored(yv, y));
                         store_scalar(y + e, yv);
                         if (codes) codes[e] = (uint8_t)code;
                     }
@@ -334,6 +338,9 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                     if constexpr (EXTRAS) {
 #pragma unroll
                         for (int i = 0; i < V; ++i) inside_bits |= ((mb[i / 4] >> (8 * (i % 4))) & 1u) << i;
+                        if constexpr (kFwd) {
+                            if (dist) dacc.add(px[j], py);
+                        }
                     }
                     if constexpr (kFwd) {
                         st_stream_16(y + e, py.raw);
@@ -373,6 +380,9 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                 }
             }
         }
+    }
+    if constexpr (EXTRAS && kFwd) {
+        if (dist) dacc.flush(dist);
     }
 }
 
@@ -465,6 +475,41 @@ __global__ void __launch_bounds__(kThreads) bwd_packmask_kernel(const T* __restr
     }
 }
 
+// ---- Table 2's raw material for an existing pair (x, q): four fp64 sums -----------------------------
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads) distortion_kernel(const T* __restrict__ x, const T* __restrict__ q,
+                                                              int64_t E, double* __restrict__ sums) {
+    DistAcc acc;
+    acc.reset();
+    const int64_t nunits = E / V;
+    const int64_t stride = (int64_t)gridDim.x * kThreads * 2;
+    for (int64_t u0 = (int64_t)blockIdx.x * kThreads * 2; u0 < nunits; u0 += stride) {
+        int64_t e[2];
+        Pack<T> px[2], pq[2];
+        float sx[2], sq[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            e[j] = (u0 + j * kThreads + threadIdx.x) * V;
+            if (e[j] < E) {
+                if constexpr (V == 1) {
+                    sx[j] = load_scalar(x + e[j]);
+                    sq[j] = load_scalar(q + e[j]);
+                } else {
+                    px[j].raw = ld_stream_16(x + e[j]);
+                    pq[j].raw = ld_stream_16(q + e[j]);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            if (e[j] >= E) continue;
+            if constexpr (V == 1) acc.add_one(sx[j], sq[j]);
+            else acc.add(px[j], pq[j]);
+        }
+    }
+    acc.flush(sums);
+}
+
 bool aligned16(const void* p) { return p == nullptr || ((uintptr_t)p & 15) == 0; }
 
 int flat_grid(const FlatGeom& f) {
@@ -519,16 +564,16 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
                ((uintptr_t)io.codes % 4 == 0) && ((uintptr_t)io.mask % 4 == 0);
     int grid = flat_grid(f);
     float qmax = (float)((1 << bits) - 1);
-    const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr;
+    const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr || io.dist != nullptr;
     if (vec && extras)
         quant_flat_kernel<T, VF, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                        (T*)io.gx, io.codes, io.mask, io.pmask, f, qmax, lo, hi);
+                                                                        (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, f, qmax, lo, hi);
     else if (vec)
         quant_flat_kernel<T, VF, MODE, false><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                         (T*)io.gx, io.codes, io.mask, io.pmask, f, qmax, lo, hi);
+                                                                         (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, f, qmax, lo, hi);
     else
         quant_flat_kernel<T, 1, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                       (T*)io.gx, io.codes, io.mask, io.pmask, f, qmax, lo, hi);
+                                                                       (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, f, qmax, lo, hi);
     return cudaGetLastError();
 }
 
@@ -617,6 +662,30 @@ cudaError_t launch_bwd_packmask(const void* gy, const uint32_t* pmask, void* gx,
         else
             bwd_packmask_kernel<__nv_bfloat16, 1><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)gy, pmask,
                                                                              (__nv_bfloat16*)gx, E);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_distortion(const void* x, const void* q, int dtype, int64_t E, double* sums, cudaStream_t st) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int VF = dtype == 0 ? 4 : 8;
+    const bool vec = aligned16(x) && aligned16(q) && (E % VF == 0);
+    const int64_t units = vec ? E / VF : E;
+    const int64_t per_cta = (int64_t)kThreads * 2;
+    const int64_t ctas = (units + per_cta - 1) / per_cta, cap = (int64_t)sms * 8;
+    const int grid = (int)(ctas < 1 ? 1 : (ctas < cap ? ctas : cap));
+    if (dtype == 0) {
+        if (vec) distortion_kernel<float, 4><<<grid, kThreads, 0, st>>>((const float*)x, (const float*)q, E, sums);
+        else distortion_kernel<float, 1><<<grid, kThreads, 0, st>>>((const float*)x, (const float*)q, E, sums);
+    } else {
+        if (vec)
+            distortion_kernel<__nv_bfloat16, 8><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)x,
+                                                                           (const __nv_bfloat16*)q, E, sums);
+        else
+            distortion_kernel<__nv_bfloat16, 1><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)x,
+                                                                           (const __nv_bfloat16*)q, E, sums);
     }
     return cudaGetLastError();
 }

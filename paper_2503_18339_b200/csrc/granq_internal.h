@@ -54,6 +54,7 @@ struct QuantIO {
     uint8_t* codes;   // optional
     uint8_t* mask;    // optional
     uint32_t* pmask;  // optional: the mask at one bit per element (forward plans that support it)
+    double* dist;     // optional: 4 running sums of Table 2's statistics, zero on entry (same plans)
 };
 
 // ---- generic ("flat") kernels: any geometry, any alignment --------------------------------
@@ -72,6 +73,8 @@ cudaError_t launch_quant_flat(const QuantIO& io, int mode, int dtype, const Geom
 // STE backward from the mask at one bit per element (bit e % 32 of word e / 32)
 cudaError_t launch_bwd_packmask(const void* gy, const uint32_t* pmask, void* gx, int dtype, int64_t E,
                                 cudaStream_t st);
+// sums[0..3] += sum x^2, sum q^2, sum x*q, sum (x-q)^2 over E elements (Table 2's raw material)
+cudaError_t launch_distortion(const void* x, const void* q, int dtype, int64_t E, double* sums, cudaStream_t st);
 // the "conventional" scheme: a host loop over groups with three launches each
 cudaError_t launch_naive(const QuantIO& io, int mode, int dtype, const Geom& g, int bits, uint32_t* kmin,
                          uint32_t* kmax, float* lo, float* hi, cudaStream_t st, int* launches);
