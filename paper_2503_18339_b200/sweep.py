@@ -7,6 +7,11 @@ CUDA-event time of one call (median of `--iters`, after warm-up, an L2-sized scr
 calls), the algorithmic GB/s (fp32: 8 / 16 B per element, bf16: 4 / 8) and its fraction of the
 measured copy bandwidth.  Inputs come from `workloads.py`; bf16 inputs are the round-to-nearest-even
 of the fp32 sample.
+
+    python -m paper_2503_18339_b200.sweep --config 2 --distortion --bits 3,4
+
+prints instead the statistics of the paper's Table 2 (cosine similarity and relative error of the
+fake-quantized activations) for layer-wise against channel-wise quantization of the same tensors.
 """
 from __future__ import annotations
 
@@ -40,8 +45,14 @@ def main() -> None:
     ap.add_argument("--modes", default="fwd,fwd+bwd")
     ap.add_argument("--only", default="", help="keep tensors whose name contains this")
     ap.add_argument("--tune", default="", help="planner knobs, e.g. l2_wave_kb=32768,l2_upl=2")
+    ap.add_argument("--distortion", action="store_true",
+                    help="instead of the bandwidth sweep: the statistics of Table 2 (cosine similarity, relative "
+                         "error) of layer-wise against channel-wise quantization on the config's tensors")
     args = ap.parse_args()
     b.lib()
+    if args.distortion:
+        distortion_table(args)
+        return
     knobs = {"l2_wave_kb": b.KNOB_L2_WAVE_KB, "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM}
     for item in filter(None, args.tune.split(",")):
         name, val = item.split("=")
@@ -82,6 +93,37 @@ def main() -> None:
                     print(f"{spec.name} {dt} {bits} {mode} {us:.1f} {gbs:.0f} {gbs / peak:.3f}", flush=True)
             del x, gy, out
         del x32, g32
+
+
+def distortion_table(args) -> None:
+    """Table 2 in kind: per tensor and averaged, layer-wise (one range per tensor) against channel-wise
+    (one range per channel) at the given bit-widths, with the time of the pass that gathers the sums."""
+    bits_list = [int(v) for v in args.bits.split(",")] if args.bits else [3]
+    print("tensor bits grouping cosine rel_error us")
+    seen = set()
+    avg = {}
+    for spec in wl.config_tensors(args.config):
+        if spec.shape in seen or args.only not in spec.name:
+            continue
+        seen.add(spec.shape)
+        x = torch.from_numpy(wl.make_activation(spec)).cuda()
+        for bits in bits_list:
+            for name, group in (("layer-wise", b.GROUP_TENSOR), ("channel-wise", b.GROUP_CHANNEL)):
+                out = b.FakeQuantOut(y=torch.empty_like(x))
+                b.granq_fakequant_fused_stats(x, bits, group=group, out=out)
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                b.granq_fakequant_fused_stats(x, bits, group=group, out=out)
+                e1.record()
+                torch.cuda.synchronize()
+                assert b.workspace_status(out.workspace) == b.OK
+                cos, rel = b.distortion_from_sums(out.sums.cpu().tolist())
+                avg.setdefault((bits, name), []).append((cos, rel))
+                print(f"{spec.name} {bits} {name} {cos:.4f} {rel:.4f} {e0.elapsed_time(e1) * 1e3:.1f}", flush=True)
+        del x
+    for (bits, name), rows in avg.items():
+        print(f"average {bits} {name} {sum(r[0] for r in rows) / len(rows):.4f} "
+              f"{sum(r[1] for r in rows) / len(rows):.4f} -")
 
 
 if __name__ == "__main__":
