@@ -235,6 +235,36 @@ int granq_fakequant_fused_stats(const void* x, int dtype, const int64_t dims[4],
                                 void* cuda_stream);
 
 /*
+ * Channel-wise fake-quantization of many weight tensors in ONE launch (Section 5.1: all weights are
+ * quantized per output channel; Eq. 1, 2, 4-6 per channel, STE backward when a gradient is given).
+ * Tensor i is a contiguous [channels, group_elems] array of `dtype` (for a convolution weight
+ * [C_out, C_in, k, k]: channels = C_out, group_elems = C_in * k * k); each leading index is one
+ * group.  Results are those of granq_fakequant_fused() with channel_axis = 0 on every tensor.
+ *   descs       HOST array of n_tensors descriptors (read before the call returns); the pointers
+ *               inside are DEVICE memory: x in, y out, gy_opt / gx_opt both or neither,
+ *               min_out / max_out `channels` floats each (required), scale_opt / zp_opt or NULL
+ *   workspace   DEVICE scratch of granq_weights_workspace_bytes(n_tensors), 256-byte aligned
+ * Limits: fewer than 2^31 groups in the batch and 2^31 elements per group.
+ */
+typedef struct granq_weight_desc {
+    const void* x;
+    const void* gy_opt;
+    void* y;
+    void* gx_opt;
+    float* min_out;
+    float* max_out;
+    float* scale_opt;
+    float* zp_opt;
+    int64_t channels;
+    int64_t group_elems;
+    int32_t bits;
+    int32_t reserved;
+} granq_weight_desc;
+size_t granq_weights_workspace_bytes(int n_tensors);
+int granq_fakequant_weights(const granq_weight_desc* descs, int n_tensors, int dtype, void* workspace,
+                            size_t workspace_bytes, uint32_t flags, void* cuda_stream);
+
+/*
  * Status word the persistent plans leave in the workspace.  Synchronises `cuda_stream`, then
  * returns GRANQ_OK, GRANQ_ERR_TIMEOUT (a bounded device-side wait ran out), or
  * GRANQ_ERR_CUDA.  `workspace` is the pointer given to the preceding call.

@@ -34,6 +34,7 @@ EXPORTS = [
     "granq_tune", "granq_selftest_division", "granq_range_noalloc", "granq_packmask_bytes",
     "granq_fakequant_fwd_packmask", "granq_fakequant_bwd_packmask", "granq_fakequant_fused_fwd_packmask",
     "granq_host_arena_status", "granq_distortion", "granq_fakequant_fused_stats",
+    "granq_weights_workspace_bytes", "granq_fakequant_weights",
 ]
 NOALLOC_MAX_GROUPS = 32768
 
@@ -45,6 +46,14 @@ class GranqError(RuntimeError):
 
 
 _lib = None
+
+
+class WeightDesc(ctypes.Structure):
+    """granq_weight_desc of include/granq.h."""
+    _fields_ = [("x", ctypes.c_void_p), ("gy_opt", ctypes.c_void_p), ("y", ctypes.c_void_p),
+                ("gx_opt", ctypes.c_void_p), ("min_out", ctypes.c_void_p), ("max_out", ctypes.c_void_p),
+                ("scale_opt", ctypes.c_void_p), ("zp_opt", ctypes.c_void_p), ("channels", ctypes.c_int64),
+                ("group_elems", ctypes.c_int64), ("bits", ctypes.c_int32), ("reserved", ctypes.c_int32)]
 
 
 def lib() -> ctypes.CDLL:
@@ -96,6 +105,10 @@ def lib() -> ctypes.CDLL:
         L.granq_distortion.argtypes = [vp, vp, ci, i64p, vp, u32, vp]
         L.granq_fakequant_fused_stats.restype = ci
         L.granq_fakequant_fused_stats.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, vp, sz, u32, vp]
+        L.granq_weights_workspace_bytes.restype = sz
+        L.granq_weights_workspace_bytes.argtypes = [ci]
+        L.granq_fakequant_weights.restype = ci
+        L.granq_fakequant_weights.argtypes = [ctypes.POINTER(WeightDesc), ci, ci, vp, sz, u32, vp]
         L.granq_packmask_bytes.restype = sz
         L.granq_packmask_bytes.argtypes = [i64p]
         L.granq_fakequant_fwd_packmask.restype = ci
@@ -422,6 +435,55 @@ def granq_fakequant_fused_stats(x: torch.Tensor, bits: int, channel_axis: int = 
         _dev(o.hi, "hi"), _dev(o.s, "s"), _dev(o.z, "z"), _dev(o.sums, "sums"), _dev(o.workspace, "workspace"),
         o.workspace.numel(), flags, _stream(stream)), "granq_fakequant_fused_stats")
     return o
+
+
+class WeightBatch:
+    """All weight tensors of a model prepared for channel-wise (leading axis) fake-quantization in one
+    launch: descriptors and outputs are built once, `run()` is a single library call.
+
+    `weights`: contiguous CUDA tensors of one dtype, any rank >= 1 (axis 0 = output channels);
+    `bits`: one int or one per tensor; `grads`: upstream gradients (all or none)."""
+
+    def __init__(self, weights, bits, grads=None, want_params: bool = False):
+        n = len(weights)
+        self.n = n
+        self.dtype = _dtype(weights[0])
+        bits = [bits] * n if isinstance(bits, int) else list(bits)
+        self.descs = (WeightDesc * n)()
+        self.outs = []
+        self._keep = (list(weights), None if grads is None else list(grads))
+        for i, w in enumerate(weights):
+            if w.dtype != weights[0].dtype:
+                raise ValueError("all tensors of a batch must have one dtype")
+            c = w.shape[0]
+            o = FakeQuantOut(y=torch.empty_like(w), lo=torch.empty(c, dtype=torch.float32, device=w.device),
+                             hi=torch.empty(c, dtype=torch.float32, device=w.device))
+            g = None if grads is None else grads[i]
+            if g is not None:
+                if g.shape != w.shape or g.dtype != w.dtype:
+                    raise ValueError("gradient must match its weight")
+                o.gx = torch.empty_like(w)
+            if want_params:
+                o.s = torch.empty(c, dtype=torch.float32, device=w.device)
+                o.z = torch.empty(c, dtype=torch.float32, device=w.device)
+            self.descs[i] = WeightDesc(_dev(w, "w"), _dev(g, "g"), _dev(o.y, "y"), _dev(o.gx, "gx"),
+                                       _dev(o.lo, "lo"), _dev(o.hi, "hi"), _dev(o.s, "s"), _dev(o.z, "z"), c,
+                                       w.numel() // max(c, 1), bits[i], 0)
+            self.outs.append(o)
+        self.workspace = torch.empty(int(lib().granq_weights_workspace_bytes(n)), dtype=torch.uint8,
+                                     device=weights[0].device)
+
+    def run(self, workspace: torch.Tensor = None, stream=None):
+        ws = self.workspace if workspace is None else workspace
+        _check(lib().granq_fakequant_weights(self.descs, self.n, self.dtype, _dev(ws, "workspace"), ws.numel(), 0,
+                                             _stream(stream)), "granq_fakequant_weights")
+        return self.outs
+
+
+def granq_fakequant_weights(weights, bits, grads=None, want_params: bool = False, workspace: torch.Tensor = None,
+                            stream=None):
+    """One-shot form of WeightBatch: returns a list of FakeQuantOut (y, gx, lo, hi, and s / z with want_params)."""
+    return WeightBatch(weights, bits, grads, want_params).run(workspace, stream)
 
 
 def selftest_division(pairs: int, seed: int = 0, stream=None) -> int:

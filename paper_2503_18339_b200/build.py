@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libgranq.so")
-SOURCES = ["granq_api.cu", "granq_flat.cu", "granq_staged.cu", "granq_l2wave.cu", "granq_colwalk.cu", "granq_selftest.cu", "granq_noalloc.cu"]
+SOURCES = ["granq_api.cu", "granq_flat.cu", "granq_staged.cu", "granq_l2wave.cu", "granq_colwalk.cu", "granq_weights.cu", "granq_selftest.cu", "granq_noalloc.cu"]
 HEADERS = ["granq_device.cuh", "granq_internal.h"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-shared", "-cudart", "static"]

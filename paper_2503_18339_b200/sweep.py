@@ -48,8 +48,14 @@ def main() -> None:
     ap.add_argument("--distortion", action="store_true",
                     help="instead of the bandwidth sweep: the statistics of Table 2 (cosine similarity, relative "
                          "error) of layer-wise against channel-wise quantization on the config's tensors")
+    ap.add_argument("--weights", default="", choices=["", "resnet20", "resnet18"],
+                    help="instead of the bandwidth sweep: all weight tensors of the network in one batched "
+                         "launch against one fused call per tensor")
     args = ap.parse_args()
     b.lib()
+    if args.weights:
+        weights_table(args)
+        return
     if args.distortion:
         distortion_table(args)
         return
@@ -93,6 +99,40 @@ def main() -> None:
                     print(f"{spec.name} {dt} {bits} {mode} {us:.1f} {gbs:.0f} {gbs / peak:.3f}", flush=True)
             del x, gy, out
         del x32, g32
+
+
+def weights_table(args) -> None:
+    """Channel-wise fake-quantization (forward + STE backward) of every weight tensor of a network:
+    one batched launch against a loop of fused calls with channel_axis = 0."""
+    ws = [torch.from_numpy(w).cuda() for w in wl.make_weights(args.weights)]
+    gs = [torch.from_numpy(g).cuda() for g in wl.make_weights(args.weights, grads=True)]
+    elems = sum(w.numel() for w in ws)
+    ws4 = [w.reshape(w.shape[0], -1, 1, 1) for w in ws]
+    gs4 = [g.reshape(g.shape[0], -1, 1, 1) for g in gs]
+    outs = [b.FakeQuantOut(y=torch.empty_like(w), gx=torch.empty_like(w), workspace=b.make_workspace(w, 0)) for w in ws4]
+    batch = b.WeightBatch(ws, 4, grads=gs)
+
+    def batched():
+        batch.run()
+
+    def looped():
+        for w, g, o in zip(ws4, gs4, outs):
+            b.granq_fakequant_fused(w, 4, gy=g, channel_axis=0, out=o)
+
+    print("network tensors elements variant us GB/s(16 B/element)")
+    for name, fn in (("batched", batched), ("one call per tensor", looped)):
+        for _ in range(3):
+            fn()
+        times = []
+        for _ in range(max(args.iters, 5)):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            fn()
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1) * 1e3)
+        us = statistics.median(times)
+        print(f"{args.weights} {len(ws)} {elems} {name} {us:.1f} {elems * 16 / us / 1e3:.0f}", flush=True)
 
 
 def distortion_table(args) -> None:

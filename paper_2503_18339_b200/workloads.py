@@ -157,3 +157,50 @@ def to_bf16_bits(a: np.ndarray) -> np.ndarray:
 def bf16_bits_to_f32(h: np.ndarray) -> np.ndarray:
     """bf16 bit patterns (uint16) -> float32, exact."""
     return (np.ascontiguousarray(h, np.uint16).astype(np.uint32) << np.uint32(16)).view(np.float32)
+
+
+# ---------------------------------------------------------------------------------------
+# Weight tensors (Section 5.1: channel-wise quantization of all weights).  Shapes of the
+# convolution and classifier weights of ResNet-20 (CIFAR) and ResNet-18 (ImageNet); values
+# He-normal with a per-output-channel log-normal spread (trained weights are not available).
+# ---------------------------------------------------------------------------------------
+_STREAM_W, _STREAM_GW = 5, 6
+
+
+def weight_shapes(net: str) -> List[Tuple[int, ...]]:
+    """[C_out, C_in, k, k] (or [C_out, C_in]) of every quantized weight tensor of the network."""
+    if net == "resnet20":
+        shapes = [(16, 3, 3, 3)]
+        cin = 16
+        for cout in (16, 32, 64):
+            for blk in range(3):
+                shapes += [(cout, cin, 3, 3), (cout, cout, 3, 3)]
+                if blk == 0 and cin != cout:
+                    shapes.append((cout, cin, 1, 1))
+                cin = cout
+        return shapes + [(100, 64)]
+    if net == "resnet18":
+        shapes = [(64, 3, 7, 7)]
+        cin = 64
+        for cout in (64, 128, 256, 512):
+            for blk in range(2):
+                shapes += [(cout, cin, 3, 3), (cout, cout, 3, 3)]
+                if blk == 0 and cin != cout:
+                    shapes.append((cout, cin, 1, 1))
+                cin = cout
+        return shapes + [(1000, 512)]
+    raise ValueError(net)
+
+
+def make_weights(net: str, seed: int = 7000, grads: bool = False) -> List[np.ndarray]:
+    """fp32 weight tensors (or their upstream gradients ~ N(0, 1e-2)) of `net`, seeded per tensor."""
+    out = []
+    for i, shape in enumerate(weight_shapes(net)):
+        fan_in = int(np.prod(shape[1:]))
+        if grads:
+            w = _rng(seed, _STREAM_GW, i).standard_normal(shape) * 0.1
+        else:
+            spread = np.exp(0.5 * _rng(seed, _STREAM_SIGMA, i).standard_normal((shape[0],) + (1,) * (len(shape) - 1)))
+            w = _rng(seed, _STREAM_W, i).standard_normal(shape) * np.sqrt(2.0 / fan_in) * spread
+        out.append((w.astype(np.float32) + np.float32(0)))
+    return out
