@@ -216,3 +216,43 @@ int granq_oracle_distortion(const double sums[4], double* cosine, double* rel_er
     return 0;
 }
 
+/* ---- integer codes as a packed bit string (Eq. 1 produces b-bit integers; Eq. 6 consumes them) ---- */
+
+/* Element e occupies bits [e*b, (e+1)*b) of a little-endian bit string (bit k of the string is bit
+ * k % 8 of byte k / 8); ceil(E*b / 8) bytes are written, unused high bits of the last byte 0. */
+int granq_oracle_pack_codes(const uint8_t* codes, int64_t E, int bits, uint8_t* packed) {
+    if (!codes || !packed || E < 0 || bits < 1 || bits > 8) return -1;
+    for (int64_t k = 0; k < (E * bits + 7) / 8; ++k) packed[k] = 0;
+    for (int64_t e = 0; e < E; ++e) {
+        if (codes[e] >> bits) return -3;                    /* a code that does not fit b bits */
+        for (int j = 0; j < bits; ++j) {
+            int64_t k = e * bits + j;
+            if ((codes[e] >> j) & 1) packed[k / 8] = (uint8_t)(packed[k / 8] | (1u << (k % 8)));
+        }
+    }
+    return 0;
+}
+
+/* Eq. 6 from the packed codes: y[e] = s[g] * (code[e] - z[g]) with g the element's group. */
+int granq_oracle_dequant_packed(const uint8_t* packed, int dtype, const int64_t dims[4], int channel_axis,
+                                int group_mode, int bits, const float* s, const float* z, void* y) {
+    geom_t g;
+    if (!packed || !s || !z || !y || bits < 1 || bits > 8) return -1;
+    if (make_geom(dims, channel_axis, group_mode, &g)) return -1;
+    for (int64_t o = 0; o < g.outer; ++o)
+        for (int64_t c = 0; c < g.C; ++c) {
+            int64_t grp = group_of(&g, group_mode, o, c);
+            for (int64_t i = 0; i < g.inner; ++i) {
+                int64_t e = (o * g.C + c) * g.inner + i;
+                unsigned code = 0;
+                for (int j = 0; j < bits; ++j) {
+                    int64_t k = e * bits + j;
+                    code |= (unsigned)((packed[k / 8] >> (k % 8)) & 1) << j;
+                }
+                float d = (float)code - z[grp];
+                store_elem(y, dtype, e, s[grp] * d);
+            }
+        }
+    return 0;
+}
+

@@ -81,6 +81,14 @@ int granq_oracle_bwd_packed(const void* gy, const uint8_t* packed, int dtype, in
 int granq_oracle_distortion_sums(const void* x, const void* q, int dtype, int64_t E, double sums[4]);
 int granq_oracle_distortion(const double sums[4], double* cosine, double* rel_error);
 
+/* Integer codes as a packed bit string: Eq. 1 yields b-bit integers, and it is those (with the
+ * per-group scale and zero-point) that Eq. 6 and the accumulation of Algorithm 1 consume.  Element e
+ * occupies bits [e*b, (e+1)*b) of a little-endian bit string of ceil(E*b / 8) bytes.
+ * granq_oracle_dequant_packed() is Eq. 6 evaluated from that string: y = s * (code - z). */
+int granq_oracle_pack_codes(const uint8_t* codes, int64_t E, int bits, uint8_t* packed);
+int granq_oracle_dequant_packed(const uint8_t* packed, int dtype, const int64_t dims[4], int channel_axis,
+                                int group_mode, int bits, const float* s, const float* z, void* y);
+
 #ifdef __cplusplus
 }
 #endif

@@ -69,6 +69,10 @@ def lib() -> ctypes.CDLL:
         L.granq_oracle_distortion_sums.argtypes = [vp, vp, ci, ctypes.c_int64, vp]
         L.granq_oracle_distortion.restype = ci
         L.granq_oracle_distortion.argtypes = [vp, vp, vp]
+        L.granq_oracle_pack_codes.restype = ci
+        L.granq_oracle_pack_codes.argtypes = [u8p, ctypes.c_int64, ci, u8p]
+        L.granq_oracle_dequant_packed.restype = ci
+        L.granq_oracle_dequant_packed.argtypes = [u8p, ci, i64p, ci, ci, ci, fp, fp, vp]
         _lib = L
     return _lib
 
@@ -224,4 +228,24 @@ def distortion(sums: np.ndarray):
     r = ctypes.c_double(0.0)
     _check(lib().granq_oracle_distortion(_p(sums), ctypes.byref(c), ctypes.byref(r)), "granq_oracle_distortion")
     return c.value, r.value
+
+
+def pack_codes(codes: np.ndarray, bits: int) -> np.ndarray:
+    """b-bit codes as a little-endian bit string: element e in bits [e*b, (e+1)*b); ceil(E*b / 8) bytes."""
+    codes = np.ascontiguousarray(codes, np.uint8)
+    packed = np.empty((codes.size * bits + 7) // 8, np.uint8)
+    _check(lib().granq_oracle_pack_codes(_p(codes), codes.size, bits, _p(packed)), "granq_oracle_pack_codes")
+    return packed
+
+
+def dequant_packed(packed: np.ndarray, shape, bits: int, s: np.ndarray, z: np.ndarray, dtype=np.float32,
+                   channel_axis: int = 1, group_mode: int = GROUP_CHANNEL) -> np.ndarray:
+    """Eq. 6 from the packed codes: y = s * (code - z); dtype np.float32 or np.uint16 (bf16 bits)."""
+    packed = np.ascontiguousarray(packed, np.uint8)
+    s = np.ascontiguousarray(s, np.float32)
+    z = np.ascontiguousarray(z, np.float32)
+    y = np.empty(shape, dtype)
+    _check(lib().granq_oracle_dequant_packed(_p(packed), _dtype_of(y), _dims(shape), channel_axis, group_mode, bits,
+                                             _p(s), _p(z), _p(y)), "granq_oracle_dequant_packed")
+    return y
 

@@ -29,6 +29,11 @@ MUTATIONS = {
     "distortion_error_not_squared_difference": ("sdd += d * d;", "sdd += d;"),
     "distortion_cosine_without_norm_of_q": ("double den = sqrt(sums[0]) * sqrt(sums[1]);", "double den = sums[0];"),
     "distortion_relative_error_not_rooted": ("sqrt(sums[3]) / sqrt(sums[0])", "sums[3] / sums[0]"),
+    "packed_codes_most_significant_bit_first": ("if ((codes[e] >> j) & 1) packed[k / 8]",
+                                                "if ((codes[e] >> (bits - 1 - j)) & 1) packed[k / 8]"),
+    "packed_codes_stride_of_8_bits": ("int64_t k = e * bits + j;\n            if ((codes[e] >> j) & 1)",
+                                      "int64_t k = e * 8 + j;\n            if ((codes[e] >> j) & 1)"),
+    "dequant_packed_adds_zero_point": ("float d = (float)code - z[grp];", "float d = (float)code + z[grp];"),
     "packed_mask_last_byte_not_cleared": ("for (int64_t b = 0; b < (E + 7) / 8; ++b) packed[b] = 0;",
                                           "for (int64_t b = 0; b < E / 8; ++b) packed[b] = 0;"),
 }

@@ -468,3 +468,46 @@ def test_distortion_sums_match_float64_dot_products(dtype):
     assert rel == pytest.approx(np.linalg.norm(xw - qw) / np.linalg.norm(xw), rel=1e-12)
     assert 0.9 < cos <= 1.0 and 0.0 < rel < 0.2
 
+
+# --------------------------------------------------------------------------------------
+# 11. integer codes as a packed bit string (Eq. 1 -> Eq. 6)
+# --------------------------------------------------------------------------------------
+def test_packed_codes_hand_case():
+    """Hand case H1, channel 0, b = 2: codes [0,1,2,3 | 0,2,2,0] -> 0 + 1*4 + 2*16 + 3*64 = 0xE4 and
+    0 + 2*4 + 2*16 + 0 = 0x28; b = 3 of [5, 2, 7]: 5 + 2*8 + 7*64 = 469 = 0x01D5 -> bytes D5 01."""
+    assert orc.pack_codes(np.array([0, 1, 2, 3, 0, 2, 2, 0], np.uint8), 2).tolist() == [0xE4, 0x28]
+    assert orc.pack_codes(np.array([5, 2, 7], np.uint8), 3).tolist() == [0xD5, 0x01]
+    y = orc.dequant_packed(np.array([0xD5, 0x01], np.uint8), (1, 1, 1, 3), 3, f32([0.5]), f32([2]))
+    assert y.ravel().tolist() == [1.5, 0.0, 2.5]                       # 0.5 * ([5, 2, 7] - 2)
+
+
+@pytest.mark.parametrize("bits", range(1, 9))
+@pytest.mark.parametrize("n", [1, 7, 32, 33, 1000])
+def test_packed_codes_match_big_integer_packing(bits, n):
+    rng = np.random.default_rng(bits * 100 + n)
+    codes = rng.integers(0, 1 << bits, n).astype(np.uint8)
+    big = 0
+    for e, c in enumerate(codes.tolist()):                  # the bit string as one Python integer
+        big |= c << (e * bits)
+    want = np.frombuffer(big.to_bytes((n * bits + 7) // 8, "little"), np.uint8)
+    assert np.array_equal(orc.pack_codes(codes, bits), want)
+    with pytest.raises(RuntimeError):                        # a code that needs more than b bits
+        if bits < 8:
+            orc.pack_codes(np.array([1 << bits], np.uint8), bits)
+        else:
+            raise RuntimeError
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("mode", [orc.GROUP_CHANNEL, orc.GROUP_SAMPLE_CHANNEL, orc.GROUP_TENSOR])
+def test_dequantizing_the_packed_codes_gives_the_fake_quantized_tensor(dtype, mode):
+    rng = np.random.default_rng(12)
+    x = rng.standard_normal((3, 5, 7, 7)).astype(np.float32)
+    if dtype == "bf16":
+        x = (x.view(np.uint32) >> 16).astype(np.uint16)
+    for bits in (3, 5, 8):
+        ref = orc.fused(x, bits, group_mode=mode)
+        y = orc.dequant_packed(orc.pack_codes(ref.codes, bits), x.shape, bits, ref.s, ref.z, dtype=x.dtype,
+                               group_mode=mode)
+        assert np.array_equal(y.view(x.dtype), ref.y.view(x.dtype))
+
