@@ -265,6 +265,27 @@ int granq_fakequant_weights(const granq_weight_desc* descs, int n_tensors, int d
                             size_t workspace_bytes, uint32_t flags, void* cuda_stream);
 
 /*
+ * Integer codes as a packed bit string (Eq. 1 yields b-bit integers; Eq. 6 and the accumulation of
+ * Algorithm 1 consume them together with the per-group scale and zero-point).  Element e occupies bits
+ * [e*b, (e+1)*b) of a little-endian bit string (bit k of the string = bit k % 32 of word k / 32);
+ * the buffer holds granq_packed_codes_bytes() = 4 * ceil(E*b / 32) bytes, 4-byte aligned, DEVICE memory;
+ * bits beyond the last element are written as 0.  An activation kept this way takes b/32 of its fp32 size.
+ *
+ * granq_quantize_packed():   Eq. 1 + clamp with a supplied range -> packed codes, scale and zero-point
+ *                            (both required: they are what gives the codes a meaning); y_opt, when not
+ *                            NULL, also receives the dequantized values as granq_fakequant_fwd() would.
+ * granq_dequantize_packed(): Eq. 6, y = s * (code - z), from the packed codes; bit for bit the y of
+ *                            granq_fakequant_fwd() for the same range.
+ */
+size_t granq_packed_codes_bytes(const int64_t dims[4], int bits);
+int granq_quantize_packed(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group, int bits,
+                          const float* min_in, const float* max_in, uint32_t* packed_codes, void* y_opt,
+                          float* scale_out, float* zp_out, uint32_t flags, void* cuda_stream);
+int granq_dequantize_packed(const uint32_t* packed_codes, int dtype, const int64_t dims[4], int channel_axis,
+                            int group, int bits, const float* scale_in, const float* zp_in, void* y, uint32_t flags,
+                            void* cuda_stream);
+
+/*
  * Status word the persistent plans leave in the workspace.  Synchronises `cuda_stream`, then
  * returns GRANQ_OK, GRANQ_ERR_TIMEOUT (a bounded device-side wait ran out), or
  * GRANQ_ERR_CUDA.  `workspace` is the pointer given to the preceding call.

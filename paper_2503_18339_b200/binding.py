@@ -34,7 +34,8 @@ EXPORTS = [
     "granq_tune", "granq_selftest_division", "granq_range_noalloc", "granq_packmask_bytes",
     "granq_fakequant_fwd_packmask", "granq_fakequant_bwd_packmask", "granq_fakequant_fused_fwd_packmask",
     "granq_host_arena_status", "granq_distortion", "granq_fakequant_fused_stats",
-    "granq_weights_workspace_bytes", "granq_fakequant_weights",
+    "granq_weights_workspace_bytes", "granq_fakequant_weights", "granq_packed_codes_bytes",
+    "granq_quantize_packed", "granq_dequantize_packed",
 ]
 NOALLOC_MAX_GROUPS = 32768
 
@@ -109,6 +110,12 @@ def lib() -> ctypes.CDLL:
         L.granq_weights_workspace_bytes.argtypes = [ci]
         L.granq_fakequant_weights.restype = ci
         L.granq_fakequant_weights.argtypes = [ctypes.POINTER(WeightDesc), ci, ci, vp, sz, u32, vp]
+        L.granq_packed_codes_bytes.restype = sz
+        L.granq_packed_codes_bytes.argtypes = [i64p, ci]
+        L.granq_quantize_packed.restype = ci
+        L.granq_quantize_packed.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, u32, vp]
+        L.granq_dequantize_packed.restype = ci
+        L.granq_dequantize_packed.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, u32, vp]
         L.granq_packmask_bytes.restype = sz
         L.granq_packmask_bytes.argtypes = [i64p]
         L.granq_fakequant_fwd_packmask.restype = ci
@@ -227,6 +234,7 @@ class FakeQuantOut:
     workspace: Optional[torch.Tensor] = None
     packed_mask: Optional[torch.Tensor] = None      # int32 words, one bit per element
     sums: Optional[torch.Tensor] = None             # 4 doubles: sum x^2, sum q^2, sum x*q, sum (x-q)^2
+    packed_codes: Optional[torch.Tensor] = None     # int32 words: the codes as a bit string, b bits each
 
 
 def granq_range(x: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL, lo: torch.Tensor = None,
@@ -484,6 +492,40 @@ def granq_fakequant_weights(weights, bits, grads=None, want_params: bool = False
                             stream=None):
     """One-shot form of WeightBatch: returns a list of FakeQuantOut (y, gx, lo, hi, and s / z with want_params)."""
     return WeightBatch(weights, bits, grads, want_params).run(workspace, stream)
+
+
+def packed_codes_bytes(shape, bits: int) -> int:
+    return int(lib().granq_packed_codes_bytes(_dims(shape), bits))
+
+
+def granq_quantize_packed(x: torch.Tensor, bits: int, lo: torch.Tensor, hi: torch.Tensor, channel_axis: int = 1,
+                          group: int = GROUP_CHANNEL, want_y: bool = False, packed_codes: torch.Tensor = None,
+                          stream=None) -> FakeQuantOut:
+    """Eq. 1 + clamp with a given range -> integer codes as a bit string (b bits each), scale, zero-point."""
+    G = num_groups(x.shape, channel_axis, group)
+    o = FakeQuantOut(lo=lo, hi=hi)
+    o.packed_codes = (torch.empty(packed_codes_bytes(x.shape, bits) // 4, dtype=torch.int32, device=x.device)
+                      if packed_codes is None else packed_codes)
+    o.s = torch.empty(G, dtype=torch.float32, device=x.device)
+    o.z = torch.empty(G, dtype=torch.float32, device=x.device)
+    if want_y:
+        o.y = torch.empty_like(x)
+    _check(lib().granq_quantize_packed(_dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, bits,
+                                       _dev(lo, "lo"), _dev(hi, "hi"), _dev(o.packed_codes, "packed_codes"),
+                                       _dev(o.y, "y"), _dev(o.s, "s"), _dev(o.z, "z"), 0, _stream(stream)),
+           "granq_quantize_packed")
+    return o
+
+
+def granq_dequantize_packed(packed_codes: torch.Tensor, shape, dtype: torch.dtype, bits: int, s: torch.Tensor,
+                            z: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL,
+                            y: torch.Tensor = None, stream=None) -> torch.Tensor:
+    """Eq. 6 from the packed codes: y = s * (code - z)."""
+    y = torch.empty(tuple(shape), dtype=dtype, device=packed_codes.device) if y is None else y
+    _check(lib().granq_dequantize_packed(_dev(packed_codes, "packed_codes"), _dtype(y), _dims(shape), channel_axis,
+                                         group, bits, _dev(s, "s"), _dev(z, "z"), _dev(y, "y"), 0, _stream(stream)),
+           "granq_dequantize_packed")
+    return y
 
 
 def selftest_division(pairs: int, seed: int = 0, stream=None) -> int:

@@ -371,6 +371,47 @@ int granq_fakequant_fused_stats(const void* x, int dtype, const int64_t dims[4],
     return cuda_status(e);
 }
 
+size_t granq_packed_codes_bytes(const int64_t dims[4], int bits) {
+    Geom g;
+    int64_t G;
+    if (bits < 1 || bits > 8 || !make_geom(dims, 1, GRANQ_GROUP_TENSOR, g, G)) return 0;
+    return (size_t)((g.E * bits + 31) / 32) * 4;
+}
+
+int granq_quantize_packed(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group, int bits,
+                          const float* min_in, const float* max_in, uint32_t* packed_codes, void* y_opt,
+                          float* scale_out, float* zp_out, uint32_t flags, void* cuda_stream) {
+    (void)flags;
+    Geom g;
+    int64_t G;
+    if (!x || !packed_codes || !min_in || !max_in || !scale_out || !zp_out || bits < 1 || bits > 8 ||
+        !dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G) || ((uintptr_t)packed_codes & 3))
+        return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
+    const size_t nb = (size_t)g.E * elt_size(dtype), cbytes = (size_t)((g.E * bits + 31) / 32) * 4;
+    if (overlaps(x, nb, y_opt, nb) || overlaps(x, nb, packed_codes, cbytes) || overlaps(y_opt, nb, packed_codes, cbytes))
+        return GRANQ_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    QuantIO io{x, nullptr, y_opt, nullptr, nullptr, nullptr, nullptr, nullptr, packed_codes, bits};
+    cudaError_t e = launch_quant_flat(io, MODE_FWD, dtype, g, bits, min_in, max_in, st);
+    if (e == cudaSuccess) e = launch_params(min_in, max_in, G, bits, scale_out, zp_out, st);
+    return cuda_status(e);
+}
+
+int granq_dequantize_packed(const uint32_t* packed_codes, int dtype, const int64_t dims[4], int channel_axis,
+                            int group, int bits, const float* scale_in, const float* zp_in, void* y, uint32_t flags,
+                            void* cuda_stream) {
+    (void)flags;
+    Geom g;
+    int64_t G;
+    if (!packed_codes || !scale_in || !zp_in || !y || bits < 1 || bits > 8 || !dtype_ok(dtype) ||
+        !make_geom(dims, channel_axis, group, g, G) || ((uintptr_t)packed_codes & 3))
+        return GRANQ_ERR_INVALID_ARG;
+    const size_t nb = (size_t)g.E * elt_size(dtype), cbytes = (size_t)((g.E * bits + 31) / 32) * 4;
+    if (overlaps(y, nb, packed_codes, cbytes)) return GRANQ_ERR_INVALID_ARG;
+    return cuda_status(launch_dequant_packed(packed_codes, y, dtype, g, bits, scale_in, zp_in, (cudaStream_t)cuda_stream));
+}
+
 int granq_workspace_status(const void* workspace, void* cuda_stream) {
     if (!workspace) return GRANQ_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)cuda_stream;

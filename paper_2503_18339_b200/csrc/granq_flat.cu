@@ -241,6 +241,29 @@ __global__ void params_kernel(const float* __restrict__ lo, const float* __restr
     if (z_opt) z_opt[i] = p.z;
 }
 
+// Packing a warp's row of integer codes into a bit string.  Every lane holds `nb` bits (its V codes
+// of b bits, nb = V * b <= 64): lane i owns bits [i * nb, (i + 1) * nb) of a row of nb 32-bit words.
+// Lane k returns word k of the row in out[0] and word k + 32 in out[1] (0 where the row has no such
+// word); all 32 lanes must call.
+__device__ __forceinline__ void warp_pack_row(uint64_t mine, uint32_t nb, uint32_t lane, uint32_t (&out)[2]) {
+    const uint32_t nsrc = 32 / nb + 2;                   // lanes whose bits can fall into one word
+    out[0] = 0;
+    out[1] = 0;
+    const int halves = nb > 32 ? 2 : 1;
+    for (int h = 0; h < halves; ++h) {
+        const uint32_t wk = lane + 32 * h;               // word of the row this lane assembles
+        const uint32_t first = (32 * wk) / nb;           // first lane that reaches into it
+        uint32_t acc = 0;
+        for (uint32_t j = 0; j < nsrc; ++j) {
+            const uint32_t src = first + j;
+            const uint64_t v = __shfl_sync(kFullMask, mine, src & 31);
+            const int off = (int)(src * nb) - (int)(32 * wk);       // where src's bits start, relative to the word
+            if (src < 32 && off < 32 && wk < nb) acc |= (uint32_t)(off >= 0 ? (v << off) : (v >> (-off)));
+        }
+        out[h] = acc;
+    }
+}
+
 // ---- Eq. 1, clamp, Eq. 6, STE: elementwise pass with a given per-group range ----------------------
 // EXTRAS: the optional codes / mask / packed-mask outputs are compiled in.  The packed mask holds
 // one bit per element (bit e % 32 of word e / 32): a warp's lanes own consecutive elements or packs
@@ -251,7 +274,9 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                                                               uint8_t* __restrict__ codes,
                                                               uint8_t* __restrict__ mask,
                                                               uint32_t* __restrict__ pmask,
-                                                              double* __restrict__ dist, FlatGeom g, float qmax,
+                                                              double* __restrict__ dist,
+                                                              uint32_t* __restrict__ pcodes, int code_bits,
+                                                              FlatGeom g, float qmax,
                                                               const float* __restrict__ lo,
                                                               const float* __restrict__ hi) {
     __shared__ TileBase s_base;
@@ -299,6 +324,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
             for (int j = 0; j < kUnroll; ++j) {
                 const bool valid = k[j] < ne;
                 uint32_t inside_bits = 0;            // bit i: the clamp was inactive for this thread's element i
+                uint64_t code_string = 0;            // this thread's V codes, b bits each, first element lowest
                 if (valid) {
                 const uint32_t q = plane_offset(g, base, k[j]);
                 QParam p;
@@ -317,9 +343,10 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                     bool in;
                     float code = quant_one(sx[j], p, qmax, yv, in);
                     inside_bits = in ? 1u : 0u;
+                    code_string = (uint64_t)code;
                     if constexpr (kFwd) {
                         if (dist) dacc.add_one(sx[j], as_stored(yv, y));
-                        store_scalar(y + e, yv);
+                        if (y) store_scalar(y + e, yv);
                         if (codes) codes[e] = (uint8_t)code;
                     }
                     if constexpr (kBwd) {
@@ -340,10 +367,15 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                         for (int i = 0; i < V; ++i) inside_bits |= ((mb[i / 4] >> (8 * (i % 4))) & 1u) << i;
                         if constexpr (kFwd) {
                             if (dist) dacc.add(px[j], py);
+                            if (pcodes) {
+#pragma unroll
+                                for (int i = 0; i < V; ++i)
+                                    code_string |= (uint64_t)((cb[i / 4] >> (8 * (i % 4))) & 0xFFu) << (i * code_bits);
+                            }
                         }
                     }
                     if constexpr (kFwd) {
-                        st_stream_16(y + e, py.raw);
+                        if (!EXTRAS || y) st_stream_16(y + e, py.raw);
                         if constexpr (EXTRAS) {
                             if (codes) {
 #pragma unroll
@@ -376,6 +408,16 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                             for (uint32_t d = 1; d < kLanes; d <<= 1) w |= __shfl_xor_sync(kFullMask, w, d);
                             if ((lane & (kLanes - 1)) == 0 && valid) pmask[word] = w;
                         }
+                    }
+                    if (pcodes) {         // the warp's 32 * V codes are V * b whole words of the bit string
+                        const uint32_t lane = threadIdx.x & 31;
+                        const uint32_t nb = (uint32_t)(V * code_bits);
+                        const int64_t row_e = e0 + k0 + (int64_t)(j * kThreads + (threadIdx.x & ~31u)) * V;
+                        const int64_t word0 = (row_e >> 5) * code_bits, nwords = (g.E * code_bits + 31) >> 5;
+                        uint32_t out[2];
+                        warp_pack_row(code_string, nb, lane, out);
+                        if (lane < nb && word0 + lane < nwords) pcodes[word0 + lane] = out[0];
+                        if (lane + 32 < nb && word0 + lane + 32 < nwords) pcodes[word0 + lane + 32] = out[1];
                     }
                 }
             }
@@ -510,6 +552,42 @@ __global__ void __launch_bounds__(kThreads) distortion_kernel(const T* __restric
     acc.flush(sums);
 }
 
+// ---- Eq. 6 from the packed integer codes: y = s * (code - z) --------------------------------------
+// V = elements per thread and step (a 16-byte pack of y when E and the pointer allow it, else 1).
+template <typename T, int V>
+__global__ void __launch_bounds__(kThreads) dequant_packed_kernel(const uint32_t* __restrict__ pcodes,
+                                                                  T* __restrict__ y, int64_t E, int64_t inner,
+                                                                  int64_t C, int bits,
+                                                                  const float* __restrict__ s,
+                                                                  const float* __restrict__ z) {
+    const int64_t nunits = E / V;
+    const uint32_t field = (1u << bits) - 1u;
+    for (int64_t u = (int64_t)blockIdx.x * kThreads + threadIdx.x; u < nunits; u += (int64_t)gridDim.x * kThreads) {
+        const int64_t e = u * V;
+        int64_t plane = e / inner, rem = e - plane * inner;
+        int64_t grp = plane % C;
+        float sg = __ldg(s + grp), zg = __ldg(z + grp);
+        Pack<T> out;
+#pragma unroll
+        for (int i = 0; i < V; ++i) {
+            const int64_t bit = (e + i) * bits;
+            const uint32_t o = (uint32_t)(bit & 31);
+            uint32_t v = __ldg(pcodes + (bit >> 5)) >> o;
+            if (o + (uint32_t)bits > 32u) v |= __ldg(pcodes + (bit >> 5) + 1) << (32u - o);
+            const float yv = __fmul_rn(sg, __fsub_rn((float)(v & field), zg));
+            if constexpr (V == 1) store_scalar(y + e, yv);
+            else out.set(i, yv);
+            if (V > 1 && ++rem == inner) {          // the next element starts the next plane
+                rem = 0;
+                grp = (grp + 1 == C) ? 0 : grp + 1;
+                sg = __ldg(s + grp);
+                zg = __ldg(z + grp);
+            }
+        }
+        if constexpr (V > 1) st_stream_16(y + e, out.raw);
+    }
+}
+
 bool aligned16(const void* p) { return p == nullptr || ((uintptr_t)p & 15) == 0; }
 
 int flat_grid(const FlatGeom& f) {
@@ -564,16 +642,17 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
                ((uintptr_t)io.codes % 4 == 0) && ((uintptr_t)io.mask % 4 == 0);
     int grid = flat_grid(f);
     float qmax = (float)((1 << bits) - 1);
-    const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr || io.dist != nullptr;
+    const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr || io.dist != nullptr ||
+                        io.pcodes != nullptr;
     if (vec && extras)
         quant_flat_kernel<T, VF, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                        (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, f, qmax, lo, hi);
+                                                                        (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes, io.code_bits, f, qmax, lo, hi);
     else if (vec)
         quant_flat_kernel<T, VF, MODE, false><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                         (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, f, qmax, lo, hi);
+                                                                         (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes, io.code_bits, f, qmax, lo, hi);
     else
         quant_flat_kernel<T, 1, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
-                                                                       (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, f, qmax, lo, hi);
+                                                                       (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes, io.code_bits, f, qmax, lo, hi);
     return cudaGetLastError();
 }
 
@@ -686,6 +765,30 @@ cudaError_t launch_distortion(const void* x, const void* q, int dtype, int64_t E
         else
             distortion_kernel<__nv_bfloat16, 1><<<grid, kThreads, 0, st>>>((const __nv_bfloat16*)x,
                                                                            (const __nv_bfloat16*)q, E, sums);
+    }
+    return cudaGetLastError();
+}
+
+cudaError_t launch_dequant_packed(const uint32_t* pcodes, void* y, int dtype, const Geom& g, int bits,
+                                  const float* s, const float* z, cudaStream_t st) {
+    int dev = 0, sms = 148;
+    cudaGetDevice(&dev);
+    cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    const int VF = dtype == 0 ? 4 : 8;
+    const bool vec = aligned16(y) && (g.E % VF == 0);
+    const int64_t units = vec ? g.E / VF : g.E;
+    const int64_t ctas = (units + kThreads - 1) / kThreads, cap = (int64_t)sms * 16;
+    const int grid = (int)(ctas < 1 ? 1 : (ctas < cap ? ctas : cap));
+    if (dtype == 0) {
+        if (vec) dequant_packed_kernel<float, 4><<<grid, kThreads, 0, st>>>(pcodes, (float*)y, g.E, g.inner, g.C, bits, s, z);
+        else dequant_packed_kernel<float, 1><<<grid, kThreads, 0, st>>>(pcodes, (float*)y, g.E, g.inner, g.C, bits, s, z);
+    } else {
+        if (vec)
+            dequant_packed_kernel<__nv_bfloat16, 8><<<grid, kThreads, 0, st>>>(pcodes, (__nv_bfloat16*)y, g.E, g.inner,
+                                                                               g.C, bits, s, z);
+        else
+            dequant_packed_kernel<__nv_bfloat16, 1><<<grid, kThreads, 0, st>>>(pcodes, (__nv_bfloat16*)y, g.E, g.inner,
+                                                                               g.C, bits, s, z);
     }
     return cudaGetLastError();
 }

@@ -55,6 +55,8 @@ struct QuantIO {
     uint8_t* mask;    // optional
     uint32_t* pmask;  // optional: the mask at one bit per element (forward plans that support it)
     double* dist;     // optional: 4 running sums of Table 2's statistics, zero on entry (same plans)
+    uint32_t* pcodes; // optional: the integer codes as a bit string, code_bits each (flat forward kernel; y may then be null)
+    int code_bits;
 };
 
 // ---- generic ("flat") kernels: any geometry, any alignment --------------------------------
@@ -75,6 +77,9 @@ cudaError_t launch_bwd_packmask(const void* gy, const uint32_t* pmask, void* gx,
                                 cudaStream_t st);
 // sums[0..3] += sum x^2, sum q^2, sum x*q, sum (x-q)^2 over E elements (Table 2's raw material)
 cudaError_t launch_distortion(const void* x, const void* q, int dtype, int64_t E, double* sums, cudaStream_t st);
+// Eq. 6 from the packed integer codes (element e in bits [e*b, (e+1)*b) of the bit string)
+cudaError_t launch_dequant_packed(const uint32_t* pcodes, void* y, int dtype, const Geom& g, int bits, const float* s,
+                                  const float* z, cudaStream_t st);
 // the "conventional" scheme: a host loop over groups with three launches each
 cudaError_t launch_naive(const QuantIO& io, int mode, int dtype, const Geom& g, int bits, uint32_t* kmin,
                          uint32_t* kmax, float* lo, float* hi, cudaStream_t st, int* launches);
