@@ -245,19 +245,40 @@ __global__ void params_kernel(const float* __restrict__ lo, const float* __restr
 // of b bits, nb = V * b <= 64): lane i owns bits [i * nb, (i + 1) * nb) of a row of nb 32-bit words.
 // Lane k returns word k of the row in out[0] and word k + 32 in out[1] (0 where the row has no such
 // word); all 32 lanes must call.
-__device__ __forceinline__ void warp_pack_row(uint64_t mine, uint32_t nb, uint32_t lane, uint32_t (&out)[2]) {
-    const uint32_t nsrc = 32 / nb + 2;                   // lanes whose bits can fall into one word
+__device__ __forceinline__ void warp_pack_row(uint64_t mine, uint32_t nb, uint32_t lane, uint32_t first0,
+                                              uint32_t first1, uint32_t (&out)[2]) {
+    // first0 / first1 = (32 * lane) / nb and (32 * (lane + 32)) / nb: the first lane that reaches into the
+    // word(s) this lane assembles (lane constants, worked out once per kernel)
     out[0] = 0;
     out[1] = 0;
-    const int halves = nb > 32 ? 2 : 1;
-    for (int h = 0; h < halves; ++h) {
+    if ((nb & (nb - 1)) == 0 && nb <= 32) {              // 32 / nb lanes make up one word exactly
+        const uint32_t lpw = 32 / nb;
+        uint32_t w = (uint32_t)mine << (nb * (lane & (lpw - 1)));
+        for (uint32_t d = 1; d < lpw; d <<= 1) w |= __shfl_xor_sync(kFullMask, w, d);
+        out[0] = __shfl_sync(kFullMask, w, (lane * lpw) & 31);      // word k sits in lanes k * lpw ...
+        return;
+    }
+    const uint32_t nsrc = 32 / nb + 2;                   // lanes whose bits can fall into one word
+    if (nb <= 32) {                                      // one word per lane at most, 32-bit shuffles
+        const uint32_t lo = (uint32_t)mine;
+        uint32_t acc = 0;
+        for (uint32_t j = 0; j < nsrc; ++j) {
+            const uint32_t src = first0 + j;
+            const uint32_t v = __shfl_sync(kFullMask, lo, src & 31);
+            const int off = (int)(src * nb) - (int)(32 * lane);     // where src's bits start, relative to the word
+            if (src < 32 && off < 32 && lane < nb) acc |= off >= 0 ? (v << off) : (v >> (-off));
+        }
+        out[0] = acc;
+        return;
+    }
+    for (int h = 0; h < 2; ++h) {
         const uint32_t wk = lane + 32 * h;               // word of the row this lane assembles
-        const uint32_t first = (32 * wk) / nb;           // first lane that reaches into it
+        const uint32_t first = h ? first1 : first0;
         uint32_t acc = 0;
         for (uint32_t j = 0; j < nsrc; ++j) {
             const uint32_t src = first + j;
             const uint64_t v = __shfl_sync(kFullMask, mine, src & 31);
-            const int off = (int)(src * nb) - (int)(32 * wk);       // where src's bits start, relative to the word
+            const int off = (int)(src * nb) - (int)(32 * wk);
             if (src < 32 && off < 32 && wk < nb) acc |= (uint32_t)(off >= 0 ? (v << off) : (v >> (-off)));
         }
         out[h] = acc;
@@ -284,6 +305,8 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
     constexpr bool kFwd = (MODE & MODE_FWD) != 0, kBwd = (MODE & MODE_BWD) != 0;
     DistAcc dacc;
     dacc.reset();
+    const uint32_t pk_nb = (uint32_t)(V * (code_bits > 0 ? code_bits : 1));
+    const uint32_t pk_first0 = (32 * (threadIdx.x & 31)) / pk_nb, pk_first1 = (32 * ((threadIdx.x & 31) + 32)) / pk_nb;
     for (int64_t tile = blockIdx.x; tile < g.ntiles; tile += gridDim.x) {
         const int64_t e0 = tile * (int64_t)kTile;
         const uint32_t ne = (uint32_t)min((int64_t)kTile, g.E - e0);
@@ -415,7 +438,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                         const int64_t row_e = e0 + k0 + (int64_t)(j * kThreads + (threadIdx.x & ~31u)) * V;
                         const int64_t word0 = (row_e >> 5) * code_bits, nwords = (g.E * code_bits + 31) >> 5;
                         uint32_t out[2];
-                        warp_pack_row(code_string, nb, lane, out);
+                        warp_pack_row(code_string, nb, lane, pk_first0, pk_first1, out);
                         if (lane < nb && word0 + lane < nwords) pcodes[word0 + lane] = out[0];
                         if (lane + 32 < nb && word0 + lane + 32 < nwords) pcodes[word0 + lane + 32] = out[1];
                     }
@@ -564,16 +587,30 @@ __global__ void __launch_bounds__(kThreads) dequant_packed_kernel(const uint32_t
     const uint32_t field = (1u << bits) - 1u;
     for (int64_t u = (int64_t)blockIdx.x * kThreads + threadIdx.x; u < nunits; u += (int64_t)gridDim.x * kThreads) {
         const int64_t e = u * V;
-        int64_t plane = e / inner, rem = e - plane * inner;
-        int64_t grp = plane % C;
+        int64_t rem, grp;
+        if (E < (1ll << 31)) {                       // 32-bit divisions are several times cheaper
+            const uint32_t plane = (uint32_t)e / (uint32_t)inner;
+            rem = (uint32_t)e - plane * (uint32_t)inner;
+            grp = plane % (uint32_t)C;
+        } else {
+            const int64_t plane = e / inner;
+            rem = e - plane * inner;
+            grp = plane % C;
+        }
         float sg = __ldg(s + grp), zg = __ldg(z + grp);
         Pack<T> out;
+        // the thread's V * b <= 64 bits lie in at most three consecutive words
+        const int64_t first_bit = e * bits, last_word = (E * bits - 1) >> 5;
+        const uint32_t bit0 = (uint32_t)(first_bit & 31);
+        const int64_t w0 = first_bit >> 5;
+        const uint32_t q0 = __ldg(pcodes + w0);
+        const uint32_t q1 = w0 + 1 <= last_word ? __ldg(pcodes + w0 + 1) : 0u;
+        const uint32_t q2 = (V * 8 > 32 && w0 + 2 <= last_word) ? __ldg(pcodes + w0 + 2) : 0u;
+        const uint64_t lo64 = ((uint64_t)q1 << 32) | q0, hi64 = ((uint64_t)q2 << 32) | q1;
 #pragma unroll
         for (int i = 0; i < V; ++i) {
-            const int64_t bit = (e + i) * bits;
-            const uint32_t o = (uint32_t)(bit & 31);
-            uint32_t v = __ldg(pcodes + (bit >> 5)) >> o;
-            if (o + (uint32_t)bits > 32u) v |= __ldg(pcodes + (bit >> 5) + 1) << (32u - o);
+            const uint32_t pos = bit0 + (uint32_t)(i * bits);               // < 96
+            const uint32_t v = pos < 32u ? (uint32_t)(lo64 >> pos) : (uint32_t)(hi64 >> (pos - 32u));
             const float yv = __fmul_rn(sg, __fsub_rn((float)(v & field), zg));
             if constexpr (V == 1) store_scalar(y + e, yv);
             else out.set(i, yv);

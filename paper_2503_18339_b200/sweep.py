@@ -48,6 +48,8 @@ def main() -> None:
     ap.add_argument("--distortion", action="store_true",
                     help="instead of the bandwidth sweep: the statistics of Table 2 (cosine similarity, relative "
                          "error) of layer-wise against channel-wise quantization on the config's tensors")
+    ap.add_argument("--packed", action="store_true",
+                    help="instead of the bandwidth sweep: quantize to packed b-bit codes and dequantize from them")
     ap.add_argument("--weights", default="", choices=["", "resnet20", "resnet18"],
                     help="instead of the bandwidth sweep: all weight tensors of the network in one batched "
                          "launch against one fused call per tensor")
@@ -55,6 +57,9 @@ def main() -> None:
     b.lib()
     if args.weights:
         weights_table(args)
+        return
+    if args.packed:
+        packed_table(args)
         return
     if args.distortion:
         distortion_table(args)
@@ -99,6 +104,42 @@ def main() -> None:
                     print(f"{spec.name} {dt} {bits} {mode} {us:.1f} {gbs:.0f} {gbs / peak:.3f}", flush=True)
             del x, gy, out
         del x32, g32
+
+
+def packed_table(args) -> None:
+    """Packed b-bit codes: time and algorithmic GB/s (fp32: 4 + b/8 bytes per element each way) of
+    granq_quantize_packed (range given) and granq_dequantize_packed on the config's tensors."""
+    peak = _peak()
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    print("tensor bits op us GB/s frac_of_measured")
+    seen = set()
+    for spec in wl.config_tensors(args.config):
+        if spec.shape in seen or args.only not in spec.name:
+            continue
+        seen.add(spec.shape)
+        x = torch.from_numpy(wl.make_activation(spec)).cuda()
+        lo, hi = b.granq_range(x)
+        y = torch.empty_like(x)
+        for bits in ([int(v) for v in args.bits.split(",")] if args.bits else spec.bits):
+            pc = torch.empty(b.packed_codes_bytes(x.shape, bits) // 4, dtype=torch.int32, device="cuda")
+            out = b.granq_quantize_packed(x, bits, lo, hi, packed_codes=pc)
+            ops = (("quantize_packed", lambda: b.granq_quantize_packed(x, bits, lo, hi, packed_codes=pc)),
+                   ("dequantize_packed", lambda: b.granq_dequantize_packed(pc, x.shape, x.dtype, bits, out.s, out.z, y=y)))
+            for name, fn in ops:
+                fn()
+                times = []
+                for _ in range(args.iters):
+                    flush.fill_(1)
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    fn()
+                    e1.record()
+                    torch.cuda.synchronize()
+                    times.append(e0.elapsed_time(e1) * 1e3)
+                us = statistics.median(times)
+                gbs = x.numel() * (4 + bits / 8) / us / 1e3
+                print(f"{spec.name} {bits} {name} {us:.1f} {gbs:.0f} {gbs / peak:.3f}", flush=True)
+        del x, y
 
 
 def weights_table(args) -> None:
