@@ -500,7 +500,7 @@ ColPlan plan_colwalk(int dtype, const Geom& g, const QuantIO& io, const StagedTu
         const uint32_t grid = c_assumed_grid(tune.l2_ctas_per_sm);
         // the search is host work on every call: remember the last few answers
         struct Memo {
-            uint32_t V, inner, C, grid;
+            uint32_t V, inner, C, grid, q;
             int64_t outer;
             uint64_t target;
             uint32_t cw;
@@ -512,7 +512,7 @@ ColPlan plan_colwalk(int dtype, const Geom& g, const QuantIO& io, const StagedTu
         {
             std::lock_guard<std::mutex> hold(memo_lock);
             for (const Memo& e : memo)
-                if (e.cw && e.V == V && e.inner == inner && e.C == C && e.grid == grid && e.outer == g.outer &&
+                if (e.cw && e.V == V && e.inner == inner && e.C == C && e.grid == grid && e.q == q && e.outer == g.outer &&
                     e.target == target) {
                     p.cw = e.cw;
                     found = true;
@@ -537,7 +537,7 @@ ColPlan plan_colwalk(int dtype, const Geom& g, const QuantIO& io, const StagedTu
         }
         if (!found) {
             std::lock_guard<std::mutex> hold(memo_lock);
-            memo[memo_next++ % 8] = Memo{V, inner, C, grid, g.outer, target, p.cw};
+            memo[memo_next++ % 8] = Memo{V, inner, C, grid, q, g.outer, target, p.cw};
         }
     }
     p.nwaves = (C + p.cw - 1) / p.cw;
@@ -586,6 +586,12 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
     a.expected = (uint32_t)(tune.extra_arrivals > 0 ? tune.extra_arrivals : 0);   // + grid, added at launch
     const uint32_t c_last = C - (plan.nwaves - 1) * plan.cw;
     const uint32_t ch[2] = {plan.nwaves > 1 ? plan.cw : c_last, c_last};
+    // The packed mask is assembled by groups of lanes that must be present together: every slab and
+    // every wave has to be a whole number of 32-element mask words (the planner sees to it; a plan
+    // that is not is refused here rather than launched).
+    if (io.pmask && (((uint64_t)C * inner) % 32 != 0 || ((uint64_t)plan.cw * inner) % 32 != 0 ||
+                     ((uint64_t)c_last * inner) % 32 != 0))
+        return cudaErrorInvalidValue;
     const bool aligned = (inner % V) == 0;
     for (int i = 0; i < 2; ++i) {
         CShape& s = a.shape[i];

@@ -111,3 +111,20 @@ def test_packmask_configs_3_4_full_size(b, spec):
     assert np.array_equal(packed_np(got.packed_mask), packed_ref(ref.mask))
     gx = b.granq_fakequant_bwd_packmask(to_dev(gy), got.packed_mask)
     assert same_bits(to_np(gx), ref.gx)
+
+
+def test_wave_cut_of_the_packed_mask_call_is_its_own(b):
+    """The planner remembers wave cuts per geometry; the cut of a call with a packed mask (waves of whole
+    mask words) must not be the one remembered for a call without (waves of whole 16-byte packs).
+    [256,1024,14,14]: several waves, 196-element planes, so the two cuts differ."""
+    spec = wl.config_tensors(5)[2]
+    x, gy = wl.make_activation(spec), wl.make_upstream_grad(spec)
+    ref = orc.fused(x, 4, gy=gy, want_codes=True)
+    dx = to_dev(x)
+    first = b.granq_fakequant_fused(dx, 4, gy=to_dev(gy))                     # remembers the plain cut
+    assert same_bits(to_np(first.y), ref.y)
+    got = b.granq_fakequant_fused_fwd_packmask(dx, 4, flags=b.FLAG_FORCE_COLWALK)
+    assert b.workspace_status(got.workspace) == b.OK
+    assert same_bits(to_np(got.y), ref.y)
+    assert np.array_equal(packed_np(got.packed_mask), packed_ref(ref.mask))
+
