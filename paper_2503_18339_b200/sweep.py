@@ -48,6 +48,10 @@ def main() -> None:
     ap.add_argument("--distortion", action="store_true",
                     help="instead of the bandwidth sweep: the statistics of Table 2 (cosine similarity, relative "
                          "error) of layer-wise against channel-wise quantization on the config's tensors")
+    ap.add_argument("--table5", action="store_true",
+                    help="instead of the bandwidth sweep: the three rows of the paper's Table 5 in kind - forward "
+                         "fake-quantization of all 19 ResNet-20 activation tensors at batch 16, 3 bits: layer-wise, "
+                         "channel-wise by the per-channel loop, channel-wise by the default plan")
     ap.add_argument("--packed", action="store_true",
                     help="instead of the bandwidth sweep: quantize to packed b-bit codes and dequantize from them")
     ap.add_argument("--weights", default="", choices=["", "resnet20", "resnet18"],
@@ -60,6 +64,9 @@ def main() -> None:
         return
     if args.packed:
         packed_table(args)
+        return
+    if args.table5:
+        table5(args)
         return
     if args.distortion:
         distortion_table(args)
@@ -104,6 +111,35 @@ def main() -> None:
                     print(f"{spec.name} {dt} {bits} {mode} {us:.1f} {gbs:.0f} {gbs / peak:.3f}", flush=True)
             del x, gy, out
         del x32, g32
+
+
+def table5(args) -> None:
+    """Quantization latency of one forward pass over the ResNet-20 activation set at batch 16 (the setting of
+    Table 5): wall time of the 19 calls including their launches, median of `--iters` repetitions."""
+    import dataclasses
+    import time
+    specs = [dataclasses.replace(s, shape=(16,) + tuple(s.shape[1:])) for s in wl.config_tensors(2)]
+    xs = [torch.from_numpy(wl.make_activation(s)).cuda() for s in specs]
+    rows = (("layer-wise (one range per tensor)", b.GROUP_TENSOR, 0),
+            ("channel-wise, per-channel loop (3 launches per channel)", b.GROUP_CHANNEL, b.FLAG_FORCE_NAIVE),
+            ("channel-wise, default plan (1 launch per tensor)", b.GROUP_CHANNEL, 0))
+    print("scheme ms_per_pass launches")
+    for name, group, flags in rows:
+        outs = [b.FakeQuantOut(y=torch.empty_like(x), workspace=b.make_workspace(x, 1, group)) for x in xs]
+        launches = sum(b.fused_plan(b.F32, x.shape, group=group, with_backward=False, flags=flags)[1] for x in xs)
+
+        def one_pass():
+            for x, o in zip(xs, outs):
+                b.granq_fakequant_fused(x, 3, group=group, out=o, flags=flags)
+        one_pass()
+        torch.cuda.synchronize()
+        times = []
+        for _ in range(max(args.iters, 5)):
+            t0 = time.perf_counter()
+            one_pass()
+            torch.cuda.synchronize()
+            times.append((time.perf_counter() - t0) * 1e3)
+        print(f"{name}: {statistics.median(times):.3f} {launches}", flush=True)
 
 
 def packed_table(args) -> None:
