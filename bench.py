@@ -440,7 +440,19 @@ def main():
         for _ in range(repeats - 1):
             s2, e2 = time_oracle(sample, arrays)
             s, e = s + s2, e + e2
+        # the same oracle calls spread over the host's cores (one call per thread at a time; ctypes releases the GIL)
+        from concurrent.futures import ThreadPoolExecutor
+        from oracle import granq_oracle as orc
+        threads = max(1, min(os.cpu_count() or 1, len(sample)))
+        tp0 = time.perf_counter()
+        with ThreadPoolExecutor(max_workers=threads) as pool:
+            list(pool.map(lambda sb: orc.fused(arrays[sb[0].name][0], sb[1], gy=arrays[sb[0].name][1], want_codes=False),
+                          sample))
+        tp = time.perf_counter() - tp0
+        par_elems = sum(sp.numel for sp, _ in sample)
         cpu = {"value": e * BYTES_PER_ELEM / s / 1e9, "unit": UNIT, "cores": 1, "kind": "oracle",
+               "all_cores": {"value": par_elems * BYTES_PER_ELEM / tp / 1e9, "unit": UNIT, "threads": threads,
+                             "how": "the sample's calls once over, one oracle call per thread at a time"},
                "sample": "every workload tensor of at most 60 M elements, b=4 and b=5 (%d calls), %d times over: %d M elements"
                          % (len(sample), repeats, e // 1_000_000), "seconds": round(s, 2), "elements_per_s": e / s,
                "host_cores_available": os.cpu_count()}
