@@ -203,6 +203,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=2)
+    ap.add_argument("--e2e-lanes", type=int, default=2, help="streams (each with its own arena) the end-to-end "
+                                                             "calls rotate over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="also print a per-tensor table to stderr")
     ap.add_argument("--tune", default="", help="planner overrides for experiments, e.g. depth=3,max_buf_units=4000")
@@ -382,7 +384,7 @@ def main():
         big = max(specs, key=lambda s: s.numel)
         cmax = max(s.shape[1] for s in specs)
         lanes = []
-        for _ in range(2):
+        for _ in range(max(1, args.e2e_lanes)):
             lanes.append({
                 "stream": torch.cuda.Stream(),
                 "arena": torch.empty(b.host_arena_bytes(b.F32, big.shape), dtype=torch.uint8, device="cuda"),
@@ -392,7 +394,7 @@ def main():
 
         def e2e_step():
             for k, (i, bits) in enumerate(calls):
-                ln = lanes[k % 2]
+                ln = lanes[k % len(lanes)]
                 xs, gs = host[i]
                 n, c = specs[i].numel, specs[i].shape[1]
                 b.granq_fakequant_fused_host(xs, bits, gs, ln["y"].view(-1)[:n].view(specs[i].shape),
@@ -427,8 +429,8 @@ def main():
                "h2d_bytes_per_step": elems_per_step * 8, "d2h_bytes_per_step": elems_per_step * 8 +
                sum(specs[i].shape[1] * 8 for i, _ in calls),
                "steps": args.e2e_steps, "ms_per_step": e_ms / args.e2e_steps,
-               "api": "granq_fakequant_fused_host (pinned host buffers; calls alternate between two streams and arenas, "
-                      "so one call's downloads overlap the next call's uploads)"}
+               "api": ("granq_fakequant_fused_host (pinned host buffers; calls rotate over %d streams and arenas, "
+                       "so one call's downloads overlap the next call's uploads)" % len(lanes))}
 
     # ---- the CPU oracle on a bounded sample, rank 0 at N = 1 only ----
     cpu = None
