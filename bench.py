@@ -291,7 +291,7 @@ def main():
         for ci, (i, bits) in enumerate(calls):
             x, gy, out = dev[i]
             if events is not None:
-                events[ci][0].record(stream)
+                events[ci].record(stream)
             if args.op == "fused":
                 b.granq_fakequant_fused(x, bits, gy=gy, out=out, flags=flags, stream=stream)
             elif args.op == "range":
@@ -304,8 +304,8 @@ def main():
                 b.granq_fakequant_bwd_packmask(gy, out.packed_mask, gx=out.gx, stream=stream)
             else:
                 b.granq_fakequant_bwd(gy, x, bits, out.lo, out.hi, gx=out.gx, stream=stream)
-            if events is not None:
-                events[ci][1].record(stream)
+        if events is not None:
+            events[len(calls)].record(stream)
 
     for _ in range(warmup):
         step()
@@ -319,8 +319,8 @@ def main():
         torch.cuda.synchronize()
 
     # ---- timed region: K steps, device time, max over ranks ----
-    ev = [[(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in calls]
-          for _ in range(args.steps)]
+    # one event before every call and one after the last: a call's time runs to the start of the next
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)] for _ in range(args.steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sampler = ClockSampler(local)
     sampler.start()
@@ -347,7 +347,7 @@ def main():
     value = whole_job_gbs(bytes_per_step, world, ms_per_step)
 
     # ---- per-call device times inside the timed region -> roofline of the dominant kernel ----
-    per_call_ms = [statistics.mean(ev[k][ci][0].elapsed_time(ev[k][ci][1]) for k in range(args.steps))
+    per_call_ms = [statistics.mean(ev[k][ci].elapsed_time(ev[k][ci + 1]) for k in range(args.steps))
                    for ci in range(len(calls))]
     # dominant kernel: the column-walk instantiation for planes that are whole 16-byte packs (all but the 7x7 ones)
     dominant = [ci for ci, (i, _) in enumerate(calls) if (specs[i].shape[2] * specs[i].shape[3]) % 4 == 0
@@ -367,7 +367,7 @@ def main():
         "traffic": (rec["dram_bytes_per_algorithmic_byte"] * dom_bytes / max(1, len(dominant)) if rec else None),
         "traffic_source": (rec["source"] if rec else None),
         "share_of_step_time": dom_ms / sum(per_call_ms),
-        "note": "achieved = algorithmic bytes of the launches / their CUDA-event time (launch gaps included)",
+        "note": "achieved = algorithmic bytes of the launches / their CUDA-event time (from the event before a call to the event before the next: launch gaps included)",
     }
     per_tensor = []
     for ci, (i, bits) in enumerate(calls):
