@@ -289,7 +289,8 @@ __device__ __forceinline__ void warp_pack_row(uint64_t mine, uint32_t nb, uint32
 // EXTRAS: the optional codes / mask / packed-mask outputs are compiled in.  The packed mask holds
 // one bit per element (bit e % 32 of word e / 32): a warp's lanes own consecutive elements or packs
 // starting at a multiple of 32 elements, so whole words are assembled with warp shuffles.
-template <typename T, int V, int MODE, bool EXTRAS>
+// PACKONLY: the packed integer codes are the only output (everything else is compiled out).
+template <typename T, int V, int MODE, bool EXTRAS, bool PACKONLY = false>
 __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restrict__ x, const T* __restrict__ gy,
                                                               T* __restrict__ y, T* __restrict__ gx,
                                                               uint8_t* __restrict__ codes,
@@ -386,18 +387,22 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                     GroupParam gp{p.s, p.z, (amax <= 1152921504606846976.0f) ? rcp : 0.0f};
                     quantize_pack<T, kBwd, false, EXTRAS>(px[j], pg[j], gp, gp, V, qmax, py, pgx, cb, mb);
                     if constexpr (EXTRAS) {
+                        if constexpr (!PACKONLY) {
 #pragma unroll
-                        for (int i = 0; i < V; ++i) inside_bits |= ((mb[i / 4] >> (8 * (i % 4))) & 1u) << i;
+                            for (int i = 0; i < V; ++i) inside_bits |= ((mb[i / 4] >> (8 * (i % 4))) & 1u) << i;
+                        }
                         if constexpr (kFwd) {
-                            if (dist) dacc.add(px[j], py);
-                            if (pcodes) {
+                            if constexpr (!PACKONLY) {
+                                if (dist) dacc.add(px[j], py);
+                            }
+                            if (PACKONLY || pcodes) {
 #pragma unroll
                                 for (int i = 0; i < V; ++i)
                                     code_string |= (uint64_t)((cb[i / 4] >> (8 * (i % 4))) & 0xFFu) << (i * code_bits);
                             }
                         }
                     }
-                    if constexpr (kFwd) {
+                    if constexpr (kFwd && !PACKONLY) {
                         if (!EXTRAS || y) st_stream_16(y + e, py.raw);
                         if constexpr (EXTRAS) {
                             if (codes) {
@@ -418,7 +423,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                 }
                 }
                 if constexpr (EXTRAS && kFwd) {
-                    if (pmask) {          // every lane of the warp is here: assemble whole 32-bit words
+                    if (!PACKONLY && pmask) {          // every lane of the warp is here: assemble whole 32-bit words
                         const uint32_t lane = threadIdx.x & 31;
                         const int64_t word = (e0 + k[j]) >> 5;
                         if constexpr (V == 1) {
@@ -432,7 +437,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                             if ((lane & (kLanes - 1)) == 0 && valid) pmask[word] = w;
                         }
                     }
-                    if (pcodes) {         // the warp's 32 * V codes are V * b whole words of the bit string
+                    if (PACKONLY || pcodes) {         // the warp's 32 * V codes are V * b whole words of the bit string
                         const uint32_t lane = threadIdx.x & 31;
                         const uint32_t nb = (uint32_t)(V * code_bits);
                         const int64_t row_e = e0 + k0 + (int64_t)(j * kThreads + (threadIdx.x & ~31u)) * V;
@@ -446,7 +451,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
             }
         }
     }
-    if constexpr (EXTRAS && kFwd) {
+    if constexpr (EXTRAS && kFwd && !PACKONLY) {
         if (dist) dacc.flush(dist);
     }
 }
@@ -681,6 +686,16 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
     float qmax = (float)((1 << bits) - 1);
     const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr || io.dist != nullptr ||
                         io.pcodes != nullptr;
+    const bool pack_only = io.pcodes != nullptr && io.y == nullptr && io.codes == nullptr && io.mask == nullptr &&
+                           io.pmask == nullptr && io.dist == nullptr;
+    if constexpr (MODE == MODE_FWD) {
+        if (vec && pack_only) {
+            quant_flat_kernel<T, VF, MODE, true, true><<<grid, kThreads, 0, st>>>(
+                (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
+                io.code_bits, f, qmax, lo, hi);
+            return cudaGetLastError();
+        }
+    }
     if (vec && extras)
         quant_flat_kernel<T, VF, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
                                                                         (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes, io.code_bits, f, qmax, lo, hi);
