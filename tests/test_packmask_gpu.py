@@ -128,3 +128,15 @@ def test_wave_cut_of_the_packed_mask_call_is_its_own(b):
     assert same_bits(to_np(got.y), ref.y)
     assert np.array_equal(packed_np(got.packed_mask), packed_ref(ref.mask))
 
+
+
+def test_batch_sharded_step_on_one_rank_equals_the_fused_path(b):
+    """data_parallel.fakequant_forward / fakequant_backward (range -> exchange -> forward with packed mask,
+    backward from the mask) with a single rank, where the exchange is a no-op: the fused path's results."""
+    from paper_2503_18339_b200 import data_parallel as dp
+    shape = (16, 24, 14, 14)
+    x, gy = make_case(shape, seed=31)
+    ref = orc.fused(x, 4, gy=gy)
+    fwd = dp.fakequant_forward(to_dev(x), 4)
+    assert same_bits(to_np(fwd.lo), ref.lo) and same_bits(to_np(fwd.hi), ref.hi) and same_bits(to_np(fwd.y), ref.y)
+    assert same_bits(to_np(dp.fakequant_backward(to_dev(gy), fwd.packed_mask)), ref.gx)
