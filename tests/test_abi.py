@@ -94,6 +94,36 @@ def test_argument_errors_are_detected_before_any_launch(lib):
     assert r == b.ERR_INVALID_ARG
     assert lib.granq_tune(99, 0) == b.ERR_INVALID_ARG
     assert lib.granq_workspace_status(None, None) == b.ERR_INVALID_ARG
+    # the later entry points: missing outputs, misaligned buffers, bad bit-widths
+    odd = ctypes.c_void_p(3 << 28 | 2)
+    r = lib.granq_fakequant_fwd_packmask(fake, b.F32, dims, 1, 0, 4, fake, fake, far, None, None, None, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # packed mask missing
+    r = lib.granq_fakequant_fwd_packmask(fake, b.F32, dims, 1, 0, 4, fake, fake, far, odd, None, None, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # packed mask not on a 4-byte boundary
+    r = lib.granq_fakequant_bwd_packmask(fake, ctypes.c_void_p(3 << 28), b.F32, dims, fake, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # gx on top of gy
+    r = lib.granq_fakequant_fused_fwd_packmask(fake, b.F32, dims, 1, 0, 4, far, ctypes.c_void_p(3 << 28), fake, fake,
+                                               None, None, None, 0, 0, None)
+    assert r == b.ERR_WORKSPACE
+    r = lib.granq_distortion(fake, far, b.F32, dims, odd, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # sums not on an 8-byte boundary
+    r = lib.granq_fakequant_fused_stats(fake, b.F32, dims, 1, 0, 4, far, fake, fake, None, None, None, fake, 4096, 0,
+                                        None)
+    assert r == b.ERR_INVALID_ARG                     # sums missing
+    r = lib.granq_quantize_packed(fake, b.F32, dims, 1, 0, 9, fake, fake, far, None, fake, fake, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # 9 bits
+    r = lib.granq_quantize_packed(fake, b.F32, dims, 1, 0, 4, fake, fake, far, None, None, fake, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # scale output missing
+    r = lib.granq_dequantize_packed(far, b.F32, dims, 1, 0, 4, fake, None, fake, 0, None)
+    assert r == b.ERR_INVALID_ARG                     # zero-point missing
+    assert b.packmask_bytes((2, 3, 4, 4)) == 12 and b.packed_codes_bytes((2, 3, 4, 4), 3) == 36
+    desc = (b.WeightDesc * 1)(b.WeightDesc(256 * 1024, None, 3 << 28, None, 256 * 1024, 256 * 1024, None, None, 4, 8,
+                                           0, 0))
+    assert lib.granq_fakequant_weights(desc, 1, b.F32, fake, 4096, 0, None) == b.ERR_INVALID_ARG      # 0 bits
+    desc[0].bits = 4
+    assert lib.granq_fakequant_weights(desc, 1, b.F32, None, 0, 0, None) == b.ERR_WORKSPACE
+    assert lib.granq_fakequant_weights(desc, 0, b.F32, fake, 4096, 0, None) == b.ERR_INVALID_ARG
+    assert lib.granq_host_arena_status(b.F32, dims, 1, 0, 1, None, None) == b.ERR_INVALID_ARG
 
 
 def test_binding_refuses_cpu_tensors(lib):
