@@ -7,6 +7,9 @@
  *   2. scale and zero-point for b bits ........................... Eq. 2 / Eq. 5
  *   3. quantize -> clamp -> dequantize ("pre-scaling") ........... Eq. 1, Eq. 6, Algorithm 1
  *   4. straight-through-estimator backward ....................... Section 2.1
+ * and, built on the same arithmetic: the forward / backward split that carries a 1-bit mask,
+ * the distortion statistics of Table 2, all weight tensors of a model in one launch
+ * (Section 5.1) and the integer codes as a packed bit string.
  *
  * Arithmetic (identical for every entry point), per group g with members x_i, in IEEE
  * fp32, round-to-nearest-even, no fused multiply-add:
@@ -39,8 +42,10 @@
  *
  * Execution.  All work is enqueued on `cuda_stream` (a cudaStream_t passed as void*;
  * NULL = the default stream); no entry point synchronises with the host except
- * granq_fakequant_fused_host() and granq_workspace_status().  Results are bit-identical
- * from run to run.
+ * granq_fakequant_fused_host() (unless GRANQ_FLAG_HOST_ASYNC), granq_host_arena_status(),
+ * granq_workspace_status() and granq_fakequant_weights() (which reads its host descriptor
+ * array before it returns).  Results are bit-identical from run to run, except the last bits
+ * of the distortion sums, whose fp64 atomics arrive in no fixed order.
  *
  * Errors.  Every function returning int returns a granq_status code.  Argument errors
  * (null required pointer, bits outside 1..8, non-positive dim, more than 2^40 elements,
