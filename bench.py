@@ -214,6 +214,8 @@ def main():
                                                       "bwd_packmask"],
                     help="time another entry point instead of the fused one (bytes/element 4, 8, 12; 8.125 for the "
                          "two halves of the mask-carrying split)")
+    ap.add_argument("--no-graph", action="store_true", help="launch every timed step eagerly instead of replaying "
+                                                            "the captured step for the steps without per-call events")
     ap.add_argument("--clear-workspace", action="store_true",
                     help="let every call clear its workspace (one more memset node per call) instead of "
                          "passing GRANQ_FLAG_WORKSPACE_ZEROED")
@@ -274,7 +276,9 @@ def main():
     bytes_per_step = elems_per_step * BYTES_PER_ELEM
     plans = [b.fused_plan(b.F32, specs[i].shape, flags=plan_flags) for i, _ in calls]
     launches_per_step = sum(n for _, n in plans)
-    stream = torch.cuda.current_stream()
+    torch.cuda.synchronize()
+    stream = torch.cuda.Stream()          # a stream of its own: the legacy default stream cannot be captured
+    torch.cuda.set_stream(stream)
 
     bpe = {"fused": 16, "range": 4, "fwd": 8, "bwd": 12, "fused_fwd_packmask": 8.125, "bwd_packmask": 8.125}[args.op]
     bytes_per_step = int(elems_per_step * bpe)
@@ -325,6 +329,22 @@ def main():
     event_steps = min(args.steps, 3)
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)] for _ in range(event_steps)]
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    # The steps without per-call events are replays of the step captured once in a CUDA graph (the same 24
+    # library calls; it spares the launch gaps between them).  --no-graph, or a capture that fails, launches eagerly.
+    graph = None
+    if not args.no_graph and args.op == "fused" and args.steps > event_steps:
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                step()
+            graph.replay()
+            torch.cuda.synchronize()
+            for _, _, out in dev:
+                assert b.workspace_status(out.workspace) == b.OK
+        except Exception as err:       # noqa: BLE001
+            print(f"CUDA graph capture failed ({err}); launching eagerly", file=sys.stderr)
+            graph = None
+            torch.cuda.synchronize()
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.25)
@@ -332,7 +352,10 @@ def main():
     t0 = time.time()
     e0.record(stream)
     for k in range(args.steps):
-        step(ev[k] if k < event_steps else None)
+        if k < event_steps or graph is None:
+            step(ev[k] if k < event_steps else None)
+        else:
+            graph.replay()
     e1.record(stream)
     barrier()
     t1 = time.time()
@@ -470,6 +493,9 @@ def main():
             "config": {"workload": WORKLOAD, "elements_per_step_per_gpu": elems_per_step,
                        "calls_per_step": len(calls), "l2": "inputs larger than L2 (7.3 GB working set per step)",
                        "group_mode": "channel",
+                       "launch": ("steps %d..%d replay the step captured in a CUDA graph, steps 1..%d are launched eagerly "
+                                  "with one CUDA event per call" % (event_steps + 1, args.steps, event_steps)
+                                  if graph is not None else "every step launched eagerly"),
                        "workspace": ("cleared by every call" if args.clear_workspace else
                                      "cleared once at allocation, GRANQ_FLAG_WORKSPACE_ZEROED on every call"), "parallelism": f"replicas x{world} (independent batches, no exchange)"},
             "elements_per_s": world * elems_per_step / (ms_per_step * 1e-3),
