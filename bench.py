@@ -208,7 +208,7 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--table", action="store_true", help="also print a per-tensor table to stderr")
     ap.add_argument("--tune", default="", help="planner overrides for experiments, e.g. depth=3,max_buf_units=4000")
-    ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged", "l2wave", "colwalk"],
+    ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged", "l2wave", "colwalk", "cluster"],
                     help="force an execution plan of the fused entry point (experiments)")
     ap.add_argument("--op", default="fused", choices=["fused", "range", "fwd", "bwd", "fused_fwd_packmask",
                                                       "bwd_packmask"],
@@ -241,14 +241,16 @@ def main():
     knob_ids = {"depth": b.KNOB_STAGED_DEPTH, "max_buf_units": b.KNOB_STAGED_MAX_BUF_UNITS,
                 "grid": b.KNOB_STAGED_GRID, "ctas_per_sm": b.KNOB_STAGED_CTAS_PER_SM,
                 "l2_wave_kb": b.KNOB_L2_WAVE_KB, "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM,
-                "l2_lag": b.KNOB_L2_LAG}
+                "l2_lag": b.KNOB_L2_LAG, "cl_tile_kb": b.KNOB_CLUSTER_TILE_KB, "cl_ctas": b.KNOB_CLUSTER_CTAS,
+                "cl_threads": b.KNOB_CLUSTER_THREADS, "cl_load": b.KNOB_CLUSTER_LOAD,
+                "cl_prefetch": b.KNOB_CLUSTER_PREFETCH, "cl_kmul": b.KNOB_CLUSTER_KMUL}
     for item in filter(None, args.tune.split(",")):
         name, val = item.split("=")
         b.tune(knob_ids[name], int(val))
     warmup = max(args.warmup, 3)
     flags = {"auto": 0, "two_pass": b.FLAG_FORCE_TWO_PASS, "naive": b.FLAG_FORCE_NAIVE,
              "staged": b.FLAG_FORCE_STAGED, "l2wave": b.FLAG_FORCE_L2WAVE,
-             "colwalk": b.FLAG_FORCE_COLWALK}[args.plan]
+             "colwalk": b.FLAG_FORCE_COLWALK, "cluster": b.FLAG_FORCE_CLUSTER}[args.plan]
     plan_flags = flags
     if not args.clear_workspace:      # the workspaces are cleared once below and every call leaves them clear
         flags |= b.FLAG_WORKSPACE_ZEROED

@@ -45,7 +45,11 @@
  * granq_fakequant_fused_host() (unless GRANQ_FLAG_HOST_ASYNC), granq_host_arena_status(),
  * granq_workspace_status() and granq_fakequant_weights() (which reads its host descriptor
  * array before it returns).  Results are bit-identical from run to run, except the last bits
- * of the distortion sums, whose fp64 atomics arrive in no fixed order.
+ * of the distortion sums, whose fp64 atomics arrive in no fixed order.  The library keeps no
+ * results and no per-call state; the only process-wide state is (a) the planner overrides set with
+ * granq_tune() (all zero unless a test or a tuning run sets them; they never change results),
+ * (b) memoised answers of pure functions of (geometry, device): occupancy per kernel and device,
+ * the column-walk planner's wave cut, the device address of granq_range_noalloc()'s array.
  *
  * Errors.  Every function returning int returns a granq_status code.  Argument errors
  * (null required pointer, bits outside 1..8, non-positive dim, more than 2^40 elements,
@@ -94,10 +98,12 @@ enum granq_flags {
                                         this flag that ended with status GRANQ_OK); the call then skips
                                         its own clearing step and leaves the workspace zero again on
                                         success.  After GRANQ_ERR_TIMEOUT clear it before the next use. */
-    GRANQ_FLAG_HOST_ASYNC = 64u       /* granq_fakequant_fused_host(): enqueue only, do not wait for the stream
+    GRANQ_FLAG_HOST_ASYNC = 64u,      /* granq_fakequant_fused_host(): enqueue only, do not wait for the stream
                                         (host outputs are valid once the stream has passed the call; ask
                                         granq_host_arena_status() then).  Lets calls on two streams with two
                                         arenas overlap one call's uploads with the other's downloads.       */
+    GRANQ_FLAG_FORCE_CLUSTER = 128u   /* fused: cluster-local kernel (a run of channels staged once in the shared
+                                        memory of one thread-block cluster) or GRANQ_ERR_UNSUPPORTED        */
 };
 
 /* Human-readable name of a status code (static storage, never NULL). */
@@ -234,6 +240,10 @@ int granq_fakequant_fused_fwd_packmask(const void* x, int dtype, const int64_t d
  */
 int granq_distortion(const void* x, const void* q, int dtype, const int64_t dims[4], double* sums_out,
                      uint32_t flags, void* cuda_stream);
+/* Host-only: Table 2's two statistics from the four sums (HOST memory, as copied back from sums_out):
+ *   cosine = sum X*Q / (sqrt(sum X^2) * sqrt(sum Q^2)),   rel_error = sqrt(sum (X-Q)^2) / sqrt(sum X^2),
+ * each 0 when its denominator is 0.  cosine_out / rel_error_out may be NULL. */
+int granq_distortion_stats(const double sums[4], double* cosine_out, double* rel_error_out);
 int granq_fakequant_fused_stats(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
                                 int bits, void* y, float* min_out, float* max_out, float* scale_opt, float* zp_opt,
                                 double* sums_out, void* workspace, size_t workspace_bytes, uint32_t flags,
@@ -249,7 +259,9 @@ int granq_fakequant_fused_stats(const void* x, int dtype, const int64_t dims[4],
  *               inside are DEVICE memory: x in, y out, gy_opt / gx_opt both or neither,
  *               min_out / max_out `channels` floats each (required), scale_opt / zp_opt or NULL
  *   workspace   DEVICE scratch of granq_weights_workspace_bytes(n_tensors), 256-byte aligned
- * Limits: fewer than 2^31 groups in the batch and 2^31 elements per group.
+ * Limits: fewer than 2^31 groups in the batch and 2^31 elements per group.  The call stages the
+ * descriptors through host memory it owns only until it returns, so it cannot be recorded into a CUDA
+ * graph: on a capturing stream it returns GRANQ_ERR_UNSUPPORTED and enqueues nothing.
  */
 typedef struct granq_weight_desc {
     const void* x;
@@ -324,7 +336,7 @@ int granq_host_arena_status(int dtype, const int64_t dims[4], int channel_axis, 
 /*
  * Plan that granq_fakequant_fused() would take for this geometry and flags on the current
  * device: 0 = two-pass, 1 = naive per-channel loop, 2 = on-chip staged, 3 = L2-resident waves,
- * 4 = column walk; negative = -status.
+ * 4 = column walk, 5 = cluster-local; negative = -status.
  * `launches_out` (HOST, may be NULL) receives the number of kernel launches of that plan.
  */
 int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,
@@ -339,6 +351,16 @@ int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int gro
  */
 int granq_staged_geometry(int dtype, const int64_t dims[4], int channel_axis, int group, int sm_count,
                           int smem_bytes, int64_t out[8]);
+
+/*
+ * Host-only query: how the cluster-local plan would cut this tensor (no counterpart in the paper).
+ * out = { CTAs, threads per CTA, CTAs per cluster, shared-memory bytes per CTA, bytes of one staged
+ *         tile, channels per run, staging (0 = plain loads, 1 = bulk copies for x, 2 = bulk copies
+ *         for x and gy), 1 if gy is prefetched into the L2 }.
+ * Returns GRANQ_ERR_UNSUPPORTED when the geometry does not qualify.
+ */
+int granq_cluster_geometry(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,
+                           int64_t out[8]);
 
 /*
  * Device self-test (no counterpart in the paper).  The staged kernel divides by the
@@ -368,7 +390,15 @@ enum granq_knob {
     GRANQ_KNOB_L2_WAVE_KB = 6,            /* L2-wave plan: x bytes of one wave, in KiB             */
     GRANQ_KNOB_L2_UPL = 7,                /* L2-wave plan: 16-byte units per lane and step (2, 4)  */
     GRANQ_KNOB_L2_CTAS_PER_SM = 8,        /* L2-wave / column-walk plans: cap on resident CTAs per SM */
-    GRANQ_KNOB_L2_LAG = 9                 /* column-walk plan: waves the range phase runs ahead (1..3) */
+    GRANQ_KNOB_L2_LAG = 9,                /* column-walk plan: waves the range phase runs ahead (1..3) */
+    GRANQ_KNOB_CLUSTER_TILE_KB = 10,      /* cluster plan: limit on the staged tile of one CTA, in KiB */
+    GRANQ_KNOB_CLUSTER_CTAS = 11,         /* cluster plan: CTAs per cluster (1, 2, 4, 8)               */
+    GRANQ_KNOB_CLUSTER_THREADS = 12,      /* cluster plan: threads per CTA (a multiple of 32, <= 512)  */
+    GRANQ_KNOB_CLUSTER_LOAD = 13,         /* cluster plan: 1 = bulk copies for x, 2 = plain loads,
+                                             3 = bulk copies for x and gy                              */
+    GRANQ_KNOB_CLUSTER_PREFETCH = 14,     /* cluster plan: 1 = L2 prefetch of gy, 2 = none             */
+    GRANQ_KNOB_CLUSTER_KMUL = 15,         /* cluster plan: multiplier of a run's minimal channel count */
+    GRANQ_KNOB_CLUSTER_EARLY_LAUNCH = 16  /* cluster plan: 2 = launch without programmatic dependent launch */
 };
 int granq_tune(int knob, int value);
 

@@ -21,10 +21,13 @@ GROUP_CHANNEL, GROUP_SAMPLE_CHANNEL, GROUP_TENSOR = 0, 1, 2
 FLAG_FORCE_TWO_PASS, FLAG_FORCE_NAIVE, FLAG_FORCE_STAGED, FLAG_FORCE_L2WAVE, FLAG_FORCE_COLWALK = 1, 2, 4, 8, 16
 FLAG_WORKSPACE_ZEROED = 32
 FLAG_HOST_ASYNC = 64
-PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED, PLAN_L2WAVE, PLAN_COLWALK = 0, 1, 2, 3, 4
+FLAG_FORCE_CLUSTER = 128
+PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED, PLAN_L2WAVE, PLAN_COLWALK, PLAN_CLUSTER = 0, 1, 2, 3, 4, 5
 (KNOB_STAGED_DEPTH, KNOB_STAGED_MAX_BUF_UNITS, KNOB_STAGED_GRID, KNOB_SPIN_LIMIT, KNOB_TEST_EXTRA_ARRIVALS,
- KNOB_STAGED_CTAS_PER_SM, KNOB_L2_WAVE_KB, KNOB_L2_UPL, KNOB_L2_CTAS_PER_SM, KNOB_L2_LAG) = range(10)
-N_KNOBS = 10
+ KNOB_STAGED_CTAS_PER_SM, KNOB_L2_WAVE_KB, KNOB_L2_UPL, KNOB_L2_CTAS_PER_SM, KNOB_L2_LAG,
+ KNOB_CLUSTER_TILE_KB, KNOB_CLUSTER_CTAS, KNOB_CLUSTER_THREADS, KNOB_CLUSTER_LOAD, KNOB_CLUSTER_PREFETCH,
+ KNOB_CLUSTER_KMUL, KNOB_CLUSTER_EARLY_LAUNCH) = range(17)
+N_KNOBS = 17
 OK, ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE, ERR_CUDA, ERR_TIMEOUT = range(6)
 
 EXPORTS = [
@@ -35,7 +38,7 @@ EXPORTS = [
     "granq_fakequant_fwd_packmask", "granq_fakequant_bwd_packmask", "granq_fakequant_fused_fwd_packmask",
     "granq_host_arena_status", "granq_distortion", "granq_fakequant_fused_stats",
     "granq_weights_workspace_bytes", "granq_fakequant_weights", "granq_packed_codes_bytes",
-    "granq_quantize_packed", "granq_dequantize_packed",
+    "granq_quantize_packed", "granq_dequantize_packed", "granq_cluster_geometry", "granq_distortion_stats",
 ]
 NOALLOC_MAX_GROUPS = 32768
 
@@ -94,6 +97,11 @@ def lib() -> ctypes.CDLL:
         L.granq_fused_plan.argtypes = [ci, i64p, ci, ci, ci, u32, ctypes.POINTER(ci)]
         L.granq_staged_geometry.restype = ci
         L.granq_staged_geometry.argtypes = [ci, i64p, ci, ci, ci, ci, i64p]
+        L.granq_distortion_stats.restype = ci
+        L.granq_distortion_stats.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
+                                             ctypes.POINTER(ctypes.c_double)]
+        L.granq_cluster_geometry.restype = ci
+        L.granq_cluster_geometry.argtypes = [ci, i64p, ci, ci, ci, i64p]
         L.granq_selftest_division.restype = ci
         L.granq_selftest_division.argtypes = [ctypes.c_uint64, ctypes.c_uint64, vp, vp]
         L.granq_range_noalloc.restype = ci
@@ -218,6 +226,18 @@ def staged_geometry(dtype: int, shape, channel_axis: int = 1, group: int = GROUP
         return None
     _check(rc, "granq_staged_geometry")
     keys = ["grid", "threads", "depth", "smem_bytes", "buf_units", "cw", "cu", "nwaves"]
+    return dict(zip(keys, [int(v) for v in out]))
+
+
+def cluster_geometry(dtype: int, shape, channel_axis: int = 1, group: int = GROUP_CHANNEL,
+                     with_backward: bool = True):
+    """Host-only: the cut of the cluster-local plan, or None if the geometry does not qualify."""
+    out = (ctypes.c_int64 * 8)()
+    rc = lib().granq_cluster_geometry(dtype, _dims(shape), channel_axis, group, int(with_backward), out)
+    if rc == ERR_UNSUPPORTED:
+        return None
+    _check(rc, "granq_cluster_geometry")
+    keys = ["grid", "threads", "cluster", "smem_bytes", "tile_bytes", "channels_per_run", "staging", "prefetch_gy"]
     return dict(zip(keys, [int(v) for v in out]))
 
 
@@ -412,10 +432,11 @@ def granq_distortion(x: torch.Tensor, q: torch.Tensor, sums: torch.Tensor = None
 
 
 def distortion_from_sums(sums):
-    """(cosine similarity, relative error) of Table 2 from the four sums (host arithmetic on 4 numbers)."""
-    sxx, sqq, sxq, sdd = (float(v) for v in sums)
-    den = (sxx ** 0.5) * (sqq ** 0.5)
-    return (sxq / den if den > 0 else 0.0), ((sdd ** 0.5) / (sxx ** 0.5) if sxx > 0 else 0.0)
+    """(cosine similarity, relative error) of Table 2 from the four sums (granq_distortion_stats)."""
+    arr = (ctypes.c_double * 4)(*[float(v) for v in sums])
+    cos, rel = ctypes.c_double(0.0), ctypes.c_double(0.0)
+    _check(lib().granq_distortion_stats(arr, ctypes.byref(cos), ctypes.byref(rel)), "granq_distortion_stats")
+    return cos.value, rel.value
 
 
 def granq_fakequant_fused_stats(x: torch.Tensor, bits: int, channel_axis: int = 1, group: int = GROUP_CHANNEL,

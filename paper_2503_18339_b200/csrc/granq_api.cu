@@ -4,38 +4,13 @@
 
 #include "granq_internal.h"
 
+#include <math.h>
+
 using namespace granq;
 
 namespace {
 
-constexpr int64_t kMaxElements = 1ll << 40;
-
-StagedTuning g_tune = {0, 0, 0, 0, 0, 0, 0, 0, 0, 0};
-
-bool make_geom(const int64_t dims[4], int axis, int group, Geom& g, int64_t& G) {
-    if (!dims || axis < 0 || axis > 3 || group < 0 || group > 2) return false;
-    int64_t E = 1;
-    for (int d = 0; d < 4; ++d) {
-        if (dims[d] <= 0 || dims[d] > kMaxElements) return false;
-        if (E > kMaxElements / dims[d]) return false;
-        E *= dims[d];
-    }
-    if (E > kMaxElements) return false;
-    int64_t outer = 1, inner = 1;
-    for (int d = 0; d < axis; ++d) outer *= dims[d];
-    for (int d = axis + 1; d < 4; ++d) inner *= dims[d];
-    const int64_t C = dims[axis];
-    g.E = E;
-    if (group == GRANQ_GROUP_CHANNEL) {
-        g.outer = outer; g.C = C; g.inner = inner;
-    } else if (group == GRANQ_GROUP_SAMPLE_CHANNEL) {
-        g.outer = 1; g.C = outer * C; g.inner = inner;
-    } else {
-        g.outer = 1; g.C = 1; g.inner = E;
-    }
-    G = g.C;
-    return true;
-}
+StagedTuning g_tune = {};
 
 bool dtype_ok(int dtype) { return dtype == GRANQ_F32 || dtype == GRANQ_BF16; }
 size_t elt_size(int dtype) { return dtype == GRANQ_F32 ? 4 : 2; }
@@ -55,13 +30,19 @@ int check_workspace(const void* ws, size_t bytes, int64_t G) {
 
 int cuda_status(cudaError_t e) { return e == cudaSuccess ? GRANQ_OK : GRANQ_ERR_CUDA; }
 
-enum { PLAN_TWO_PASS = 0, PLAN_NAIVE = 1, PLAN_STAGED = 2, PLAN_L2WAVE = 3, PLAN_COLWALK = 4 };
+enum { PLAN_TWO_PASS = 0, PLAN_NAIVE = 1, PLAN_STAGED = 2, PLAN_L2WAVE = 3, PLAN_COLWALK = 4, PLAN_CLUSTER = 5 };
 
 // plan of the fused entry point; `plan_out` is filled when the staged plan is taken
-int choose_plan(int dtype, const Geom& g, const QuantIO& io, uint32_t flags, StagedPlan* plan_out,
-                L2Plan* l2_out, ColPlan* col_out) {
+int choose_plan(int dtype, const Geom& g, const QuantIO& io, bool backward, uint32_t flags, StagedPlan* plan_out,
+                L2Plan* l2_out, ColPlan* col_out, ClusterPlan* cl_out) {
     if (flags & GRANQ_FLAG_FORCE_NAIVE) return PLAN_NAIVE;
     if (flags & GRANQ_FLAG_FORCE_TWO_PASS) return PLAN_TWO_PASS;
+    if (flags & GRANQ_FLAG_FORCE_CLUSTER) {
+        ClusterPlan kp = plan_cluster(dtype, g, io, backward, g_tune);
+        if (!kp.ok) return -GRANQ_ERR_UNSUPPORTED;
+        if (cl_out) *cl_out = kp;
+        return PLAN_CLUSTER;
+    }
     if (flags & GRANQ_FLAG_FORCE_COLWALK) {
         ColPlan cp = plan_colwalk(dtype, g, io, g_tune);
         if (!cp.ok) return -GRANQ_ERR_UNSUPPORTED;
@@ -82,8 +63,14 @@ int choose_plan(int dtype, const Geom& g, const QuantIO& io, uint32_t flags, Sta
         if (plan_out) *plan_out = p;
         return PLAN_STAGED;
     }
-    // default: the column-walk kernel where there are slabs to walk, else the L2-resident-wave
-    // kernel (both have measured faster than the shared-memory-staged kernel on every workload tensor)
+    // default: the cluster-local kernel where a run of channels fits the shared memory of one cluster
+    // (x is then read once and nothing waits on the grid), else the column-walk kernel where there are
+    // slabs to walk, else the L2-resident-wave kernel
+    ClusterPlan kp = plan_cluster(dtype, g, io, backward, g_tune);
+    if (kp.ok) {
+        if (cl_out) *cl_out = kp;
+        return PLAN_CLUSTER;
+    }
     ColPlan cp = plan_colwalk(dtype, g, io, g_tune);
     if (cp.ok) {
         if (col_out) *col_out = cp;
@@ -206,18 +193,27 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
     StagedPlan sp{};
     L2Plan lp{};
     ColPlan cp{};
-    const int plan = choose_plan(dtype, g, io, flags, &sp, &lp, &cp);
+    ClusterPlan kp{};
+    const int plan = choose_plan(dtype, g, io, gy_opt != nullptr, flags, &sp, &lp, &cp, &kp);
     if (plan < 0) return -plan;
 
     Workspace ws = carve_workspace(workspace, G);
-    // The column-walk kernel leaves a zeroed workspace zeroed; with the caller's word that it is
-    // zero on entry nothing has to be cleared.  The other plans clear before and, to keep that
-    // word true for the next call, after.
+    // The column-walk kernel leaves a zeroed workspace zeroed and the cluster-local kernel writes
+    // nothing but the status word (and that only when a wait ran out); with the caller's word that
+    // the workspace is zero on entry nothing has to be cleared.  The other plans clear before and, to
+    // keep that word true for the next call, after.
     const bool zeroed = (flags & GRANQ_FLAG_WORKSPACE_ZEROED) != 0;
+    const bool keeps_zero = plan == PLAN_COLWALK || plan == PLAN_CLUSTER;
     cudaError_t e = cudaSuccess;
-    if (!(zeroed && plan == PLAN_COLWALK)) e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
+    if (plan == PLAN_CLUSTER) {
+        if (!zeroed) e = cudaMemsetAsync(workspace, 0, sizeof(uint32_t), st);      // the status word
+    } else if (!(zeroed && keeps_zero)) {
+        e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
+    }
     if (e != cudaSuccess) return GRANQ_ERR_CUDA;
-    if (plan == PLAN_STAGED) {
+    if (plan == PLAN_CLUSTER) {
+        e = launch_cluster(kp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
+    } else if (plan == PLAN_STAGED) {
         e = launch_staged(sp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
     } else if (plan == PLAN_L2WAVE) {
         e = launch_l2wave(lp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
@@ -233,7 +229,7 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
             e = launch_finalize_range(ws.kmin, ws.kmax, G, min_out, max_out, bits, scale_opt, zp_opt, st);
         if (e == cudaSuccess) e = launch_quant_flat(io, mode, dtype, g, bits, min_out, max_out, st);
     }
-    if (e == cudaSuccess && zeroed && plan != PLAN_COLWALK)
+    if (e == cudaSuccess && zeroed && !keeps_zero)
         e = cudaMemsetAsync((char*)workspace + sizeof(uint32_t), 0, ws.clear_bytes - sizeof(uint32_t), st);
     return cuda_status(e);
 }
@@ -330,6 +326,15 @@ int granq_distortion(const void* x, const void* q, int dtype, const int64_t dims
     cudaError_t e = cudaMemsetAsync(sums_out, 0, 4 * sizeof(double), st);
     if (e == cudaSuccess) e = launch_distortion(x, q, dtype, g.E, sums_out, st);
     return cuda_status(e);
+}
+
+int granq_distortion_stats(const double sums[4], double* cosine_out, double* rel_error_out) {
+    if (!sums) return GRANQ_ERR_INVALID_ARG;
+    const double sxx = sums[0], sqq = sums[1], sxq = sums[2], sdd = sums[3];
+    const double den = sqrt(sxx) * sqrt(sqq);
+    if (cosine_out) *cosine_out = den > 0.0 ? sxq / den : 0.0;
+    if (rel_error_out) *rel_error_out = sxx > 0.0 ? sqrt(sdd) / sqrt(sxx) : 0.0;
+    return GRANQ_OK;
 }
 
 int granq_fakequant_fused_stats(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
@@ -437,10 +442,11 @@ int granq_fakequant_fused_host(const void* x_host, const void* gy_host_opt, int 
                                void* device_arena, size_t arena_bytes, uint32_t flags, void* cuda_stream) {
     Geom g;
     int64_t G;
-    if (!x_host || !y_host || !min_host || !max_host || !dtype_ok(dtype) ||
+    if (!x_host || !y_host || !min_host || !max_host || bits < 1 || bits > 8 || !dtype_ok(dtype) ||
         !make_geom(dims, channel_axis, group, g, G))
         return GRANQ_ERR_INVALID_ARG;
     if ((gy_host_opt == nullptr) != (gx_host_opt == nullptr)) return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
     const int bwd = gy_host_opt ? 1 : 0;
     if (!device_arena || ((uintptr_t)device_arena & 255) ||
         arena_bytes < granq_host_arena_bytes(dtype, dims, channel_axis, group, bwd))
@@ -491,11 +497,10 @@ int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int gro
     Geom g;
     int64_t G;
     if (!dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G)) return -GRANQ_ERR_INVALID_ARG;
-    (void)with_backward;
     QuantIO io{};   // null pointers: alignment is assumed
-    const int plan = choose_plan(dtype, g, io, flags, nullptr, nullptr, nullptr);
+    const int plan = choose_plan(dtype, g, io, with_backward != 0, flags, nullptr, nullptr, nullptr, nullptr);
     if (launches_out) {
-        if (plan == PLAN_STAGED || plan == PLAN_L2WAVE || plan == PLAN_COLWALK) *launches_out = 1;
+        if (plan == PLAN_STAGED || plan == PLAN_L2WAVE || plan == PLAN_COLWALK || plan == PLAN_CLUSTER) *launches_out = 1;
         else if (plan == PLAN_NAIVE) *launches_out = (int)(3 * g.C);
         else if (plan == PLAN_TWO_PASS) *launches_out = 3;
     }
@@ -515,6 +520,19 @@ int granq_staged_geometry(int dtype, const int64_t dims[4], int channel_axis, in
     return GRANQ_OK;
 }
 
+int granq_cluster_geometry(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,
+                           int64_t out[8]) {
+    Geom g;
+    int64_t G;
+    if (!out || !dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G)) return GRANQ_ERR_INVALID_ARG;
+    QuantIO io{};
+    ClusterPlan p = plan_cluster(dtype, g, io, with_backward != 0, g_tune);
+    if (!p.ok) return GRANQ_ERR_UNSUPPORTED;
+    out[0] = (int64_t)((g.C + p.k - 1) / p.k) * p.R; out[1] = p.threads; out[2] = p.R; out[3] = p.smem_bytes;
+    out[4] = p.tile_bytes; out[5] = p.k; out[6] = p.load; out[7] = p.prefetch_gy ? 1 : 0;
+    return GRANQ_OK;
+}
+
 int granq_tune(int knob, int value) {
     switch (knob) {
         case GRANQ_KNOB_STAGED_DEPTH: g_tune.depth = value; return GRANQ_OK;
@@ -527,6 +545,13 @@ int granq_tune(int knob, int value) {
         case GRANQ_KNOB_L2_UPL: g_tune.l2_upl = value; return GRANQ_OK;
         case GRANQ_KNOB_L2_CTAS_PER_SM: g_tune.l2_ctas_per_sm = value; return GRANQ_OK;
         case GRANQ_KNOB_L2_LAG: g_tune.l2_lag = value; return GRANQ_OK;
+        case GRANQ_KNOB_CLUSTER_TILE_KB: g_tune.cl_tile_kb = value; return GRANQ_OK;
+        case GRANQ_KNOB_CLUSTER_CTAS: g_tune.cl_r = value; return GRANQ_OK;
+        case GRANQ_KNOB_CLUSTER_THREADS: g_tune.cl_threads = value; return GRANQ_OK;
+        case GRANQ_KNOB_CLUSTER_LOAD: g_tune.cl_load = value; return GRANQ_OK;
+        case GRANQ_KNOB_CLUSTER_PREFETCH: g_tune.cl_prefetch = value; return GRANQ_OK;
+        case GRANQ_KNOB_CLUSTER_KMUL: g_tune.cl_kmul = value; return GRANQ_OK;
+        case GRANQ_KNOB_CLUSTER_EARLY_LAUNCH: g_tune.cl_pdl = value; return GRANQ_OK;
         default: return GRANQ_ERR_INVALID_ARG;
     }
 }

@@ -23,6 +23,7 @@
 #include "granq_internal.h"
 
 #include <algorithm>
+#include <atomic>
 #include <mutex>
 
 namespace granq {
@@ -437,14 +438,19 @@ uint32_t c_assumed_grid(int cta_cap) {
 template <typename T, int MODE, bool ALIGNED, bool EXTRAS>
 cudaError_t c_launch_t(CArgs& args, int sm_count, int cta_cap, cudaStream_t st) {
     auto kern = colwalk_kernel<T, MODE, ALIGNED, EXTRAS, 4, 2>;
-    static int per_sm_cached = 0;      // one value per instantiation: every device here is the same part
-    if (per_sm_cached == 0) {
+    // resident CTAs per SM of this instantiation, remembered per device (a pure function of both)
+    static std::atomic<int> per_sm_cached[64] = {};
+    int dev = 0;
+    cudaError_t de = cudaGetDevice(&dev);
+    if (de != cudaSuccess) return de;
+    int per_sm = (dev >= 0 && dev < 64) ? per_sm_cached[dev].load(std::memory_order_relaxed) : 0;
+    if (per_sm == 0) {
         int n = 0;
         if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kern, kCThreads, 0) != cudaSuccess || n <= 0)
             return cudaErrorLaunchOutOfResources;
-        per_sm_cached = n;
+        per_sm = n;
+        if (dev >= 0 && dev < 64) per_sm_cached[dev].store(n, std::memory_order_relaxed);
     }
-    int per_sm = per_sm_cached;
     if (cta_cap > 0 && per_sm > cta_cap) per_sm = cta_cap;
     const uint32_t grid = (uint32_t)(sm_count * per_sm);
     for (int i = 0; i < 2; ++i) {

@@ -19,6 +19,34 @@ struct Geom {
     int64_t inner;  // contiguous elements of one (slab, group) plane
 };
 
+// (dims, channel axis, group mode) -> channel-group form and the number of groups; false when the
+// arguments are invalid (null dims, axis or mode out of range, a non-positive dim, more than 2^40 elements).
+constexpr int64_t kMaxElements = 1ll << 40;
+inline bool make_geom(const int64_t dims[4], int axis, int group, Geom& g, int64_t& G) {
+    if (!dims || axis < 0 || axis > 3 || group < 0 || group > 2) return false;
+    int64_t E = 1;
+    for (int d = 0; d < 4; ++d) {
+        if (dims[d] <= 0 || dims[d] > kMaxElements) return false;
+        if (E > kMaxElements / dims[d]) return false;
+        E *= dims[d];
+    }
+    if (E > kMaxElements) return false;
+    int64_t outer = 1, inner = 1;
+    for (int d = 0; d < axis; ++d) outer *= dims[d];
+    for (int d = axis + 1; d < 4; ++d) inner *= dims[d];
+    const int64_t C = dims[axis];
+    g.E = E;
+    if (group == 0) {            // GRANQ_GROUP_CHANNEL
+        g.outer = outer; g.C = C; g.inner = inner;
+    } else if (group == 1) {     // GRANQ_GROUP_SAMPLE_CHANNEL
+        g.outer = 1; g.C = outer * C; g.inner = inner;
+    } else {                     // GRANQ_GROUP_TENSOR
+        g.outer = 1; g.C = 1; g.inner = E;
+    }
+    G = g.C;
+    return true;
+}
+
 // Workspace layout (all plans): a 256-byte header whose first word is the device status,
 // then G min-keys, G max-keys, then G + 1 wave arrival counters.
 constexpr size_t kWsHeaderBytes = 256;
@@ -106,6 +134,13 @@ struct StagedTuning {
     int l2_upl;           // L2-wave plan: 16-byte units per lane and step (2 or 4)
     int l2_ctas_per_sm;   // L2-wave and column-walk plans: cap on resident CTAs per SM
     int l2_lag;           // column-walk plan: waves of phase 1 running ahead of phase 2 (1..3)
+    int cl_tile_kb;       // cluster plan: limit on the staged tile of one CTA, in KiB
+    int cl_r;             // cluster plan: CTAs per cluster (1, 2, 4, 8)
+    int cl_threads;       // cluster plan: threads per CTA
+    int cl_load;          // cluster plan: 1 = bulk copies for x, 2 = plain loads that reduce on the way, 3 = bulk copies for x and gy
+    int cl_prefetch;      // cluster plan: 1 = ask the L2 for gy while x is loading, 2 = do not
+    int cl_kmul;          // cluster plan: multiplier of the minimal channel count of a run
+    int cl_pdl;           // cluster plan: 2 = no programmatic dependent launch
 };
 StagedPlan plan_staged(int dtype, const Geom& g, const QuantIO& io, int device, const StagedTuning& tune);
 StagedPlan plan_staged_on(int dtype, const Geom& g, const QuantIO& io, int sm_count, int smem_optin,
@@ -136,6 +171,23 @@ struct ColPlan {
 };
 ColPlan plan_colwalk(int dtype, const Geom& g, const QuantIO& io, const StagedTuning& tune);
 cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int dtype, const Geom& g, int bits,
+                           const Workspace& ws, float* lo, float* hi, float* s_opt, float* z_opt,
+                           const StagedTuning& tune, cudaStream_t st);
+
+// ---- cluster-local kernel (a run of channels staged once in the shared memory of one cluster) ----
+struct ClusterPlan {
+    bool ok;
+    uint32_t k;              // channels per run
+    uint32_t R;              // CTAs per cluster
+    uint32_t threads;        // threads per CTA
+    uint32_t tile_bytes;     // staged tile of one CTA
+    uint32_t smem_bytes;     // dynamic shared memory per CTA (tile + keys + parameters)
+    int load;                // 0 = plain loads, 1 = x staged by bulk copies, 2 = x and gy staged by bulk copies
+    bool prefetch_gy;
+    bool early_launch;       // programmatic dependent launch: set the grid up while the kernel ahead drains
+};
+ClusterPlan plan_cluster(int dtype, const Geom& g, const QuantIO& io, bool backward, const StagedTuning& tune);
+cudaError_t launch_cluster(const ClusterPlan& plan, const QuantIO& io, int mode, int dtype, const Geom& g, int bits,
                            const Workspace& ws, float* lo, float* hi, float* s_opt, float* z_opt,
                            const StagedTuning& tune, cudaStream_t st);
 

@@ -11,6 +11,8 @@
 
 #include "granq_internal.h"
 
+#include <atomic>
+
 namespace {
 
 constexpr int64_t kNoAllocMaxGroups = GRANQ_NOALLOC_MAX_GROUPS;
@@ -20,9 +22,10 @@ static __device__ __align__(256) uint32_t g_noalloc_keys[2 * kNoAllocMaxGroups];
 
 // Device address of the array, looked up once per device with that device current.  In host
 // code `g_noalloc_keys` itself is only a handle for the runtime, not something a kernel can
-// dereference.
+// dereference.  Two host threads that make the first call on a device together both look the
+// address up and store the same value (the entries are atomic, the lookup is idempotent).
 uint32_t* noalloc_keys_on_current_device(cudaError_t* err) {
-    static uint32_t* cached[64] = {};
+    static std::atomic<uint32_t*> cached[64] = {};
     int dev = 0;
     *err = cudaGetDevice(&dev);
     if (*err != cudaSuccess) return nullptr;
@@ -30,13 +33,15 @@ uint32_t* noalloc_keys_on_current_device(cudaError_t* err) {
         *err = cudaErrorInvalidDevice;
         return nullptr;
     }
-    if (!cached[dev]) {
+    uint32_t* keys = cached[dev].load(std::memory_order_acquire);
+    if (!keys) {
         void* p = nullptr;
         *err = cudaGetSymbolAddress(&p, g_noalloc_keys);
         if (*err != cudaSuccess) return nullptr;
-        cached[dev] = static_cast<uint32_t*>(p);
+        keys = static_cast<uint32_t*>(p);
+        cached[dev].store(keys, std::memory_order_release);
     }
-    return cached[dev];
+    return keys;
 }
 
 }  // namespace
@@ -46,22 +51,10 @@ extern "C" int granq_range_noalloc(const void* x, int dtype, const int64_t dims[
     using namespace granq;
     if (!x || !min_out || !max_out || !dims || (dtype != GRANQ_F32 && dtype != GRANQ_BF16))
         return GRANQ_ERR_INVALID_ARG;
-    const int64_t G = granq_num_groups(dims, channel_axis, group);
-    if (G <= 0) return GRANQ_ERR_INVALID_ARG;
-    if (G > kNoAllocMaxGroups) return GRANQ_ERR_UNSUPPORTED;      // more groups than the built-in scratch holds
-    int64_t E = 1, outer = 1, inner = 1;
-    for (int d = 0; d < 4; ++d) E *= dims[d];
-    for (int d = 0; d < channel_axis; ++d) outer *= dims[d];
-    for (int d = channel_axis + 1; d < 4; ++d) inner *= dims[d];
     Geom g;
-    g.E = E;
-    if (group == GRANQ_GROUP_CHANNEL) {
-        g.outer = outer; g.C = dims[channel_axis]; g.inner = inner;
-    } else if (group == GRANQ_GROUP_SAMPLE_CHANNEL) {
-        g.outer = 1; g.C = outer * dims[channel_axis]; g.inner = inner;
-    } else {
-        g.outer = 1; g.C = 1; g.inner = E;
-    }
+    int64_t G = 0;
+    if (!make_geom(dims, channel_axis, group, g, G)) return GRANQ_ERR_INVALID_ARG;
+    if (G > kNoAllocMaxGroups) return GRANQ_ERR_UNSUPPORTED;      // more groups than the built-in scratch holds
     cudaError_t e = cudaSuccess;
     uint32_t* keys = noalloc_keys_on_current_device(&e);
     if (!keys) return GRANQ_ERR_CUDA;

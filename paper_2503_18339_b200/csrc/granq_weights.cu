@@ -162,6 +162,12 @@ int granq_fakequant_weights(const granq_weight_desc* descs, int n_tensors, int d
         if (total >= (1ull << 31)) return GRANQ_ERR_UNSUPPORTED;
     }
     cudaStream_t st = (cudaStream_t)cuda_stream;
+    // The table below is pageable host memory that lives until this call returns: fine for an eager copy (the
+    // runtime has read it by then), wrong for a captured one (a replay would read freed memory) - so a
+    // capturing stream is refused.
+    cudaStreamCaptureStatus capturing = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &capturing) != cudaSuccess) return GRANQ_ERR_CUDA;
+    if (capturing != cudaStreamCaptureStatusNone) return GRANQ_ERR_UNSUPPORTED;
     // the table is pageable host memory: the copy has read it by the time the call returns
     cudaError_t e = cudaMemcpyAsync(workspace, table.data(), table.size() * sizeof(WDesc), cudaMemcpyHostToDevice, st);
     if (e != cudaSuccess) return GRANQ_ERR_CUDA;

@@ -2,8 +2,9 @@
 quantize with ONE per-channel range, that of the whole batch (Eq. 4 over the global batch).
 
 The path has exactly one exchange step, between the range (Eq. 4) and the scale / zero-point
-(Eq. 5): an all-reduce of 2 * G floats.  Everything before and after is local.  The exchange uses
-`torch.distributed` (NCCL on GPUs, gloo on CPU); the arithmetic is the library's.
+(Eq. 5): the per-group minima and maxima (G floats each) are all-reduced, MIN and MAX.  Everything
+before and after is local.  The exchange uses `torch.distributed` (NCCL on GPUs, gloo on CPU) on the
+buffers the library wrote, in place; no arithmetic happens outside the library and the collective.
 
 Without this module each rank quantizes with the range of its own slice (independent replicas),
 which is what `bench.py --gpus N` times.
@@ -16,16 +17,20 @@ import torch
 import torch.distributed as dist
 
 
-def sync_range(lo: torch.Tensor, hi: torch.Tensor, group=None) -> None:
-    """In place: lo <- min over ranks, hi <- max over ranks, with one all-reduce (MAX over [-lo, hi]).
-    A no-op without an initialised process group or with a single rank."""
+def sync_range(lo: torch.Tensor, hi: torch.Tensor, group=None, stream=None) -> None:
+    """In place: lo <- min over ranks, hi <- max over ranks (two all-reduces of G floats, issued back to
+    back; the messages are a few KB, so both are latency-bound).  On CUDA tensors the collectives are
+    ordered after what `stream` holds - the range kernel that wrote lo / hi - and the stream then waits
+    for them.  A no-op without an initialised process group or with a single rank."""
     if not (dist.is_available() and dist.is_initialized()) or dist.get_world_size(group) == 1:
         return
-    G = lo.numel()
-    packed = torch.cat([-lo.reshape(-1), hi.reshape(-1)])
-    dist.all_reduce(packed, op=dist.ReduceOp.MAX, group=group)
-    lo.copy_((-packed[:G]).reshape(lo.shape))
-    hi.copy_(packed[G:].reshape(hi.shape))
+    if lo.is_cuda and stream is not None:
+        with torch.cuda.stream(stream):       # the process group orders its work after the current stream
+            dist.all_reduce(lo, op=dist.ReduceOp.MIN, group=group)
+            dist.all_reduce(hi, op=dist.ReduceOp.MAX, group=group)
+        return
+    dist.all_reduce(lo, op=dist.ReduceOp.MIN, group=group)
+    dist.all_reduce(hi, op=dist.ReduceOp.MAX, group=group)
 
 
 def fakequant_forward(x: torch.Tensor, bits: int, channel_axis: int = 1, group_mode: int = 0, group=None,
@@ -34,7 +39,7 @@ def fakequant_forward(x: torch.Tensor, bits: int, channel_axis: int = 1, group_m
     STE mask with the global range.  Returns the binding's FakeQuantOut (y, packed_mask, lo, hi)."""
     from . import binding as b
     lo, hi = b.granq_range(x, channel_axis=channel_axis, group=group_mode, stream=stream)
-    sync_range(lo, hi, group)
+    sync_range(lo, hi, group, stream)
     return b.granq_fakequant_fwd_packmask(x, bits, lo, hi, channel_axis=channel_axis, group=group_mode,
                                           stream=stream)
 

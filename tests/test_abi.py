@@ -184,6 +184,67 @@ def test_staged_plan_under_forced_small_buffers(lib):
                 planned += 1
                 _check_geometry(shape, dt, 0, geo)
     finally:
-        for k in range(9):
+        for k in range(b.N_KNOBS):
             b.tune(k, 0)
     assert planned > 500
+
+
+def test_distortion_stats_against_the_oracle_and_closed_forms(lib):
+    """Table 2's two statistics from the four sums: the C entry point against the oracle's and against
+    closed forms (Q = X, Q = 0, a 3-4-5 pair), and its degenerate cases."""
+    from oracle import granq_oracle as orc
+    from paper_2503_18339_b200 import binding as b
+    assert b.distortion_from_sums([4.0, 4.0, 4.0, 0.0]) == (1.0, 0.0)               # Q = X
+    assert b.distortion_from_sums([4.0, 0.0, 0.0, 4.0]) == (0.0, 1.0)               # Q = 0
+    assert b.distortion_from_sums([0.0, 0.0, 0.0, 0.0]) == (0.0, 0.0)               # X = 0
+    cos, rel = b.distortion_from_sums([9.0, 16.0, 0.0, 25.0])                       # X = (3, 0), Q = (0, 4)
+    assert cos == 0.0 and abs(rel - 5.0 / 3.0) < 1e-15
+    rnd = random.Random(3)
+    for _ in range(50):
+        sxx, sqq = rnd.uniform(0.1, 1e6), rnd.uniform(0.1, 1e6)
+        sxq = rnd.uniform(-1, 1) * (sxx * sqq) ** 0.5
+        sums = [sxx, sqq, sxq, sxx + sqq - 2 * sxq]
+        got, want = b.distortion_from_sums(sums), orc.distortion(sums)
+        assert abs(got[0] - want[0]) <= 1e-15 * max(1.0, abs(want[0])) and abs(got[1] - want[1]) <= 1e-15 * max(1.0, want[1])
+    assert lib.granq_distortion_stats(None, None, None) == b.ERR_INVALID_ARG
+
+
+def test_cluster_plan_cuts_within_its_limits(lib):
+    """Host-only: whatever the cluster-local planner answers respects its own invariants - a run is a whole
+    number of 16-byte units in every slab, a CTA's tiles fit the shared memory of an SM twice over (or the
+    forced limit), the cluster size is a portable power of two no larger than the number of slabs."""
+    from paper_2503_18339_b200 import binding as b
+    rnd = random.Random(11)
+    planned = 0
+    try:
+        for _ in range(3000):
+            shape = (rnd.choice([1, 2, 3, 8, 13, 64, 128, 256]), rnd.randint(1, 600),
+                     rnd.choice([1, 2, 4, 7, 8, 14, 28, 56]), rnd.choice([1, 4, 7, 8, 14, 16, 28, 56]))
+            dt, mode, bwd = rnd.choice([0, 1]), rnd.choice([0, 1]), rnd.choice([False, True])
+            V, esize = (4, 4) if dt == 0 else (8, 2)
+            b.tune(b.KNOB_CLUSTER_CTAS, rnd.choice([0, 0, 0, 1, 2, 4, 8]))
+            b.tune(b.KNOB_CLUSTER_TILE_KB, rnd.choice([0, 0, 8, 32, 200]))
+            b.tune(b.KNOB_CLUSTER_LOAD, rnd.choice([0, 0, 1, 2, 3, 4, 5]))
+            b.tune(b.KNOB_CLUSTER_KMUL, rnd.choice([0, 0, 0, 2, 5]))
+            geo = b.cluster_geometry(dt, shape, group=mode, with_backward=bwd)
+            inner = shape[2] * shape[3]
+            outer, C = (shape[0], shape[1]) if mode == 0 else (1, shape[0] * shape[1])
+            if (C * inner) % V or inner < V:
+                assert geo is None
+                continue
+            if geo is None:
+                continue
+            planned += 1
+            k, R = geo["channels_per_run"], geo["cluster"]
+            assert (k * inner) % V == 0 and k >= 1
+            assert R in (1, 2, 4, 8) and R <= outer
+            assert geo["grid"] == -(-C // k) * R
+            assert geo["tile_bytes"] == -(-outer // R) * min(k, C if k > C else k) * inner * esize or k > C
+            tiles = 2 if geo["staging"] in (2, 4) else 1
+            assert tiles == 1 or bwd
+            assert geo["smem_bytes"] >= tiles * geo["tile_bytes"] and geo["smem_bytes"] <= 227 * 1024
+            assert geo["threads"] % 32 == 0 and 32 <= geo["threads"] <= 512
+    finally:
+        for k in range(b.N_KNOBS):
+            b.tune(k, 0)
+    assert planned > 300

@@ -140,3 +140,12 @@ def test_batch_sharded_step_on_one_rank_equals_the_fused_path(b):
     fwd = dp.fakequant_forward(to_dev(x), 4)
     assert same_bits(to_np(fwd.lo), ref.lo) and same_bits(to_np(fwd.hi), ref.hi) and same_bits(to_np(fwd.y), ref.y)
     assert same_bits(to_np(dp.fakequant_backward(to_dev(gy), fwd.packed_mask)), ref.gx)
+    # the same on a stream that is not the current one (the exchange is ordered on that stream too)
+    import torch
+    st = torch.cuda.Stream()
+    xd, gyd = to_dev(x), to_dev(gy)
+    torch.cuda.synchronize()
+    fwd = dp.fakequant_forward(xd, 4, stream=st)
+    gx = dp.fakequant_backward(gyd, fwd.packed_mask, stream=st)
+    st.synchronize()
+    assert same_bits(to_np(fwd.lo), ref.lo) and same_bits(to_np(fwd.y), ref.y) and same_bits(to_np(gx), ref.gx)

@@ -137,14 +137,16 @@ def test_fused_small_all_plans(b, shape, mode, dtype):
     bits = 2 + (sum(shape) + mode) % 7
     x, gy = make_case(shape, seed=sum(shape) * 7 + mode, dtype=dtype, relu=(shape[0] % 2 == 0))
     ref = orc.fused(x, bits, gy=gy, group_mode=mode)
-    for flags in (0, b.FLAG_FORCE_TWO_PASS, b.FLAG_FORCE_NAIVE, b.FLAG_FORCE_L2WAVE, b.FLAG_FORCE_COLWALK):
+    for flags in (0, b.FLAG_FORCE_TWO_PASS, b.FLAG_FORCE_NAIVE, b.FLAG_FORCE_L2WAVE, b.FLAG_FORCE_COLWALK,
+                  b.FLAG_FORCE_CLUSTER):
         if flags == b.FLAG_FORCE_NAIVE and b.num_groups(shape, 1, mode) > 300:
             continue
         try:
             got = b.granq_fakequant_fused(to_dev(x), bits, gy=to_dev(gy), group=mode, want_codes=True,
                                           want_mask=True, want_params=True, flags=flags)
         except b.GranqError as err:      # the persistent plans do not take every geometry
-            assert flags in (b.FLAG_FORCE_L2WAVE, b.FLAG_FORCE_COLWALK) and err.status == b.ERR_UNSUPPORTED
+            assert flags in (b.FLAG_FORCE_L2WAVE, b.FLAG_FORCE_COLWALK, b.FLAG_FORCE_CLUSTER)
+            assert err.status == b.ERR_UNSUPPORTED
             continue
         assert b.workspace_status(got.workspace) == b.OK
         assert_parity(got, ref, shape, 1, mode, backward=True)
@@ -259,9 +261,13 @@ def test_colwalk_needs_slabs_to_walk(b):
     with pytest.raises(b.GranqError) as err:
         b.granq_fakequant_fused(to_dev(make_case((2, 8, 8, 8), seed=1)[0]), 4, flags=b.FLAG_FORCE_COLWALK)
     assert err.value.status == b.ERR_UNSUPPORTED
-    assert b.fused_plan(b.F32, (2, 8, 8, 8))[0] == b.PLAN_L2WAVE
-    assert b.fused_plan(b.F32, (64, 8, 8, 8))[0] == b.PLAN_COLWALK
-    assert b.fused_plan(b.F32, (64, 8, 8, 8), group=b.GROUP_SAMPLE_CHANNEL)[0] == b.PLAN_L2WAVE
+    # defaults: groups that fit the shared memory of a cluster go to the cluster-local kernel; larger ones to
+    # the column walk when the batch has slabs to walk, else to the L2-resident waves
+    assert b.fused_plan(b.F32, (2, 8, 8, 8))[0] == b.PLAN_CLUSTER
+    assert b.fused_plan(b.F32, (64, 8, 8, 8), group=b.GROUP_SAMPLE_CHANNEL)[0] == b.PLAN_CLUSTER
+    assert b.fused_plan(b.F32, (64, 8, 112, 112))[0] == b.PLAN_COLWALK
+    assert b.fused_plan(b.F32, (2, 8, 512, 512))[0] == b.PLAN_L2WAVE
+    assert b.fused_plan(b.F32, (64, 8, 2, 2, ))[0] == b.PLAN_CLUSTER
 
 
 def test_colwalk_workspace_stays_zeroed(b, knobs):

@@ -7,7 +7,20 @@ import numpy as np
 import pytest
 import torch
 
+from oracle import granq_oracle as orc
+
 pytestmark = pytest.mark.gpu
+
+
+def _bits(t: torch.Tensor) -> np.ndarray:
+    return t.detach().cpu().numpy().view(np.uint32)
+
+
+def _oracle_range(x: torch.Tensor, group: int):
+    """Eq. 4 by the CPU oracle on the same values (bf16 tensors go in as their bit patterns)."""
+    if x.dtype == torch.bfloat16:
+        return orc.range_(x.view(torch.int16).cpu().numpy().view(np.uint16), group_mode=group)
+    return orc.range_(x.cpu().numpy(), group_mode=group)
 
 
 @pytest.fixture(scope="module")
@@ -35,6 +48,8 @@ def test_two_calls_in_a_row_match_the_workspace_entry_point(b, dtype):
     for x, group in ((first, b.GROUP_SAMPLE_CHANNEL), (second, b.GROUP_CHANNEL), (first, b.GROUP_TENSOR)):
         lo, hi, lo_ref, hi_ref = _pair(b, x, group)
         assert torch.equal(lo, lo_ref) and torch.equal(hi, hi_ref)          # min / max are bit-exact in every test here
+        lo_orc, hi_orc = _oracle_range(x, group)                            # ... and against the CPU oracle
+        assert np.array_equal(_bits(lo), lo_orc.view(np.uint32)) and np.array_equal(_bits(hi), hi_orc.view(np.uint32))
         xf = x.float()
         if group == b.GROUP_CHANNEL:
             assert torch.equal(lo, xf.amin(dim=(0, 2, 3))) and torch.equal(hi, xf.amax(dim=(0, 2, 3)))
