@@ -5,14 +5,20 @@ One step = fused forward + backward fake-quantization (range -> scale / zero-poi
 quantize / clamp / dequantize -> STE backward, one library call per tensor) of every tensor
 of the ResNet-18 and MobileNetV2 ImageNet-shaped activation sets (12 fp32 tensors, batch
 128) at both of their bit-widths (4 and 5): 24 calls, 914 M elements, 14.6 GB of
-algorithmic traffic (16 B per element: read x, read gy, write y, write gx).
+algorithmic traffic (16 B per element: read x, read gy, write y, write gx).  A step runs all
+twelve tensors at 4 bits, then all twelve at 5 bits, so no tensor is touched by two
+consecutive calls and every call finds its tensor cold (7.3 GB pass through between them).
 
-Prints ONE JSON line.  `value` is algorithmic GB/s with all tensors resident in HBM;
-`e2e` is the same metric through the host-buffer entry point (pinned host memory, copies
-inside the timed region); `roofline` relates the dominant kernel to the measured HBM copy
-bandwidth; `cpu_baseline` is the CPU oracle timed on a bounded sample of the same workload.
+Prints ONE JSON line.  `value` is algorithmic GB/s over K eagerly launched steps with all
+tensors resident in HBM (mean; median and best step beside it); `e2e` is the same metric
+through the host-buffer entry point (pinned host memory, copies inside the timed region);
+`roofline` relates the dominant kernel to the measured HBM copy bandwidth; `per_tensor` is each
+call's sustained cold time (back-to-back calls over rotating copies of the tensor, no event
+between them); `sub` holds bounded runs of the other configurations, entry points, group modes
+and plans; `cpu_baseline` is the CPU oracle timed on a bounded sample of the same workload.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+With --gpus N > 1 and no torchrun environment the script starts its N ranks itself.
 """
 from __future__ import annotations
 
@@ -57,7 +63,7 @@ def measured_peak():
         return FALLBACK_HBM_GBS, "fallback (6.65 TB/s, earlier measurement on this pool)"
 
 
-DOMINANT_KERNEL_SOURCES = ("granq_colwalk.cu", "granq_device.cuh", "granq_internal.h")
+DOMINANT_KERNEL_SOURCES = ("granq_colwalk.cu", "granq_device.cuh")
 
 
 def kernel_source_hash() -> str:
@@ -196,6 +202,46 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def free_port() -> int:
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        return sk.getsockname()[1]
+
+
+def spawn_ranks(n: int, argv, extra_env=None, timeout=None):
+    """Start `n` ranks of `argv` on this node (RANK / LOCAL_RANK / WORLD_SIZE / MASTER_* set as torchrun
+    would) and wait for them; returns their exit codes.  Rank 0 inherits stdout."""
+    port = free_port()
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port), **(extra_env or {}))
+        procs.append(subprocess.Popen(list(argv), env=env, stdout=None if r == 0 else subprocess.DEVNULL))
+    codes = []
+    for pr in procs:
+        try:
+            codes.append(pr.wait(timeout=timeout))
+        except subprocess.TimeoutExpired:
+            pr.kill()
+            codes.append(-9)
+    return codes
+
+
+def rank_selftest():
+    """The multi-rank plumbing without a GPU: gloo ranks agree on the slowest rank's time and rank 0 prints
+    the aggregate (what the spawn path of --gpus N is tested with on CPU)."""
+    import torch.distributed as dist
+    rank, world = int(os.environ["RANK"]), int(os.environ["WORLD_SIZE"])
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    ms = max_over_ranks(10.0 * (rank + 1), device="cpu")
+    if rank == 0:
+        print(json.dumps({"selftest": True, "n_gpus": world, "ms_per_step": ms,
+                          "value": whole_job_gbs(1_000_000_000, world, ms)}))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -206,26 +252,42 @@ def main():
     ap.add_argument("--e2e-lanes", type=int, default=2, help="streams (each with its own arena) the end-to-end "
                                                              "calls rotate over")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-sub", action="store_true", help="skip the bounded sub-records and the per-tensor pass")
     ap.add_argument("--table", action="store_true", help="also print a per-tensor table to stderr")
     ap.add_argument("--tune", default="", help="planner overrides for experiments, e.g. depth=3,max_buf_units=4000")
-    ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged", "l2wave", "colwalk", "cluster"],
+    ap.add_argument("--plan", default="auto", choices=["auto", "two_pass", "naive", "staged", "l2wave", "colwalk",
+                                                       "cluster"],
                     help="force an execution plan of the fused entry point (experiments)")
     ap.add_argument("--op", default="fused", choices=["fused", "range", "fwd", "bwd", "fused_fwd_packmask",
                                                       "bwd_packmask"],
                     help="time another entry point instead of the fused one (bytes/element 4, 8, 12; 8.125 for the "
                          "two halves of the mask-carrying split)")
-    ap.add_argument("--no-graph", action="store_true", help="launch every timed step eagerly instead of replaying "
-                                                            "the captured step for the steps without per-call events")
+    ap.add_argument("--no-graph", action="store_true", help="skip the CUDA-graph replay figure")
     ap.add_argument("--clear-workspace", action="store_true",
                     help="let every call clear its workspace (one more memset node per call) instead of "
                          "passing GRANQ_FLAG_WORKSPACE_ZEROED")
+    ap.add_argument("--sharded", action="store_true", help="also time the batch-sharded forward / backward "
+                                                           "(range, all-reduce of the range, forward with packed "
+                                                           "mask, backward from the mask)")
     ap.add_argument("--only", default="", help="profiling aid: keep only workload tensors whose name contains this")
+    ap.add_argument("--rank-selftest", action="store_true", help=argparse.SUPPRESS)
     args = ap.parse_args()
+    if args.rank_selftest:
+        if "RANK" not in os.environ:
+            codes = spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:])
+            sys.exit(max(abs(c) for c in codes))
+        rank_selftest()
+        return
     if args.impl == "reference":
         if args.steps > 3:
             args.steps = 3          # each step is ~10 s of CPU work
         run_reference(args)
         return
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        # a plain `python bench.py --gpus N`: start the N ranks here (one per GPU, NCCL for the barrier and the
+        # maximum over ranks only: the path has no exchange step)
+        codes = spawn_ranks(args.gpus, [sys.executable, os.path.abspath(__file__)] + sys.argv[1:])
+        sys.exit(max(abs(c) for c in codes))
 
     import torch
     import torch.distributed as dist
@@ -243,17 +305,19 @@ def main():
                 "l2_wave_kb": b.KNOB_L2_WAVE_KB, "l2_upl": b.KNOB_L2_UPL, "l2_ctas_per_sm": b.KNOB_L2_CTAS_PER_SM,
                 "l2_lag": b.KNOB_L2_LAG, "cl_tile_kb": b.KNOB_CLUSTER_TILE_KB, "cl_ctas": b.KNOB_CLUSTER_CTAS,
                 "cl_threads": b.KNOB_CLUSTER_THREADS, "cl_load": b.KNOB_CLUSTER_LOAD,
-                "cl_prefetch": b.KNOB_CLUSTER_PREFETCH, "cl_kmul": b.KNOB_CLUSTER_KMUL}
+                "cl_prefetch": b.KNOB_CLUSTER_PREFETCH, "cl_kmul": b.KNOB_CLUSTER_KMUL,
+                "cl_early_launch": b.KNOB_CLUSTER_EARLY_LAUNCH}
     for item in filter(None, args.tune.split(",")):
         name, val = item.split("=")
         b.tune(knob_ids[name], int(val))
     warmup = max(args.warmup, 3)
-    flags = {"auto": 0, "two_pass": b.FLAG_FORCE_TWO_PASS, "naive": b.FLAG_FORCE_NAIVE,
-             "staged": b.FLAG_FORCE_STAGED, "l2wave": b.FLAG_FORCE_L2WAVE,
-             "colwalk": b.FLAG_FORCE_COLWALK, "cluster": b.FLAG_FORCE_CLUSTER}[args.plan]
-    plan_flags = flags
+    plan_flags = {"auto": 0, "two_pass": b.FLAG_FORCE_TWO_PASS, "naive": b.FLAG_FORCE_NAIVE,
+                  "staged": b.FLAG_FORCE_STAGED, "l2wave": b.FLAG_FORCE_L2WAVE,
+                  "colwalk": b.FLAG_FORCE_COLWALK, "cluster": b.FLAG_FORCE_CLUSTER}[args.plan]
+    flags = plan_flags
     if not args.clear_workspace:      # the workspaces are cleared once below and every call leaves them clear
         flags |= b.FLAG_WORKSPACE_ZEROED
+    peak, peak_src = measured_peak()
 
     specs = [s for s in workload_specs() if args.only in s.name]
     # ---- host (pinned) inputs and outputs; every rank has its own batch (weak scaling, no exchange) ----
@@ -264,21 +328,24 @@ def main():
         wl.make_activation(s, out=xs.numpy(), block_offset=1000 * rank)
         wl.make_upstream_grad(s, out=gs.numpy(), block_offset=1000 * rank)
         host.append((xs, gs))
+
+    def outputs_for(x, groups, group=b.GROUP_CHANNEL):
+        return b.FakeQuantOut(y=torch.empty_like(x), gx=torch.empty_like(x),
+                              lo=torch.empty(groups, device="cuda"), hi=torch.empty(groups, device="cuda"),
+                              workspace=b.make_workspace(x, group=group, zeroed=True))
+
     dev = []
     for s, (xs, gs) in zip(specs, host):
         x = xs.cuda(non_blocking=True)
         gy = gs.cuda(non_blocking=True)
-        out = b.FakeQuantOut(y=torch.empty_like(x), gx=torch.empty_like(x),
-                             lo=torch.empty(s.shape[1], device="cuda"), hi=torch.empty(s.shape[1], device="cuda"),
-                             workspace=b.make_workspace(x, zeroed=True))
-        dev.append((x, gy, out))
+        dev.append((x, gy, outputs_for(x, s.shape[1])))
     torch.cuda.synchronize()
-    calls = [(i, bits) for i, s in enumerate(specs) for bits in s.bits]
+    # all tensors at their first bit-width, then all at their second: consecutive calls never share a tensor
+    nbits = max(len(s.bits) for s in specs)
+    calls = [(i, s.bits[k]) for k in range(nbits) for i, s in enumerate(specs) if k < len(s.bits)]
     elems_per_step = sum(specs[i].numel for i, _ in calls)
-    bytes_per_step = elems_per_step * BYTES_PER_ELEM
     plans = [b.fused_plan(b.F32, specs[i].shape, flags=plan_flags) for i, _ in calls]
     launches_per_step = sum(n for _, n in plans)
-    torch.cuda.synchronize()
     stream = torch.cuda.Stream()          # a stream of its own: the legacy default stream cannot be captured
     torch.cuda.set_stream(stream)
 
@@ -293,75 +360,68 @@ def main():
             if args.op == "bwd_packmask":
                 b.granq_fakequant_fused_fwd_packmask(x, 4, out=out, stream=stream)
 
+    def one_call(x, gy, out, bits, op=None, fl=None, group=b.GROUP_CHANNEL):
+        op = args.op if op is None else op
+        fl = flags if fl is None else fl
+        if op == "fused":
+            b.granq_fakequant_fused(x, bits, gy=gy, group=group, out=out, flags=fl, stream=stream)
+        elif op == "fused_fwd":
+            b.granq_fakequant_fused(x, bits, group=group, out=out, flags=fl, stream=stream)
+        elif op == "range":
+            b.granq_range(x, lo=out.lo, hi=out.hi, workspace=out.workspace, stream=stream)
+        elif op == "fwd":
+            b.granq_fakequant_fwd(x, bits, out.lo, out.hi, y=out.y, stream=stream)
+        elif op == "fused_fwd_packmask":
+            b.granq_fakequant_fused_fwd_packmask(x, bits, out=out, flags=fl, stream=stream)
+        elif op == "bwd_packmask":
+            b.granq_fakequant_bwd_packmask(gy, out.packed_mask, gx=out.gx, stream=stream)
+        else:
+            b.granq_fakequant_bwd(gy, x, bits, out.lo, out.hi, gx=out.gx, stream=stream)
+
     def step(events=None):
         for ci, (i, bits) in enumerate(calls):
             x, gy, out = dev[i]
             if events is not None:
                 events[ci].record(stream)
-            if args.op == "fused":
-                b.granq_fakequant_fused(x, bits, gy=gy, out=out, flags=flags, stream=stream)
-            elif args.op == "range":
-                b.granq_range(x, lo=out.lo, hi=out.hi, workspace=out.workspace, stream=stream)
-            elif args.op == "fwd":
-                b.granq_fakequant_fwd(x, bits, out.lo, out.hi, y=out.y, stream=stream)
-            elif args.op == "fused_fwd_packmask":
-                b.granq_fakequant_fused_fwd_packmask(x, bits, out=out, flags=flags, stream=stream)
-            elif args.op == "bwd_packmask":
-                b.granq_fakequant_bwd_packmask(gy, out.packed_mask, gx=out.gx, stream=stream)
-            else:
-                b.granq_fakequant_bwd(gy, x, bits, out.lo, out.hi, gx=out.gx, stream=stream)
+            one_call(x, gy, out, bits)
         if events is not None:
             events[len(calls)].record(stream)
 
+    def check_status():
+        torch.cuda.synchronize()
+        for _, _, out in dev:
+            assert b.workspace_status(out.workspace) == b.OK
+
     for _ in range(warmup):
         step()
-    torch.cuda.synchronize()
-    for _, _, out in dev:
-        assert b.workspace_status(out.workspace) == b.OK
+    check_status()
 
     def barrier():
         if world > 1:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- timed region: K steps, device time, max over ranks ----
-    # Per-call events cost device time themselves (about 3 % of a step when every step has them), so only the
-    # first steps of the timed region carry them: one event before every call and one after the last, a call's
-    # time running to the start of the next.
+    # ---- timed region: K eagerly launched steps, device time, max over ranks ----
+    # One event per step boundary gives the per-step times (median, best).  The first steps also carry one event
+    # before every call (a call's time then runs to the start of the next call) for the roofline of the dominant
+    # kernel; these events cost a little device time themselves and keep a call from being set up while its
+    # predecessor drains, so the steps that carry them are a bit slower than the others - they are part of `value`.
     event_steps = min(args.steps, 3)
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(calls) + 1)] for _ in range(event_steps)]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    # The steps without per-call events are replays of the step captured once in a CUDA graph (the same 24
-    # library calls; it spares the launch gaps between them).  --no-graph, or a capture that fails, launches eagerly.
-    graph = None
-    if not args.no_graph and args.op == "fused" and args.steps > event_steps:
-        try:
-            graph = torch.cuda.CUDAGraph()
-            with torch.cuda.graph(graph, stream=stream):
-                step()
-            graph.replay()
-            torch.cuda.synchronize()
-            for _, _, out in dev:
-                assert b.workspace_status(out.workspace) == b.OK
-        except Exception as err:       # noqa: BLE001
-            print(f"CUDA graph capture failed ({err}); launching eagerly", file=sys.stderr)
-            graph = None
-            torch.cuda.synchronize()
+    marks = [torch.cuda.Event(enable_timing=True) for _ in range(args.steps + 1)]
     sampler = ClockSampler(local)
     sampler.start()
     time.sleep(0.25)
     barrier()
     t0 = time.time()
-    e0.record(stream)
+    marks[0].record(stream)
     for k in range(args.steps):
-        if k < event_steps or graph is None:
-            step(ev[k] if k < event_steps else None)
-        else:
-            graph.replay()
-    e1.record(stream)
+        step(ev[k] if k < event_steps else None)
+        marks[k + 1].record(stream)
     barrier()
     t1 = time.time()
-    total_ms = e0.elapsed_time(e1)
+    total_ms = marks[0].elapsed_time(marks[args.steps])
+    step_ms = [marks[k].elapsed_time(marks[k + 1]) for k in range(args.steps)]
     # keep the GPU under the same load a little longer so the clock sampler sees it
     if t1 - t0 < 0.6:
         tend = time.time() + 0.6
@@ -373,16 +433,40 @@ def main():
     total_ms = max_over_ranks(total_ms)
     ms_per_step = total_ms / args.steps
     value = whole_job_gbs(bytes_per_step, world, ms_per_step)
+    plain_steps = step_ms[event_steps:] or step_ms
+    check_status()
+
+    # ---- the same step replayed from a CUDA graph (spares the launch gaps; reported beside `value`) ----
+    graph_rec = None
+    if not args.no_graph and args.op == "fused":
+        try:
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                step()
+            graph.replay()
+            check_status()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            g0.record(stream)
+            for _ in range(5):
+                graph.replay()
+            g1.record(stream)
+            torch.cuda.synchronize()
+            g_ms = g0.elapsed_time(g1) / 5
+            graph_rec = {"ms_per_step": g_ms, "value": whole_job_gbs(bytes_per_step, 1, g_ms), "unit": UNIT,
+                         "steps": 5, "note": "the step captured once and replayed; this rank only"}
+            del graph
+        except Exception as err:       # noqa: BLE001
+            graph_rec = {"unavailable": str(err)[:200]}
+            torch.cuda.synchronize()
 
     # ---- per-call device times inside the timed region -> roofline of the dominant kernel ----
     per_call_ms = [statistics.mean(ev[k][ci].elapsed_time(ev[k][ci + 1]) for k in range(event_steps))
                    for ci in range(len(calls))]
-    # dominant kernel: the column-walk instantiation for planes that are whole 16-byte packs (all but the 7x7 ones)
+    # dominant kernel: the column-walk instantiation for planes that are whole 16-byte packs
     dominant = [ci for ci, (i, _) in enumerate(calls) if (specs[i].shape[2] * specs[i].shape[3]) % 4 == 0
                 and plans[ci][0] == b.PLAN_COLWALK]
     dom_bytes = sum(specs[calls[ci][0]].numel for ci in dominant) * bpe
     dom_ms = sum(per_call_ms[ci] for ci in dominant)
-    peak, peak_src = measured_peak()
     achieved = dom_bytes / (dom_ms * 1e-3) / 1e9 if dominant else None
     rec = recorded_traffic()
     roofline = {
@@ -397,12 +481,194 @@ def main():
         "share_of_step_time": dom_ms / sum(per_call_ms),
         "note": "achieved = algorithmic bytes of the launches / their CUDA-event time (from the event before a call to the event before the next: launch gaps included; events in the first 3 timed steps)",
     }
-    per_tensor = []
+    in_step = []
     for ci, (i, bits) in enumerate(calls):
         gbs = specs[i].numel * bpe / (per_call_ms[ci] * 1e-3) / 1e9
-        per_tensor.append({"tensor": specs[i].name, "bits": bits, "us": round(per_call_ms[ci] * 1e3, 2),
-                           "GBps": round(gbs, 1), "frac_measured": round(gbs / peak, 3),
-                           "frac_8TBs": round(gbs / NOMINAL_HBM_GBS, 3), "plan": plans[ci][0]})
+        in_step.append({"tensor": specs[i].name, "bits": bits, "us": round(per_call_ms[ci] * 1e3, 2),
+                        "GBps": round(gbs, 1), "frac_measured": round(gbs / peak, 3), "plan": plans[ci][0]})
+
+    # ---- helpers for the bounded records below ----
+    def sustained_us(run, n_calls, reps=3):
+        """Median and best time per call of `run(k)` for k in range(n_calls), launched back to back with no
+        event between the calls."""
+        run_all = lambda: [run(k) for k in range(n_calls)]      # noqa: E731
+        run_all()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a0, a1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a0.record(stream)
+            run_all()
+            a1.record(stream)
+            torch.cuda.synchronize()
+            ts.append(a0.elapsed_time(a1) * 1e3 / n_calls)
+        return statistics.median(ts), min(ts)
+
+    def rotating(x, gy, groups, group=b.GROUP_CHANNEL, min_bytes=400_000_000):
+        """Copies of (x, gy, outputs) whose four arrays together exceed three times the L2: calls that walk
+        over them find their tensor cold.  A tensor that large by itself is its own single copy."""
+        n = max(1, -(-min_bytes // (4 * x.numel() * x.element_size())))
+        sets = [(x, gy, outputs_for(x, groups, group))]
+        for _ in range(n - 1):
+            sets.append((x.clone(), gy.clone(), outputs_for(x, groups, group)))
+        return sets
+
+    def frac(elems, bytes_per_elem, us):
+        return elems * bytes_per_elem / us / 1e3 / peak
+
+    per_tensor, per_bits, sub = [], {}, {}
+    if not args.no_sub and args.op == "fused":
+        # ---- every call of the step by itself: sustained, cold, no event between calls ----
+        for i, s in enumerate(specs):
+            x, gy, _ = dev[i]
+            sets = rotating(x, gy, s.shape[1])
+            n_calls = max(4, 2 * len(sets))
+            for bits in s.bits:
+                med, best = sustained_us(lambda k: one_call(*sets[k % len(sets)], bits), n_calls)
+                per_tensor.append({"tensor": s.name, "bits": bits, "us": round(med, 2), "best_us": round(best, 2),
+                                   "GBps": round(s.numel * 16 / med / 1e3, 1), "frac_measured": round(frac(s.numel, 16, med), 3),
+                                   "frac_8TBs": round(s.numel * 16 / med / 1e3 / NOMINAL_HBM_GBS, 3),
+                                   "elements_per_s": s.numel / (med * 1e-6), "copies": len(sets),
+                                   "plan": b.fused_plan(b.F32, s.shape, flags=plan_flags)[0]})
+                acc = per_bits.setdefault(bits, [0, 0.0])
+                acc[0] += s.numel
+                acc[1] += med
+            del sets
+        check_status()
+
+        # ---- other group mode, plan, contract on tensors of the step ----
+        def pick(name):
+            for i, s in enumerate(specs):
+                if name in s.name:
+                    return i, s
+            return None, None
+        for name in ("cfg3.2", "cfg3.4"):
+            i, s = pick(name)
+            if s is None:
+                continue
+            x, gy, _ = dev[i]
+            G = b.num_groups(s.shape, 1, b.GROUP_SAMPLE_CHANNEL)
+            sets = rotating(x, gy, G, b.GROUP_SAMPLE_CHANNEL)
+            med, best = sustained_us(lambda k: one_call(*sets[k % len(sets)], 4, group=b.GROUP_SAMPLE_CHANNEL),
+                                     max(4, 2 * len(sets)))
+            sub.setdefault("per_sample_groups", []).append(
+                {"tensor": s.name, "groups": G, "us": round(med, 2), "frac_measured": round(frac(s.numel, 16, med), 3),
+                 "plan": b.fused_plan(b.F32, s.shape, group=b.GROUP_SAMPLE_CHANNEL)[0]})
+            del sets
+        i, s = pick("cfg3.4")
+        if s is not None:          # the 'conventional' per-channel loop: three launches per channel
+            x, gy, out = dev[i]
+            med, best = sustained_us(lambda k: one_call(x, gy, out, 4, fl=b.FLAG_FORCE_NAIVE), 2, reps=2)
+            sub["naive_per_channel_loop"] = [{"tensor": s.name, "launches": 3 * s.shape[1], "us": round(med, 1),
+                                              "frac_measured": round(frac(s.numel, 16, med), 4)}]
+        # default contract: every call clears its own workspace (no GRANQ_FLAG_WORKSPACE_ZEROED)
+        for _ in range(2):
+            for ci, (i, bits) in enumerate(calls):
+                one_call(*dev[i], bits, fl=plan_flags)
+        d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        d0.record(stream)
+        for _ in range(3):
+            for ci, (i, bits) in enumerate(calls):
+                one_call(*dev[i], bits, fl=plan_flags)
+        d1.record(stream)
+        torch.cuda.synchronize()
+        d_ms = d0.elapsed_time(d1) / 3
+        sub["default_workspace_contract"] = {"ms_per_step": d_ms, "value": whole_job_gbs(bytes_per_step, 1, d_ms),
+                                             "frac_measured": whole_job_gbs(bytes_per_step, 1, d_ms) / peak,
+                                             "note": "every call clears its workspace itself (one memset node more "
+                                                     "per call); 3 eager steps"}
+        check_status()
+
+        if rank == 0 and not args.only:
+            # ---- configs 1, 2, 5 (bounded: a few calls each) ----
+            s1 = wl.config_tensors(1)[0]
+            x1 = torch.from_numpy(wl.make_activation(s1)).cuda()
+            g1_ = torch.from_numpy(wl.make_upstream_grad(s1)).cuda()
+            sets = rotating(x1, g1_, s1.shape[1])
+            cold, _ = sustained_us(lambda k: one_call(*sets[k % len(sets)], 3), len(sets))
+            warm, _ = sustained_us(lambda k: one_call(*sets[0], 3), 50)
+            sub["config1"] = {"tensor": s1.name, "bits": 3, "cold_us": round(cold, 2), "warm_us": round(warm, 2),
+                              "cold_frac_measured": round(frac(s1.numel, 16, cold), 4),
+                              "warm_frac_measured": round(frac(s1.numel, 16, warm), 4),
+                              "note": "1 MB tensor: launch-bound (the host needs about 10 us per call)"}
+            del sets
+            c2 = wl.config_tensors(2)
+            t2 = []
+            for s in c2:
+                x = torch.from_numpy(wl.make_activation(s)).cuda()
+                gy = torch.from_numpy(wl.make_upstream_grad(s)).cuda()
+                t2.append((x, gy, outputs_for(x, s.shape[1])))
+            calls2 = [(j, bits) for bits in (3, 4) for j in range(len(c2))]
+            e2 = sum(c2[j].numel for j, _ in calls2)
+            cold, _ = sustained_us(lambda k: one_call(*t2[calls2[k][0]], calls2[k][1]), len(calls2))
+            small = [j for j, s in enumerate(c2) if s.shape[1] == 64][:2]       # 2 x 4 x 4.2 MB: stays in the L2
+            warm, _ = sustained_us(lambda k: one_call(*t2[small[k % 2]], 3), 40)
+            sub["config2"] = {"calls": len(calls2), "elements": e2, "ms_per_set": cold * len(calls2) / 1e3,
+                              "cold_frac_measured": round(frac(e2, 16, cold * len(calls2)), 3),
+                              "warm_small_tensor_us": round(warm, 2),
+                              "warm_small_tensor_frac_measured": round(frac(c2[small[0]].numel, 16, warm), 3),
+                              "note": "19 tensors x b in {3,4}, 772 MB working set (cold between calls); the 4 MB "
+                                      "tensors alternating in pairs stay in the L2 (warm) and are launch-bound"}
+            del t2
+            torch.cuda.empty_cache()
+            gen = torch.Generator(device="cuda").manual_seed(5000)
+            rows5 = []
+            for s in wl.config_tensors(5):
+                # values of the same recipe generated on the device (Student-t(3), per-channel log-normal spread)
+                sig = torch.exp(torch.randn(1, s.shape[1], 1, 1, device="cuda", generator=gen))
+                x32 = torch.randn(s.shape, device="cuda", generator=gen)
+                den = torch.zeros(s.shape, device="cuda")
+                for _ in range(3):
+                    den += torch.randn(s.shape, device="cuda", generator=gen) ** 2
+                x32 = x32 / torch.sqrt(den / 3.0).clamp_min(1e-6) * sig
+                del den
+                g32 = torch.randn(s.shape, device="cuda", generator=gen)
+                for dt in ("f32", "bf16"):
+                    x = x32 if dt == "f32" else x32.bfloat16()
+                    gy = g32 if dt == "f32" else g32.bfloat16()
+                    out = outputs_for(x, s.shape[1])
+                    e = x.element_size()
+                    fused, _ = sustained_us(lambda k: one_call(x, gy, out, 2 + k % 7), 7, reps=2)
+                    fwd, _ = sustained_us(lambda k: one_call(x, None, out, 2 + k % 7, op="fused_fwd"), 7, reps=2)
+                    rows5.append({"tensor": s.name, "dtype": dt, "bits": "2..8 (one call each)",
+                                  "fused_us": round(fused, 1), "fused_frac_measured": round(frac(s.numel, 4 * e, fused), 3),
+                                  "fwd_only_us": round(fwd, 1), "fwd_only_frac_measured": round(frac(s.numel, 2 * e, fwd), 3),
+                                  "elements_per_s_fused": s.numel / (fused * 1e-6),
+                                  "plan": b.fused_plan(b.F32 if dt == "f32" else b.BF16, s.shape)[0]})
+                    del out
+                del x32, g32
+                torch.cuda.empty_cache()
+            sub["config5"] = {"rows": rows5, "data": "device-generated Student-t(3) x per-channel log-normal spread "
+                                                     "(same recipe as the parity inputs); each tensor is larger "
+                                                     "than the L2, so every call is cold"}
+
+    sharded = None
+    if args.sharded:
+        from paper_2503_18339_b200 import data_parallel as dp
+        for x, gy, out in dev:
+            out.packed_mask = b.make_packed_mask(x)
+
+        def sharded_step():
+            for i, bits in calls:
+                x, gy, out = dev[i]
+                lo, hi = b.granq_range(x, lo=out.lo, hi=out.hi, workspace=out.workspace, stream=stream)
+                dp.sync_range(lo, hi, stream=stream)
+                b.granq_fakequant_fwd_packmask(x, bits, lo, hi, y=out.y, packed_mask=out.packed_mask, stream=stream)
+                b.granq_fakequant_bwd_packmask(gy, out.packed_mask, gx=out.gx, stream=stream)
+        sharded_step()
+        barrier()
+        h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        h0.record(stream)
+        for _ in range(3):
+            sharded_step()
+        h1.record(stream)
+        barrier()
+        h_ms = max_over_ranks(h0.elapsed_time(h1) / 3)
+        sharded = {"ms_per_step": h_ms, "value": whole_job_gbs(int(elems_per_step * 20.25), world, h_ms), "unit": UNIT,
+                   "bytes_per_element": 20.25, "scaling": "strong in the batch: every rank holds 1/N of a global batch "
+                   "and all ranks quantize with its range",
+                   "note": "range (4 B) + all-reduce of 2*C floats + forward with packed mask (8.125 B) + backward "
+                           "from the mask (8.125 B)"}
 
     # ---- end to end through the host-buffer entry point (pinned memory, copies timed) ----
     e2e = None
@@ -493,24 +759,31 @@ def main():
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
             "config": {"workload": WORKLOAD, "elements_per_step_per_gpu": elems_per_step,
-                       "calls_per_step": len(calls), "l2": "inputs larger than L2 (7.3 GB working set per step)",
+                       "calls_per_step": len(calls),
+                       "l2": "inputs larger than L2: a step is all 12 tensors at 4 bits, then all 12 at 5 bits, so "
+                             "3.6 GB pass through the 126 MB L2 between two calls on the same tensor (every call is cold)",
                        "group_mode": "channel",
-                       "launch": ("steps %d..%d replay the step captured in a CUDA graph, steps 1..%d are launched eagerly "
-                                  "with one CUDA event per call" % (event_steps + 1, args.steps, event_steps)
-                                  if graph is not None else "every step launched eagerly"),
+                       "launch": ("every step launched eagerly through the C ABI; steps 1..%d carry one CUDA event per "
+                                  "call" % event_steps),
                        "workspace": ("cleared by every call" if args.clear_workspace else
-                                     "cleared once at allocation, GRANQ_FLAG_WORKSPACE_ZEROED on every call"), "parallelism": f"replicas x{world} (independent batches, no exchange)"},
+                                     "cleared once at allocation, GRANQ_FLAG_WORKSPACE_ZEROED on every call"),
+                       "parallelism": f"replicas x{world} (independent batches, no exchange)"},
+            "step_ms": {"mean": ms_per_step, "median": statistics.median(step_ms), "best": min(step_ms),
+                        "median_without_call_events": statistics.median(plain_steps), "rank": 0},
+            "value_median_step": whole_job_gbs(bytes_per_step, world, statistics.median(step_ms)),
+            "value_best_step": whole_job_gbs(bytes_per_step, world, min(step_ms)),
             "elements_per_s": world * elems_per_step / (ms_per_step * 1e-3),
+            "elements_per_s_by_bits": {str(k): v[0] / (v[1] * 1e-6) for k, v in sorted(per_bits.items())},
             "frac_of_measured_hbm": value / world / peak, "frac_of_nominal_8TBs": value / world / NOMINAL_HBM_GBS,
             "gpu_launches": launches_per_step * args.steps, "clocks": clocks, "e2e": e2e, "roofline": roofline,
-            "cpu_baseline": cpu, "per_tensor": per_tensor,
+            "cpu_baseline": cpu, "graph_replay": graph_rec, "per_tensor": per_tensor, "in_step": in_step, "sub": sub,
+            "sharded": sharded,
         }
         print(json.dumps(line))
         if args.table:
-            for r in per_tensor:
+            for r in (per_tensor or in_step):
                 print(f"{r['tensor']:28s} b={r['bits']} {r['us']:9.1f} us {r['GBps']:8.1f} GB/s "
-                      f"{100 * r['frac_measured']:5.1f}% of measured {100 * r['frac_8TBs']:5.1f}% of 8 TB/s",
-                      file=sys.stderr)
+                      f"{100 * r['frac_measured']:5.1f}% of measured plan {r['plan']}", file=sys.stderr)
     if world > 1:
         dist.destroy_process_group()
 

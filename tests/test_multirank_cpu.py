@@ -47,3 +47,23 @@ def test_single_process_is_the_identity():
     import bench
     assert bench.max_over_ranks(3.5, device="cpu") == 3.5
     assert np.isclose(bench.whole_job_gbs(16_000_000_000, 1, 4.0), 4000.0)
+
+
+def test_plain_command_with_gpus_2_starts_its_own_ranks():
+    """`python bench.py --gpus 2` without a torchrun environment spawns the ranks itself: here with the
+    GPU-free self-test (gloo), rank 0 printing the aggregate over both ranks and the slower rank's time."""
+    import json
+    import subprocess
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "LOCAL_RANK", "WORLD_SIZE", "MASTER_ADDR", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--gpus", "2", "--rank-selftest"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    line = json.loads(res.stdout.strip().splitlines()[-1])
+    assert line["n_gpus"] == 2 and line["ms_per_step"] == 20.0 and line["value"] == 2 * 1e9 / 20e-3 / 1e9
+
+
+def test_spawn_ranks_sets_the_torchrun_environment():
+    sys.path.insert(0, ROOT)
+    import bench
+    code = "import os,sys; sys.exit(0 if (os.environ['WORLD_SIZE'], os.environ['MASTER_ADDR']) == ('3', '127.0.0.1') and os.environ['RANK'] == os.environ['LOCAL_RANK'] else 1)"
+    assert bench.spawn_ranks(3, [sys.executable, "-c", code], timeout=60) == [0, 0, 0]
