@@ -642,6 +642,98 @@ def main():
                                                      "(same recipe as the parity inputs); each tensor is larger "
                                                      "than the L2, so every call is cold"}
 
+        if rank == 0 and not args.only:
+            # ---- the other entry points over the step's tensors (one pass each, b = 4) ----
+            for x, gy, out in dev:
+                out.packed_mask = b.make_packed_mask(x)
+                one_call(x, gy, out, 4)          # a range for the calls that take one
+            rows = {}
+            for op, bytes_pe in (("range", 4), ("fwd", 8), ("bwd", 12), ("fused_fwd", 8), ("fused_fwd_packmask", 8.125),
+                                 ("bwd_packmask", 8.125)):
+                med, _ = sustained_us(lambda k: one_call(*dev[k], 4, op=op), len(dev), reps=2)
+                tot = sum(s.numel for s in specs)
+                big = [i for i, s in enumerate(specs) if s.numel * 4 >= 100_000_000]
+                med_big, _ = sustained_us(lambda k: one_call(*dev[big[k]], 4, op=op), len(big), reps=2)
+                rows[op] = {"bytes_per_element": bytes_pe, "frac_measured_all_12": round(frac(tot, bytes_pe, med * len(dev)), 3),
+                            "frac_measured_100MB_and_up": round(frac(sum(specs[i].numel for i in big), bytes_pe,
+                                                                     med_big * len(big)), 3)}
+            sub["entry_points"] = rows
+            check_status()
+            # ---- packed integer codes on one tensor (4 + b/8 bytes per element each way) ----
+            i, s = pick("cfg3.1")
+            x, gy, out = dev[i]
+            rows = []
+            for bits in (3, 4, 5):
+                pc = torch.empty(b.packed_codes_bytes(x.shape, bits) // 4, dtype=torch.int32, device="cuda")
+                q = b.granq_quantize_packed(x, bits, out.lo, out.hi, packed_codes=pc, stream=stream)
+                tq, _ = sustained_us(lambda k: b.granq_quantize_packed(x, bits, out.lo, out.hi, packed_codes=pc,
+                                                                       stream=stream), 3, reps=2)
+                td, _ = sustained_us(lambda k: b.granq_dequantize_packed(pc, x.shape, x.dtype, bits, q.s, q.z, y=out.y,
+                                                                         stream=stream), 3, reps=2)
+                rows.append({"tensor": s.name, "bits": bits, "quantize_us": round(tq, 1),
+                             "quantize_frac_measured": round(frac(s.numel, 4 + bits / 8, tq), 3),
+                             "dequantize_us": round(td, 1), "dequantize_frac_measured": round(frac(s.numel, 4 + bits / 8, td), 3)})
+            sub["packed_codes"] = rows
+            # ---- all weight tensors of a network in one launch against one fused call per tensor ----
+            rows = []
+            for net in ("resnet20", "resnet18"):
+                ws = [torch.from_numpy(w).cuda() for w in wl.make_weights(net)]
+                gs = [torch.from_numpy(g).cuda() for g in wl.make_weights(net, grads=True)]
+                ws4 = [w.reshape(w.shape[0], -1, 1, 1) for w in ws]
+                gs4 = [g.reshape(g.shape[0], -1, 1, 1) for g in gs]
+                wouts = [b.FakeQuantOut(y=torch.empty_like(w), gx=torch.empty_like(w), workspace=b.make_workspace(w, 0))
+                         for w in ws4]
+                batch = b.WeightBatch(ws, 4, grads=gs)
+                tb, _ = sustained_us(lambda k: batch.run(stream=stream), 5)
+                tl, _ = sustained_us(lambda k: b.granq_fakequant_fused(ws4[k], 4, gy=gs4[k], channel_axis=0, out=wouts[k],
+                                                                       stream=stream), len(ws4))
+                rows.append({"network": net, "tensors": len(ws), "elements": sum(w.numel() for w in ws),
+                             "batched_us": round(tb, 1), "one_call_per_tensor_us": round(tl * len(ws4), 1)})
+            sub["weights"] = rows
+            # ---- Table 2 in kind: layer-wise against channel-wise at 3 bits on the ResNet-20-shaped set ----
+            rows, seen = [], set()
+            for s2 in wl.config_tensors(2):
+                if s2.shape in seen:
+                    continue
+                seen.add(s2.shape)
+                x2 = torch.from_numpy(wl.make_activation(s2)).cuda()
+                row = {"tensor": s2.name, "bits": 3}
+                for name, group in (("layer_wise", b.GROUP_TENSOR), ("channel_wise", b.GROUP_CHANNEL)):
+                    o2 = b.FakeQuantOut(y=torch.empty_like(x2))
+                    b.granq_fakequant_fused_stats(x2, 3, group=group, out=o2, stream=stream)
+                    torch.cuda.synchronize()
+                    cos, rel = b.distortion_from_sums(o2.sums.cpu().tolist())
+                    row[name] = {"cosine": round(cos, 4), "rel_error": round(rel, 4)}
+                rows.append(row)
+                del x2
+            sub["table2_in_kind"] = {"rows": rows, "paper": "ResNet-20, 3 bits: layer-wise 0.5111 / 0.3129, channel-wise "
+                                                            "0.6835 / 0.1063 (cosine / relative error; other data)"}
+            # ---- Table 5 in kind: one forward pass over the 19 ResNet-20 activation tensors at batch 16, 3 bits ----
+            import dataclasses
+            s16 = [dataclasses.replace(s2, shape=(16,) + tuple(s2.shape[1:])) for s2 in wl.config_tensors(2)]
+            x16 = [torch.from_numpy(wl.make_activation(s2)).cuda() for s2 in s16]
+            rows = []
+            for name, group, fl in (("layer-wise", b.GROUP_TENSOR, 0),
+                                    ("channel-wise, per-channel loop", b.GROUP_CHANNEL, b.FLAG_FORCE_NAIVE),
+                                    ("channel-wise, default plan", b.GROUP_CHANNEL, 0)):
+                o16 = [b.FakeQuantOut(y=torch.empty_like(x), workspace=b.make_workspace(x, 1, group)) for x in x16]
+                launches = sum(b.fused_plan(b.F32, x.shape, group=group, with_backward=False, flags=fl)[1] for x in x16)
+
+                def one_pass():
+                    for x, o in zip(x16, o16):
+                        b.granq_fakequant_fused(x, 3, group=group, out=o, flags=fl, stream=stream)
+                one_pass()
+                torch.cuda.synchronize()
+                walls = []
+                for _ in range(5):
+                    w0 = time.perf_counter()
+                    one_pass()
+                    torch.cuda.synchronize()
+                    walls.append((time.perf_counter() - w0) * 1e3)
+                rows.append({"scheme": name, "ms_per_pass_wall": round(statistics.median(walls), 3), "launches": launches})
+            sub["table5_in_kind"] = {"rows": rows, "paper_ms": {"layer-wise": 0.227, "channel-wise (conventional)": 103.671,
+                                                                "GranQ": 0.236}, "paper_hardware": "not stated"}
+
     sharded = None
     if args.sharded:
         from paper_2503_18339_b200 import data_parallel as dp

@@ -434,7 +434,7 @@ __global__ void __launch_bounds__(kKMaxThreads, 2) cluster_kernel(const KArgs a)
         auto emit = [&](const Pack<T>& px, const Pack<T>& pg, size_t at) {
             Pack<T> py, pgx;
             uint32_t cb[V / 4], mb[V / 4];
-            quantize_pack<T, kBwd, !ALIGNED, EXTRAS>(px, pg, g1, g2, ne, qmax, py, pgx, cb, mb);
+            quantize_pack<T, kBwd, !ALIGNED, EXTRAS, true>(px, pg, g1, g2, ne, qmax, py, pgx, cb, mb);
             st_hint_16(yg + at, py.raw, drop);
             if constexpr (kBwd) st_hint_16(gxg + at, pgx.raw, drop);
             if constexpr (EXTRAS) {

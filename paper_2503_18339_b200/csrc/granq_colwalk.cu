@@ -307,7 +307,7 @@ __global__ void __launch_bounds__(kCThreads, 4) colwalk_kernel(const CArgs a) {
             auto emit = [&](const Pack<T>& px, const Pack<T>& pg, size_t at) {
                 Pack<T> py, pgx;
                 uint32_t cb[V / 4], mb[V / 4];
-                quantize_pack<T, kBwd, !ALIGNED, EXTRAS>(px, pg, g1, g2, it.ne, qmax, py, pgx, cb, mb);
+                quantize_pack<T, kBwd, !ALIGNED, EXTRAS, true>(px, pg, g1, g2, it.ne, qmax, py, pgx, cb, mb);
                 st_hint_16(yg + at, py.raw, drop);
                 if constexpr (kBwd) st_hint_16(gxg + at, pgx.raw, drop);
                 if constexpr (EXTRAS) {

@@ -242,44 +242,71 @@ __device__ __forceinline__ GroupParam group_param_from_keys(const uint32_t* kmin
     return gp;
 }
 
+// The rounded value r = round(x / s + z) from ONE fused multiply-add, where that is provably the same integer.
+// Only r enters the results (code = clamp(r), y = s * (code - z), mask = (r == code)); the quotient and the sum
+// are intermediates.  With rcp = RN(1 / s), up = RN(x * rcp + z) lies within E = 2^-24 * (|x / s| + |up|) of the
+// real number v = x / s + z, and so does the exactly rounded u = RN(RN(x / s) + z).  |x / s| <= |v| + |z|, and
+// values beyond the clamp range [-1, qmax + 1] round to the same clamped integer either way, so inside it
+// E <= 2^-24 * (|z| + 2 * 258) < M = 2^-23 * (|z| + 1024).  If up is farther than 2 M from every half-integer,
+// v is farther than M from it, u lies on the same side, and round(u) = round(up).  tie_threshold() returns
+// 0.5 - 2 M: an element whose distance |up - round(up)| reaches it takes the exact sequence instead (for
+// |z| >= 2^21 the threshold is <= 0 and every element does).
+__device__ __forceinline__ float tie_threshold(float z) {
+    return __fmaf_rn(-2.384185791015625e-07f, __fadd_rn(fabsf(z), 1024.0f), 0.5f);      // 0.5 - 2^-22 * (|z| + 1024)
+}
+
 // Quantize one pack: elements [0, n1) belong to the group with parameters g1, the rest to
 // g2 (n1 = V when the pack lies in one group).  EXTRAS also packs the codes and the mask
-// (one byte per element).
-template <typename T, bool BWD, bool SPLIT, bool EXTRAS>
+// (one byte per element).  SELF: the range is that of the tensor itself, so x / s + z lies within
+// [-1, qmax + 1] already (x in [lo, hi] gives RN(x / s) - round(RN(lo / s)) >= -1/2, and at most qmax plus a few
+// units in the last place of hi / s < 2^33 above that) and the clamp before the rounding can go.
+template <typename T, bool BWD, bool SPLIT, bool EXTRAS, bool SELF = false>
 __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& pg, const GroupParam& g1,
                                               const GroupParam& g2, int n1, float qmax, Pack<T>& py, Pack<T>& pgx,
                                               uint32_t (&cb)[Pack<T>::V / 4], uint32_t (&mb)[Pack<T>::V / 4]) {
     constexpr int V = Pack<T>::V;
+    const float kMagic = 12582912.0f;  // 1.5 * 2^23
 #pragma unroll
     for (int i = 0; i < V / 4; ++i) {
         cb[i] = 0;
         mb[i] = 0;
     }
-    auto element = [&](int i, float t, float s, float z) {
-        float yv;
-        bool in;
-        const float code = quant_from_quotient(t, s, z, qmax, yv, in);
-        py.set(i, yv);
+    auto finish = [&](int i, float r, float s, float z) {      // r: the rounded value, within [-1, qmax + 1]
+        const float q = fminf(fmaxf(r, 0.0f), qmax);
+        const bool in = (r == q);
+        py.set(i, __fmul_rn(s, __fsub_rn(q, z)));
         if constexpr (BWD) pgx.set(i, in ? pg.get(i) : 0.0f);
         if constexpr (EXTRAS) {
-            cb[i / 4] |= (uint32_t)code << (8 * (i % 4));
+            cb[i / 4] |= (uint32_t)q << (8 * (i % 4));
             mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
         }
     };
+    auto exact_round = [&](float t, float z) -> float {        // t = RN(x / s): the sequence as defined
+        const float u = __fadd_rn(t, z);
+        const float uc = fminf(fmaxf(u, -1.0f), __fadd_rn(qmax, 1.0f));
+        return __fsub_rn(__fadd_rn(uc, kMagic), kMagic);
+    };
     const bool fast = SPLIT ? (g1.r != 0.0f && g2.r != 0.0f) : (g1.r != 0.0f);
     if (fast) {
+        const float thr1 = tie_threshold(g1.z), thr2 = SPLIT ? tie_threshold(g2.z) : thr1;
 #pragma unroll
         for (int i = 0; i < V; ++i) {
             const bool first = !SPLIT || i < n1;
             const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z, rc = first ? g1.r : g2.r;
-            element(i, div_by_scale(px.get(i), s, rc), s, z);
+            const float x = px.get(i);
+            float up = __fmaf_rn(x, rc, z);
+            if constexpr (!SELF) up = fminf(fmaxf(up, -1.0f), __fadd_rn(qmax, 1.0f));
+            float r = __fsub_rn(__fadd_rn(up, kMagic), kMagic);
+            if (!(fabsf(__fsub_rn(up, r)) < (first ? thr1 : thr2)))     // rare: too close to a tie for the shortcut
+                r = exact_round(div_by_scale(x, s, rc), z);
+            finish(i, r, s, z);
         }
     } else {
 #pragma unroll
         for (int i = 0; i < V; ++i) {
             const bool first = !SPLIT || i < n1;
             const float s = first ? g1.s : g2.s, z = first ? g1.z : g2.z;
-            element(i, __fdiv_rn(px.get(i), s), s, z);
+            finish(i, exact_round(__fdiv_rn(px.get(i), s), z), s, z);
         }
     }
 }

@@ -272,7 +272,7 @@ __global__ void __launch_bounds__(kLThreads, UPL == 2 ? 4 : 3) l2wave_kernel(con
                 if (!valid) continue;
                 Pack<T> py, pgx;
                 uint32_t cb[V / 4], mb[V / 4];
-                quantize_pack<T, kBwd, !ALIGNED, EXTRAS>(px[j], pg[j], g1, g2, n1, qmax, py, pgx, cb, mb);
+                quantize_pack<T, kBwd, !ALIGNED, EXTRAS, true>(px[j], pg[j], g1, g2, n1, qmax, py, pgx, cb, mb);
                 const uint32_t gu = gbase + uo;
                 st_hint_16(yg + gu, py.raw, drop);
                 if constexpr (kBwd) st_hint_16(gxg + gu, pgx.raw, drop);
