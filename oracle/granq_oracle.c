@@ -256,3 +256,54 @@ int granq_oracle_dequant_packed(const uint8_t* packed, int dtype, const int64_t 
     return 0;
 }
 
+
+/* ---- the accumulation over the pre-scaled activations (Eq. 6 left-hand side, Algorithm 1 output step) ---- */
+
+/* Pointwise (1 x 1) case.  codes: the integer codes of Eq. 1, [N, C, P] (channels_last = 0: the paper's
+ * C x (HW) matrix per sample) or [N, P, C] (channels_last = 1); s, z: per-channel scale and zero-point (Eq. 5);
+ * w: fp32 [O, C]; y: fp64, [N, O, P] or [N, P, O].
+ * Eq. 6 / Algorithm 1: the pre-scaled activation A~ = s_c * (code - z_c) is formed first, in fp32 exactly as
+ * the pre-scale step forms it (one subtract, one multiply), then y = sum_c w[o][c] * A~[c], products and sum
+ * in fp64, c ascending. */
+int granq_oracle_accumulate(const uint8_t* codes, const int64_t dims[3], int channels_last, const float* s,
+                            const float* z, const float* w, int64_t O, double* y) {
+    if (!codes || !dims || !s || !z || !w || !y || O <= 0) return -1;
+    const int64_t N = dims[0], C = dims[1], P = dims[2];
+    if (N <= 0 || C <= 0 || P <= 0) return -1;
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t o = 0; o < O; ++o)
+            for (int64_t p = 0; p < P; ++p) {
+                double acc = 0.0;
+                for (int64_t c = 0; c < C; ++c) {
+                    const uint8_t code = channels_last ? codes[(n * P + p) * C + c] : codes[(n * C + c) * P + p];
+                    float d = (float)code - z[c];
+                    float a = s[c] * d;                           /* the pre-scaled activation */
+                    acc += (double)w[o * C + c] * (double)a;
+                }
+                if (channels_last) y[(n * P + p) * O + o] = acc;
+                else y[(n * O + o) * P + p] = acc;
+            }
+    return 0;
+}
+
+/* Eq. 3, the conventional order the paper contrasts with: the per-channel scale is applied inside the
+ * accumulation, y = sum_c w_c * s_c * (code_c - z_c), every operation in fp64.  The same real number as
+ * Eq. 6 gives; only the order of the operations differs. */
+int granq_oracle_accumulate_inloop(const uint8_t* codes, const int64_t dims[3], int channels_last, const float* s,
+                                   const float* z, const float* w, int64_t O, double* y) {
+    if (!codes || !dims || !s || !z || !w || !y || O <= 0) return -1;
+    const int64_t N = dims[0], C = dims[1], P = dims[2];
+    if (N <= 0 || C <= 0 || P <= 0) return -1;
+    for (int64_t n = 0; n < N; ++n)
+        for (int64_t o = 0; o < O; ++o)
+            for (int64_t p = 0; p < P; ++p) {
+                double acc = 0.0;
+                for (int64_t c = 0; c < C; ++c) {
+                    const uint8_t code = channels_last ? codes[(n * P + p) * C + c] : codes[(n * C + c) * P + p];
+                    acc += (double)w[o * C + c] * (double)s[c] * ((double)code - (double)z[c]);
+                }
+                if (channels_last) y[(n * P + p) * O + o] = acc;
+                else y[(n * O + o) * P + p] = acc;
+            }
+    return 0;
+}

@@ -89,6 +89,16 @@ int granq_oracle_pack_codes(const uint8_t* codes, int64_t E, int bits, uint8_t* 
 int granq_oracle_dequant_packed(const uint8_t* packed, int dtype, const int64_t dims[4], int channel_axis,
                                 int group_mode, int bits, const float* s, const float* z, void* y);
 
+/* The accumulation over the pre-scaled activations, pointwise (1 x 1) case: Eq. 6 left-hand side and the
+ * output step of Algorithm 1, y[n][o][p] = sum_c w[o][c] * A~[n][c][p] with A~ = s_c * (code - z_c) formed
+ * first in fp32 (the pre-scale step), the sum in fp64 with c ascending.  dims = {N, C, P}; codes are
+ * [N, C, P] (channels_last = 0) or [N, P, C] (1); y is [N, O, P] or [N, P, O].  The _inloop form is Eq. 3,
+ * the conventional order with the scale inside the loop, all in fp64: the same real number. */
+int granq_oracle_accumulate(const uint8_t* codes, const int64_t dims[3], int channels_last, const float* s,
+                            const float* z, const float* w, int64_t O, double* y);
+int granq_oracle_accumulate_inloop(const uint8_t* codes, const int64_t dims[3], int channels_last, const float* s,
+                                   const float* z, const float* w, int64_t O, double* y);
+
 #ifdef __cplusplus
 }
 #endif

@@ -249,3 +249,32 @@ def dequant_packed(packed: np.ndarray, shape, bits: int, s: np.ndarray, z: np.nd
                                              _p(s), _p(z), _p(y)), "granq_oracle_dequant_packed")
     return y
 
+
+
+def accumulate(codes: np.ndarray, s: np.ndarray, z: np.ndarray, w: np.ndarray, channels_last: bool = False,
+               inloop: bool = False) -> np.ndarray:
+    """Eq. 6 left-hand side / Algorithm 1 output step, pointwise case: y = sum_c w[o, c] * s_c * (code - z_c).
+    codes: uint8 [N, C, H, W] (or [N, H, W, C] with channels_last); w: float32 [O, C]; returns float64
+    [N, O, H, W] (or [N, H, W, O]).  inloop=True evaluates Eq. 3's order instead (scale inside the loop)."""
+    codes = np.ascontiguousarray(codes, np.uint8)
+    w = np.ascontiguousarray(w, np.float32)
+    s = np.ascontiguousarray(s, np.float32)
+    z = np.ascontiguousarray(z, np.float32)
+    if codes.ndim != 4 or w.ndim != 2:
+        raise ValueError("codes must be 4-d and w 2-d")
+    if channels_last:
+        n, h, wd, c = codes.shape
+    else:
+        n, c, h, wd = codes.shape
+    o = w.shape[0]
+    if w.shape[1] != c or s.size != c or z.size != c:
+        raise ValueError("w, s, z must have one entry per channel")
+    y = np.empty((n, h, wd, o) if channels_last else (n, o, h, wd), np.float64)
+    dims = (ctypes.c_int64 * 3)(n, c, h * wd)
+    L = lib()
+    fn = L.granq_oracle_accumulate_inloop if inloop else L.granq_oracle_accumulate
+    fn.restype = ctypes.c_int
+    fn.argtypes = [ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p,
+                   ctypes.c_void_p, ctypes.c_int64, ctypes.c_void_p]
+    _check(fn(_p(codes), dims, int(channels_last), _p(s), _p(z), _p(w), o, _p(y)), "granq_oracle_accumulate")
+    return y

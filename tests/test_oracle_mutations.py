@@ -34,6 +34,12 @@ MUTATIONS = {
     "packed_codes_stride_of_8_bits": ("int64_t k = e * bits + j;\n            if ((codes[e] >> j) & 1)",
                                       "int64_t k = e * 8 + j;\n            if ((codes[e] >> j) & 1)"),
     "dequant_packed_adds_zero_point": ("float d = (float)code - z[grp];", "float d = (float)code + z[grp];"),
+    "accumulate_without_zero_point": ("float d = (float)code - z[c];\n                    float a = s[c] * d;", "float d = (float)code;\n                    float a = s[c] * d;"),
+    "accumulate_weight_indexed_transposed": ("acc += (double)w[o * C + c] * (double)a;", "acc += (double)w[c * O + o] * (double)a;"),
+    "accumulate_inloop_scale_of_the_output_channel": ("acc += (double)w[o * C + c] * (double)s[c] * ((double)code - (double)z[c]);",
+                                                      "acc += (double)w[o * C + c] * (double)s[o % C] * ((double)code - (double)z[c]);"),
+    "accumulate_skips_the_last_channel": ("for (int64_t c = 0; c < C; ++c) {\n                    const uint8_t code = channels_last ? codes[(n * P + p) * C + c] : codes[(n * C + c) * P + p];\n                    float d",
+                                          "for (int64_t c = 0; c + 1 < C; ++c) {\n                    const uint8_t code = channels_last ? codes[(n * P + p) * C + c] : codes[(n * C + c) * P + p];\n                    float d"),
     "packed_mask_last_byte_not_cleared": ("for (int64_t b = 0; b < (E + 7) / 8; ++b) packed[b] = 0;",
                                           "for (int64_t b = 0; b < E / 8; ++b) packed[b] = 0;"),
 }

@@ -511,3 +511,46 @@ def test_dequantizing_the_packed_codes_gives_the_fake_quantized_tensor(dtype, mo
                                group_mode=mode)
         assert np.array_equal(y.view(x.dtype), ref.y.view(x.dtype))
 
+
+
+# ---- the accumulation over the pre-scaled activations (Eq. 6 left-hand side, Algorithm 1 output step) ----
+def test_accumulate_hand_case_from_the_first_hand_case():
+    """Codes, scales and zero-points of hand case H1 (channel mode, b = 2): channel 0 has s = 1, z = 0 and codes
+    [0,1,2,3 | 0,2,2,0], channel 1 has s = 1, z = 1 and codes [0,1,2,3 | 1,2,3,1], so the pre-scaled activations are
+    [0,1,2,3 | 0,2,2,0] and [-1,0,1,2 | 0,1,2,0].  With w = [[2, -1], [0.5, 0.25]] (all products exact):
+    y[o=0] = 2 A0 - A1 = [1,2,3,4 | 0,3,2,0],  y[o=1] = A0 / 2 + A1 / 4 = [-.25,.5,1.25,2 | 0,1.25,1.5,0]."""
+    codes = np.array([[[[0, 1], [2, 3]], [[0, 1], [2, 3]]], [[[0, 2], [2, 0]], [[1, 2], [3, 1]]]], np.uint8)
+    s, z = np.array([1, 1], np.float32), np.array([0, 1], np.float32)
+    w = np.array([[2, -1], [0.5, 0.25]], np.float32)
+    want = np.array([[[1, 2, 3, 4], [-0.25, 0.5, 1.25, 2.0]], [[0, 3, 2, 0], [0, 1.25, 1.5, 0]]], np.float64)
+    for inloop in (False, True):
+        y = orc.accumulate(codes, s, z, w, inloop=inloop)
+        assert y.shape == (2, 2, 2, 2) and np.array_equal(y.reshape(2, 2, 4), want)
+        ycl = orc.accumulate(np.ascontiguousarray(codes.transpose(0, 2, 3, 1)), s, z, w, channels_last=True, inloop=inloop)
+        assert np.array_equal(ycl.transpose(0, 3, 1, 2), y)
+
+
+def test_accumulate_special_weights_and_library_contraction():
+    rng = np.random.default_rng(77)
+    n, c, h, wd, o = 3, 13, 5, 7, 6
+    x = (rng.standard_normal((n, c, h, wd)) * np.exp(rng.standard_normal((1, c, 1, 1)))).astype(np.float32)
+    res = orc.fused(x, 4)
+    w = rng.standard_normal((o, c)).astype(np.float32)
+    # zero weights give zero, one-hot weights pick the pre-scaled activation of one channel (the fake-quantized tensor)
+    assert not orc.accumulate(res.codes, res.s, res.z, np.zeros((o, c), np.float32)).any()
+    onehot = np.zeros((c, c), np.float32)
+    onehot[np.arange(c), np.arange(c)[::-1]] = 1
+    y1 = orc.accumulate(res.codes, res.s, res.z, onehot)
+    assert np.array_equal(y1, res.y[:, ::-1].astype(np.float64))
+    # a library contraction in float64 over the fake-quantized tensor (Eq. 6 read as a matrix product)
+    y = orc.accumulate(res.codes, res.s, res.z, w)
+    lib = np.einsum("oc,nchw->nohw", w.astype(np.float64), res.y.astype(np.float64))
+    scale = np.einsum("oc,nchw->nohw", np.abs(w).astype(np.float64), np.abs(res.y).astype(np.float64))
+    assert np.all(np.abs(y - lib) <= 1e-13 * scale + 1e-300)
+    # Eq. 3 (scale inside the loop) is the same real number: equal up to the fp32 rounding of the pre-scaled value
+    y3 = orc.accumulate(res.codes, res.s, res.z, w, inloop=True)
+    assert np.all(np.abs(y - y3) <= 2.0 ** -23 * scale + 1e-300) and not np.array_equal(y, y3)
+    # and Eq. 3 against its own float64 contraction: w * s folded into the weights, the zero-point as a rank-one term
+    ws = w.astype(np.float64) * res.s.astype(np.float64)
+    alt = np.einsum("oc,nchw->nohw", ws, res.codes.astype(np.float64)) - (ws @ res.z.astype(np.float64)).reshape(1, o, 1, 1)
+    assert np.all(np.abs(y3 - alt) <= 1e-12 * (scale + np.abs(ws @ res.z.astype(np.float64)).reshape(1, o, 1, 1)))
