@@ -674,6 +674,24 @@ def main():
                              "quantize_frac_measured": round(frac(s.numel, 4 + bits / 8, tq), 3),
                              "dequantize_us": round(td, 1), "dequantize_frac_measured": round(frac(s.numel, 4 + bits / 8, td), 3)})
             sub["packed_codes"] = rows
+            # ---- the accumulation over the codes on the tensor cores (Eq. 6 left-hand side, pointwise case) ----
+            rows = []
+            for name, oc in (("cfg3.1", 64), ("cfg3.3", 256)):
+                i, s = pick(name)
+                x, gy, out = dev[i]
+                qp = b.granq_quantize_packed(x, 4, out.lo, out.hi, stream=stream)
+                wt = torch.randn(oc, s.shape[1], device="cuda") / 8
+                ya, wsa = b.granq_accumulate_codes(qp.packed_codes, s.shape, 4, qp.s, qp.z, wt, stream=stream)
+                ta, _ = sustained_us(lambda k: b.granq_accumulate_codes(qp.packed_codes, s.shape, 4, qp.s, qp.z, wt, y=ya,
+                                                                        workspace=wsa, stream=stream), 3, reps=2)
+                assert b.workspace_status(wsa) == b.OK
+                pix = s.numel // s.shape[1]
+                alg = s.numel * 0.5 + pix * oc * 4 + oc * s.shape[1] * 4          # packed codes in, y out, weights in
+                flops = 2.0 * pix * s.shape[1] * oc * 2                          # two bf16 halves of the weights
+                rows.append({"tensor": s.name, "out_channels": oc, "us": round(ta, 1),
+                             "frac_measured_hbm": round(alg / ta / 1e3 / peak, 3), "tflops": round(flops / ta / 1e6, 1),
+                             "note": "three launches: weights, codes -> bf16 channels-last, contraction"})
+            sub["accumulate_codes"] = rows
             # ---- all weight tensors of a network in one launch against one fused call per tensor ----
             rows = []
             for net in ("resnet20", "resnet18"):

@@ -303,6 +303,31 @@ int granq_dequantize_packed(const uint32_t* packed_codes, int dtype, const int64
                             void* cuda_stream);
 
 /*
+ * The accumulation over the integer codes, pointwise (1 x 1) case: Eq. 6 left-hand side and the output
+ * step of Algorithm 1 (Eq. 3 is the order the paper contrasts it with),
+ *     y[n][o][p] = sum_c w[o][c] * s_c * (code[n][c][p] - z_c)
+ * evaluated as  sum_c (w[o][c] * s_c) * code  -  sum_c (w[o][c] * s_c) * z_c : the scale is folded into the
+ * weights once, the sum runs over the integer codes on the tensor cores (bf16 operands - the codes are exact,
+ * the scaled weights are split into two bf16 halves - with fp32 accumulation), the zero-points become one
+ * bias per output channel.
+ *   packed_codes  in   the codes as written by granq_quantize_packed() for a tensor of `dims`
+ *                      (channel_axis 1: NCHW;  channel_axis 3: channels-last, N H W C), GRANQ_GROUP_CHANNEL
+ *   scale, zp     in   C floats each (per-channel, as written by granq_quantize_packed())
+ *   weights       in   fp32 [out_channels, C], row-major
+ *   y             out  fp32, [N, out_channels, H, W] for channel_axis 1, [N, H, W, out_channels] for 3
+ *   workspace          DEVICE scratch of granq_accumulate_workspace_bytes(), 256-byte aligned; its first word
+ *                      is a status word as described at granq_workspace_status()
+ * Result: within (2^-17 + C * 2^-22) * sum_c |w s_c| (code + |z_c|) + 2^-21 * (|bias| + |y|) of the exact sum
+ * (the split of the scaled weights, fp32 accumulation of 2 C products in any order, one rounding each of bias
+ * and y).
+ * Limits: fewer than 2^31 pixels in the batch, C < 2^20, out_channels < 2^24; otherwise GRANQ_ERR_INVALID_ARG.
+ */
+size_t granq_accumulate_workspace_bytes(const int64_t dims[4], int channel_axis, int64_t out_channels);
+int granq_accumulate_codes(const uint32_t* packed_codes, const int64_t dims[4], int channel_axis, int bits,
+                           const float* scale, const float* zp, const float* weights, int64_t out_channels,
+                           float* y, void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream);
+
+/*
  * Status word the persistent plans leave in the workspace.  Synchronises `cuda_stream`, then
  * returns GRANQ_OK, GRANQ_ERR_TIMEOUT (a bounded device-side wait ran out), or
  * GRANQ_ERR_CUDA.  `workspace` is the pointer given to the preceding call.

@@ -39,6 +39,7 @@ EXPORTS = [
     "granq_host_arena_status", "granq_distortion", "granq_fakequant_fused_stats",
     "granq_weights_workspace_bytes", "granq_fakequant_weights", "granq_packed_codes_bytes",
     "granq_quantize_packed", "granq_dequantize_packed", "granq_cluster_geometry", "granq_distortion_stats",
+    "granq_accumulate_workspace_bytes", "granq_accumulate_codes",
 ]
 NOALLOC_MAX_GROUPS = 32768
 
@@ -100,6 +101,10 @@ def lib() -> ctypes.CDLL:
         L.granq_distortion_stats.restype = ci
         L.granq_distortion_stats.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                              ctypes.POINTER(ctypes.c_double)]
+        L.granq_accumulate_workspace_bytes.restype = sz
+        L.granq_accumulate_workspace_bytes.argtypes = [i64p, ci, ctypes.c_int64]
+        L.granq_accumulate_codes.restype = ci
+        L.granq_accumulate_codes.argtypes = [vp, i64p, ci, ci, vp, vp, vp, ctypes.c_int64, vp, vp, sz, u32, vp]
         L.granq_cluster_geometry.restype = ci
         L.granq_cluster_geometry.argtypes = [ci, i64p, ci, ci, ci, i64p]
         L.granq_selftest_division.restype = ci
@@ -547,6 +552,33 @@ def granq_dequantize_packed(packed_codes: torch.Tensor, shape, dtype: torch.dtyp
                                          group, bits, _dev(s, "s"), _dev(z, "z"), _dev(y, "y"), 0, _stream(stream)),
            "granq_dequantize_packed")
     return y
+
+
+def accumulate_workspace_bytes(shape, channel_axis: int, out_channels: int) -> int:
+    return int(lib().granq_accumulate_workspace_bytes(_dims(shape), channel_axis, out_channels))
+
+
+def granq_accumulate_codes(packed_codes: torch.Tensor, shape, bits: int, s: torch.Tensor, z: torch.Tensor,
+                           weights: torch.Tensor, channel_axis: int = 1, y: torch.Tensor = None,
+                           workspace: torch.Tensor = None, stream=None):
+    """Eq. 6 left-hand side / Algorithm 1 output step, pointwise case, from the packed integer codes of a
+    tensor of `shape` (NCHW for channel_axis 1, N H W C for 3): y = sum_c w[o, c] * s_c * (code - z_c), fp32.
+    Returns (y, workspace); the workspace's status word tells whether a bounded wait ran out."""
+    shape = tuple(int(d) for d in shape)
+    if weights.dtype != torch.float32 or weights.dim() != 2 or weights.shape[1] != shape[channel_axis]:
+        raise ValueError("weights must be float32 [out_channels, C]")
+    o = int(weights.shape[0])
+    if y is None:
+        out_shape = (shape[0], o, shape[2], shape[3]) if channel_axis == 1 else (shape[0], shape[1], shape[2], o)
+        y = torch.empty(out_shape, dtype=torch.float32, device=packed_codes.device)
+    if workspace is None:
+        workspace = torch.empty(accumulate_workspace_bytes(shape, channel_axis, o), dtype=torch.uint8,
+                                device=packed_codes.device)
+    _check(lib().granq_accumulate_codes(_dev(packed_codes, "packed_codes"), _dims(shape), channel_axis, bits,
+                                        _dev(s, "s"), _dev(z, "z"), _dev(weights, "weights"), o, _dev(y, "y"),
+                                        _dev(workspace, "workspace"), workspace.numel(), 0, _stream(stream)),
+           "granq_accumulate_codes")
+    return y, workspace
 
 
 def selftest_division(pairs: int, seed: int = 0, stream=None) -> int:

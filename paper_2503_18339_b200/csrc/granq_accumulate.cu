@@ -1,0 +1,416 @@
+// The accumulation over the integer codes, pointwise (1 x 1) case: Eq. 6 left-hand side and the
+// output step of Algorithm 1,
+//     y[n][o][p] = sum_c w[o][c] * s_c * (code[n][c][p] - z_c),
+// regrouped so that the sum runs over the integer codes themselves (the paper's "pure integer-domain"
+// accumulation; Eq. 3 is the contrast, with s_c inside the loop):
+//     y = sum_c W'[o][c] * code[c]  -  bias[o],     W' = w * s (scale folded in ONCE, up front),
+//                                                   bias[o] = sum_c W'[o][c] * z_c (a rank-one term).
+// The first sum is a dense contraction and runs on the 5th-generation tensor cores:
+//   - the codes (0 .. 255) are exact in bf16; W' is split into two bf16 matrices hi + lo (hi = the
+//     rounding of W', lo = the rounding of the rest; what is left is below 2^-17 |W'|), so two
+//     tcgen05.mma per K step accumulate into the same fp32 accumulator in tensor memory;
+//   - operands are staged in shared memory by TMA tile loads of this GPU's own memory (128-byte
+//     swizzle, no multicast), a ring of stages handed back and forth through mbarriers;
+//   - one elected thread issues the MMAs; the accumulator (128 pixels x BN output channels) lives in
+//     tensor memory and is read back with tcgen05.ld for the epilogue, which subtracts the bias and
+//     stores y in the layout of the input (NCHW or channels-last).
+// Three launches: weights (W' hi / lo, bias), codes (packed bit string -> bf16, channels-last matrix
+// [pixels, C]: for an NCHW tensor a tiled transpose), contraction.  Every wait on an mbarrier is
+// bounded; a wait that runs out records GRANQ_ERR_TIMEOUT in the workspace's status word, the CTA
+// skips its remaining work, frees its tensor memory and returns.
+#include "../../include/granq.h"
+
+#include "granq_internal.h"
+
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include <algorithm>
+
+namespace granq {
+
+namespace {
+
+constexpr int kABm = 128;                 // pixels per tile (rows of the accumulator = tensor-memory lanes)
+constexpr int kABk = 64;                  // channels per stage: 64 bf16 = one 128-byte swizzle row
+constexpr int kAStages = 4;
+constexpr int kAThreads = 128;            // warp 0: TMA producer, warp 1: MMA issuer; all four: epilogue
+constexpr uint32_t kASpin = 1u << 22;     // bounded mbarrier wait
+constexpr uint32_t kATimeout = 5;         // GRANQ_ERR_TIMEOUT
+
+__device__ __forceinline__ uint32_t a_smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void a_mbar_init(uint64_t* bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(a_smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void a_mbar_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(a_smem_u32(bar)), "r"(bytes)
+                 : "memory");
+}
+__device__ __forceinline__ bool a_mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(a_smem_u32(bar)), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// 2-d tile load of this GPU's own memory (no multicast): coordinates (x = innermost element, y = row)
+__device__ __forceinline__ void a_tma_load_2d(void* dst_smem, const CUtensorMap* map, int x, int y, uint64_t* bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::
+            "r"(a_smem_u32(dst_smem)),
+        "l"(map), "r"(a_smem_u32(bar)), "r"(x), "r"(y)
+        : "memory");
+}
+// K-major operand tile in shared memory, 128-byte swizzle: rows of 64 bf16, groups of 8 rows 1024 bytes apart
+__device__ __forceinline__ uint64_t a_smem_desc(const void* tile) {
+    uint64_t d = 0;
+    d |= (uint64_t)((a_smem_u32(tile) >> 4) & 0x3FFF);      // start address, 16-byte units
+    d |= (uint64_t)1 << 16;                                  // leading byte offset (unused with a swizzle)
+    d |= (uint64_t)(1024 >> 4) << 32;                        // stride byte offset: next group of 8 rows
+    d |= (uint64_t)1 << 46;                                  // descriptor version of this architecture
+    d |= (uint64_t)2 << 61;                                  // 128-byte swizzle
+    return d;
+}
+// bf16 x bf16 -> fp32, both operands K-major, M = 128, N = n
+__device__ __forceinline__ uint32_t a_instr_desc(uint32_t n) {
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((n >> 3) << 17) | ((uint32_t)(kABm >> 4) << 24);
+}
+__device__ __forceinline__ void a_mma(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}" ::"r"(d_tmem),
+        "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// the mbarrier gets one arrival when every MMA issued so far by this thread has completed
+__device__ __forceinline__ void a_commit(uint64_t* bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(a_smem_u32(bar))
+                 : "memory");
+}
+
+struct AArgs {
+    float* y;
+    const float* bias;
+    uint32_t* status;
+    int64_t rows;          // pixels of the whole batch
+    int64_t P;             // pixels of one sample
+    int64_t O;             // output channels
+    int kblocks;           // ceil(C / 64)
+    int channels_last;     // layout of y
+    uint32_t spin_limit;
+};
+
+// D[128 pixels x BN] = codes[128 x C] * (hi + lo)[BN x C]^T in tensor memory; y = D - bias
+template <int BN>
+__global__ void __launch_bounds__(kAThreads, 1)
+accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_hi,
+                  const __grid_constant__ CUtensorMap map_lo, const AArgs a) {
+    constexpr uint32_t kABytes = kABm * kABk * 2, kBBytes = BN * kABk * 2, kStageBytes = kABytes + 2 * kBBytes;
+    extern __shared__ __align__(1024) unsigned char a_smem[];
+    __shared__ __align__(8) uint64_t s_full[kAStages], s_empty[kAStages], s_done;
+    __shared__ uint32_t s_tmem, s_abort;
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    // 1024-byte aligned stage buffers (the swizzle pattern is a function of the address)
+    unsigned char* stages = a_smem + ((1024u - (a_smem_u32(a_smem) & 1023u)) & 1023u);
+    const int row0 = (int)blockIdx.x * kABm, col0 = (int)blockIdx.y * BN;
+
+    if (tid == 0) {
+        for (int s = 0; s < kAStages; ++s) {
+            a_mbar_init(&s_full[s], 1);
+            a_mbar_init(&s_empty[s], 1);
+        }
+        a_mbar_init(&s_done, 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {       // BN columns of tensor memory for the accumulator (a power of two >= 32)
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(a_smem_u32(&s_tmem)),
+                     "r"((uint32_t)BN)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s_tmem;
+
+    // bounded wait; false when it ran out or another role of this CTA has given up
+    auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+        for (uint32_t i = 0; i < a.spin_limit; ++i) {
+            if (a_mbar_try_wait(bar, parity)) return true;
+            if ((i & 1023u) == 1023u && *(volatile uint32_t*)&s_abort) return false;
+        }
+        atomicExch(a.status, kATimeout);
+        *(volatile uint32_t*)&s_abort = 1;
+        return false;
+    };
+
+    if (warp == 0 && lane == 0) {
+        // ---- producer: one stage = 128 x 64 codes + BN x 64 of each weight half ----
+        for (int kb = 0; kb < a.kblocks; ++kb) {
+            const int s = kb % kAStages;
+            if (kb >= kAStages && !wait(&s_empty[s], (uint32_t)((kb / kAStages - 1) & 1))) break;
+            unsigned char* st = stages + (size_t)s * kStageBytes;
+            a_mbar_expect_tx(&s_full[s], kStageBytes);
+            a_tma_load_2d(st, &map_q, kb * kABk, row0, &s_full[s]);
+            a_tma_load_2d(st + kABytes, &map_hi, kb * kABk, col0, &s_full[s]);
+            a_tma_load_2d(st + kABytes + kBBytes, &map_lo, kb * kABk, col0, &s_full[s]);
+        }
+    } else if (warp == 1 && lane == 0) {
+        // ---- MMA issuer: per stage 4 K steps of 16, each against the hi and the lo half of the weights ----
+        const uint32_t idesc = a_instr_desc(BN);
+        bool ok = true;
+        for (int kb = 0; kb < a.kblocks && ok; ++kb) {
+            const int s = kb % kAStages;
+            ok = wait(&s_full[s], (uint32_t)((kb / kAStages) & 1));
+            if (!ok) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            unsigned char* st = stages + (size_t)s * kStageBytes;
+            const uint64_t dq = a_smem_desc(st), dh = a_smem_desc(st + kABytes), dl = a_smem_desc(st + kABytes + kBBytes);
+#pragma unroll
+            for (int k = 0; k < kABk / 16; ++k) {        // 16 bf16 = 32 bytes = 2 sixteen-byte units along K
+                a_mma(tmem, dq + 2 * k, dh + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                a_mma(tmem, dq + 2 * k, dl + 2 * k, idesc, 1u);
+            }
+            a_commit(&s_empty[s]);       // the stage may be refilled once these MMAs have read it
+        }
+        a_commit(&s_done);               // arrives when every MMA has completed: the accumulator is final
+    }
+    __syncwarp();
+
+    // ---- epilogue: warp w reads lanes 32 w .. 32 w + 31 of the accumulator, 32 columns at a time ----
+    const bool done = wait(&s_done, 0);
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const int64_t gp = (int64_t)row0 + warp * 32 + lane;      // this thread's pixel, over the whole batch
+    const int64_t n = gp / a.P, p = gp - n * a.P;
+#pragma unroll 1
+    for (int c = 0; c < BN; c += 32) {
+        uint32_t v[32];
+        const uint32_t taddr = tmem + ((warp * 32u) << 16) + (uint32_t)c;
+        asm volatile(
+            "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+            "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,"
+            "%30,%31}, [%32];"
+            : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+              "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]), "=r"(v[16]),
+              "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]), "=r"(v[24]),
+              "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+            : "r"(taddr)
+            : "memory");
+        asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+        if (done && gp < a.rows) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+                const int64_t o = (int64_t)col0 + c + j;
+                if (o < a.O) {
+                    const float val = __fsub_rn(__uint_as_float(v[j]), __ldg(a.bias + o));
+                    if (a.channels_last) a.y[gp * a.O + o] = val;
+                    else a.y[(n * a.O + o) * a.P + p] = val;
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 1)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
+}
+
+// W' = w * s in fp32, split into hi + lo (bf16 each), rows padded with zeros to Cpad; one CTA per output channel.
+// bias[o] = sum_c (hi + lo)[o][c] * z_c in fp64 (the matrix that is really multiplied), rounded once to fp32.
+__global__ void accumulate_weights_kernel(const float* __restrict__ w, const float* __restrict__ s,
+                                          const float* __restrict__ z, int C, int Cpad, __nv_bfloat16* hi,
+                                          __nv_bfloat16* lo, float* bias) {
+    const int o = blockIdx.x;
+    double acc = 0.0;
+    for (int c = threadIdx.x; c < Cpad; c += blockDim.x) {
+        float h = 0.0f, l = 0.0f;
+        if (c < C) {
+            const float wp = __fmul_rn(w[(size_t)o * C + c], s[c]);
+            const __nv_bfloat16 hb = __float2bfloat16_rn(wp);
+            h = __bfloat162float(hb);
+            const __nv_bfloat16 lb = __float2bfloat16_rn(__fsub_rn(wp, h));
+            l = __bfloat162float(lb);
+            acc += ((double)h + (double)l) * (double)z[c];
+            hi[(size_t)o * Cpad + c] = hb;
+            lo[(size_t)o * Cpad + c] = lb;
+        } else {
+            hi[(size_t)o * Cpad + c] = __float2bfloat16_rn(0.0f);
+            lo[(size_t)o * Cpad + c] = __float2bfloat16_rn(0.0f);
+        }
+    }
+    __shared__ double red[32];
+    for (int d = 16; d > 0; d >>= 1) acc += __shfl_xor_sync(0xFFFFFFFFu, acc, d);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = acc;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t = 0.0;
+        for (int i = 0; i < (int)(blockDim.x + 31) / 32; ++i) t += red[i];
+        bias[o] = (float)t;
+    }
+}
+
+// code e of a bit string of b-bit codes (element e in bits [e*b, (e+1)*b), little-endian words)
+__device__ __forceinline__ uint32_t a_code_at(const uint32_t* __restrict__ packed, int64_t e, int bits) {
+    const int64_t bit = e * bits;
+    const int64_t word = bit >> 5;
+    const int sh = (int)(bit & 31);
+    uint32_t v = __ldg(packed + word) >> sh;
+    if (sh + bits > 32) v |= __ldg(packed + word + 1) << (32 - sh);
+    return v & ((1u << bits) - 1u);
+}
+
+// NCHW codes -> bf16 matrix [N * P, Cpad] (channels-last): 32 x 32 tiles transposed through shared memory
+__global__ void accumulate_codes_nchw_kernel(const uint32_t* __restrict__ packed, int bits, int64_t C, int64_t P,
+                                             int64_t Cpad, __nv_bfloat16* __restrict__ q) {
+    __shared__ uint8_t tile[32][33];
+    const int64_t n = blockIdx.z, c0 = (int64_t)blockIdx.y * 32, p0 = (int64_t)blockIdx.x * 32;
+    for (int cc = threadIdx.y; cc < 32; cc += blockDim.y) {
+        const int64_t c = c0 + cc, p = p0 + threadIdx.x;
+        tile[cc][threadIdx.x] = (c < C && p < P) ? (uint8_t)a_code_at(packed, (n * C + c) * P + p, bits) : (uint8_t)0;
+    }
+    __syncthreads();
+    for (int pp = threadIdx.y; pp < 32; pp += blockDim.y) {
+        const int64_t p = p0 + pp, c = c0 + threadIdx.x;
+        if (p < P && c < Cpad) q[(n * P + p) * Cpad + c] = __float2bfloat16_rn((float)tile[threadIdx.x][pp]);
+    }
+}
+
+// channels-last codes -> bf16 matrix [rows, Cpad]
+__global__ void accumulate_codes_nhwc_kernel(const uint32_t* __restrict__ packed, int bits, int64_t rows, int64_t C,
+                                             int64_t Cpad, __nv_bfloat16* __restrict__ q) {
+    const int64_t total = rows * Cpad;
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t r = i / Cpad, c = i - r * Cpad;
+        q[i] = __float2bfloat16_rn(c < C ? (float)a_code_at(packed, r * C + c, bits) : 0.0f);
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// bf16 matrix [rows, cols] (cols contiguous) cut into boxes of 64 columns x box_rows rows, 128-byte swizzle;
+// columns and rows beyond the matrix read as zero
+bool a_make_map(EncodeTiledFn encode, CUtensorMap* map, const void* base, uint64_t rows, uint64_t cols,
+                uint32_t box_rows) {
+    const cuuint64_t dims[2] = {cols, rows};
+    const cuuint64_t strides[1] = {cols * 2};
+    const cuuint32_t box[2] = {(cuuint32_t)kABk, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+struct ALayout {
+    int64_t N, C, P, Cpad, rows;
+    size_t off_q, off_hi, off_lo, off_bias, total;
+};
+
+bool a_layout(const int64_t dims[4], int channel_axis, int64_t O, ALayout& L) {
+    if (!dims || (channel_axis != 1 && channel_axis != 3) || O <= 0 || O >= (1ll << 24)) return false;
+    for (int d = 0; d < 4; ++d)
+        if (dims[d] <= 0 || dims[d] >= (1ll << 31)) return false;
+    L.N = dims[0];
+    L.C = channel_axis == 1 ? dims[1] : dims[3];
+    L.P = channel_axis == 1 ? dims[2] * dims[3] : dims[1] * dims[2];
+    if (L.C >= (1ll << 20) || L.P >= (1ll << 31) || L.N * L.P >= (1ll << 31)) return false;
+    L.Cpad = (L.C + 7) & ~7ll;                 // rows of 16-byte multiples for the tile loads
+    L.rows = L.N * L.P;
+    auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
+    L.off_q = 256;
+    L.off_hi = L.off_q + up((size_t)L.rows * L.Cpad * 2);
+    L.off_lo = L.off_hi + up((size_t)O * L.Cpad * 2);
+    L.off_bias = L.off_lo + up((size_t)O * L.Cpad * 2);
+    L.total = L.off_bias + up((size_t)O * 4);
+    return true;
+}
+
+template <int BN>
+cudaError_t a_launch(const CUtensorMap& mq, const CUtensorMap& mh, const CUtensorMap& ml, const AArgs& args,
+                     cudaStream_t st) {
+    const size_t smem = (size_t)kAStages * (kABm * kABk * 2 + 2 * BN * kABk * 2) + 1024;
+    auto kern = accumulate_kernel<BN>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    const dim3 grid((unsigned)((args.rows + kABm - 1) / kABm), (unsigned)((args.O + BN - 1) / BN));
+    kern<<<grid, kAThreads, smem, st>>>(mq, mh, ml, args);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+}  // namespace granq
+
+using namespace granq;
+
+extern "C" size_t granq_accumulate_workspace_bytes(const int64_t dims[4], int channel_axis, int64_t out_channels) {
+    ALayout L;
+    if (!a_layout(dims, channel_axis, out_channels, L)) return 0;
+    return L.total;
+}
+
+extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_t dims[4], int channel_axis, int bits,
+                                      const float* scale, const float* zp, const float* weights, int64_t out_channels,
+                                      float* y, void* workspace, size_t workspace_bytes, uint32_t flags,
+                                      void* cuda_stream) {
+    (void)flags;
+    ALayout L;
+    if (!packed_codes || !scale || !zp || !weights || !y || bits < 1 || bits > 8 || ((uintptr_t)packed_codes & 3) ||
+        !a_layout(dims, channel_axis, out_channels, L))
+        return GRANQ_ERR_INVALID_ARG;
+    if (!workspace || ((uintptr_t)workspace & 255) || workspace_bytes < L.total) return GRANQ_ERR_WORKSPACE;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    // the tile-load descriptors are made by the driver: look its encoder up (no link-time dependency on the driver)
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess || !fn ||
+        qres != cudaDriverEntryPointSuccess)
+        return GRANQ_ERR_CUDA;
+    EncodeTiledFn encode = (EncodeTiledFn)fn;
+    char* ws = (char*)workspace;
+    __nv_bfloat16* q = (__nv_bfloat16*)(ws + L.off_q);
+    __nv_bfloat16* hi = (__nv_bfloat16*)(ws + L.off_hi);
+    __nv_bfloat16* lo = (__nv_bfloat16*)(ws + L.off_lo);
+    float* bias = (float*)(ws + L.off_bias);
+    const int BN = out_channels <= 64 ? 64 : 128;
+    CUtensorMap mq, mh, ml;
+    if (!a_make_map(encode, &mq, q, (uint64_t)L.rows, (uint64_t)L.Cpad, kABm) ||
+        !a_make_map(encode, &mh, hi, (uint64_t)out_channels, (uint64_t)L.Cpad, (uint32_t)BN) ||
+        !a_make_map(encode, &ml, lo, (uint64_t)out_channels, (uint64_t)L.Cpad, (uint32_t)BN))
+        return GRANQ_ERR_CUDA;
+
+    cudaError_t e = cudaMemsetAsync(workspace, 0, sizeof(uint32_t), st);       // the status word
+    if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+    accumulate_weights_kernel<<<(unsigned)out_channels, 128, 0, st>>>(weights, scale, zp, (int)L.C, (int)L.Cpad, hi, lo,
+                                                                    bias);
+    if (channel_axis == 1) {
+        const dim3 grid((unsigned)((L.P + 31) / 32), (unsigned)((L.Cpad + 31) / 32), (unsigned)L.N);
+        if (grid.y > 65535 || grid.z > 65535) return GRANQ_ERR_UNSUPPORTED;
+        accumulate_codes_nchw_kernel<<<grid, dim3(32, 8), 0, st>>>(packed_codes, bits, L.C, L.P, L.Cpad, q);
+    } else {
+        const int64_t total = L.rows * L.Cpad;
+        const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 16);
+        accumulate_codes_nhwc_kernel<<<blocks, 256, 0, st>>>(packed_codes, bits, L.rows, L.C, L.Cpad, q);
+    }
+    if (cudaGetLastError() != cudaSuccess) return GRANQ_ERR_CUDA;
+    AArgs args{};
+    args.y = y;
+    args.bias = bias;
+    args.status = (uint32_t*)workspace;
+    args.rows = L.rows;
+    args.P = L.P;
+    args.O = out_channels;
+    args.kblocks = (int)((L.Cpad + kABk - 1) / kABk);
+    args.channels_last = channel_axis == 3 ? 1 : 0;
+    args.spin_limit = kASpin;
+    e = BN == 64 ? a_launch<64>(mq, mh, ml, args, st) : a_launch<128>(mq, mh, ml, args, st);
+    return e == cudaSuccess ? GRANQ_OK : GRANQ_ERR_CUDA;
+}
