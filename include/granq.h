@@ -173,8 +173,11 @@ int granq_fakequant_bwd(const void* gy, const void* x, int dtype, const int64_t 
 /*
  * The whole path in one call (Algorithm 1, range step through pre-scale step, plus the
  * backward): range of x itself -> scale / zero-point -> y, and gx when gy_opt is given.
- * The default plan processes the tensor in waves of channel groups that stay in the L2 cache
- * between the range pass and the quantize pass, so x is read from HBM (about) once.
+ * The default plan stages a run of adjacent channels once in the shared memory of one thread-block
+ * cluster where their group fits (x is then read from HBM exactly once); larger groups are processed
+ * in waves of channel groups that stay in the L2 cache between the range pass and the quantize pass, so
+ * x is read from HBM (about) once; channels-last geometries (channel_axis = 3, or planes of one element)
+ * take a range launch and a quantize launch with one 16-byte unit column per thread.
  *   x                 in   E elements          gy_opt   in   E elements or NULL (forward only)
  *   y                 out  E elements          gx_opt   out  E elements (required iff gy_opt)
  *   min_out, max_out  out  G floats each (required)
@@ -361,7 +364,8 @@ int granq_host_arena_status(int dtype, const int64_t dims[4], int channel_axis, 
 /*
  * Plan that granq_fakequant_fused() would take for this geometry and flags on the current
  * device: 0 = two-pass, 1 = naive per-channel loop, 2 = on-chip staged, 3 = L2-resident waves,
- * 4 = column walk, 5 = cluster-local; negative = -status.
+ * 4 = column walk, 5 = cluster-local, 6 = channels-last rows (range launch + quantize launch with one
+ * 16-byte unit column per thread); negative = -status.
  * `launches_out` (HOST, may be NULL) receives the number of kernel launches of that plan.
  */
 int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int group, int with_backward,

@@ -22,7 +22,7 @@ FLAG_FORCE_TWO_PASS, FLAG_FORCE_NAIVE, FLAG_FORCE_STAGED, FLAG_FORCE_L2WAVE, FLA
 FLAG_WORKSPACE_ZEROED = 32
 FLAG_HOST_ASYNC = 64
 FLAG_FORCE_CLUSTER = 128
-PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED, PLAN_L2WAVE, PLAN_COLWALK, PLAN_CLUSTER = 0, 1, 2, 3, 4, 5
+PLAN_TWO_PASS, PLAN_NAIVE, PLAN_STAGED, PLAN_L2WAVE, PLAN_COLWALK, PLAN_CLUSTER, PLAN_ROWS = 0, 1, 2, 3, 4, 5, 6
 (KNOB_STAGED_DEPTH, KNOB_STAGED_MAX_BUF_UNITS, KNOB_STAGED_GRID, KNOB_SPIN_LIMIT, KNOB_TEST_EXTRA_ARRIVALS,
  KNOB_STAGED_CTAS_PER_SM, KNOB_L2_WAVE_KB, KNOB_L2_UPL, KNOB_L2_CTAS_PER_SM, KNOB_L2_LAG,
  KNOB_CLUSTER_TILE_KB, KNOB_CLUSTER_CTAS, KNOB_CLUSTER_THREADS, KNOB_CLUSTER_LOAD, KNOB_CLUSTER_PREFETCH,

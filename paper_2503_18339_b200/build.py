@@ -12,7 +12,7 @@ INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libgranq.so")
 OBJ_DIR = os.path.join(HERE, "_build")
 SOURCES = ["granq_api.cu", "granq_flat.cu", "granq_staged.cu", "granq_l2wave.cu", "granq_colwalk.cu",
-           "granq_cluster.cu", "granq_accumulate.cu", "granq_weights.cu", "granq_selftest.cu", "granq_noalloc.cu"]
+           "granq_cluster.cu", "granq_accumulate.cu", "granq_rows.cu", "granq_weights.cu", "granq_selftest.cu", "granq_noalloc.cu"]
 HEADERS = ["granq_device.cuh", "granq_internal.h"]
 NVCC_FLAGS = ["-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC"]

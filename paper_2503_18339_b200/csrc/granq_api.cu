@@ -30,7 +30,7 @@ int check_workspace(const void* ws, size_t bytes, int64_t G) {
 
 int cuda_status(cudaError_t e) { return e == cudaSuccess ? GRANQ_OK : GRANQ_ERR_CUDA; }
 
-enum { PLAN_TWO_PASS = 0, PLAN_NAIVE = 1, PLAN_STAGED = 2, PLAN_L2WAVE = 3, PLAN_COLWALK = 4, PLAN_CLUSTER = 5 };
+enum { PLAN_TWO_PASS = 0, PLAN_NAIVE = 1, PLAN_STAGED = 2, PLAN_L2WAVE = 3, PLAN_COLWALK = 4, PLAN_CLUSTER = 5, PLAN_ROWS = 6 };
 
 // plan of the fused entry point; `plan_out` is filled when the staged plan is taken
 int choose_plan(int dtype, const Geom& g, const QuantIO& io, bool backward, uint32_t flags, StagedPlan* plan_out,
@@ -63,6 +63,9 @@ int choose_plan(int dtype, const Geom& g, const QuantIO& io, bool backward, uint
         if (plan_out) *plan_out = p;
         return PLAN_STAGED;
     }
+    // channels-last geometries (the channel is the innermost axis) have plans of their own: the cluster-local
+    // kernel cannot stage them (a run of channels is a few bytes per row) and there are no planes to walk
+    if (g.inner == 1 && plan_rows(dtype, g, io)) return PLAN_ROWS;
     // default: the cluster-local kernel where a run of channels fits the shared memory of one cluster
     // (x is then read once and nothing waits on the grid), else the column-walk kernel where there are
     // slabs to walk, else the L2-resident-wave kernel
@@ -213,6 +216,8 @@ int granq_fakequant_fused(const void* x, const void* gy_opt, int dtype, const in
     if (e != cudaSuccess) return GRANQ_ERR_CUDA;
     if (plan == PLAN_CLUSTER) {
         e = launch_cluster(kp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
+    } else if (plan == PLAN_ROWS) {
+        e = launch_rows(io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, st);
     } else if (plan == PLAN_STAGED) {
         e = launch_staged(sp, io, mode, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt, g_tune, st);
     } else if (plan == PLAN_L2WAVE) {
@@ -501,6 +506,7 @@ int granq_fused_plan(int dtype, const int64_t dims[4], int channel_axis, int gro
     const int plan = choose_plan(dtype, g, io, with_backward != 0, flags, nullptr, nullptr, nullptr, nullptr);
     if (launches_out) {
         if (plan == PLAN_STAGED || plan == PLAN_L2WAVE || plan == PLAN_COLWALK || plan == PLAN_CLUSTER) *launches_out = 1;
+        else if (plan == PLAN_ROWS) *launches_out = 2;
         else if (plan == PLAN_NAIVE) *launches_out = (int)(3 * g.C);
         else if (plan == PLAN_TWO_PASS) *launches_out = 3;
     }

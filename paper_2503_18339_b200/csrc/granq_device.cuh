@@ -311,6 +311,48 @@ __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& 
     }
 }
 
+// Quantize one pack whose V elements belong to V different groups (channels-last rows), the range being the
+// tensor's own: element i takes the parameters g[i].  Same arithmetic and shortcut as quantize_pack().
+template <typename T, bool BWD, bool EXTRAS>
+__device__ __forceinline__ void quantize_pack_each(const Pack<T>& px, const Pack<T>& pg,
+                                                   const GroupParam (&g)[Pack<T>::V], float qmax, Pack<T>& py,
+                                                   Pack<T>& pgx, uint32_t (&cb)[Pack<T>::V / 4],
+                                                   uint32_t (&mb)[Pack<T>::V / 4]) {
+    constexpr int V = Pack<T>::V;
+    const float kMagic = 12582912.0f;  // 1.5 * 2^23
+#pragma unroll
+    for (int i = 0; i < V / 4; ++i) {
+        cb[i] = 0;
+        mb[i] = 0;
+    }
+#pragma unroll
+    for (int i = 0; i < V; ++i) {
+        const float s = g[i].s, z = g[i].z, rc = g[i].r, x = px.get(i);
+        float r;
+        if (rc != 0.0f) {
+            const float up = __fmaf_rn(x, rc, z);
+            r = __fsub_rn(__fadd_rn(up, kMagic), kMagic);
+            if (!(fabsf(__fsub_rn(up, r)) < tie_threshold(z))) {     // rare: too close to a tie for the shortcut
+                const float u = __fadd_rn(div_by_scale(x, s, rc), z);
+                const float uc = fminf(fmaxf(u, -1.0f), __fadd_rn(qmax, 1.0f));
+                r = __fsub_rn(__fadd_rn(uc, kMagic), kMagic);
+            }
+        } else {
+            const float u = __fadd_rn(__fdiv_rn(x, s), z);
+            const float uc = fminf(fmaxf(u, -1.0f), __fadd_rn(qmax, 1.0f));
+            r = __fsub_rn(__fadd_rn(uc, kMagic), kMagic);
+        }
+        const float q = fminf(fmaxf(r, 0.0f), qmax);
+        const bool in = (r == q);
+        py.set(i, __fmul_rn(s, __fsub_rn(q, z)));
+        if constexpr (BWD) pgx.set(i, in ? pg.get(i) : 0.0f);
+        if constexpr (EXTRAS) {
+            cb[i / 4] |= (uint32_t)q << (8 * (i % 4));
+            mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
+        }
+    }
+}
+
 // per-lane min / max of elements [first, last) of one pack
 template <typename T>
 __device__ __forceinline__ void pack_minmax(const Pack<T>& p, int first, int last, float& mn, float& mx) {

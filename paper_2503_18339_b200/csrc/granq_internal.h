@@ -174,6 +174,11 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
                            const Workspace& ws, float* lo, float* hi, float* s_opt, float* z_opt,
                            const StagedTuning& tune, cudaStream_t st);
 
+// ---- channels-last kernels (the channel is the innermost axis: one 16-byte unit holds V channels of a row) ----
+bool plan_rows(int dtype, const Geom& g, const QuantIO& io);
+cudaError_t launch_rows(const QuantIO& io, int mode, int dtype, const Geom& g, int bits, const Workspace& ws,
+                        float* lo, float* hi, float* s_opt, float* z_opt, cudaStream_t st);
+
 // ---- cluster-local kernel (a run of channels staged once in the shared memory of one cluster) ----
 struct ClusterPlan {
     bool ok;
