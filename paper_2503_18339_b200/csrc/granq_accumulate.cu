@@ -33,7 +33,7 @@ namespace {
 
 constexpr int kABm = 128;                 // pixels per tile (rows of the accumulator = tensor-memory lanes)
 constexpr int kABk = 64;                  // channels per stage: 64 bf16 = one 128-byte swizzle row
-constexpr int kAStages = 4;
+constexpr int kAMaxStages = 4;         // the ring is as deep as the K blocks need, at most this
 constexpr int kAThreads = 128;            // warp 0: TMA producer, warp 1: MMA issuer; all four: epilogue
 constexpr uint32_t kASpin = 1u << 22;     // bounded mbarrier wait
 constexpr uint32_t kATimeout = 5;         // GRANQ_ERR_TIMEOUT
@@ -102,17 +102,18 @@ struct AArgs {
     int64_t O;             // output channels
     int kblocks;           // ceil(C / 64)
     int channels_last;     // layout of y
+    int stages;            // depth of the ring of operand stages
     uint32_t spin_limit;
 };
 
 // D[128 pixels x BN] = codes[128 x C] * (hi + lo)[BN x C]^T in tensor memory; y = D - bias
 template <int BN>
-__global__ void __launch_bounds__(kAThreads, 1)
+__global__ void __launch_bounds__(kAThreads, BN == 64 ? 6 : 4)
 accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_hi,
                   const __grid_constant__ CUtensorMap map_lo, const AArgs a) {
     constexpr uint32_t kABytes = kABm * kABk * 2, kBBytes = BN * kABk * 2, kStageBytes = kABytes + 2 * kBBytes;
     extern __shared__ __align__(1024) unsigned char a_smem[];
-    __shared__ __align__(8) uint64_t s_full[kAStages], s_empty[kAStages], s_done;
+    __shared__ __align__(8) uint64_t s_full[kAMaxStages], s_empty[kAMaxStages], s_done;
     __shared__ uint32_t s_tmem, s_abort;
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // 1024-byte aligned stage buffers (the swizzle pattern is a function of the address)
@@ -120,7 +121,7 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const int row0 = (int)blockIdx.x * kABm, col0 = (int)blockIdx.y * BN;
 
     if (tid == 0) {
-        for (int s = 0; s < kAStages; ++s) {
+        for (int s = 0; s < kAMaxStages; ++s) {
             a_mbar_init(&s_full[s], 1);
             a_mbar_init(&s_empty[s], 1);
         }
@@ -154,8 +155,8 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     if (warp == 0 && lane == 0) {
         // ---- producer: one stage = 128 x 64 codes + BN x 64 of each weight half ----
         for (int kb = 0; kb < a.kblocks; ++kb) {
-            const int s = kb % kAStages;
-            if (kb >= kAStages && !wait(&s_empty[s], (uint32_t)((kb / kAStages - 1) & 1))) break;
+            const int s = kb % a.stages;
+            if (kb >= a.stages && !wait(&s_empty[s], (uint32_t)((kb / a.stages - 1) & 1))) break;
             unsigned char* st = stages + (size_t)s * kStageBytes;
             a_mbar_expect_tx(&s_full[s], kStageBytes);
             a_tma_load_2d(st, &map_q, kb * kABk, row0, &s_full[s]);
@@ -167,8 +168,8 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const uint32_t idesc = a_instr_desc(BN);
         bool ok = true;
         for (int kb = 0; kb < a.kblocks && ok; ++kb) {
-            const int s = kb % kAStages;
-            ok = wait(&s_full[s], (uint32_t)((kb / kAStages) & 1));
+            const int s = kb % a.stages;
+            ok = wait(&s_full[s], (uint32_t)((kb / a.stages) & 1));
             if (!ok) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
             unsigned char* st = stages + (size_t)s * kStageBytes;
@@ -266,19 +267,40 @@ __device__ __forceinline__ uint32_t a_code_at(const uint32_t* __restrict__ packe
     return v & ((1u << bits) - 1u);
 }
 
-// NCHW codes -> bf16 matrix [N * P, Cpad] (channels-last): 32 x 32 tiles transposed through shared memory
-__global__ void accumulate_codes_nchw_kernel(const uint32_t* __restrict__ packed, int bits, int64_t C, int64_t P,
-                                             int64_t Cpad, __nv_bfloat16* __restrict__ q) {
-    __shared__ uint8_t tile[32][33];
-    const int64_t n = blockIdx.z, c0 = (int64_t)blockIdx.y * 32, p0 = (int64_t)blockIdx.x * 32;
-    for (int cc = threadIdx.y; cc < 32; cc += blockDim.y) {
-        const int64_t c = c0 + cc, p = p0 + threadIdx.x;
-        tile[cc][threadIdx.x] = (c < C && p < P) ? (uint8_t)a_code_at(packed, (n * C + c) * P + p, bits) : (uint8_t)0;
+// NCHW codes -> bf16 matrix [N * P, Cpad] (channels-last): tiles of 32 channels x 256 pixels transposed through
+// shared memory; a thread extracts 32 codes, then writes 4 times 8 channels of one pixel as one 16-byte store
+constexpr int kUPix = 256;
+__global__ void __launch_bounds__(256) accumulate_codes_nchw_kernel(const uint32_t* __restrict__ packed, int bits,
+                                                                    int64_t C, int64_t P, int64_t Cpad,
+                                                                    __nv_bfloat16* __restrict__ q) {
+    __shared__ uint8_t tile[32][kUPix + 4];
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int64_t n = blockIdx.z, c0 = (int64_t)blockIdx.y * 32, p0 = (int64_t)blockIdx.x * kUPix;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int cc = ty + 8 * i;
+        const int64_t c = c0 + cc;
+#pragma unroll
+        for (int j = 0; j < kUPix / 32; ++j) {
+            const int64_t p = p0 + j * 32 + tx;
+            tile[cc][j * 32 + tx] = (c < C && p < P) ? (uint8_t)a_code_at(packed, (n * C + c) * P + p, bits) : (uint8_t)0;
+        }
     }
     __syncthreads();
-    for (int pp = threadIdx.y; pp < 32; pp += blockDim.y) {
-        const int64_t p = p0 + pp, c = c0 + threadIdx.x;
-        if (p < P && c < Cpad) q[(n * P + p) * Cpad + c] = __float2bfloat16_rn((float)tile[threadIdx.x][pp]);
+    // 256 pixels x 4 groups of 8 channels = 1024 stores of 16 bytes, 4 per thread; the 4 groups of a pixel are 64
+    // contiguous bytes of its row
+    for (int k = threadIdx.x; k < kUPix * 4; k += 256) {
+        const int pp = k >> 2, g8 = (k & 3) * 8;
+        const int64_t p = p0 + pp, c = c0 + g8;
+        if (p >= P || c >= Cpad) continue;
+        uint32_t w[4];
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {
+            const uint32_t lo = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn((float)tile[g8 + 2 * h][pp]));
+            const uint32_t hi = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn((float)tile[g8 + 2 * h + 1][pp]));
+            w[h] = lo | (hi << 16);
+        }
+        *reinterpret_cast<uint4*>(q + (n * P + p) * Cpad + c) = make_uint4(w[0], w[1], w[2], w[3]);
     }
 }
 
@@ -336,7 +358,8 @@ bool a_layout(const int64_t dims[4], int channel_axis, int64_t O, ALayout& L) {
 template <int BN>
 cudaError_t a_launch(const CUtensorMap& mq, const CUtensorMap& mh, const CUtensorMap& ml, const AArgs& args,
                      cudaStream_t st) {
-    const size_t smem = (size_t)kAStages * (kABm * kABk * 2 + 2 * BN * kABk * 2) + 1024;
+    // a short ring leaves room for several CTAs per SM, whose load / multiply / store chains then overlap
+    const size_t smem = (size_t)args.stages * (kABm * kABk * 2 + 2 * BN * kABk * 2) + 1024;
     auto kern = accumulate_kernel<BN>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -392,9 +415,9 @@ extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_
     accumulate_weights_kernel<<<(unsigned)out_channels, 128, 0, st>>>(weights, scale, zp, (int)L.C, (int)L.Cpad, hi, lo,
                                                                     bias);
     if (channel_axis == 1) {
-        const dim3 grid((unsigned)((L.P + 31) / 32), (unsigned)((L.Cpad + 31) / 32), (unsigned)L.N);
+        const dim3 grid((unsigned)((L.P + kUPix - 1) / kUPix), (unsigned)((L.Cpad + 31) / 32), (unsigned)L.N);
         if (grid.y > 65535 || grid.z > 65535) return GRANQ_ERR_UNSUPPORTED;
-        accumulate_codes_nchw_kernel<<<grid, dim3(32, 8), 0, st>>>(packed_codes, bits, L.C, L.P, L.Cpad, q);
+        accumulate_codes_nchw_kernel<<<grid, 256, 0, st>>>(packed_codes, bits, L.C, L.P, L.Cpad, q);
     } else {
         const int64_t total = L.rows * L.Cpad;
         const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 16);
@@ -411,6 +434,7 @@ extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_
     args.kblocks = (int)((L.Cpad + kABk - 1) / kABk);
     args.channels_last = channel_axis == 3 ? 1 : 0;
     args.spin_limit = kASpin;
+    args.stages = std::min(args.kblocks, 2);
     e = BN == 64 ? a_launch<64>(mq, mh, ml, args, st) : a_launch<128>(mq, mh, ml, args, st);
     return e == cudaSuccess ? GRANQ_OK : GRANQ_ERR_CUDA;
 }
