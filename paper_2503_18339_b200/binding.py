@@ -151,6 +151,16 @@ def _check(rc: int, what: str) -> None:
         raise GranqError(rc, what)
 
 
+def _new(shape, dtype, device) -> torch.Tensor:
+    """Every output tensor the binding allocates itself comes from here (tests swap it for an allocator
+    that surrounds each tensor with guard bands)."""
+    return torch.empty(shape, dtype=dtype, device=device)
+
+
+def _new_like(t: torch.Tensor) -> torch.Tensor:
+    return _new(tuple(t.shape), t.dtype, t.device)
+
+
 def _dims(shape):
     if len(shape) != 4:
         raise ValueError("granq tensors are 4-d (NCHW)")
@@ -266,8 +276,8 @@ def granq_range(x: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANN
                 hi: torch.Tensor = None, workspace: torch.Tensor = None, flags: int = 0, stream=None):
     """Per-group (lo, hi) of x: Eq. 4."""
     G = num_groups(x.shape, channel_axis, group)
-    lo = torch.empty(G, dtype=torch.float32, device=x.device) if lo is None else lo
-    hi = torch.empty(G, dtype=torch.float32, device=x.device) if hi is None else hi
+    lo = _new(G, torch.float32, x.device) if lo is None else lo
+    hi = _new(G, torch.float32, x.device) if hi is None else hi
     ws = make_workspace(x, channel_axis, group) if workspace is None else workspace
     _check(lib().granq_range(_dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, _dev(lo, "lo"),
                              _dev(hi, "hi"), _dev(ws, "workspace"), ws.numel(), flags, _stream(stream)),
@@ -289,12 +299,12 @@ def granq_fakequant_fwd(x: torch.Tensor, bits: int, lo: torch.Tensor, hi: torch.
     """Quantize -> clamp -> dequantize with a given per-group range: Eq. 1, 2, 6."""
     G = num_groups(x.shape, channel_axis, group)
     o = FakeQuantOut(lo=lo, hi=hi)
-    o.y = torch.empty_like(x) if y is None else y
+    o.y = _new_like(x) if y is None else y
     if want_codes:
-        o.codes = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+        o.codes = _new(x.shape, torch.uint8, x.device)
     if want_params:
-        o.s = torch.empty(G, dtype=torch.float32, device=x.device)
-        o.z = torch.empty(G, dtype=torch.float32, device=x.device)
+        o.s = _new(G, torch.float32, x.device)
+        o.z = _new(G, torch.float32, x.device)
     _check(lib().granq_fakequant_fwd(_dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, bits,
                                      _dev(lo, "lo"), _dev(hi, "hi"), _dev(o.y, "y"), _dev(o.codes, "codes"),
                                      _dev(o.s, "s"), _dev(o.z, "z"), flags, _stream(stream)),
@@ -309,9 +319,9 @@ def granq_fakequant_bwd(gy: torch.Tensor, x: torch.Tensor, bits: int, lo: torch.
     if gy.shape != x.shape or gy.dtype != x.dtype:
         raise ValueError("gy must match x")
     o = FakeQuantOut(lo=lo, hi=hi)
-    o.gx = torch.empty_like(x) if gx is None else gx
+    o.gx = _new_like(x) if gx is None else gx
     if want_mask:
-        o.mask = torch.empty(x.shape, dtype=torch.uint8, device=x.device)
+        o.mask = _new(x.shape, torch.uint8, x.device)
     _check(lib().granq_fakequant_bwd(_dev(gy, "gy"), _dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group,
                                      bits, _dev(lo, "lo"), _dev(hi, "hi"), _dev(o.gx, "gx"), _dev(o.mask, "mask"),
                                      flags, _stream(stream)),
@@ -334,20 +344,20 @@ def granq_fakequant_fused(x: torch.Tensor, bits: int, gy: torch.Tensor = None, c
     o = out if out is not None else FakeQuantOut()
     dev = x.device
     if o.y is None:
-        o.y = torch.empty_like(x)
+        o.y = _new_like(x)
     if gy is not None and o.gx is None:
-        o.gx = torch.empty_like(x)
+        o.gx = _new_like(x)
     if o.lo is None:
-        o.lo = torch.empty(G, dtype=torch.float32, device=dev)
+        o.lo = _new(G, torch.float32, dev)
     if o.hi is None:
-        o.hi = torch.empty(G, dtype=torch.float32, device=dev)
+        o.hi = _new(G, torch.float32, dev)
     if want_params and o.s is None:
-        o.s = torch.empty(G, dtype=torch.float32, device=dev)
-        o.z = torch.empty(G, dtype=torch.float32, device=dev)
+        o.s = _new(G, torch.float32, dev)
+        o.z = _new(G, torch.float32, dev)
     if want_codes and o.codes is None:
-        o.codes = torch.empty(x.shape, dtype=torch.uint8, device=dev)
+        o.codes = _new(x.shape, torch.uint8, dev)
     if want_mask and gy is not None and o.mask is None:
-        o.mask = torch.empty(x.shape, dtype=torch.uint8, device=dev)
+        o.mask = _new(x.shape, torch.uint8, dev)
     if o.workspace is None:
         o.workspace = make_workspace(x, channel_axis, group)
     _check(lib().granq_fakequant_fused(
@@ -364,7 +374,7 @@ def packmask_bytes(shape) -> int:
 
 def make_packed_mask(x: torch.Tensor) -> torch.Tensor:
     """Buffer for the STE mask of x at one bit per element (int32 words)."""
-    return torch.empty(packmask_bytes(x.shape) // 4, dtype=torch.int32, device=x.device)
+    return _new(packmask_bytes(x.shape) // 4, torch.int32, x.device)
 
 
 def granq_fakequant_fwd_packmask(x: torch.Tensor, bits: int, lo: torch.Tensor, hi: torch.Tensor,
@@ -374,11 +384,11 @@ def granq_fakequant_fwd_packmask(x: torch.Tensor, bits: int, lo: torch.Tensor, h
     """Forward with a given range that also stores the STE mask at one bit per element (Section 2.1)."""
     G = num_groups(x.shape, channel_axis, group)
     o = FakeQuantOut(lo=lo, hi=hi)
-    o.y = torch.empty_like(x) if y is None else y
+    o.y = _new_like(x) if y is None else y
     o.packed_mask = make_packed_mask(x) if packed_mask is None else packed_mask
     if want_params:
-        o.s = torch.empty(G, dtype=torch.float32, device=x.device)
-        o.z = torch.empty(G, dtype=torch.float32, device=x.device)
+        o.s = _new(G, torch.float32, x.device)
+        o.z = _new(G, torch.float32, x.device)
     _check(lib().granq_fakequant_fwd_packmask(_dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, bits,
                                               _dev(lo, "lo"), _dev(hi, "hi"), _dev(o.y, "y"),
                                               _dev(o.packed_mask, "packed_mask"), _dev(o.s, "s"), _dev(o.z, "z"),
@@ -391,7 +401,7 @@ def granq_fakequant_bwd_packmask(gy: torch.Tensor, packed_mask: torch.Tensor, gx
     """STE backward from the packed mask alone: gx = gy where the bit is set, else 0."""
     if packed_mask.numel() * packed_mask.element_size() < packmask_bytes(gy.shape):
         raise ValueError("packed mask too small for gy")
-    gx = torch.empty_like(gy) if gx is None else gx
+    gx = _new_like(gy) if gx is None else gx
     _check(lib().granq_fakequant_bwd_packmask(_dev(gy, "gy"), _dev(packed_mask, "packed_mask"), _dtype(gy),
                                               _dims(gy.shape), _dev(gx, "gx"), flags, _stream(stream)),
            "granq_fakequant_bwd_packmask")
@@ -406,16 +416,16 @@ def granq_fakequant_fused_fwd_packmask(x: torch.Tensor, bits: int, channel_axis:
     o = out if out is not None else FakeQuantOut()
     dev = x.device
     if o.y is None:
-        o.y = torch.empty_like(x)
+        o.y = _new_like(x)
     if o.packed_mask is None:
         o.packed_mask = make_packed_mask(x)
     if o.lo is None:
-        o.lo = torch.empty(G, dtype=torch.float32, device=dev)
+        o.lo = _new(G, torch.float32, dev)
     if o.hi is None:
-        o.hi = torch.empty(G, dtype=torch.float32, device=dev)
+        o.hi = _new(G, torch.float32, dev)
     if want_params and o.s is None:
-        o.s = torch.empty(G, dtype=torch.float32, device=dev)
-        o.z = torch.empty(G, dtype=torch.float32, device=dev)
+        o.s = _new(G, torch.float32, dev)
+        o.z = _new(G, torch.float32, dev)
     if o.workspace is None:
         o.workspace = make_workspace(x, channel_axis, group)
     _check(lib().granq_fakequant_fused_fwd_packmask(
@@ -430,7 +440,7 @@ def granq_distortion(x: torch.Tensor, q: torch.Tensor, sums: torch.Tensor = None
     """[sum x^2, sum q^2, sum x*q, sum (x-q)^2] as 4 doubles on the device (Table 2's raw material)."""
     if q.shape != x.shape or q.dtype != x.dtype:
         raise ValueError("q must match x")
-    sums = torch.empty(4, dtype=torch.float64, device=x.device) if sums is None else sums
+    sums = _new(4, torch.float64, x.device) if sums is None else sums
     _check(lib().granq_distortion(_dev(x, "x"), _dev(q, "q"), _dtype(x), _dims(x.shape), _dev(sums, "sums"), 0,
                                   _stream(stream)), "granq_distortion")
     return sums
@@ -452,16 +462,16 @@ def granq_fakequant_fused_stats(x: torch.Tensor, bits: int, channel_axis: int = 
     o = out if out is not None else FakeQuantOut()
     dev = x.device
     if o.y is None:
-        o.y = torch.empty_like(x)
+        o.y = _new_like(x)
     if o.sums is None:
-        o.sums = torch.empty(4, dtype=torch.float64, device=dev)
+        o.sums = _new(4, torch.float64, dev)
     if o.lo is None:
-        o.lo = torch.empty(G, dtype=torch.float32, device=dev)
+        o.lo = _new(G, torch.float32, dev)
     if o.hi is None:
-        o.hi = torch.empty(G, dtype=torch.float32, device=dev)
+        o.hi = _new(G, torch.float32, dev)
     if want_params and o.s is None:
-        o.s = torch.empty(G, dtype=torch.float32, device=dev)
-        o.z = torch.empty(G, dtype=torch.float32, device=dev)
+        o.s = _new(G, torch.float32, dev)
+        o.z = _new(G, torch.float32, dev)
     if o.workspace is None:
         o.workspace = make_workspace(x, channel_axis, group)
     _check(lib().granq_fakequant_fused_stats(
@@ -490,16 +500,16 @@ class WeightBatch:
             if w.dtype != weights[0].dtype:
                 raise ValueError("all tensors of a batch must have one dtype")
             c = w.shape[0]
-            o = FakeQuantOut(y=torch.empty_like(w), lo=torch.empty(c, dtype=torch.float32, device=w.device),
-                             hi=torch.empty(c, dtype=torch.float32, device=w.device))
+            o = FakeQuantOut(y=_new_like(w), lo=_new(c, torch.float32, w.device),
+                             hi=_new(c, torch.float32, w.device))
             g = None if grads is None else grads[i]
             if g is not None:
                 if g.shape != w.shape or g.dtype != w.dtype:
                     raise ValueError("gradient must match its weight")
-                o.gx = torch.empty_like(w)
+                o.gx = _new_like(w)
             if want_params:
-                o.s = torch.empty(c, dtype=torch.float32, device=w.device)
-                o.z = torch.empty(c, dtype=torch.float32, device=w.device)
+                o.s = _new(c, torch.float32, w.device)
+                o.z = _new(c, torch.float32, w.device)
             self.descs[i] = WeightDesc(_dev(w, "w"), _dev(g, "g"), _dev(o.y, "y"), _dev(o.gx, "gx"),
                                        _dev(o.lo, "lo"), _dev(o.hi, "hi"), _dev(o.s, "s"), _dev(o.z, "z"), c,
                                        w.numel() // max(c, 1), bits[i], 0)
@@ -530,12 +540,12 @@ def granq_quantize_packed(x: torch.Tensor, bits: int, lo: torch.Tensor, hi: torc
     """Eq. 1 + clamp with a given range -> integer codes as a bit string (b bits each), scale, zero-point."""
     G = num_groups(x.shape, channel_axis, group)
     o = FakeQuantOut(lo=lo, hi=hi)
-    o.packed_codes = (torch.empty(packed_codes_bytes(x.shape, bits) // 4, dtype=torch.int32, device=x.device)
+    o.packed_codes = (_new(packed_codes_bytes(x.shape, bits) // 4, torch.int32, x.device)
                       if packed_codes is None else packed_codes)
-    o.s = torch.empty(G, dtype=torch.float32, device=x.device)
-    o.z = torch.empty(G, dtype=torch.float32, device=x.device)
+    o.s = _new(G, torch.float32, x.device)
+    o.z = _new(G, torch.float32, x.device)
     if want_y:
-        o.y = torch.empty_like(x)
+        o.y = _new_like(x)
     _check(lib().granq_quantize_packed(_dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, bits,
                                        _dev(lo, "lo"), _dev(hi, "hi"), _dev(o.packed_codes, "packed_codes"),
                                        _dev(o.y, "y"), _dev(o.s, "s"), _dev(o.z, "z"), 0, _stream(stream)),
@@ -547,7 +557,7 @@ def granq_dequantize_packed(packed_codes: torch.Tensor, shape, dtype: torch.dtyp
                             z: torch.Tensor, channel_axis: int = 1, group: int = GROUP_CHANNEL,
                             y: torch.Tensor = None, stream=None) -> torch.Tensor:
     """Eq. 6 from the packed codes: y = s * (code - z)."""
-    y = torch.empty(tuple(shape), dtype=dtype, device=packed_codes.device) if y is None else y
+    y = _new(tuple(shape), dtype, packed_codes.device) if y is None else y
     _check(lib().granq_dequantize_packed(_dev(packed_codes, "packed_codes"), _dtype(y), _dims(shape), channel_axis,
                                          group, bits, _dev(s, "s"), _dev(z, "z"), _dev(y, "y"), 0, _stream(stream)),
            "granq_dequantize_packed")
@@ -570,7 +580,7 @@ def granq_accumulate_codes(packed_codes: torch.Tensor, shape, bits: int, s: torc
     o = int(weights.shape[0])
     if y is None:
         out_shape = (shape[0], o, shape[2], shape[3]) if channel_axis == 1 else (shape[0], shape[1], shape[2], o)
-        y = torch.empty(out_shape, dtype=torch.float32, device=packed_codes.device)
+        y = _new(out_shape, torch.float32, packed_codes.device)
     if workspace is None:
         workspace = torch.empty(accumulate_workspace_bytes(shape, channel_axis, o), dtype=torch.uint8,
                                 device=packed_codes.device)

@@ -97,6 +97,16 @@ class Guarded:
             assert bool((raw[:start] == POISON).all()), "an output was written before its first byte"
             assert bool((raw[start + nbytes:] == POISON).all()), "an output was written past its last byte"
 
+    def held_bytes(self) -> int:
+        return sum(raw.numel() for raw, _, _ in self._bufs)
+
+    def check_and_release(self):
+        """Check every margin, then let go of the allocations (the tensors handed out stay valid: they hold a
+        reference to their storage)."""
+        torch.cuda.synchronize()
+        self.check()
+        self._bufs.clear()
+
 
 def guarded_out(b, g: Guarded, x: torch.Tensor, G: int, backward: bool, codes: bool = True, params: bool = True,
                 offset: int = 0):
