@@ -796,8 +796,12 @@ def main():
                 "gx": torch.empty(big.shape, dtype=torch.float32).pin_memory(),
                 "lo": torch.empty(cmax).pin_memory(), "hi": torch.empty(cmax).pin_memory(), "last": None})
 
+        # both bit-widths of a tensor back to back, one per lane: the two lanes then move equal amounts at the
+        # same time and one lane's download overlaps the other's upload best
+        e2e_calls = [(i, bits) for i, sp in enumerate(specs) for bits in sp.bits]
+
         def e2e_step():
-            for k, (i, bits) in enumerate(calls):
+            for k, (i, bits) in enumerate(e2e_calls):
                 ln = lanes[k % len(lanes)]
                 xs, gs = host[i]
                 n, c = specs[i].numel, specs[i].shape[1]
