@@ -660,10 +660,10 @@ def main():
             sub["entry_points"] = rows
             check_status()
             # ---- packed integer codes on one tensor (4 + b/8 bytes per element each way) ----
-            i, s = pick("cfg3.1")
-            x, gy, out = dev[i]
             rows = []
-            for bits in (3, 4, 5):
+            for name, bits in (("cfg3.1", 3), ("cfg3.1", 4), ("cfg3.1", 5), ("cfg4.6", 4)):      # the last one: 7x7 planes
+                i, s = pick(name)
+                x, gy, out = dev[i]
                 pc = torch.empty(b.packed_codes_bytes(x.shape, bits) // 4, dtype=torch.int32, device="cuda")
                 q = b.granq_quantize_packed(x, bits, out.lo, out.hi, packed_codes=pc, stream=stream)
                 tq, _ = sustained_us(lambda k: b.granq_quantize_packed(x, bits, out.lo, out.hi, packed_codes=pc,

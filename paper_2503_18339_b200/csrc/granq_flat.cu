@@ -290,7 +290,9 @@ __device__ __forceinline__ void warp_pack_row(uint64_t mine, uint32_t nb, uint32
 // one bit per element (bit e % 32 of word e / 32): a warp's lanes own consecutive elements or packs
 // starting at a multiple of 32 elements, so whole words are assembled with warp shuffles.
 // PACKONLY: the packed integer codes are the only output (everything else is compiled out).
-template <typename T, int V, int MODE, bool EXTRAS, bool PACKONLY = false>
+// RAGGED: planes are not whole 16-byte packs (7x7 planes), so a pack may straddle two planes and takes the
+// parameters of both (planes of at least one pack: never more than two).
+template <typename T, int V, int MODE, bool EXTRAS, bool PACKONLY = false, bool RAGGED = false>
 __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restrict__ x, const T* __restrict__ gy,
                                                               T* __restrict__ y, T* __restrict__ gx,
                                                               uint8_t* __restrict__ codes,
@@ -385,7 +387,26 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
 #pragma unroll
                     for (int i = 0; i < V; ++i) amax = fmaxf(amax, fabsf(px[j].get(i)));
                     GroupParam gp{p.s, p.z, (amax <= 1152921504606846976.0f) ? rcp : 0.0f};
-                    quantize_pack<T, kBwd, false, EXTRAS>(px[j], pg[j], gp, gp, V, qmax, py, pgx, cb, mb);
+                    GroupParam gp2 = gp;
+                    int n1 = V;
+                    if constexpr (RAGGED) {
+                        const uint32_t rem = (uint32_t)base.rem + k[j] - q * (uint32_t)g.inner;      // position inside plane q
+                        n1 = (int)min((uint32_t)V, (uint32_t)g.inner - rem);
+                        if (n1 < V) {                                                           // the rest lies in plane q + 1
+                            if (tabled) {
+                                gp2.s = s_tab_s[q + 1];
+                                gp2.z = s_tab_z[q + 1];
+                                gp2.r = (amax <= 1152921504606846976.0f) ? s_tab_r[q + 1] : 0.0f;
+                            } else {
+                                const uint32_t grp2 = group_at(g, base, q + 1);
+                                const QParam p2 = make_qparam(__fadd_rn(lo[grp2], 0.0f), __fadd_rn(hi[grp2], 0.0f), qmax);
+                                gp2.s = p2.s;
+                                gp2.z = p2.z;
+                                gp2.r = 0.0f;
+                            }
+                        }
+                    }
+                    quantize_pack<T, kBwd, RAGGED, EXTRAS>(px[j], pg[j], gp, gp2, n1, qmax, py, pgx, cb, mb);
                     if constexpr (EXTRAS) {
                         if constexpr (!PACKONLY) {
 #pragma unroll
@@ -688,13 +709,34 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
                         io.pcodes != nullptr;
     const bool pack_only = io.pcodes != nullptr && io.y == nullptr && io.codes == nullptr && io.mask == nullptr &&
                            io.pmask == nullptr && io.dist == nullptr;
+    // planes that are not whole packs, everything else in place for 16-byte accesses: the vector kernel with
+    // packs that may straddle two planes
+    const bool ragged = !vec && g.inner >= VF && g.inner % VF != 0 && g.E % VF == 0 && !f.inner_big && aligned16(io.x) &&
+                        aligned16(io.gy) && aligned16(io.y) && aligned16(io.gx) && ((uintptr_t)io.codes % 4 == 0) &&
+                        ((uintptr_t)io.mask % 4 == 0);
     if constexpr (MODE == MODE_FWD) {
-        if (vec && pack_only) {
-            quant_flat_kernel<T, VF, MODE, true, true><<<grid, kThreads, 0, st>>>(
-                (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
-                io.code_bits, f, qmax, lo, hi);
+        if ((vec || ragged) && pack_only) {
+            if (vec)
+                quant_flat_kernel<T, VF, MODE, true, true><<<grid, kThreads, 0, st>>>(
+                    (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
+                    io.code_bits, f, qmax, lo, hi);
+            else
+                quant_flat_kernel<T, VF, MODE, true, true, true><<<grid, kThreads, 0, st>>>(
+                    (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
+                    io.code_bits, f, qmax, lo, hi);
             return cudaGetLastError();
         }
+    }
+    if (ragged) {
+        if (extras)
+            quant_flat_kernel<T, VF, MODE, true, false, true><<<grid, kThreads, 0, st>>>(
+                (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
+                io.code_bits, f, qmax, lo, hi);
+        else
+            quant_flat_kernel<T, VF, MODE, false, false, true><<<grid, kThreads, 0, st>>>(
+                (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
+                io.code_bits, f, qmax, lo, hi);
+        return cudaGetLastError();
     }
     if (vec && extras)
         quant_flat_kernel<T, VF, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
