@@ -217,10 +217,11 @@ int granq_fakequant_bwd_packmask(const void* gy, const uint32_t* packed_mask, in
                                  void* gx, uint32_t flags, void* cuda_stream);
 
 /* The forward half of the whole path in one call (Algorithm 1, range step through pre-scale step):
- * range of x itself -> scale / zero-point -> y and the packed mask.  Takes the column-walk plan
- * when slabs and waves are whole mask words, else a range pass followed by an elementwise pass
- * (GRANQ_FLAG_FORCE_TWO_PASS / GRANQ_FLAG_FORCE_COLWALK select one; GRANQ_FLAG_WORKSPACE_ZEROED
- * as for granq_fakequant_fused()).
+ * range of x itself -> scale / zero-point -> y and the packed mask.  Takes the cluster-local plan
+ * where a run of channels that is whole bytes of mask fits one cluster, the column-walk plan when slabs
+ * and waves are whole mask words, else a range pass followed by an elementwise pass
+ * (GRANQ_FLAG_FORCE_TWO_PASS / GRANQ_FLAG_FORCE_COLWALK / GRANQ_FLAG_FORCE_CLUSTER select one;
+ * GRANQ_FLAG_WORKSPACE_ZEROED as for granq_fakequant_fused()).
  *   min_out, max_out out G floats each (required);  scale_opt, zp_opt G floats or NULL */
 int granq_fakequant_fused_fwd_packmask(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group,
                                        int bits, void* y, uint32_t* packed_mask, float* min_out, float* max_out,

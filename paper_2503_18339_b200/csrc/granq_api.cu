@@ -296,14 +296,26 @@ int granq_fakequant_fused_fwd_packmask(const void* x, int dtype, const int64_t d
     if (int rc = check_workspace(workspace, workspace_bytes, G)) return rc;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     QuantIO io{x, nullptr, y, nullptr, nullptr, nullptr, packed_mask};
-    // the column-walk kernel where the geometry allows whole mask words per wave, else range pass + flat pass
+    // the cluster-local kernel where a run of whole mask words fits one cluster, else the column-walk kernel
+    // where the geometry allows whole mask words per wave, else range pass + flat pass
     ColPlan cp{};
+    ClusterPlan kp{};
     const bool two_pass = (flags & GRANQ_FLAG_FORCE_TWO_PASS) != 0;
-    if (!two_pass) cp = plan_colwalk(dtype, g, io, g_tune);
+    if (!two_pass && !(flags & GRANQ_FLAG_FORCE_COLWALK)) kp = plan_cluster(dtype, g, io, false, g_tune);
+    if ((flags & GRANQ_FLAG_FORCE_CLUSTER) && !kp.ok) return GRANQ_ERR_UNSUPPORTED;
+    if (!two_pass && !kp.ok) cp = plan_colwalk(dtype, g, io, g_tune);
     if ((flags & GRANQ_FLAG_FORCE_COLWALK) && !cp.ok) return GRANQ_ERR_UNSUPPORTED;
     Workspace ws = carve_workspace(workspace, G);
     const bool zeroed = (flags & GRANQ_FLAG_WORKSPACE_ZEROED) != 0;
     cudaError_t e = cudaSuccess;
+    if (kp.ok) {
+        if (!zeroed) e = cudaMemsetAsync(workspace, 0, sizeof(uint32_t), st);      // the status word
+        // the kernel writes the mask byte by byte: the padding bits of a last, partial word are cleared here
+        if (e == cudaSuccess && g.E % 32 != 0) e = cudaMemsetAsync(packed_mask + g.E / 32, 0, sizeof(uint32_t), st);
+        if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+        return cuda_status(launch_cluster(kp, io, MODE_FWD, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt,
+                                          g_tune, st));
+    }
     if (!(zeroed && cp.ok)) e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
     if (e != cudaSuccess) return GRANQ_ERR_CUDA;
     if (cp.ok) {
@@ -361,11 +373,21 @@ int granq_fakequant_fused_stats(const void* x, int dtype, const int64_t dims[4],
     // the column-walk kernel where there are slabs to walk, else range pass + flat pass (layer-wise and
     // per-sample groups): the statistics are gathered in the pass that writes y either way
     ColPlan cp{};
-    if (!(flags & GRANQ_FLAG_FORCE_TWO_PASS)) cp = plan_colwalk(dtype, g, io, g_tune);
+    ClusterPlan kp{};
+    const bool two_pass = (flags & GRANQ_FLAG_FORCE_TWO_PASS) != 0;
+    if (!two_pass && !(flags & GRANQ_FLAG_FORCE_COLWALK)) kp = plan_cluster(dtype, g, io, false, g_tune);
+    if ((flags & GRANQ_FLAG_FORCE_CLUSTER) && !kp.ok) return GRANQ_ERR_UNSUPPORTED;
+    if (!two_pass && !kp.ok) cp = plan_colwalk(dtype, g, io, g_tune);
     if ((flags & GRANQ_FLAG_FORCE_COLWALK) && !cp.ok) return GRANQ_ERR_UNSUPPORTED;
     Workspace ws = carve_workspace(workspace, G);
     const bool zeroed = (flags & GRANQ_FLAG_WORKSPACE_ZEROED) != 0;
     cudaError_t e = cudaMemsetAsync(sums_out, 0, 4 * sizeof(double), st);
+    if (e == cudaSuccess && kp.ok) {
+        if (!zeroed) e = cudaMemsetAsync(workspace, 0, sizeof(uint32_t), st);      // the status word
+        if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+        return cuda_status(launch_cluster(kp, io, MODE_FWD, dtype, g, bits, ws, min_out, max_out, scale_opt, zp_opt,
+                                          g_tune, st));
+    }
     if (e == cudaSuccess && !(zeroed && cp.ok)) e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
     if (e != cudaSuccess) return GRANQ_ERR_CUDA;
     if (cp.ok) {

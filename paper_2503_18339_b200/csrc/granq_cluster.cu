@@ -42,6 +42,8 @@ struct KArgs {
     void* gx;
     uint8_t* codes;
     uint8_t* mask;
+    uint32_t* pmask;       // the STE mask at one bit per element, or null (forward plans with whole mask bytes per run)
+    double* dist;          // four running sums of Table 2's statistics, or null
     uint32_t* status;
     float* lo;
     float* hi;
@@ -192,7 +194,7 @@ enum : int {
 };
 
 // U1 / U2 = slabs a thread has in flight in the range walk (plain-load variant) / the quantize walk
-template <typename T, int MODE, bool ALIGNED, bool EXTRAS, int LOAD, int U1, int U2>
+template <typename T, int MODE, bool ALIGNED, int EXTRAS, int LOAD, int U1, int U2>
 __global__ void __launch_bounds__(kKMaxThreads, 2) cluster_kernel(const KArgs a) {
     constexpr int V = Pack<T>::V;
     constexpr bool kBwd = (MODE & MODE_BWD) != 0;
@@ -419,6 +421,8 @@ __global__ void __launch_bounds__(kKMaxThreads, 2) cluster_kernel(const KArgs a)
 
     // ---- quantize, clamp, dequantize from shared memory; STE backward (Eq. 1, 6, Section 2.1) ----
     const float qmax = a.qmax;
+    DistAcc dacc;               // Table 2's sums over everything this thread quantizes (EXTRAS only)
+    dacc.reset();
     if constexpr (ASYNC && GY) k_cp_async_wait<0>();
     for (uint32_t tile0 = 0; tile0 < ncol; tile0 += P) {
         const uint32_t col = tile0 + cin;
@@ -437,15 +441,24 @@ __global__ void __launch_bounds__(kKMaxThreads, 2) cluster_kernel(const KArgs a)
             quantize_pack<T, kBwd, !ALIGNED, EXTRAS, true>(px, pg, g1, g2, ne, qmax, py, pgx, cb, mb);
             st_hint_16(yg + at, py.raw, drop);
             if constexpr (kBwd) st_hint_16(gxg + at, pgx.raw, drop);
-            if constexpr (EXTRAS) {
-                const size_t w = (gbase + at) * (V / 4);
-                if (a.codes) {
+            if constexpr (EXTRAS != 0) {
+                if constexpr (EXTRAS == 1) {
+                    const size_t w = (gbase + at) * (V / 4);
+                    if (a.codes) {
 #pragma unroll
-                    for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.codes)[w + i] = cb[i];
+                        for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.codes)[w + i] = cb[i];
+                    }
+                    if (kBwd && a.mask) {
+#pragma unroll
+                        for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.mask)[w + i] = mb[i];
+                    }
+                    if (a.dist) dacc.add(px, py);
                 }
-                if (kBwd && a.mask) {
-#pragma unroll
-                    for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.mask)[w + i] = mb[i];
+                if (a.pmask) {
+                    // the mask is written byte by byte (8 elements: two fp32 packs of neighbouring lanes, one bf16
+                    // pack): the planner has made every run and slab whole bytes of mask and the rows of columns
+                    // whole pairs of lanes, so both lanes of a byte are here together, in the same slab
+                    store_mask_byte<V>(a.pmask, (gbase + at) * V, mask_bits_of<V, EXTRAS>(mb), tid & 31);
                 }
             }
         };
@@ -497,6 +510,9 @@ __global__ void __launch_bounds__(kKMaxThreads, 2) cluster_kernel(const KArgs a)
             qg += sstep;
         }
     }
+    if constexpr (EXTRAS == 1) {
+        if (a.dist) dacc.flush(a.dist);       // all lanes of every warp are here
+    }
     if constexpr (BULK) {
         // Nothing of this CTA may still be in flight when it leaves: every barrier once more (a no-op unless a
         // wait above gave up early), with the built-in limit.
@@ -520,7 +536,7 @@ uint32_t k_gcd(uint32_t a, uint32_t b) {
     return a;
 }
 
-template <typename T, int MODE, bool ALIGNED, bool EXTRAS>
+template <typename T, int MODE, bool ALIGNED, int EXTRAS>
 cudaError_t k_launch_t(const KArgs& args, const ClusterPlan& plan, uint32_t grid, cudaStream_t st) {
     auto launch = [&](auto kern) -> cudaError_t {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)plan.smem_bytes);
@@ -543,21 +559,30 @@ cudaError_t k_launch_t(const KArgs& args, const ClusterPlan& plan, uint32_t grid
         cfg.numAttrs = plan.early_launch ? 2 : 1;
         return cudaLaunchKernelEx(&cfg, kern, args);
     };
-    switch (plan.load) {
-        case K_LOAD_BULK_X: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_BULK_X, 4, 2>);
-        case K_LOAD_BULK_XG: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_BULK_XG, 4, 2>);
-        case K_LOAD_ASYNC_X: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_ASYNC_X, 4, 2>);
-        case K_LOAD_ASYNC_XG: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_ASYNC_XG, 4, 2>);
-        default: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_PLAIN, 4, 2>);
+    if constexpr (EXTRAS == 2) {      // the packed mask alone: forward plans with per-thread copies or plain loads
+        if (plan.load == K_LOAD_ASYNC_X) return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_ASYNC_X, 4, 2>);
+        return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_PLAIN, 4, 2>);
+    } else {
+        switch (plan.load) {
+            case K_LOAD_BULK_X: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_BULK_X, 4, 2>);
+            case K_LOAD_BULK_XG: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_BULK_XG, 4, 2>);
+            case K_LOAD_ASYNC_X: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_ASYNC_X, 4, 2>);
+            case K_LOAD_ASYNC_XG: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_ASYNC_XG, 4, 2>);
+            default: return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_PLAIN, 4, 2>);
+        }
     }
 }
 
 template <typename T, int MODE>
-cudaError_t k_launch_mode(const KArgs& a, const ClusterPlan& p, bool aligned, bool extras, uint32_t grid,
+cudaError_t k_launch_mode(const KArgs& a, const ClusterPlan& p, bool aligned, int extras, uint32_t grid,
                           cudaStream_t st) {
+    if constexpr (MODE == MODE_FWD) {
+        if (extras == 2)
+            return aligned ? k_launch_t<T, MODE, true, 2>(a, p, grid, st) : k_launch_t<T, MODE, false, 2>(a, p, grid, st);
+    }
     if (aligned)
-        return extras ? k_launch_t<T, MODE, true, true>(a, p, grid, st) : k_launch_t<T, MODE, true, false>(a, p, grid, st);
-    return extras ? k_launch_t<T, MODE, false, true>(a, p, grid, st) : k_launch_t<T, MODE, false, false>(a, p, grid, st);
+        return extras ? k_launch_t<T, MODE, true, 1>(a, p, grid, st) : k_launch_t<T, MODE, true, 0>(a, p, grid, st);
+    return extras ? k_launch_t<T, MODE, false, 1>(a, p, grid, st) : k_launch_t<T, MODE, false, 0>(a, p, grid, st);
 }
 
 }  // namespace
@@ -570,7 +595,8 @@ ClusterPlan plan_cluster(int dtype, const Geom& g, const QuantIO& io, bool backw
     ClusterPlan p{};
     p.ok = false;
     const uint32_t V = dtype == 0 ? 4 : 8, esize = 16 / V;
-    if (io.pmask || io.dist || io.pcodes) return p;
+    if (io.pcodes) return p;
+    if (io.pmask && (g.C * g.inner) % 8 != 0) return p;
     if (!k_aligned16(io.x) || !k_aligned16(io.gy) || !k_aligned16(io.y) || !k_aligned16(io.gx)) return p;
     if (((uintptr_t)io.codes & 3) || ((uintptr_t)io.mask & 3)) return p;
     if (g.inner < (int64_t)V || g.inner >= (1ll << 24) || g.C >= (1ll << 28) || g.outer >= (1ll << 24)) return p;
@@ -581,7 +607,9 @@ ClusterPlan plan_cluster(int dtype, const Geom& g, const QuantIO& io, bool backw
     // too for fp32 tensors with a gradient when that still fits a portable cluster (measured faster there;
     // bf16 halves the bytes per element, and reading gy in the quantize walk measured faster).
     const uint64_t limit = tune.cl_tile_kb > 0 ? (uint64_t)tune.cl_tile_kb * 1024 : 112ull * 1024;   // two CTAs per SM
-    const uint64_t group_bytes = (uint64_t)g.outer * (V / k_gcd((uint32_t)g.inner, V)) * g.inner * esize;
+    // a run is whole 16-byte units; with a packed mask also whole bytes of mask (8 elements)
+    const uint32_t unit = io.pmask ? 8u : V;
+    const uint64_t group_bytes = (uint64_t)g.outer * (unit / k_gcd((uint32_t)g.inner, unit)) * g.inner * esize;
     switch (tune.cl_load) {
         case 1: p.load = K_LOAD_BULK_X; break;
         case 2: p.load = K_LOAD_PLAIN; break;
@@ -592,8 +620,10 @@ ClusterPlan plan_cluster(int dtype, const Geom& g, const QuantIO& io, bool backw
             p.load = (backward && dtype == 0 && 2 * group_bytes <= 8 * limit) ? K_LOAD_ASYNC_XG : K_LOAD_ASYNC_X;
             break;
     }
+    // the two lanes that assemble a byte of mask must both be there: only the variants without a give-up path qualify
+    if (io.pmask && p.load != K_LOAD_ASYNC_X && p.load != K_LOAD_ASYNC_XG && p.load != K_LOAD_PLAIN) return p;
     const uint64_t tiles = (p.load == K_LOAD_BULK_XG || p.load == K_LOAD_ASYNC_XG) ? 2 : 1;   // staged tiles per CTA
-    const uint32_t k0 = V / k_gcd(inner, V);
+    const uint32_t k0 = unit / k_gcd(inner, unit);
     const uint64_t target = std::min<uint64_t>(limit, 64ull * 1024);
     const uint64_t run0 = (uint64_t)k0 * inner * esize;                  // bytes of a minimal run in one slab
     // CTAs per run: the smallest power of two (at most 8, the portable cluster size) that fits the limit
@@ -661,6 +691,8 @@ cudaError_t launch_cluster(const ClusterPlan& plan, const QuantIO& io, int mode,
     a.gx = io.gx;
     a.codes = io.codes;
     a.mask = io.mask;
+    a.pmask = io.pmask;
+    a.dist = io.dist;
     a.status = ws.status;
     a.lo = lo;
     a.hi = hi;
@@ -681,7 +713,8 @@ cudaError_t launch_cluster(const ClusterPlan& plan, const QuantIO& io, int mode,
     const uint32_t nruns = (a.C + plan.k - 1) / plan.k;
     const uint32_t grid = nruns * plan.R;
     const bool aligned = (a.inner % V) == 0;
-    const bool extras = io.codes != nullptr || io.mask != nullptr;
+    // 1: codes / mask bytes / sums compiled in; 2: the packed mask alone (a leaner instantiation of the forward kernel)
+    const int extras = (io.codes != nullptr || io.mask != nullptr || io.dist != nullptr) ? 1 : (io.pmask != nullptr ? 2 : 0);
     if (dtype == 0) {
         if (mode == MODE_FWD) return k_launch_mode<float, MODE_FWD>(a, plan, aligned, extras, grid, st);
         return k_launch_mode<float, MODE_BOTH>(a, plan, aligned, extras, grid, st);

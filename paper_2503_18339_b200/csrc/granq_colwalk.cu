@@ -116,7 +116,7 @@ struct ColRange {
 };
 
 // U1 / U2 = slabs a thread has in flight in phase 1 / phase 2
-template <typename T, int MODE, bool ALIGNED, bool EXTRAS, int U1, int U2>
+template <typename T, int MODE, bool ALIGNED, int EXTRAS, int U1, int U2>
 __global__ void __launch_bounds__(kCThreads, 4) colwalk_kernel(const CArgs a) {
     constexpr int V = Pack<T>::V;
     constexpr bool kBwd = (MODE & MODE_BWD) != 0;
@@ -310,28 +310,23 @@ __global__ void __launch_bounds__(kCThreads, 4) colwalk_kernel(const CArgs a) {
                 quantize_pack<T, kBwd, !ALIGNED, EXTRAS, true>(px, pg, g1, g2, it.ne, qmax, py, pgx, cb, mb);
                 st_hint_16(yg + at, py.raw, drop);
                 if constexpr (kBwd) st_hint_16(gxg + at, pgx.raw, drop);
-                if constexpr (EXTRAS) {
-                    if (a.codes) {
+                if constexpr (EXTRAS != 0) {
+                    if constexpr (EXTRAS == 1) {
+                        if (a.codes) {
 #pragma unroll
-                        for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.codes)[at * (V / 4) + i] = cb[i];
-                    }
-                    if (kBwd && a.mask) {
+                            for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.codes)[at * (V / 4) + i] = cb[i];
+                        }
+                        if (kBwd && a.mask) {
 #pragma unroll
-                        for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.mask)[at * (V / 4) + i] = mb[i];
+                            for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(a.mask)[at * (V / 4) + i] = mb[i];
+                        }
+                        if (a.dist) dacc.add(px, py);
                     }
-                    if (a.dist) dacc.add(px, py);
                     if (a.pmask) {
-                        // 32 / V neighbouring lanes own the 32 elements of one mask word; the planner has made
-                        // every slab and wave a whole number of words, so such a group of lanes is here together
-                        constexpr uint32_t kLanes = 32 / V;
-                        const uint32_t members = ((1u << kLanes) - 1u) << (lane & ~(kLanes - 1));
-                        uint32_t bits = 0;
-#pragma unroll
-                        for (int i = 0; i < V; ++i) bits |= ((mb[i / 4] >> (8 * (i % 4))) & 1u) << i;
-                        uint32_t wv = bits << (V * (lane & (kLanes - 1)));
-#pragma unroll
-                        for (uint32_t d = 1; d < kLanes; d <<= 1) wv |= __shfl_xor_sync(members, wv, d);
-                        if ((lane & (kLanes - 1)) == 0) a.pmask[(at * V) >> 5] = wv;
+                        // the mask is written byte by byte (8 elements: two fp32 packs of neighbouring lanes, one
+                        // bf16 pack); the planner has made every slab and wave whole mask words, so both lanes of a
+                        // byte are here together
+                        store_mask_byte<V>(a.pmask, at * V, mask_bits_of<V, EXTRAS>(mb), lane);
                     }
                 }
             };
@@ -372,7 +367,7 @@ __global__ void __launch_bounds__(kCThreads, 4) colwalk_kernel(const CArgs a) {
         phase2(w);
     }
 
-    if constexpr (EXTRAS) {
+    if constexpr (EXTRAS == 1) {
         if (a.dist) dacc.flush(a.dist);
     }
 
@@ -435,7 +430,7 @@ uint32_t c_assumed_grid(int cta_cap) {
     return (uint32_t)(sms * per_sm);
 }
 
-template <typename T, int MODE, bool ALIGNED, bool EXTRAS>
+template <typename T, int MODE, bool ALIGNED, int EXTRAS>
 cudaError_t c_launch_t(CArgs& args, int sm_count, int cta_cap, cudaStream_t st) {
     auto kern = colwalk_kernel<T, MODE, ALIGNED, EXTRAS, 4, 2>;
     // resident CTAs per SM of this instantiation, remembered per device (a pure function of both)
@@ -464,12 +459,14 @@ cudaError_t c_launch_t(CArgs& args, int sm_count, int cta_cap, cudaStream_t st) 
 }
 
 template <typename T, int MODE>
-cudaError_t c_launch_mode(CArgs& a, bool aligned, bool extras, int sms, int cap, cudaStream_t st) {
+cudaError_t c_launch_mode(CArgs& a, bool aligned, int extras, int sms, int cap, cudaStream_t st) {
+    if constexpr (MODE == MODE_FWD) {
+        if (extras == 2)       // the packed mask alone: a leaner instantiation of the forward kernel
+            return aligned ? c_launch_t<T, MODE, true, 2>(a, sms, cap, st) : c_launch_t<T, MODE, false, 2>(a, sms, cap, st);
+    }
     if (aligned)
-        return extras ? c_launch_t<T, MODE, true, true>(a, sms, cap, st)
-                      : c_launch_t<T, MODE, true, false>(a, sms, cap, st);
-    return extras ? c_launch_t<T, MODE, false, true>(a, sms, cap, st)
-                  : c_launch_t<T, MODE, false, false>(a, sms, cap, st);
+        return extras ? c_launch_t<T, MODE, true, 1>(a, sms, cap, st) : c_launch_t<T, MODE, true, 0>(a, sms, cap, st);
+    return extras ? c_launch_t<T, MODE, false, 1>(a, sms, cap, st) : c_launch_t<T, MODE, false, 0>(a, sms, cap, st);
 }
 
 }  // namespace
@@ -607,7 +604,8 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
         s.div_ncol = make_fastdiv(s.ncol);
     }
     a.div_plane = make_fastdiv(aligned ? inner / V : inner);
-    const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr || io.dist != nullptr;
+    // 1: codes / mask bytes / sums compiled in; 2: the packed mask alone
+    const int extras = (io.codes != nullptr || io.mask != nullptr || io.dist != nullptr) ? 1 : (io.pmask != nullptr ? 2 : 0);
     const int cap = tune.l2_ctas_per_sm;
     if (dtype == 0) {
         if (mode == MODE_FWD) return c_launch_mode<float, MODE_FWD>(a, aligned, extras, sms, cap, st);

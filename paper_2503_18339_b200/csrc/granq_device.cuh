@@ -256,11 +256,12 @@ __device__ __forceinline__ float tie_threshold(float z) {
 }
 
 // Quantize one pack: elements [0, n1) belong to the group with parameters g1, the rest to
-// g2 (n1 = V when the pack lies in one group).  EXTRAS also packs the codes and the mask
-// (one byte per element).  SELF: the range is that of the tensor itself, so x / s + z lies within
+// g2 (n1 = V when the pack lies in one group).  EXTRAS = 1 also packs the codes and the mask
+// (one byte per element); EXTRAS = 2 leaves the codes out and returns the mask as V bits in mb[0]
+// (bit i: the clamp was inactive for element i), which is all the packed mask needs.  SELF: the range is that of the tensor itself, so x / s + z lies within
 // [-1, qmax + 1] already (x in [lo, hi] gives RN(x / s) - round(RN(lo / s)) >= -1/2, and at most qmax plus a few
 // units in the last place of hi / s < 2^33 above that) and the clamp before the rounding can go.
-template <typename T, bool BWD, bool SPLIT, bool EXTRAS, bool SELF = false>
+template <typename T, bool BWD, bool SPLIT, int EXTRAS, bool SELF = false>
 __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& pg, const GroupParam& g1,
                                               const GroupParam& g2, int n1, float qmax, Pack<T>& py, Pack<T>& pgx,
                                               uint32_t (&cb)[Pack<T>::V / 4], uint32_t (&mb)[Pack<T>::V / 4]) {
@@ -276,9 +277,11 @@ __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& 
         const bool in = (r == q);
         py.set(i, __fmul_rn(s, __fsub_rn(q, z)));
         if constexpr (BWD) pgx.set(i, in ? pg.get(i) : 0.0f);
-        if constexpr (EXTRAS) {
+        if constexpr (EXTRAS == 1) {
             cb[i / 4] |= (uint32_t)q << (8 * (i % 4));
             mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
+        } else if constexpr (EXTRAS == 2) {
+            mb[0] |= in ? (1u << i) : 0u;
         }
     };
     auto exact_round = [&](float t, float z) -> float {        // t = RN(x / s): the sequence as defined
@@ -363,6 +366,33 @@ __device__ __forceinline__ void pack_minmax(const Pack<T>& p, int first, int las
             mn = fminf(mn, v);
             mx = fmaxf(mx, v);
         }
+    }
+}
+
+// The V mask bits of one pack, from the mask bytes of quantize_pack<EXTRAS = 1> or the bits of <EXTRAS = 2>.
+template <int V, int EXTRAS>
+__device__ __forceinline__ uint32_t mask_bits_of(const uint32_t (&mb)[V / 4]) {
+    if constexpr (EXTRAS == 2) {
+        return mb[0];
+    } else {
+        uint32_t bits = 0;
+#pragma unroll
+        for (int i = 0; i < V; ++i) bits |= ((mb[i / 4] >> (8 * (i % 4))) & 1u) << i;
+        return bits;
+    }
+}
+
+// Store the packed mask one byte (8 elements) at a time: `bits` are the V mask bits of the pack that starts at
+// element `first` (a multiple of V; for V = 4 the even lane of a pair holds the low half of a byte, and both
+// lanes of the pair must call this together with neighbouring packs).
+template <int V>
+__device__ __forceinline__ void store_mask_byte(uint32_t* pmask, size_t first, uint32_t bits, uint32_t lane) {
+    if constexpr (V == 4) {
+        const uint32_t other = __shfl_xor_sync(3u << (lane & ~1u), bits, 1);
+        if (!(lane & 1)) reinterpret_cast<uint8_t*>(pmask)[first >> 3] = (uint8_t)(bits | (other << 4));
+    } else {
+        static_assert(V == 8, "a pack is 4 or 8 elements");
+        reinterpret_cast<uint8_t*>(pmask)[first >> 3] = (uint8_t)bits;
     }
 }
 

@@ -286,13 +286,13 @@ __device__ __forceinline__ void warp_pack_row(uint64_t mine, uint32_t nb, uint32
 }
 
 // ---- Eq. 1, clamp, Eq. 6, STE: elementwise pass with a given per-group range ----------------------
-// EXTRAS: the optional codes / mask / packed-mask outputs are compiled in.  The packed mask holds
+// EXTRAS = 1: the optional codes / mask / packed-mask outputs are compiled in; 2: the packed mask alone.  The packed mask holds
 // one bit per element (bit e % 32 of word e / 32): a warp's lanes own consecutive elements or packs
 // starting at a multiple of 32 elements, so whole words are assembled with warp shuffles.
 // PACKONLY: the packed integer codes are the only output (everything else is compiled out).
 // RAGGED: planes are not whole 16-byte packs (7x7 planes), so a pack may straddle two planes and takes the
 // parameters of both (planes of at least one pack: never more than two).
-template <typename T, int V, int MODE, bool EXTRAS, bool PACKONLY = false, bool RAGGED = false>
+template <typename T, int V, int MODE, int EXTRAS, bool PACKONLY = false, bool RAGGED = false>
 __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restrict__ x, const T* __restrict__ gy,
                                                               T* __restrict__ y, T* __restrict__ gx,
                                                               uint8_t* __restrict__ codes,
@@ -407,12 +407,9 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                         }
                     }
                     quantize_pack<T, kBwd, RAGGED, EXTRAS>(px[j], pg[j], gp, gp2, n1, qmax, py, pgx, cb, mb);
-                    if constexpr (EXTRAS) {
-                        if constexpr (!PACKONLY) {
-#pragma unroll
-                            for (int i = 0; i < V; ++i) inside_bits |= ((mb[i / 4] >> (8 * (i % 4))) & 1u) << i;
-                        }
-                        if constexpr (kFwd) {
+                    if constexpr (EXTRAS != 0) {
+                        if constexpr (!PACKONLY) inside_bits = mask_bits_of<V, EXTRAS>(mb);
+                        if constexpr (kFwd && EXTRAS == 1) {
                             if constexpr (!PACKONLY) {
                                 if (dist) dacc.add(px[j], py);
                             }
@@ -424,8 +421,8 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                         }
                     }
                     if constexpr (kFwd && !PACKONLY) {
-                        if (!EXTRAS || y) st_stream_16(y + e, py.raw);
-                        if constexpr (EXTRAS) {
+                        if (EXTRAS != 1 || y) st_stream_16(y + e, py.raw);
+                        if constexpr (EXTRAS == 1) {
                             if (codes) {
 #pragma unroll
                                 for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(codes + e)[i] = cb[i];
@@ -434,7 +431,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                     }
                     if constexpr (kBwd) {
                         st_stream_16(gx + e, pgx.raw);
-                        if constexpr (EXTRAS) {
+                        if constexpr (EXTRAS == 1) {
                             if (mask) {
 #pragma unroll
                                 for (int i = 0; i < V / 4; ++i) reinterpret_cast<uint32_t*>(mask + e)[i] = mb[i];
@@ -443,7 +440,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                     }
                 }
                 }
-                if constexpr (EXTRAS && kFwd) {
+                if constexpr (EXTRAS != 0 && kFwd) {
                     if (!PACKONLY && pmask) {          // every lane of the warp is here: assemble whole 32-bit words
                         const uint32_t lane = threadIdx.x & 31;
                         const int64_t word = (e0 + k[j]) >> 5;
@@ -458,7 +455,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                             if ((lane & (kLanes - 1)) == 0 && valid) pmask[word] = w;
                         }
                     }
-                    if (PACKONLY || pcodes) {         // the warp's 32 * V codes are V * b whole words of the bit string
+                    if (EXTRAS == 1 && (PACKONLY || pcodes)) {      // the warp's 32 * V codes are V * b whole words of the bit string
                         const uint32_t lane = threadIdx.x & 31;
                         const uint32_t nb = (uint32_t)(V * code_bits);
                         const int64_t row_e = e0 + k0 + (int64_t)(j * kThreads + (threadIdx.x & ~31u)) * V;
@@ -472,7 +469,7 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
             }
         }
     }
-    if constexpr (EXTRAS && kFwd && !PACKONLY) {
+    if constexpr (EXTRAS == 1 && kFwd && !PACKONLY) {
         if (dist) dacc.flush(dist);
     }
 }
@@ -707,6 +704,9 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
     float qmax = (float)((1 << bits) - 1);
     const bool extras = io.codes != nullptr || io.mask != nullptr || io.pmask != nullptr || io.dist != nullptr ||
                         io.pcodes != nullptr;
+    // forward with y and the packed mask as the only outputs: a leaner instantiation
+    const bool pmask_only = io.pmask != nullptr && io.y != nullptr && io.codes == nullptr && io.mask == nullptr &&
+                            io.dist == nullptr && io.pcodes == nullptr;
     const bool pack_only = io.pcodes != nullptr && io.y == nullptr && io.codes == nullptr && io.mask == nullptr &&
                            io.pmask == nullptr && io.dist == nullptr;
     // planes that are not whole packs, everything else in place for 16-byte accesses: the vector kernel with
@@ -717,11 +717,22 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
     if constexpr (MODE == MODE_FWD) {
         if ((vec || ragged) && pack_only) {
             if (vec)
-                quant_flat_kernel<T, VF, MODE, true, true><<<grid, kThreads, 0, st>>>(
+                quant_flat_kernel<T, VF, MODE, 1, true><<<grid, kThreads, 0, st>>>(
                     (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
                     io.code_bits, f, qmax, lo, hi);
             else
-                quant_flat_kernel<T, VF, MODE, true, true, true><<<grid, kThreads, 0, st>>>(
+                quant_flat_kernel<T, VF, MODE, 1, true, true><<<grid, kThreads, 0, st>>>(
+                    (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
+                    io.code_bits, f, qmax, lo, hi);
+            return cudaGetLastError();
+        }
+        if ((vec || ragged) && pmask_only) {
+            if (vec)
+                quant_flat_kernel<T, VF, MODE, 2><<<grid, kThreads, 0, st>>>(
+                    (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
+                    io.code_bits, f, qmax, lo, hi);
+            else
+                quant_flat_kernel<T, VF, MODE, 2, false, true><<<grid, kThreads, 0, st>>>(
                     (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
                     io.code_bits, f, qmax, lo, hi);
             return cudaGetLastError();
@@ -729,23 +740,23 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
     }
     if (ragged) {
         if (extras)
-            quant_flat_kernel<T, VF, MODE, true, false, true><<<grid, kThreads, 0, st>>>(
+            quant_flat_kernel<T, VF, MODE, 1, false, true><<<grid, kThreads, 0, st>>>(
                 (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
                 io.code_bits, f, qmax, lo, hi);
         else
-            quant_flat_kernel<T, VF, MODE, false, false, true><<<grid, kThreads, 0, st>>>(
+            quant_flat_kernel<T, VF, MODE, 0, false, true><<<grid, kThreads, 0, st>>>(
                 (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
                 io.code_bits, f, qmax, lo, hi);
         return cudaGetLastError();
     }
     if (vec && extras)
-        quant_flat_kernel<T, VF, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
+        quant_flat_kernel<T, VF, MODE, 1><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
                                                                         (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes, io.code_bits, f, qmax, lo, hi);
     else if (vec)
-        quant_flat_kernel<T, VF, MODE, false><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
+        quant_flat_kernel<T, VF, MODE, 0><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
                                                                          (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes, io.code_bits, f, qmax, lo, hi);
     else
-        quant_flat_kernel<T, 1, MODE, true><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
+        quant_flat_kernel<T, 1, MODE, 1><<<grid, kThreads, 0, st>>>((const T*)io.x, (const T*)io.gy, (T*)io.y,
                                                                        (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes, io.code_bits, f, qmax, lo, hi);
     return cudaGetLastError();
 }

@@ -49,12 +49,12 @@ def test_fused_stats_every_grouping_and_plan(b, knobs, shape, dtype):
     for mode in (orc.GROUP_CHANNEL, orc.GROUP_SAMPLE_CHANNEL, orc.GROUP_TENSOR):
         ref = orc.fused(x, bits, group_mode=mode)
         ref_sums = orc.distortion_sums(x, ref.y)
-        for flags, wave_kb in ((0, 0), (b.FLAG_FORCE_TWO_PASS, 0), (b.FLAG_FORCE_COLWALK, 1)):
+        for flags, wave_kb in ((0, 0), (b.FLAG_FORCE_TWO_PASS, 0), (b.FLAG_FORCE_COLWALK, 1), (b.FLAG_FORCE_CLUSTER, 0)):
             knobs(l2_wave_kb=wave_kb)
             try:
                 got = b.granq_fakequant_fused_stats(to_dev(x), bits, group=mode, want_params=True, flags=flags)
             except b.GranqError as err:
-                assert flags == b.FLAG_FORCE_COLWALK and err.status == b.ERR_UNSUPPORTED
+                assert flags in (b.FLAG_FORCE_COLWALK, b.FLAG_FORCE_CLUSTER) and err.status == b.ERR_UNSUPPORTED
                 continue
             assert b.workspace_status(got.workspace) == b.OK
             assert_parity(got, ref, shape, 1, mode, backward=False)

@@ -15,7 +15,8 @@ SHAPES = [
     (1, 1, 1, 9),        # scalar path, one partial word
     (3, 5, 7, 7),        # 735 elements, ragged planes, scalar path
     (4, 16, 14, 14),     # vector path
-    (16, 8, 7, 7),       # 7x7 planes, slab of 392 elements: not whole mask words -> two-pass in the fused call
+    (16, 8, 7, 7),       # 7x7 planes, slab of 392 elements = 49 bytes of mask: cluster plan, else two-pass
+    (3, 8, 7, 7),        # the same with a last mask word that is half padding
     (16, 32, 7, 7),      # 7x7 planes, slab of 1568 = 49 words: column walk with 32-channel waves
     (9, 24, 12, 12),     # column walk, aligned planes
     (8, 3, 4, 4),        # 48 elements per slab
@@ -66,21 +67,30 @@ def test_fused_fwd_packmask(b, knobs, shape, dtype):
     ref = orc.fused(x, bits, gy=gy)
     expect = packed_ref(ref.mask)
     dt = b.BF16 if dtype == "bf16" else b.F32
-    for flags, wave_kb in ((0, 0), (b.FLAG_FORCE_TWO_PASS, 0), (b.FLAG_FORCE_COLWALK, 1), (b.FLAG_FORCE_COLWALK, 0)):
+    for flags, wave_kb in ((0, 0), (b.FLAG_FORCE_TWO_PASS, 0), (b.FLAG_FORCE_COLWALK, 1), (b.FLAG_FORCE_COLWALK, 0),
+                           (b.FLAG_FORCE_CLUSTER, 0), (b.FLAG_FORCE_CLUSTER, 2)):
         knobs(l2_wave_kb=wave_kb)
+        if flags == b.FLAG_FORCE_CLUSTER:
+            b.tune(b.KNOB_CLUSTER_CTAS, wave_kb)          # the cluster plan: automatic cut, then clusters of 2
         try:
             got = b.granq_fakequant_fused_fwd_packmask(to_dev(x), bits, want_params=True, flags=flags)
         except b.GranqError as err:
-            assert flags == b.FLAG_FORCE_COLWALK and err.status == b.ERR_UNSUPPORTED
+            assert flags in (b.FLAG_FORCE_COLWALK, b.FLAG_FORCE_CLUSTER) and err.status == b.ERR_UNSUPPORTED
             continue
+        finally:
+            b.tune(b.KNOB_CLUSTER_CTAS, 0)
         assert b.workspace_status(got.workspace) == b.OK
         assert_parity(got, ref, shape, 1, orc.GROUP_CHANNEL, backward=False)
         assert np.array_equal(packed_np(got.packed_mask), expect), f"packed mask differs (flags {flags})"
         gx = b.granq_fakequant_bwd_packmask(to_dev(gy), got.packed_mask)
         assert same_bits(to_np(gx), ref.gx)
-    # the column walk must really be taken where slabs and waves are whole mask words
-    if shape[0] >= 8 and (shape[1] * shape[2] * shape[3]) % 32 == 0 and shape[2] * shape[3] >= (8 if dtype == "bf16" else 4):
+    # the column walk must really be taken where slabs and waves are whole mask words, the cluster plan where
+    # slabs are whole bytes of mask
+    wide = shape[2] * shape[3] >= (8 if dtype == "bf16" else 4)
+    if shape[0] >= 8 and (shape[1] * shape[2] * shape[3]) % 32 == 0 and wide:
         b.granq_fakequant_fused_fwd_packmask(to_dev(x), bits, flags=b.FLAG_FORCE_COLWALK)
+    if (shape[1] * shape[2] * shape[3]) % 8 == 0 and wide:
+        b.granq_fakequant_fused_fwd_packmask(to_dev(x), bits, flags=b.FLAG_FORCE_CLUSTER)
 
 
 def test_packmask_rejects_bad_arguments(b):
