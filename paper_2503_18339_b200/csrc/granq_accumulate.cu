@@ -9,15 +9,17 @@
 //   - the codes (0 .. 255) are exact in bf16; W' is split into two bf16 matrices hi + lo (hi = the
 //     rounding of W', lo = the rounding of the rest; what is left is below 2^-17 |W'|), so two
 //     tcgen05.mma per K step accumulate into the same fp32 accumulator in tensor memory;
-//   - operands are staged in shared memory by TMA tile loads of this GPU's own memory (128-byte
-//     swizzle, no multicast), a ring of stages handed back and forth through mbarriers;
+//   - the codes never exist as a matrix in HBM: the threads of a CTA read the packed bit string, expand the
+//     codes of a tile (128 pixels x 64 channels) to bf16 and store them into shared memory in the layout the
+//     tensor core reads (rows of 64 bf16, 128-byte swizzle), then make the stores visible to the asynchronous
+//     proxy; the two weight halves come by TMA tile loads of this GPU's own memory (same swizzle, no
+//     multicast); a ring of stages is handed back and forth through mbarriers;
 //   - one elected thread issues the MMAs; the accumulator (128 pixels x BN output channels) lives in
 //     tensor memory and is read back with tcgen05.ld for the epilogue, which subtracts the bias and
 //     stores y in the layout of the input (NCHW or channels-last).
-// Three launches: weights (W' hi / lo, bias), codes (packed bit string -> bf16, channels-last matrix
-// [pixels, C]: for an NCHW tensor a tiled transpose), contraction.  Every wait on an mbarrier is
-// bounded; a wait that runs out records GRANQ_ERR_TIMEOUT in the workspace's status word, the CTA
-// skips its remaining work, frees its tensor memory and returns.
+// Two launches: weights (W' hi / lo, bias), then expansion + contraction + epilogue in one kernel.  Every wait
+// on an mbarrier is bounded; a wait that runs out records GRANQ_ERR_TIMEOUT in the workspace's status word,
+// the CTA skips its remaining work, frees its tensor memory and returns.
 #include "../../include/granq.h"
 
 #include "granq_internal.h"
@@ -34,7 +36,8 @@ namespace {
 constexpr int kABm = 128;                 // pixels per tile (rows of the accumulator = tensor-memory lanes)
 constexpr int kABk = 64;                  // channels per stage: 64 bf16 = one 128-byte swizzle row
 constexpr int kAMaxStages = 4;         // the ring is as deep as the K blocks need, at most this
-constexpr int kAThreads = 128;            // warp 0: TMA producer, warp 1: MMA issuer; all four: epilogue
+constexpr int kAThreads = 128;            // all four warps expand codes and run the epilogue; thread 0 loads the
+                                          // weights, thread 32 issues the MMAs
 constexpr uint32_t kASpin = 1u << 22;     // bounded mbarrier wait
 constexpr uint32_t kATimeout = 5;         // GRANQ_ERR_TIMEOUT
 
@@ -97,20 +100,71 @@ struct AArgs {
     float* y;
     const float* bias;
     uint32_t* status;
-    int64_t rows;          // pixels of the whole batch
-    int64_t P;             // pixels of one sample
-    int64_t O;             // output channels
-    int kblocks;           // ceil(C / 64)
-    int channels_last;     // layout of y
-    int stages;            // depth of the ring of operand stages
+    const uint32_t* packed;   // the codes as a bit string, b bits each, in the storage order of the tensor
+    int64_t nwords;           // 32-bit words of the bit string
+    int64_t rows;             // pixels of the whole batch
+    int64_t P;                // pixels of one sample
+    int64_t C;                // input channels
+    int64_t O;                // output channels
+    int bits;
+    int kblocks;              // ceil(C / 64)
+    int stages;               // depth of the ring of operand stages
     uint32_t spin_limit;
 };
 
-// D[128 pixels x BN] = codes[128 x C] * (hi + lo)[BN x C]^T in tensor memory; y = D - bias
-template <int BN>
+// code e of a bit string of b-bit codes (element e in bits [e*b, (e+1)*b), little-endian words)
+__device__ __forceinline__ uint32_t a_code_at(const uint32_t* __restrict__ packed, int64_t e, int bits) {
+    const int64_t bit = e * bits;
+    const int64_t word = bit >> 5;
+    const int sh = (int)(bit & 31);
+    uint32_t v = __ldg(packed + word) >> sh;
+    if (sh + bits > 32) v |= __ldg(packed + word + 1) << (32 - sh);
+    return v & ((1u << bits) - 1u);
+}
+
+// the `count` (1 .. 8) codes of elements e, e + 1, ... as one 64-bit string (code j in bits [j*b, (j+1)*b)),
+// zero above them; reads at most three words, none beyond the end of the bit string
+__device__ __forceinline__ uint64_t a_codes8(const uint32_t* __restrict__ packed, int64_t e, int bits, int count,
+                                             int64_t nwords) {
+    const int64_t bit = e * bits;
+    const int64_t w = bit >> 5;
+    const uint32_t sh = (uint32_t)(bit & 31);
+    const uint32_t need = sh + (uint32_t)(count * bits);
+    const uint32_t w0 = __ldg(packed + w);
+    uint32_t w1 = 0, w2 = 0;
+    if (need > 32 && w + 1 < nwords) w1 = __ldg(packed + w + 1);
+    if (need > 64 && w + 2 < nwords) w2 = __ldg(packed + w + 2);
+    const uint64_t v = ((uint64_t)__funnelshift_r(w1, w2, sh) << 32) | __funnelshift_r(w0, w1, sh);
+    const int keep = count * bits;
+    return keep >= 64 ? v : (v & ((1ull << keep) - 1ull));
+}
+
+// two codes -> two bf16 in one word (the first in the low half), exact.  Codes below 128: 0x4300 | code is the
+// bf16 number 128 + code, and one packed subtraction of 128 gives the code; 8-bit codes go through fp32.
+__device__ __forceinline__ uint32_t a_pair_bf16(uint32_t c0, uint32_t c1, bool wide) {
+    if (!wide) {
+        const uint32_t biased = c0 | (c1 << 16) | 0x43004300u, bias = 0x43004300u;
+        const __nv_bfloat162 d = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&biased),
+                                         *reinterpret_cast<const __nv_bfloat162*>(&bias));
+        return *reinterpret_cast<const uint32_t*>(&d);
+    }
+    const float f0 = __fsub_rn(__uint_as_float(0x4B000000u | c0), 8388608.0f);
+    const float f1 = __fsub_rn(__uint_as_float(0x4B000000u | c1), 8388608.0f);
+    const __nv_bfloat162 d = __floats2bfloat162_rn(f0, f1);
+    return *reinterpret_cast<const uint32_t*>(&d);
+}
+
+// 16 bytes of an operand row: chunk `chunk` (8 bf16) of row `row` of a K-major tile with the 128-byte swizzle
+// (rows of 128 bytes; within each group of 8 rows chunk c of row r sits at position c ^ (r & 7))
+__device__ __forceinline__ void a_store_chunk(unsigned char* tile, uint32_t row, uint32_t chunk, const uint32_t (&w)[4]) {
+    *reinterpret_cast<uint4*>(tile + row * 128u + ((chunk ^ (row & 7u)) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+}
+
+// D[128 pixels x BN] = codes[128 x C] * (hi + lo)[BN x C]^T in tensor memory; y = D - bias.
+// NHWC: the bit string is in channels-last order (and so is y), else in NCHW order.
+template <int BN, bool NHWC>
 __global__ void __launch_bounds__(kAThreads, BN == 64 ? 6 : 4)
-accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_hi,
-                  const __grid_constant__ CUtensorMap map_lo, const AArgs a) {
+accumulate_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo, const AArgs a) {
     constexpr uint32_t kABytes = kABm * kABk * 2, kBBytes = BN * kABk * 2, kStageBytes = kABytes + 2 * kBBytes;
     extern __shared__ __align__(1024) unsigned char a_smem[];
     __shared__ __align__(8) uint64_t s_full[kAMaxStages], s_empty[kAMaxStages], s_done;
@@ -118,7 +172,8 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // 1024-byte aligned stage buffers (the swizzle pattern is a function of the address)
     unsigned char* stages = a_smem + ((1024u - (a_smem_u32(a_smem) & 1023u)) & 1023u);
-    const int row0 = (int)blockIdx.x * kABm, col0 = (int)blockIdx.y * BN;
+    const int64_t row0 = (int64_t)blockIdx.x * kABm;
+    const int col0 = (int)blockIdx.y * BN;
 
     if (tid == 0) {
         for (int s = 0; s < kAMaxStages; ++s) {
@@ -141,7 +196,7 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const uint32_t tmem = s_tmem;
 
-    // bounded wait; false when it ran out or another role of this CTA has given up
+    // bounded wait; false when it ran out or another thread of this CTA has given up
     auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
         for (uint32_t i = 0; i < a.spin_limit; ++i) {
             if (a_mbar_try_wait(bar, parity)) return true;
@@ -152,43 +207,110 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         return false;
     };
 
-    if (warp == 0 && lane == 0) {
-        // ---- producer: one stage = 128 x 64 codes + BN x 64 of each weight half ----
-        for (int kb = 0; kb < a.kblocks; ++kb) {
-            const int s = kb % a.stages;
-            if (kb >= a.stages && !wait(&s_empty[s], (uint32_t)((kb / a.stages - 1) & 1))) break;
-            unsigned char* st = stages + (size_t)s * kStageBytes;
-            a_mbar_expect_tx(&s_full[s], kStageBytes);
-            a_tma_load_2d(st, &map_q, kb * kABk, row0, &s_full[s]);
+    // ---- this thread's share of a tile of codes: 8 of its 1024 sixteen-byte chunks ----
+    const int bits = a.bits;
+    const bool wide = bits == 8;
+    const uint32_t code_mask = (1u << bits) - 1u;
+    const uint32_t cg = tid & 7;                 // which 8 of the stage's 64 channels
+    // NCHW: rows 8 q .. 8 q + 7 (q = tid / 8), whose codes are consecutive in the bit string for each channel when
+    // they lie in one sample
+    const int64_t gp0 = row0 + 8 * (int64_t)(tid >> 3);
+    const int64_t n0 = gp0 / a.P, p0 = gp0 - n0 * a.P;
+    const bool together = (p0 + 7 < a.P) && (gp0 + 7 < a.rows);
+    auto expand = [&](unsigned char* tile, int kb) {
+        const int64_t c0 = (int64_t)kb * kABk + 8 * cg;
+        if constexpr (NHWC) {
+            const int count = (int)min((int64_t)8, a.C - c0);
+#pragma unroll
+            for (int r = 0; r < 8; ++r) {
+                const uint32_t row = (tid >> 3) + 16u * r;
+                const int64_t gp = row0 + row;
+                uint64_t v = 0;
+                if (gp < a.rows && count > 0) v = a_codes8(a.packed, gp * a.C + c0, bits, count, a.nwords);
+                uint32_t w[4];
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    const uint32_t e0 = (uint32_t)v & code_mask;
+                    v >>= bits;
+                    const uint32_t e1 = (uint32_t)v & code_mask;
+                    v >>= bits;
+                    w[h] = a_pair_bf16(e0, e1, wide);
+                }
+                a_store_chunk(tile, row, cg, w);
+            }
+        } else {
+            uint64_t v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i) {
+                const int64_t c = c0 + i;
+                v[i] = 0;
+                if (c < a.C && gp0 < a.rows) {
+                    if (together) {
+                        v[i] = a_codes8(a.packed, (n0 * a.C + c) * a.P + p0, bits, 8, a.nwords);
+                    } else {                                     // a sample boundary or the end of the batch inside
+                        for (int j = 0; j < 8; ++j) {
+                            const int64_t gp = gp0 + j;
+                            if (gp < a.rows) {
+                                const int64_t n = gp / a.P, p = gp - n * a.P;
+                                v[i] |= (uint64_t)a_code_at(a.packed, (n * a.C + c) * a.P + p, bits) << (j * bits);
+                            }
+                        }
+                    }
+                }
+            }
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                uint32_t w[4];
+#pragma unroll
+                for (int h = 0; h < 4; ++h) {
+                    w[h] = a_pair_bf16((uint32_t)v[2 * h] & code_mask, (uint32_t)v[2 * h + 1] & code_mask, wide);
+                    v[2 * h] >>= bits;
+                    v[2 * h + 1] >>= bits;
+                }
+                a_store_chunk(tile, 8u * (tid >> 3) + j, cg, w);
+            }
+        }
+    };
+
+    // ---- main loop over the K blocks: expand the codes, load the weights, multiply ----
+    const uint32_t idesc = a_instr_desc(BN);
+    bool ok = true;
+    for (int kb = 0; kb < a.kblocks; ++kb) {
+        const int s = kb % a.stages;
+        if (kb >= a.stages) {            // the MMAs that read this stage have completed
+            ok = __syncthreads_and(wait(&s_empty[s], (uint32_t)((kb / a.stages - 1) & 1)) ? 1 : 0) != 0;
+            if (!ok) break;
+        }
+        unsigned char* st = stages + (size_t)s * kStageBytes;
+        if (tid == 0) {
+            a_mbar_expect_tx(&s_full[s], 2 * kBBytes);
             a_tma_load_2d(st + kABytes, &map_hi, kb * kABk, col0, &s_full[s]);
             a_tma_load_2d(st + kABytes + kBBytes, &map_lo, kb * kABk, col0, &s_full[s]);
         }
-    } else if (warp == 1 && lane == 0) {
-        // ---- MMA issuer: per stage 4 K steps of 16, each against the hi and the lo half of the weights ----
-        const uint32_t idesc = a_instr_desc(BN);
-        bool ok = true;
-        for (int kb = 0; kb < a.kblocks && ok; ++kb) {
-            const int s = kb % a.stages;
-            ok = wait(&s_full[s], (uint32_t)((kb / a.stages) & 1));
-            if (!ok) break;
-            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-            unsigned char* st = stages + (size_t)s * kStageBytes;
-            const uint64_t dq = a_smem_desc(st), dh = a_smem_desc(st + kABytes), dl = a_smem_desc(st + kABytes + kBBytes);
+        expand(st, kb);
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the stores above, for the tensor core
+        __syncthreads();
+        if (tid == 32) {
+            // per stage 4 K steps of 16, each against the hi and the lo half of the weights
+            if (wait(&s_full[s], (uint32_t)((kb / a.stages) & 1))) {
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t dq = a_smem_desc(st), dh = a_smem_desc(st + kABytes), dl = a_smem_desc(st + kABytes + kBBytes);
 #pragma unroll
-            for (int k = 0; k < kABk / 16; ++k) {        // 16 bf16 = 32 bytes = 2 sixteen-byte units along K
-                a_mma(tmem, dq + 2 * k, dh + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                a_mma(tmem, dq + 2 * k, dl + 2 * k, idesc, 1u);
+                for (int k = 0; k < kABk / 16; ++k) {        // 16 bf16 = 32 bytes = 2 sixteen-byte units along K
+                    a_mma(tmem, dq + 2 * k, dh + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    a_mma(tmem, dq + 2 * k, dl + 2 * k, idesc, 1u);
+                }
+                a_commit(&s_empty[s]);       // the stage may be refilled once these MMAs have read it
+                if (kb + 1 == a.kblocks) a_commit(&s_done);      // the accumulator is final when this arrives
             }
-            a_commit(&s_empty[s]);       // the stage may be refilled once these MMAs have read it
         }
-        a_commit(&s_done);               // arrives when every MMA has completed: the accumulator is final
     }
     __syncwarp();
 
     // ---- epilogue: warp w reads lanes 32 w .. 32 w + 31 of the accumulator, 32 columns at a time ----
-    const bool done = wait(&s_done, 0);
+    const bool done = ok && wait(&s_done, 0);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-    const int64_t gp = (int64_t)row0 + warp * 32 + lane;      // this thread's pixel, over the whole batch
+    const int64_t gp = row0 + warp * 32 + lane;      // this thread's pixel, over the whole batch
     const int64_t n = gp / a.P, p = gp - n * a.P;
 #pragma unroll 1
     for (int c = 0; c < BN; c += 32) {
@@ -211,7 +333,7 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 const int64_t o = (int64_t)col0 + c + j;
                 if (o < a.O) {
                     const float val = __fsub_rn(__uint_as_float(v[j]), __ldg(a.bias + o));
-                    if (a.channels_last) a.y[gp * a.O + o] = val;
+                    if constexpr (NHWC) a.y[gp * a.O + o] = val;
                     else a.y[(n * a.O + o) * a.P + p] = val;
                 }
             }
@@ -257,63 +379,6 @@ __global__ void accumulate_weights_kernel(const float* __restrict__ w, const flo
     }
 }
 
-// code e of a bit string of b-bit codes (element e in bits [e*b, (e+1)*b), little-endian words)
-__device__ __forceinline__ uint32_t a_code_at(const uint32_t* __restrict__ packed, int64_t e, int bits) {
-    const int64_t bit = e * bits;
-    const int64_t word = bit >> 5;
-    const int sh = (int)(bit & 31);
-    uint32_t v = __ldg(packed + word) >> sh;
-    if (sh + bits > 32) v |= __ldg(packed + word + 1) << (32 - sh);
-    return v & ((1u << bits) - 1u);
-}
-
-// NCHW codes -> bf16 matrix [N * P, Cpad] (channels-last): tiles of 32 channels x 256 pixels transposed through
-// shared memory; a thread extracts 32 codes, then writes 4 times 8 channels of one pixel as one 16-byte store
-constexpr int kUPix = 256;
-__global__ void __launch_bounds__(256) accumulate_codes_nchw_kernel(const uint32_t* __restrict__ packed, int bits,
-                                                                    int64_t C, int64_t P, int64_t Cpad,
-                                                                    __nv_bfloat16* __restrict__ q) {
-    __shared__ uint8_t tile[32][kUPix + 4];
-    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-    const int64_t n = blockIdx.z, c0 = (int64_t)blockIdx.y * 32, p0 = (int64_t)blockIdx.x * kUPix;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const int cc = ty + 8 * i;
-        const int64_t c = c0 + cc;
-#pragma unroll
-        for (int j = 0; j < kUPix / 32; ++j) {
-            const int64_t p = p0 + j * 32 + tx;
-            tile[cc][j * 32 + tx] = (c < C && p < P) ? (uint8_t)a_code_at(packed, (n * C + c) * P + p, bits) : (uint8_t)0;
-        }
-    }
-    __syncthreads();
-    // 256 pixels x 4 groups of 8 channels = 1024 stores of 16 bytes, 4 per thread; the 4 groups of a pixel are 64
-    // contiguous bytes of its row
-    for (int k = threadIdx.x; k < kUPix * 4; k += 256) {
-        const int pp = k >> 2, g8 = (k & 3) * 8;
-        const int64_t p = p0 + pp, c = c0 + g8;
-        if (p >= P || c >= Cpad) continue;
-        uint32_t w[4];
-#pragma unroll
-        for (int h = 0; h < 4; ++h) {
-            const uint32_t lo = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn((float)tile[g8 + 2 * h][pp]));
-            const uint32_t hi = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn((float)tile[g8 + 2 * h + 1][pp]));
-            w[h] = lo | (hi << 16);
-        }
-        *reinterpret_cast<uint4*>(q + (n * P + p) * Cpad + c) = make_uint4(w[0], w[1], w[2], w[3]);
-    }
-}
-
-// channels-last codes -> bf16 matrix [rows, Cpad]
-__global__ void accumulate_codes_nhwc_kernel(const uint32_t* __restrict__ packed, int bits, int64_t rows, int64_t C,
-                                             int64_t Cpad, __nv_bfloat16* __restrict__ q) {
-    const int64_t total = rows * Cpad;
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t r = i / Cpad, c = i - r * Cpad;
-        q[i] = __float2bfloat16_rn(c < C ? (float)a_code_at(packed, r * C + c, bits) : 0.0f);
-    }
-}
-
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -333,7 +398,7 @@ bool a_make_map(EncodeTiledFn encode, CUtensorMap* map, const void* base, uint64
 
 struct ALayout {
     int64_t N, C, P, Cpad, rows;
-    size_t off_q, off_hi, off_lo, off_bias, total;
+    size_t off_hi, off_lo, off_bias, total;
 };
 
 bool a_layout(const int64_t dims[4], int channel_axis, int64_t O, ALayout& L) {
@@ -347,24 +412,22 @@ bool a_layout(const int64_t dims[4], int channel_axis, int64_t O, ALayout& L) {
     L.Cpad = (L.C + 7) & ~7ll;                 // rows of 16-byte multiples for the tile loads
     L.rows = L.N * L.P;
     auto up = [](size_t v) { return (v + 255) & ~(size_t)255; };
-    L.off_q = 256;
-    L.off_hi = L.off_q + up((size_t)L.rows * L.Cpad * 2);
+    L.off_hi = 256;
     L.off_lo = L.off_hi + up((size_t)O * L.Cpad * 2);
     L.off_bias = L.off_lo + up((size_t)O * L.Cpad * 2);
     L.total = L.off_bias + up((size_t)O * 4);
     return true;
 }
 
-template <int BN>
-cudaError_t a_launch(const CUtensorMap& mq, const CUtensorMap& mh, const CUtensorMap& ml, const AArgs& args,
-                     cudaStream_t st) {
+template <int BN, bool NHWC>
+cudaError_t a_launch(const CUtensorMap& mh, const CUtensorMap& ml, const AArgs& args, cudaStream_t st) {
     // a short ring leaves room for several CTAs per SM, whose load / multiply / store chains then overlap
     const size_t smem = (size_t)args.stages * (kABm * kABk * 2 + 2 * BN * kABk * 2) + 1024;
-    auto kern = accumulate_kernel<BN>;
+    auto kern = accumulate_kernel<BN, NHWC>;
     cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     const dim3 grid((unsigned)((args.rows + kABm - 1) / kABm), (unsigned)((args.O + BN - 1) / BN));
-    kern<<<grid, kAThreads, smem, st>>>(mq, mh, ml, args);
+    kern<<<grid, kAThreads, smem, st>>>(mh, ml, args);
     return cudaGetLastError();
 }
 
@@ -399,14 +462,12 @@ extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_
         return GRANQ_ERR_CUDA;
     EncodeTiledFn encode = (EncodeTiledFn)fn;
     char* ws = (char*)workspace;
-    __nv_bfloat16* q = (__nv_bfloat16*)(ws + L.off_q);
     __nv_bfloat16* hi = (__nv_bfloat16*)(ws + L.off_hi);
     __nv_bfloat16* lo = (__nv_bfloat16*)(ws + L.off_lo);
     float* bias = (float*)(ws + L.off_bias);
     const int BN = out_channels <= 64 ? 64 : 128;
-    CUtensorMap mq, mh, ml;
-    if (!a_make_map(encode, &mq, q, (uint64_t)L.rows, (uint64_t)L.Cpad, kABm) ||
-        !a_make_map(encode, &mh, hi, (uint64_t)out_channels, (uint64_t)L.Cpad, (uint32_t)BN) ||
+    CUtensorMap mh, ml;
+    if (!a_make_map(encode, &mh, hi, (uint64_t)out_channels, (uint64_t)L.Cpad, (uint32_t)BN) ||
         !a_make_map(encode, &ml, lo, (uint64_t)out_channels, (uint64_t)L.Cpad, (uint32_t)BN))
         return GRANQ_ERR_CUDA;
 
@@ -414,27 +475,24 @@ extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_
     if (e != cudaSuccess) return GRANQ_ERR_CUDA;
     accumulate_weights_kernel<<<(unsigned)out_channels, 128, 0, st>>>(weights, scale, zp, (int)L.C, (int)L.Cpad, hi, lo,
                                                                     bias);
-    if (channel_axis == 1) {
-        const dim3 grid((unsigned)((L.P + kUPix - 1) / kUPix), (unsigned)((L.Cpad + 31) / 32), (unsigned)L.N);
-        if (grid.y > 65535 || grid.z > 65535) return GRANQ_ERR_UNSUPPORTED;
-        accumulate_codes_nchw_kernel<<<grid, 256, 0, st>>>(packed_codes, bits, L.C, L.P, L.Cpad, q);
-    } else {
-        const int64_t total = L.rows * L.Cpad;
-        const unsigned blocks = (unsigned)std::min<int64_t>((total + 255) / 256, 148 * 16);
-        accumulate_codes_nhwc_kernel<<<blocks, 256, 0, st>>>(packed_codes, bits, L.rows, L.C, L.Cpad, q);
-    }
     if (cudaGetLastError() != cudaSuccess) return GRANQ_ERR_CUDA;
     AArgs args{};
     args.y = y;
     args.bias = bias;
     args.status = (uint32_t*)workspace;
+    args.packed = packed_codes;
+    args.nwords = (L.rows * L.C * bits + 31) / 32;
     args.rows = L.rows;
     args.P = L.P;
+    args.C = L.C;
     args.O = out_channels;
+    args.bits = bits;
     args.kblocks = (int)((L.Cpad + kABk - 1) / kABk);
-    args.channels_last = channel_axis == 3 ? 1 : 0;
     args.spin_limit = kASpin;
     args.stages = std::min(args.kblocks, 2);
-    e = BN == 64 ? a_launch<64>(mq, mh, ml, args, st) : a_launch<128>(mq, mh, ml, args, st);
+    if (channel_axis == 3)
+        e = BN == 64 ? a_launch<64, true>(mh, ml, args, st) : a_launch<128, true>(mh, ml, args, st);
+    else
+        e = BN == 64 ? a_launch<64, false>(mh, ml, args, st) : a_launch<128, false>(mh, ml, args, st);
     return e == cudaSuccess ? GRANQ_OK : GRANQ_ERR_CUDA;
 }
