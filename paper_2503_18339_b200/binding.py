@@ -570,10 +570,11 @@ def accumulate_workspace_bytes(shape, channel_axis: int, out_channels: int) -> i
 
 def granq_accumulate_codes(packed_codes: torch.Tensor, shape, bits: int, s: torch.Tensor, z: torch.Tensor,
                            weights: torch.Tensor, channel_axis: int = 1, y: torch.Tensor = None,
-                           workspace: torch.Tensor = None, stream=None):
+                           workspace: torch.Tensor = None, flags: int = 0, stream=None):
     """Eq. 6 left-hand side / Algorithm 1 output step, pointwise case, from the packed integer codes of a
     tensor of `shape` (NCHW for channel_axis 1, N H W C for 3): y = sum_c w[o, c] * s_c * (code - z_c), fp32.
-    Returns (y, workspace); the workspace's status word tells whether a bounded wait ran out."""
+    Returns (y, workspace); the workspace's status word tells whether a bounded wait ran out.
+    flags: FLAG_FORCE_TWO_PASS takes the kernel with one tile per CTA instead of the persistent one."""
     shape = tuple(int(d) for d in shape)
     if weights.dtype != torch.float32 or weights.dim() != 2 or weights.shape[1] != shape[channel_axis]:
         raise ValueError("weights must be float32 [out_channels, C]")
@@ -586,7 +587,7 @@ def granq_accumulate_codes(packed_codes: torch.Tensor, shape, bits: int, s: torc
                                 device=packed_codes.device)
     _check(lib().granq_accumulate_codes(_dev(packed_codes, "packed_codes"), _dims(shape), channel_axis, bits,
                                         _dev(s, "s"), _dev(z, "z"), _dev(weights, "weights"), o, _dev(y, "y"),
-                                        _dev(workspace, "workspace"), workspace.numel(), 0, _stream(stream)),
+                                        _dev(workspace, "workspace"), workspace.numel(), flags, _stream(stream)),
            "granq_accumulate_codes")
     return y, workspace
 

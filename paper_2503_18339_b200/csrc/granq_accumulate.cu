@@ -60,6 +60,9 @@ __device__ __forceinline__ bool a_mbar_try_wait(uint64_t* bar, uint32_t parity) 
         : "memory");
     return ok != 0;
 }
+__device__ __forceinline__ void a_mbar_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(a_smem_u32(bar)) : "memory");
+}
 // 2-d tile load of this GPU's own memory (no multicast): coordinates (x = innermost element, y = row)
 __device__ __forceinline__ void a_tma_load_2d(void* dst_smem, const CUtensorMap* map, int x, int y, uint64_t* bar) {
     asm volatile(
@@ -139,6 +142,24 @@ __device__ __forceinline__ uint64_t a_codes8(const uint32_t* __restrict__ packed
     return keep >= 64 ? v : (v & ((1ull << keep) - 1ull));
 }
 
+// The same in two steps, so that the loads can be issued long before their words are needed: a_codes8_load() only
+// loads (up to three words, none beyond the end of the bit string) and returns the shift; a_codes8_finish() lines
+// the codes up at bit 0 and clears what lies above them.
+__device__ __forceinline__ uint32_t a_codes8_load(const uint32_t* __restrict__ packed, uint64_t bit, uint32_t nbits,
+                                                  int64_t nwords, uint32_t& w0, uint32_t& w1, uint32_t& w2) {
+    const int64_t w = (int64_t)(bit >> 5);
+    const uint32_t sh = (uint32_t)bit & 31u;
+    const uint32_t need = sh + nbits;
+    w0 = __ldg(packed + w);
+    w1 = (need > 32 && w + 1 < nwords) ? __ldg(packed + w + 1) : 0u;
+    w2 = (need > 64 && w + 2 < nwords) ? __ldg(packed + w + 2) : 0u;
+    return sh;
+}
+__device__ __forceinline__ uint64_t a_codes8_finish(uint32_t w0, uint32_t w1, uint32_t w2, uint32_t sh, int keep_bits) {
+    const uint64_t v = ((uint64_t)__funnelshift_r(w1, w2, sh) << 32) | __funnelshift_r(w0, w1, sh);
+    return keep_bits >= 64 ? v : (v & ((1ull << keep_bits) - 1ull));
+}
+
 // two codes -> two bf16 in one word (the first in the low half), exact.  Codes below 128: 0x4300 | code is the
 // bf16 number 128 + code, and one packed subtraction of 128 gives the code; 8-bit codes go through fp32.
 __device__ __forceinline__ uint32_t a_pair_bf16(uint32_t c0, uint32_t c1, bool wide) {
@@ -205,6 +226,13 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_const
         atomicExch(a.status, kATimeout);
         *(volatile uint32_t*)&s_abort = 1;
         return false;
+    };
+    // the same for a whole warp: one lane polls (hundreds of threads polling one barrier word keep the shared-memory
+    // atomic unit busy for a microsecond per hand-over), the shuffle hands the outcome and the ordering to the rest
+    auto warp_wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+        uint32_t ok = 0;
+        if (lane == 0) ok = wait(bar, parity) ? 1u : 0u;
+        return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
     };
 
     // ---- this thread's share of a tile of codes: 8 of its 1024 sixteen-byte chunks ----
@@ -278,7 +306,7 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_const
     for (int kb = 0; kb < a.kblocks; ++kb) {
         const int s = kb % a.stages;
         if (kb >= a.stages) {            // the MMAs that read this stage have completed
-            ok = __syncthreads_and(wait(&s_empty[s], (uint32_t)((kb / a.stages - 1) & 1)) ? 1 : 0) != 0;
+            ok = __syncthreads_and(warp_wait(&s_empty[s], (uint32_t)((kb / a.stages - 1) & 1)) ? 1 : 0) != 0;
             if (!ok) break;
         }
         unsigned char* st = stages + (size_t)s * kStageBytes;
@@ -308,7 +336,7 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_const
     __syncwarp();
 
     // ---- epilogue: warp w reads lanes 32 w .. 32 w + 31 of the accumulator, 32 columns at a time ----
-    const bool done = ok && wait(&s_done, 0);
+    const bool done = ok && warp_wait(&s_done, 0);
     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
     const int64_t gp = row0 + warp * 32 + lane;      // this thread's pixel, over the whole batch
     const int64_t n = gp / a.P, p = gp - n * a.P;
@@ -343,6 +371,321 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_const
     __syncthreads();
     if (warp == 1)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
+}
+
+// ---- the persistent form: one CTA per SM walks over row tiles, its warps split into three roles ----
+//   warps 0 .. 7   two groups of 128 threads expand codes into a ring of operand stages, turn and turn about
+//                  (the words of a group's next stage are loaded before the current one is converted);
+//   warp  8        one thread loads both weight halves for all K blocks once (TMA) and issues every MMA;
+//   warps 9 .. 16  read a finished accumulator out of tensor memory (a warp reads the 32 lanes of its quarter,
+//                  warp % 4, and one half of the columns), subtract the bias and store y.
+// The CTA owns all 512 columns of its SM's tensor memory: 512 / BN accumulators in turn, so the MMAs run several
+// tiles ahead of the epilogue (a hand-over from the tensor core to the epilogue and back costs about a
+// microsecond; with two accumulators that latency, not the work, set the pace).  Needs the weight halves of
+// all K blocks resident in shared memory.
+constexpr int kPStages = 6;               // operand stages of 128 x 64 codes
+constexpr int kPTmemCols = 512;           // all of an SM's tensor memory
+constexpr int kPProducers = 256;          // threads that expand codes
+constexpr int kPEpilogue = 256;           // threads that read accumulators out and store y
+constexpr int kPThreads = kPProducers + 32 + kPEpilogue;
+constexpr size_t kPWeightBytes = 128 * 1024;      // resident weight halves at most
+
+struct PBars {
+    uint64_t a_full[kPStages], a_empty[kPStages], acc_full[8], acc_empty[8], b_full;
+};
+
+template <int BN, bool NHWC>
+__global__ void __launch_bounds__(kPThreads, 1)
+accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
+                             const AArgs a) {
+    constexpr uint32_t kABytes = kABm * kABk * 2, kBBytes = BN * kABk * 2;
+    constexpr int kAcc = kPTmemCols / BN;          // accumulators
+    static_assert(kAcc <= 8, "barriers for at most 8 accumulators");
+    extern __shared__ __align__(1024) unsigned char a_smem[];
+    __shared__ __align__(8) PBars bars;
+    __shared__ float s_bias[BN];
+    __shared__ uint32_t s_tmem, s_abort;
+    const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    unsigned char* ring = a_smem + ((1024u - (a_smem_u32(a_smem) & 1023u)) & 1023u);
+    unsigned char* wts = ring + (size_t)kPStages * kABytes;          // per K block: hi half, lo half
+    const int col0 = (int)blockIdx.y * BN;
+    const int64_t row_tiles = (a.rows + kABm - 1) / kABm;
+    const int kblocks = a.kblocks;
+    // this CTA's row tiles: blockIdx.x, blockIdx.x + gridDim.x, ...
+    const int my_tiles = (int)((row_tiles - (int64_t)blockIdx.x + gridDim.x - 1) / gridDim.x);
+    const int my_iters = my_tiles * kblocks;
+
+    if (tid == 0) {
+        for (int s = 0; s < kPStages; ++s) {
+            a_mbar_init(&bars.a_full[s], 4);                 // one arrival per warp of a producer group
+            a_mbar_init(&bars.a_empty[s], 1);
+        }
+        for (int b = 0; b < kAcc; ++b) {
+            a_mbar_init(&bars.acc_full[b], 1);
+            a_mbar_init(&bars.acc_empty[b], kPEpilogue / 32);     // one arrival per epilogue warp
+        }
+        a_mbar_init(&bars.b_full, 1);
+        s_abort = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    for (int i = tid; i < BN; i += kPThreads) s_bias[i] = (col0 + i < a.O) ? a.bias[col0 + i] : 0.0f;
+    if (warp == 8) {       // kAcc accumulators of BN columns each
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(a_smem_u32(&s_tmem)),
+                     "r"((uint32_t)kPTmemCols)
+                     : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = s_tmem;
+
+    // bounded wait; false when it ran out or another thread of this CTA has given up
+    auto wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+        for (uint32_t i = 0; i < a.spin_limit; ++i) {
+            if (a_mbar_try_wait(bar, parity)) return true;
+            if ((i & 1023u) == 1023u && *(volatile uint32_t*)&s_abort) return false;
+        }
+        atomicExch(a.status, kATimeout);
+        *(volatile uint32_t*)&s_abort = 1;
+        return false;
+    };
+    // the same for a whole warp: one lane polls (hundreds of threads polling one barrier word keep the shared-memory
+    // atomic unit busy for a microsecond per hand-over), the shuffle hands the outcome and the ordering to the rest
+    auto warp_wait = [&](uint64_t* bar, uint32_t parity) -> bool {
+        uint32_t ok = 0;
+        if (lane == 0) ok = wait(bar, parity) ? 1u : 0u;
+        return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
+    };
+
+    if (warp < 8) {
+        // ---- producers: group g takes the iterations (tile, K block) with it % 2 == g ----
+        const uint32_t group = tid >> 7, pt = tid & 127;
+        const int bits = a.bits;
+        const bool wide = bits == 8;
+        const uint32_t code_mask = (1u << bits) - 1u;
+        const uint32_t cg = pt & 7, rq = pt >> 3;          // 8 channels of the stage's 64; row group
+        // The eight code strings of this thread for iteration `it`, as loaded words (three per string) and shifts
+        // (5 bits each).  NCHW: 8 channels x rows 8 rq .. 8 rq + 7 (code j of string i = channel i, row j);
+        // channels-last: rows rq + 16 r x 8 channels (string r = row).
+        struct Raw {
+            uint32_t w0[8], w1[8], w2[8];
+            uint64_t shifts;
+            int keep;                 // bits of a string that hold codes
+        };
+        // (pixel counts are below 2^31: 32-bit index arithmetic; only bit offsets need 64 bits)
+        const uint32_t rows32 = (uint32_t)a.rows, P32 = (uint32_t)a.P, C32 = (uint32_t)a.C;
+        auto fetch = [&](int it, Raw& r) {
+            const int ti = it / kblocks, kb = it - ti * kblocks;
+            const uint32_t row0 = (blockIdx.x + (uint32_t)ti * gridDim.x) * (uint32_t)kABm;
+            const uint32_t c0 = (uint32_t)kb * kABk + 8u * cg;
+            r.shifts = 0;
+            if constexpr (NHWC) {
+                const uint32_t count = c0 < C32 ? min(8u, C32 - c0) : 0u;
+                r.keep = (int)count * bits;
+                uint64_t bit = ((uint64_t)(row0 + rq) * C32 + c0) * (uint32_t)bits;
+                const uint64_t step = (uint64_t)16 * C32 * (uint32_t)bits;           // 16 rows on
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    r.w0[i] = r.w1[i] = r.w2[i] = 0;
+                    if (row0 + rq + 16u * i < rows32 && count > 0)
+                        r.shifts |= (uint64_t)a_codes8_load(a.packed, bit, (uint32_t)r.keep, a.nwords, r.w0[i], r.w1[i], r.w2[i])
+                                    << (5 * i);
+                    bit += step;
+                }
+            } else {
+                const uint32_t gp0 = row0 + 8u * rq;
+                const uint32_t n0 = gp0 / P32, p0 = gp0 - n0 * P32;
+                const bool together = (p0 + 7 < P32) && (gp0 + 7 < rows32);
+                r.keep = 8 * bits;
+                uint64_t bit = (((uint64_t)n0 * C32 + c0) * P32 + p0) * (uint32_t)bits;
+                const uint64_t step = (uint64_t)P32 * (uint32_t)bits;                 // one channel on
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const uint32_t c = c0 + i;
+                    r.w0[i] = r.w1[i] = r.w2[i] = 0;
+                    if (c < C32 && gp0 < rows32) {
+                        if (together) {
+                            r.shifts |= (uint64_t)a_codes8_load(a.packed, bit, (uint32_t)r.keep, a.nwords, r.w0[i], r.w1[i],
+                                                                r.w2[i])
+                                        << (5 * i);
+                        } else {                                 // a sample boundary or the end of the batch inside
+                            uint64_t v = 0;
+                            for (uint32_t j = 0; j < 8; ++j) {
+                                const uint32_t gp = gp0 + j;
+                                if (gp < rows32) {
+                                    const uint32_t n = gp / P32, p = gp - n * P32;
+                                    v |= (uint64_t)a_code_at(a.packed, ((int64_t)n * C32 + c) * P32 + p, bits) << (j * bits);
+                                }
+                            }
+                            r.w0[i] = (uint32_t)v;
+                            r.w1[i] = (uint32_t)(v >> 32);
+                        }
+                    }
+                    bit += step;
+                }
+            }
+        };
+        auto store = [&](unsigned char* tile, const Raw& r) {
+            uint64_t v[8];
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+                v[i] = a_codes8_finish(r.w0[i], r.w1[i], r.w2[i], (uint32_t)(r.shifts >> (5 * i)) & 31u, r.keep);
+            if constexpr (NHWC) {
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        const uint32_t e0 = (uint32_t)v[i] & code_mask;
+                        v[i] >>= bits;
+                        const uint32_t e1 = (uint32_t)v[i] & code_mask;
+                        v[i] >>= bits;
+                        w[h] = a_pair_bf16(e0, e1, wide);
+                    }
+                    a_store_chunk(tile, rq + 16u * i, cg, w);
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < 8; ++j) {
+                    uint32_t w[4];
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {
+                        w[h] = a_pair_bf16((uint32_t)v[2 * h] & code_mask, (uint32_t)v[2 * h + 1] & code_mask, wide);
+                        v[2 * h] >>= bits;
+                        v[2 * h + 1] >>= bits;
+                    }
+                    a_store_chunk(tile, 8u * rq + j, cg, w);
+                }
+            }
+        };
+        // the words of this group's next iteration are in flight while the current one is converted and stored
+        // (two sets of registers, used turn and turn about)
+        Raw ra, rb;
+        auto step = [&](int it, Raw& now, Raw& next) -> bool {
+            if (it + 2 < my_iters) fetch(it + 2, next);
+            const int s = it % kPStages;
+            // the MMAs that read this stage kPStages iterations ago have completed (passes at once the first time round)
+            if (!warp_wait(&bars.a_empty[s], (uint32_t)(((it / kPStages) & 1) ^ 1))) return false;
+            store(ring + (size_t)s * kABytes, now);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the stores above, for the tensor core
+            __syncwarp();
+            if (lane == 0) a_mbar_arrive(&bars.a_full[s]);
+            return true;
+        };
+        int it = (int)group;
+        if (it < my_iters) fetch(it, ra);
+        for (; it < my_iters; it += 4) {
+            if (!step(it, ra, rb)) break;
+            if (it + 2 < my_iters && !step(it + 2, rb, ra)) break;
+        }
+    } else if (warp == 8) {
+        if (lane == 0) {
+            // ---- weights once, then every MMA: per K block 4 steps of 16, each against the hi and the lo half ----
+            a_mbar_expect_tx(&bars.b_full, (uint32_t)(2 * kBBytes) * (uint32_t)kblocks);
+            for (int kb = 0; kb < kblocks; ++kb) {
+                a_tma_load_2d(wts + (size_t)kb * 2 * kBBytes, &map_hi, kb * kABk, col0, &bars.b_full);
+                a_tma_load_2d(wts + (size_t)kb * 2 * kBBytes + kBBytes, &map_lo, kb * kABk, col0, &bars.b_full);
+            }
+            const uint32_t idesc = a_instr_desc(BN);
+            bool ok = wait(&bars.b_full, 0);
+            int it = 0;
+            for (int t = 0; t < my_tiles && ok; ++t) {
+                const uint32_t buf = (uint32_t)(t % kAcc);
+                // the epilogue has read this accumulator out (passes at once the first time round)
+                ok = wait(&bars.acc_empty[buf], (uint32_t)(((t / kAcc) & 1) ^ 1));
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                for (int kb = 0; kb < kblocks; ++kb, ++it) {
+                    const int s = it % kPStages;
+                    ok = wait(&bars.a_full[s], (uint32_t)((it / kPStages) & 1));
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t dq = a_smem_desc(ring + (size_t)s * kABytes);
+                    const uint64_t dh = a_smem_desc(wts + (size_t)kb * 2 * kBBytes);
+                    const uint64_t dl = a_smem_desc(wts + (size_t)kb * 2 * kBBytes + kBBytes);
+#pragma unroll
+                    for (int k = 0; k < kABk / 16; ++k) {    // 16 bf16 = 32 bytes = 2 sixteen-byte units along K
+                        a_mma(tmem + buf * BN, dq + 2 * k, dh + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        a_mma(tmem + buf * BN, dq + 2 * k, dl + 2 * k, idesc, 1u);
+                    }
+                    a_commit(&bars.a_empty[s]);       // the stage may be refilled once these MMAs have read it
+                }
+                if (ok) a_commit(&bars.acc_full[buf]);       // the accumulator is final when this arrives
+            }
+        }
+        __syncwarp();
+    } else {
+        // ---- epilogue: a warp reads lanes 32 q .. 32 q + 31 (q = warp % 4) and one half of the columns ----
+        const uint32_t q = warp & 3u;
+        const int chalf = (int)((warp - 9u) >> 2) * (BN / 2);
+        for (int t = 0; t < my_tiles; ++t) {
+            const uint32_t buf = (uint32_t)(t % kAcc);
+            if (!warp_wait(&bars.acc_full[buf], (uint32_t)((t / kAcc) & 1))) break;
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const uint32_t gp = (blockIdx.x + (uint32_t)t * gridDim.x) * (uint32_t)kABm + q * 32u + lane;      // this thread's pixel
+            const uint32_t n = gp / (uint32_t)a.P, p = gp - n * (uint32_t)a.P;
+            const bool live = gp < (uint32_t)a.rows;
+            // this thread's element of output channel col0: the next channel is P (NCHW) or 1 (channels-last) further
+            float* const yrow = NHWC ? a.y + (size_t)gp * (size_t)a.O + col0
+                                     : a.y + ((size_t)n * (size_t)a.O + col0) * (size_t)a.P + p;
+#pragma unroll 1
+            for (int c = chalf; c < chalf + BN / 2; c += 32) {
+                uint32_t v[32];
+                const uint32_t taddr = tmem + ((q * 32u) << 16) + buf * BN + (uint32_t)c;
+                asm volatile(
+                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+                    "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
+                    "%29,%30,%31}, [%32];"
+                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+                      "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+                      "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+                      "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+                    : "r"(taddr)
+                    : "memory");
+                asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+                if (c + 32 >= chalf + BN / 2) {          // this warp's part is in registers: hand the accumulator back
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0) a_mbar_arrive(&bars.acc_empty[buf]);
+                }
+                if (live) {
+                    if constexpr (NHWC) {
+                        float* out = yrow + c;
+                        if ((a.O & 3) == 0 && col0 + c + 32 <= a.O && ((uintptr_t)a.y & 15) == 0) {      // 16-byte aligned rows
+#pragma unroll
+                            for (int j = 0; j < 32; j += 4) {
+                                float4 f;
+                                f.x = __fsub_rn(__uint_as_float(v[j]), s_bias[c + j]);
+                                f.y = __fsub_rn(__uint_as_float(v[j + 1]), s_bias[c + j + 1]);
+                                f.z = __fsub_rn(__uint_as_float(v[j + 2]), s_bias[c + j + 2]);
+                                f.w = __fsub_rn(__uint_as_float(v[j + 3]), s_bias[c + j + 3]);
+                                *reinterpret_cast<float4*>(out + j) = f;
+                            }
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (col0 + c + j < a.O) out[j] = __fsub_rn(__uint_as_float(v[j]), s_bias[c + j]);
+                        }
+                    } else {
+                        float* out = yrow + (size_t)c * (size_t)a.P;
+                        const int left = (int)a.O - col0 - c;          // channels of this chunk that exist
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) {
+                            if (j < left) *out = __fsub_rn(__uint_as_float(v[j]), s_bias[c + j]);
+                            out += (uint32_t)a.P;
+                        }
+                    }
+                }
+            }
+        }
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 8)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kPTmemCols)
+                     : "memory");
 }
 
 // W' = w * s in fp32, split into hi + lo (bf16 each), rows padded with zeros to Cpad; one CTA per output channel.
@@ -431,6 +774,25 @@ cudaError_t a_launch(const CUtensorMap& mh, const CUtensorMap& ml, const AArgs& 
     return cudaGetLastError();
 }
 
+// the persistent form, when the weight halves of all K blocks fit beside the ring of stages
+template <int BN, bool NHWC>
+cudaError_t p_launch(const CUtensorMap& mh, const CUtensorMap& ml, const AArgs& args, cudaStream_t st) {
+    const size_t smem = (size_t)kPStages * kABm * kABk * 2 + (size_t)args.kblocks * 2 * BN * kABk * 2 + 1024;
+    auto kern = accumulate_persistent_kernel<BN, NHWC>;
+    cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    int dev = 0, sms = 0;
+    if ((e = cudaGetDevice(&dev)) != cudaSuccess) return e;
+    if ((e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const int64_t row_tiles = (args.rows + kABm - 1) / kABm;
+    const unsigned col_tiles = (unsigned)((args.O + BN - 1) / BN);
+    // one CTA per SM, shared out among the column tiles; no CTA without a row tile
+    const unsigned per_col = (unsigned)std::max<int64_t>(1, std::min<int64_t>(row_tiles, sms / (int)std::min<unsigned>(col_tiles, (unsigned)sms)));
+    const dim3 grid(per_col, col_tiles);
+    kern<<<grid, kPThreads, smem, st>>>(mh, ml, args);
+    return cudaGetLastError();
+}
+
 }  // namespace
 
 }  // namespace granq
@@ -447,7 +809,6 @@ extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_
                                       const float* scale, const float* zp, const float* weights, int64_t out_channels,
                                       float* y, void* workspace, size_t workspace_bytes, uint32_t flags,
                                       void* cuda_stream) {
-    (void)flags;
     ALayout L;
     if (!packed_codes || !scale || !zp || !weights || !y || bits < 1 || bits > 8 || ((uintptr_t)packed_codes & 3) ||
         !a_layout(dims, channel_axis, out_channels, L))
@@ -490,9 +851,17 @@ extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_
     args.kblocks = (int)((L.Cpad + kABk - 1) / kABk);
     args.spin_limit = kASpin;
     args.stages = std::min(args.kblocks, 2);
-    if (channel_axis == 3)
+    const bool persistent = !(flags & GRANQ_FLAG_FORCE_TWO_PASS) &&
+                            (size_t)args.kblocks * 2 * BN * kABk * 2 <= kPWeightBytes;
+    if (persistent) {
+        if (channel_axis == 3)
+            e = BN == 64 ? p_launch<64, true>(mh, ml, args, st) : p_launch<128, true>(mh, ml, args, st);
+        else
+            e = BN == 64 ? p_launch<64, false>(mh, ml, args, st) : p_launch<128, false>(mh, ml, args, st);
+    } else if (channel_axis == 3) {
         e = BN == 64 ? a_launch<64, true>(mh, ml, args, st) : a_launch<128, true>(mh, ml, args, st);
-    else
+    } else {
         e = BN == 64 ? a_launch<64, false>(mh, ml, args, st) : a_launch<128, false>(mh, ml, args, st);
+    }
     return e == cudaSuccess ? GRANQ_OK : GRANQ_ERR_CUDA;
 }

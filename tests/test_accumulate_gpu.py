@@ -34,7 +34,7 @@ def packed_words(codes: np.ndarray, bits: int) -> torch.Tensor:
     return torch.from_numpy(by.view(np.int32).copy()).cuda()
 
 
-def run(b, codes_nchw, bits, s, z, w, channels_last):
+def run(b, codes_nchw, bits, s, z, w, channels_last, flags=0):
     n, c, h, wd = codes_nchw.shape
     o = w.shape[0]
     src = np.ascontiguousarray(codes_nchw.transpose(0, 2, 3, 1)) if channels_last else codes_nchw
@@ -42,7 +42,7 @@ def run(b, codes_nchw, bits, s, z, w, channels_last):
     y = g.empty((n, h, wd, o) if channels_last else (n, o, h, wd), torch.float32)
     got, ws = b.granq_accumulate_codes(packed_words(src, bits), src.shape, bits, torch.from_numpy(s).cuda(),
                                        torch.from_numpy(z).cuda(), torch.from_numpy(w).cuda(),
-                                       channel_axis=3 if channels_last else 1, y=y)
+                                       channel_axis=3 if channels_last else 1, y=y, flags=flags)
     assert b.workspace_status(ws) == b.OK
     g.check()
     got = got.cpu().numpy().astype(np.float64)
@@ -63,6 +63,9 @@ SHAPES = [   # (N, C, H, W, O)
     (1, 256, 28, 28, 200),    # 4 K blocks (one full turn of the ring), 7 pixel tiles, 2 channel tiles
     (2, 384, 14, 14, 72),     # 6 K blocks: the ring wraps
     (5, 128, 7, 7, 512),      # tiles that straddle samples, 4 channel tiles
+    (32, 64, 56, 56, 64),     # 784 pixel tiles: a persistent CTA takes five or six, both accumulators and every
+                              # stage of the ring come round several times
+    (9, 72, 28, 28, 40),      # 56 tiles, 2 K blocks each (the second one 8 channels wide)
 ]
 
 
@@ -76,12 +79,13 @@ def test_accumulate_matches_the_oracle_within_the_derived_bound(b, shape, channe
     res = orc.fused(x, bits)                                       # codes, s, z by the oracle (signed data: z != 0)
     w = (rng.standard_normal((o, c)) / np.sqrt(c)).astype(np.float32)
     ref = orc.accumulate(res.codes, res.s, res.z, w)
-    got = run(b, res.codes, bits, res.s, res.z, w, channels_last)
     S, bias = bound(res.codes, res.s, res.z, w)
     tol = (2.0 ** -17 + c * 2.0 ** -22) * S + 2.0 ** -21 * (bias + np.abs(ref))
-    err = np.abs(got - ref)
-    assert np.all(err <= tol), f"max err/tol {np.max(err / np.maximum(tol, 1e-300)):.3f}"
-    assert np.max(err / np.maximum(tol, 1e-300)) < 0.5            # and in practice well inside it
+    for flags in (0, b.FLAG_FORCE_TWO_PASS):       # the persistent kernel (where the weights fit), one tile per CTA
+        got = run(b, res.codes, bits, res.s, res.z, w, channels_last, flags)
+        err = np.abs(got - ref)
+        assert np.all(err <= tol), f"max err/tol {np.max(err / np.maximum(tol, 1e-300)):.3f} (flags {flags})"
+        assert np.max(err / np.maximum(tol, 1e-300)) < 0.5            # and in practice well inside it
     # a dropped K block, a transposed operand or a missing bias would be far outside: the error is not trivially small
     assert np.max(np.abs(ref)) > 100 * np.max(tol)
 
@@ -98,8 +102,9 @@ def test_accumulate_is_exact_on_small_integers(b, channels_last):
     z = rng.integers(0, 2 ** bits, c).astype(np.float32)
     w = rng.integers(-8, 9, (o, c)).astype(np.float32)
     ref = orc.accumulate(codes, s, z, w)
-    got = run(b, codes, bits, s, z, w, channels_last)
-    assert np.array_equal(got, ref)
+    for flags in (0, b.FLAG_FORCE_TWO_PASS):
+        got = run(b, codes, bits, s, z, w, channels_last, flags)
+        assert np.array_equal(got, ref)
     # one-hot weights select the pre-scaled activation of one channel
     onehot = np.zeros((c, c), np.float32)
     onehot[np.arange(c), (np.arange(c) * 7) % c] = 1
