@@ -373,19 +373,35 @@ accumulate_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_const
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
 }
 
+// 16 consecutive columns of this warp's 32 lanes of tensor memory (lane = thread), not yet waited for
+__device__ __forceinline__ void a_tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15}, [%16];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]), "=r"(v[8]),
+          "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15])
+        : "r"(taddr)
+        : "memory");
+}
+
 // ---- the persistent form: one CTA per SM walks over row tiles, its warps split into three roles ----
-//   warps 0 .. 7   two groups of 128 threads expand codes into a ring of operand stages, turn and turn about
-//                  (the words of a group's next stage are loaded before the current one is converted);
-//   warp  8        one thread loads both weight halves for all K blocks once (TMA) and issues every MMA;
-//   warps 9 .. 16  read a finished accumulator out of tensor memory (a warp reads the 32 lanes of its quarter,
+//   warps 0 .. 15  four groups of 128 threads expand codes into a ring of operand stages, turn and turn about
+//                  (loading and converting is a chain of dependent integer instructions and memory latency, so
+//                  it is warps, not issue slots, that are short);
+//   warp  16       one thread loads both weight halves for all K blocks once (TMA) and issues every MMA
+//                  (4 per K block);
+//   warps 17 .. 24 read a finished accumulator out of tensor memory (a warp reads the 32 lanes of its quarter,
 //                  warp % 4, and one half of the columns), subtract the bias and store y.
-// The CTA owns all 512 columns of its SM's tensor memory: 512 / BN accumulators in turn, so the MMAs run several
+// Both weight halves sit one after the other in shared memory and are multiplied as ONE operand of 2 BN columns
+// (an MMA of 128 x 64 x 16 spends its time fetching the 128 x 16 code operand, not computing: with both halves
+// behind one fetch the tensor core is busy half as long); the epilogue adds the two column blocks.
+// The CTA owns all 512 columns of its SM's tensor memory: 512 / (2 BN) accumulators in turn, so the MMAs run
 // tiles ahead of the epilogue (a hand-over from the tensor core to the epilogue and back costs about a
 // microsecond; with two accumulators that latency, not the work, set the pace).  Needs the weight halves of
 // all K blocks resident in shared memory.
 constexpr int kPStages = 6;               // operand stages of 128 x 64 codes
 constexpr int kPTmemCols = 512;           // all of an SM's tensor memory
-constexpr int kPProducers = 256;          // threads that expand codes
+constexpr int kPGroups = 4;                // groups of 128 threads that expand codes, turn and turn about
+constexpr int kPProducers = 128 * kPGroups;
 constexpr int kPEpilogue = 256;           // threads that read accumulators out and store y
 constexpr int kPThreads = kPProducers + 32 + kPEpilogue;
 constexpr size_t kPWeightBytes = 128 * 1024;      // resident weight halves at most
@@ -399,7 +415,7 @@ __global__ void __launch_bounds__(kPThreads, 1)
 accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
                              const AArgs a) {
     constexpr uint32_t kABytes = kABm * kABk * 2, kBBytes = BN * kABk * 2;
-    constexpr int kAcc = kPTmemCols / BN;          // accumulators
+    constexpr int kAcc = kPTmemCols / (2 * BN);    // accumulators (each: BN columns for the hi half, BN for the lo half)
     static_assert(kAcc <= 8, "barriers for at most 8 accumulators");
     extern __shared__ __align__(1024) unsigned char a_smem[];
     __shared__ __align__(8) PBars bars;
@@ -430,7 +446,7 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     }
     for (int i = tid; i < BN; i += kPThreads) s_bias[i] = (col0 + i < a.O) ? a.bias[col0 + i] : 0.0f;
-    if (warp == 8) {       // kAcc accumulators of BN columns each
+    if (warp == kPProducers / 32) {       // kAcc accumulators of BN columns each
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(a_smem_u32(&s_tmem)),
                      "r"((uint32_t)kPTmemCols)
                      : "memory");
@@ -459,8 +475,8 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
         return __shfl_sync(0xFFFFFFFFu, ok, 0) != 0;
     };
 
-    if (warp < 8) {
-        // ---- producers: group g takes the iterations (tile, K block) with it % 2 == g ----
+    if (warp < kPProducers / 32) {
+        // ---- producers: group g takes the iterations (tile, K block) with it % kPGroups == g ----
         const uint32_t group = tid >> 7, pt = tid & 127;
         const int bits = a.bits;
         const bool wide = bits == 8;
@@ -476,11 +492,38 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
         };
         // (pixel counts are below 2^31: 32-bit index arithmetic; only bit offsets need 64 bits)
         const uint32_t rows32 = (uint32_t)a.rows, P32 = (uint32_t)a.P, C32 = (uint32_t)a.C;
+        // 4-bit codes and strings (8 codes) that are whole words of the bit string: planes (NCHW) or pixels'
+        // channel vectors (channels-last) of a multiple of 8 elements
+        const bool words4 = bits == 4 && ((NHWC ? C32 : P32) & 7u) == 0;
         auto fetch = [&](int it, Raw& r) {
             const int ti = it / kblocks, kb = it - ti * kblocks;
             const uint32_t row0 = (blockIdx.x + (uint32_t)ti * gridDim.x) * (uint32_t)kABm;
             const uint32_t c0 = (uint32_t)kb * kABk + 8u * cg;
             r.shifts = 0;
+            if (words4) {
+                // 4-bit codes whose strings are whole, aligned words: one load per string, 32-bit arithmetic throughout
+                r.keep = 32;
+                if constexpr (NHWC) {
+                    const uint32_t* src = a.packed + ((size_t)(row0 + rq) * (C32 >> 3) + (c0 >> 3));
+                    const uint32_t stepw = 16u * (C32 >> 3);
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        r.w0[i] = (row0 + rq + 16u * i < rows32 && c0 < C32) ? __ldg(src + (size_t)i * stepw) : 0u;
+                        r.w1[i] = r.w2[i] = 0;
+                    }
+                } else {
+                    const uint32_t gp0 = row0 + 8u * rq;
+                    const uint32_t n0 = gp0 / P32, p0 = gp0 - n0 * P32;
+                    const uint32_t* src = a.packed + ((((size_t)n0 * C32 + c0) * P32 + p0) >> 3);
+                    const uint32_t stepw = P32 >> 3;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {
+                        r.w0[i] = (gp0 < rows32 && c0 + i < C32) ? __ldg(src + (size_t)i * stepw) : 0u;
+                        r.w1[i] = r.w2[i] = 0;
+                    }
+                }
+                return;
+            }
             if constexpr (NHWC) {
                 const uint32_t count = c0 < C32 ? min(8u, C32 - c0) : 0u;
                 r.keep = (int)count * bits;
@@ -528,6 +571,53 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
             }
         };
         auto store = [&](unsigned char* tile, const Raw& r) {
+            if (bits == 4) {
+                // 4-bit codes: a string is the 8 nibbles of one word.  Even and odd nibbles are spread to bytes with two
+                // masks, byte permutes put a pair of codes beside the constant 0x43 (0x43cc is the bf16 number 128 + cc),
+                // and one packed subtraction of 128 leaves the two codes as bf16: 13 instructions for 8 codes.
+                const uint32_t k43 = 0x43434343u, k128 = 0x43004300u;
+                auto two = [&](uint32_t x, uint32_t sel) -> uint32_t {
+                    const uint32_t biased = __byte_perm(x, k43, sel);
+                    const __nv_bfloat162 d = __hsub2(*reinterpret_cast<const __nv_bfloat162*>(&biased),
+                                                     *reinterpret_cast<const __nv_bfloat162*>(&k128));
+                    return *reinterpret_cast<const uint32_t*>(&d);
+                };
+                uint32_t u[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    u[i] = __funnelshift_r(r.w0[i], r.w1[i], (uint32_t)(r.shifts >> (5 * i)) & 31u);
+                    if (r.keep < 32) u[i] &= (1u << r.keep) - 1u;
+                }
+                if constexpr (NHWC) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) {          // string i = row rq + 16 i, its nibbles = 8 channels
+                        const uint32_t lo = u[i] & 0x0F0F0F0Fu, hi = (u[i] >> 4) & 0x0F0F0F0Fu;
+                        const uint32_t x01 = __byte_perm(lo, hi, 0x5140), x23 = __byte_perm(lo, hi, 0x7362);
+                        const uint32_t w[4] = {two(x01, 0x4140), two(x01, 0x4342), two(x23, 0x4140), two(x23, 0x4342)};
+                        a_store_chunk(tile, rq + 16u * i, cg, w);
+                    }
+                } else {
+                    uint32_t w[8][4];                      // [row][pair of channels]
+#pragma unroll
+                    for (int h = 0; h < 4; ++h) {          // strings 2h, 2h + 1 = two channels, nibble j = row 8 rq + j
+                        const uint32_t alo = u[2 * h] & 0x0F0F0F0Fu, ahi = (u[2 * h] >> 4) & 0x0F0F0F0Fu;
+                        const uint32_t blo = u[2 * h + 1] & 0x0F0F0F0Fu, bhi = (u[2 * h + 1] >> 4) & 0x0F0F0F0Fu;
+                        const uint32_t e01 = __byte_perm(alo, blo, 0x5140), e23 = __byte_perm(alo, blo, 0x7362);    // rows 0 2 | 4 6
+                        const uint32_t o01 = __byte_perm(ahi, bhi, 0x5140), o23 = __byte_perm(ahi, bhi, 0x7362);    // rows 1 3 | 5 7
+                        w[0][h] = two(e01, 0x4140);
+                        w[2][h] = two(e01, 0x4342);
+                        w[4][h] = two(e23, 0x4140);
+                        w[6][h] = two(e23, 0x4342);
+                        w[1][h] = two(o01, 0x4140);
+                        w[3][h] = two(o01, 0x4342);
+                        w[5][h] = two(o23, 0x4140);
+                        w[7][h] = two(o23, 0x4342);
+                    }
+#pragma unroll
+                    for (int j = 0; j < 8; ++j) a_store_chunk(tile, 8u * rq + j, cg, w[j]);
+                }
+                return;
+            }
             uint64_t v[8];
 #pragma unroll
             for (int i = 0; i < 8; ++i)
@@ -560,27 +650,21 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
                 }
             }
         };
-        // the words of this group's next iteration are in flight while the current one is converted and stored
-        // (two sets of registers, used turn and turn about)
-        Raw ra, rb;
-        auto step = [&](int it, Raw& now, Raw& next) -> bool {
-            if (it + 2 < my_iters) fetch(it + 2, next);
+        // One iteration: load the words, wait for the stage, convert and store, publish.  The latency of the loads is
+        // covered by the other groups' turns, not by loading ahead: a second set of registers for words in flight
+        // cost more (register pressure, and the proxy fence below waits for them anyway) than it brought.
+        Raw r;
+        for (int it = (int)group; it < my_iters; it += kPGroups) {
+            fetch(it, r);
             const int s = it % kPStages;
             // the MMAs that read this stage kPStages iterations ago have completed (passes at once the first time round)
-            if (!warp_wait(&bars.a_empty[s], (uint32_t)(((it / kPStages) & 1) ^ 1))) return false;
-            store(ring + (size_t)s * kABytes, now);
+            if (!warp_wait(&bars.a_empty[s], (uint32_t)(((it / kPStages) & 1) ^ 1))) break;
+            store(ring + (size_t)s * kABytes, r);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");      // the stores above, for the tensor core
             __syncwarp();
             if (lane == 0) a_mbar_arrive(&bars.a_full[s]);
-            return true;
-        };
-        int it = (int)group;
-        if (it < my_iters) fetch(it, ra);
-        for (; it < my_iters; it += 4) {
-            if (!step(it, ra, rb)) break;
-            if (it + 2 < my_iters && !step(it + 2, rb, ra)) break;
         }
-    } else if (warp == 8) {
+    } else if (warp == kPProducers / 32) {
         if (lane == 0) {
             // ---- weights once, then every MMA: per K block 4 steps of 16, each against the hi and the lo half ----
             a_mbar_expect_tx(&bars.b_full, (uint32_t)(2 * kBBytes) * (uint32_t)kblocks);
@@ -588,7 +672,7 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
                 a_tma_load_2d(wts + (size_t)kb * 2 * kBBytes, &map_hi, kb * kABk, col0, &bars.b_full);
                 a_tma_load_2d(wts + (size_t)kb * 2 * kBBytes + kBBytes, &map_lo, kb * kABk, col0, &bars.b_full);
             }
-            const uint32_t idesc = a_instr_desc(BN);
+            const uint32_t idesc = a_instr_desc(2 * BN);        // hi and lo halves as one operand
             bool ok = wait(&bars.b_full, 0);
             int it = 0;
             for (int t = 0; t < my_tiles && ok; ++t) {
@@ -603,13 +687,10 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t dq = a_smem_desc(ring + (size_t)s * kABytes);
-                    const uint64_t dh = a_smem_desc(wts + (size_t)kb * 2 * kBBytes);
-                    const uint64_t dl = a_smem_desc(wts + (size_t)kb * 2 * kBBytes + kBBytes);
+                    const uint64_t dw = a_smem_desc(wts + (size_t)kb * 2 * kBBytes);      // 2 BN rows: hi, then lo
 #pragma unroll
-                    for (int k = 0; k < kABk / 16; ++k) {    // 16 bf16 = 32 bytes = 2 sixteen-byte units along K
-                        a_mma(tmem + buf * BN, dq + 2 * k, dh + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                        a_mma(tmem + buf * BN, dq + 2 * k, dl + 2 * k, idesc, 1u);
-                    }
+                    for (int k = 0; k < kABk / 16; ++k)      // 16 bf16 = 32 bytes = 2 sixteen-byte units along K
+                        a_mma(tmem + buf * (2 * BN), dq + 2 * k, dw + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
                     a_commit(&bars.a_empty[s]);       // the stage may be refilled once these MMAs have read it
                 }
                 if (ok) a_commit(&bars.acc_full[buf]);       // the accumulator is final when this arrives
@@ -619,7 +700,7 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
     } else {
         // ---- epilogue: a warp reads lanes 32 q .. 32 q + 31 (q = warp % 4) and one half of the columns ----
         const uint32_t q = warp & 3u;
-        const int chalf = (int)((warp - 9u) >> 2) * (BN / 2);
+        const int chalf = (int)((warp - (kPProducers / 32 + 1)) >> 2) * (BN / 2);
         for (int t = 0; t < my_tiles; ++t) {
             const uint32_t buf = (uint32_t)(t % kAcc);
             if (!warp_wait(&bars.acc_full[buf], (uint32_t)((t / kAcc) & 1))) break;
@@ -631,49 +712,39 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
             float* const yrow = NHWC ? a.y + (size_t)gp * (size_t)a.O + col0
                                      : a.y + ((size_t)n * (size_t)a.O + col0) * (size_t)a.P + p;
 #pragma unroll 1
-            for (int c = chalf; c < chalf + BN / 2; c += 32) {
-                uint32_t v[32];
-                const uint32_t taddr = tmem + ((q * 32u) << 16) + buf * BN + (uint32_t)c;
-                asm volatile(
-                    "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-                    "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,"
-                    "%29,%30,%31}, [%32];"
-                    : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-                      "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-                      "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-                      "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-                    : "r"(taddr)
-                    : "memory");
+            for (int c = chalf; c < chalf + BN / 2; c += 16) {
+                uint32_t vh[16], vl[16];
+                const uint32_t taddr = tmem + ((q * 32u) << 16) + buf * (2 * BN) + (uint32_t)c;
+                a_tmem_ld16(taddr, vh);              // the hi half's sums
+                a_tmem_ld16(taddr + BN, vl);         // the lo half's
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (c + 32 >= chalf + BN / 2) {          // this warp's part is in registers: hand the accumulator back
+                if (c + 16 >= chalf + BN / 2) {          // this warp's part is in registers: hand the accumulator back
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) a_mbar_arrive(&bars.acc_empty[buf]);
                 }
+                float f[16];
+#pragma unroll
+                for (int j = 0; j < 16; ++j)
+                    f[j] = __fsub_rn(__fadd_rn(__uint_as_float(vh[j]), __uint_as_float(vl[j])), s_bias[c + j]);
                 if (live) {
                     if constexpr (NHWC) {
                         float* out = yrow + c;
-                        if ((a.O & 3) == 0 && col0 + c + 32 <= a.O && ((uintptr_t)a.y & 15) == 0) {      // 16-byte aligned rows
+                        if ((a.O & 3) == 0 && col0 + c + 16 <= a.O && ((uintptr_t)a.y & 15) == 0) {      // 16-byte aligned rows
 #pragma unroll
-                            for (int j = 0; j < 32; j += 4) {
-                                float4 f;
-                                f.x = __fsub_rn(__uint_as_float(v[j]), s_bias[c + j]);
-                                f.y = __fsub_rn(__uint_as_float(v[j + 1]), s_bias[c + j + 1]);
-                                f.z = __fsub_rn(__uint_as_float(v[j + 2]), s_bias[c + j + 2]);
-                                f.w = __fsub_rn(__uint_as_float(v[j + 3]), s_bias[c + j + 3]);
-                                *reinterpret_cast<float4*>(out + j) = f;
-                            }
+                            for (int j = 0; j < 16; j += 4)
+                                *reinterpret_cast<float4*>(out + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
                         } else {
 #pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (col0 + c + j < a.O) out[j] = __fsub_rn(__uint_as_float(v[j]), s_bias[c + j]);
+                            for (int j = 0; j < 16; ++j)
+                                if (col0 + c + j < a.O) out[j] = f[j];
                         }
                     } else {
                         float* out = yrow + (size_t)c * (size_t)a.P;
                         const int left = (int)a.O - col0 - c;          // channels of this chunk that exist
 #pragma unroll
-                        for (int j = 0; j < 32; ++j) {
-                            if (j < left) *out = __fsub_rn(__uint_as_float(v[j]), s_bias[c + j]);
+                        for (int j = 0; j < 16; ++j) {
+                            if (j < left) *out = f[j];
                             out += (uint32_t)a.P;
                         }
                     }
@@ -683,7 +754,7 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
-    if (warp == 8)
+    if (warp == kPProducers / 32)
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)kPTmemCols)
                      : "memory");
 }
@@ -826,7 +897,13 @@ extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_
     __nv_bfloat16* hi = (__nv_bfloat16*)(ws + L.off_hi);
     __nv_bfloat16* lo = (__nv_bfloat16*)(ws + L.off_lo);
     float* bias = (float*)(ws + L.off_bias);
-    const int BN = out_channels <= 64 ? 64 : 128;
+    // Output channels per tile: 128 when there are more than 64 of them, unless only the narrower tile lets the
+    // weight halves of all K blocks stay resident in shared memory (the persistent kernel's condition).
+    const int kblocks = (int)((L.Cpad + kABk - 1) / kABk);
+    auto resident = [&](int bn) { return (size_t)kblocks * 2 * bn * kABk * 2 <= kPWeightBytes; };
+    const bool one_tile_per_cta = (flags & GRANQ_FLAG_FORCE_TWO_PASS) != 0;
+    int BN = out_channels <= 64 ? 64 : 128;
+    if (!one_tile_per_cta && BN == 128 && !resident(128) && resident(64)) BN = 64;
     CUtensorMap mh, ml;
     if (!a_make_map(encode, &mh, hi, (uint64_t)out_channels, (uint64_t)L.Cpad, (uint32_t)BN) ||
         !a_make_map(encode, &ml, lo, (uint64_t)out_channels, (uint64_t)L.Cpad, (uint32_t)BN))
@@ -848,11 +925,10 @@ extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_
     args.C = L.C;
     args.O = out_channels;
     args.bits = bits;
-    args.kblocks = (int)((L.Cpad + kABk - 1) / kABk);
+    args.kblocks = kblocks;
     args.spin_limit = kASpin;
     args.stages = std::min(args.kblocks, 2);
-    const bool persistent = !(flags & GRANQ_FLAG_FORCE_TWO_PASS) &&
-                            (size_t)args.kblocks * 2 * BN * kABk * 2 <= kPWeightBytes;
+    const bool persistent = !one_tile_per_cta && resident(BN);
     if (persistent) {
         if (channel_axis == 3)
             e = BN == 64 ? p_launch<64, true>(mh, ml, args, st) : p_launch<128, true>(mh, ml, args, st);
