@@ -319,11 +319,18 @@ int granq_dequantize_packed(const uint32_t* packed_codes, int dtype, const int64
  *   scale, zp     in   C floats each (per-channel, as written by granq_quantize_packed())
  *   weights       in   fp32 [out_channels, C], row-major
  *   y             out  fp32, [N, out_channels, H, W] for channel_axis 1, [N, H, W, out_channels] for 3
- *   workspace          DEVICE scratch of granq_accumulate_workspace_bytes(), 256-byte aligned; its first word
- *                      is a status word as described at granq_workspace_status()
+ *   workspace          DEVICE scratch of granq_accumulate_workspace_bytes() (the two weight halves and the bias:
+ *                      the codes are expanded to bf16 inside the contraction kernel and never exist as a matrix
+ *                      in device memory), 256-byte aligned; its first word is a status word as described at
+ *                      granq_workspace_status()
+ *   flags              0, or GRANQ_FLAG_FORCE_TWO_PASS for the kernel with one pixel tile per CTA instead of the
+ *                      persistent one (which is taken whenever the weight halves of all channels fit in shared
+ *                      memory, and holds all of an SM's tensor memory while it runs)
+ * Two launches on `cuda_stream` (weights, then expansion + contraction + epilogue) after a 4-byte clear of the
+ * status word.
  * Result: within (2^-17 + C * 2^-22) * sum_c |w s_c| (code + |z_c|) + 2^-21 * (|bias| + |y|) of the exact sum
- * (the split of the scaled weights, fp32 accumulation of 2 C products in any order, one rounding each of bias
- * and y).
+ * (the split of the scaled weights, fp32 accumulation of the C products of each half in any order, the sum of
+ * the two halves, one rounding each of bias and y).
  * Limits: fewer than 2^31 pixels in the batch, C < 2^20, out_channels < 2^24; otherwise GRANQ_ERR_INVALID_ARG.
  */
 size_t granq_accumulate_workspace_bytes(const int64_t dims[4], int channel_axis, int64_t out_channels);
