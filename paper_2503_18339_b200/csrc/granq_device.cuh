@@ -258,7 +258,9 @@ __device__ __forceinline__ float tie_threshold(float z) {
 // Quantize one pack: elements [0, n1) belong to the group with parameters g1, the rest to
 // g2 (n1 = V when the pack lies in one group).  EXTRAS = 1 also packs the codes and the mask
 // (one byte per element); EXTRAS = 2 leaves the codes out and returns the mask as V bits in mb[0]
-// (bit i: the clamp was inactive for element i), which is all the packed mask needs.  SELF: the range is that of the tensor itself, so x / s + z lies within
+// (bit i: the clamp was inactive for element i), which is all the packed mask needs; EXTRAS = 3 returns
+// only the codes, one byte per element, taken from the low mantissa bits of code + 2^23 instead of a
+// float-to-integer conversion (packed-code output).  SELF: the range is that of the tensor itself, so x / s + z lies within
 // [-1, qmax + 1] already (x in [lo, hi] gives RN(x / s) - round(RN(lo / s)) >= -1/2, and at most qmax plus a few
 // units in the last place of hi / s < 2^33 above that) and the clamp before the rounding can go.
 template <typename T, bool BWD, bool SPLIT, int EXTRAS, bool SELF = false>
@@ -282,6 +284,8 @@ __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& 
             mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
         } else if constexpr (EXTRAS == 2) {
             mb[0] |= in ? (1u << i) : 0u;
+        } else if constexpr (EXTRAS == 3) {
+            cb[i / 4] |= (__float_as_uint(__fadd_rn(q, 8388608.0f)) & 0xFFu) << (8 * (i % 4));
         }
     };
     auto exact_round = [&](float t, float z) -> float {        // t = RN(x / s): the sequence as defined

@@ -289,7 +289,9 @@ __device__ __forceinline__ void warp_pack_row(uint64_t mine, uint32_t nb, uint32
 // EXTRAS = 1: the optional codes / mask / packed-mask outputs are compiled in; 2: the packed mask alone.  The packed mask holds
 // one bit per element (bit e % 32 of word e / 32): a warp's lanes own consecutive elements or packs
 // starting at a multiple of 32 elements, so whole words are assembled with warp shuffles.
-// PACKONLY: the packed integer codes are the only output (everything else is compiled out).
+// PACKONLY: the packed integer codes are the only output (everything else is compiled out).  With EXTRAS = 3
+// (tensors of a multiple of 32 elements) the bit string is written 8 codes = b bytes at a time by every second
+// fp32 lane (every bf16 lane) with plain stores: no word assembly across the warp.
 // RAGGED: planes are not whole 16-byte packs (7x7 planes), so a pack may straddle two planes and takes the
 // parameters of both (planes of at least one pack: never more than two).
 template <typename T, int V, int MODE, int EXTRAS, bool PACKONLY = false, bool RAGGED = false>
@@ -407,7 +409,21 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                         }
                     }
                     quantize_pack<T, kBwd, RAGGED, EXTRAS>(px[j], pg[j], gp, gp2, n1, qmax, py, pgx, cb, mb);
-                    if constexpr (EXTRAS != 0) {
+                    if constexpr (EXTRAS == 3) {
+                        // V codes of b bits from V bytes (32-bit arithmetic while the string fits one word)
+                        if (code_bits == 8) {
+                            code_string = cb[0];
+                            if constexpr (V == 8) code_string |= (uint64_t)cb[1] << 32;
+                        } else {
+#pragma unroll
+                            for (int h = 0; h < V / 4; ++h) {
+                                uint32_t four = 0;
+#pragma unroll
+                                for (int i = 0; i < 4; ++i) four |= ((cb[h] >> (8 * i)) & 0xFFu) << (i * code_bits);
+                                code_string |= (uint64_t)four << (h * 4 * code_bits);
+                            }
+                        }
+                    } else if constexpr (EXTRAS != 0) {
                         if constexpr (!PACKONLY) inside_bits = mask_bits_of<V, EXTRAS>(mb);
                         if constexpr (kFwd && EXTRAS == 1) {
                             if constexpr (!PACKONLY) {
@@ -455,7 +471,34 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                             if ((lane & (kLanes - 1)) == 0 && valid) pmask[word] = w;
                         }
                     }
-                    if (EXTRAS == 1 && (PACKONLY || pcodes)) {      // the warp's 32 * V codes are V * b whole words of the bit string
+                    if constexpr (EXTRAS == 3) {
+                        // 8 consecutive codes are b whole bytes of the bit string, at byte (first element / 8) * b
+                        const uint32_t lane = threadIdx.x & 31;
+                        uint64_t eight = code_string;
+                        if constexpr (V == 4) {
+                            const uint32_t next = __shfl_down_sync(kFullMask, (uint32_t)code_string, 1);
+                            eight |= (uint64_t)next << (4 * code_bits);
+                        }
+                        if (valid && (V == 8 || !(lane & 1))) {
+                            uint8_t* dst = reinterpret_cast<uint8_t*>(pcodes) + ((e0 + k[j]) >> 3) * code_bits;
+                            switch (code_bits) {
+                                case 8:          // (the buffer is only known to be 4-byte aligned)
+                                    reinterpret_cast<uint32_t*>(dst)[0] = (uint32_t)eight;
+                                    reinterpret_cast<uint32_t*>(dst)[1] = (uint32_t)(eight >> 32);
+                                    break;
+                                case 4: *reinterpret_cast<uint32_t*>(dst) = (uint32_t)eight; break;
+                                case 2: *reinterpret_cast<uint16_t*>(dst) = (uint16_t)eight; break;
+                                case 6:
+                                    reinterpret_cast<uint16_t*>(dst)[0] = (uint16_t)eight;
+                                    reinterpret_cast<uint16_t*>(dst)[1] = (uint16_t)(eight >> 16);
+                                    reinterpret_cast<uint16_t*>(dst)[2] = (uint16_t)(eight >> 32);
+                                    break;
+                                default:
+                                    for (int t = 0; t < code_bits; ++t) dst[t] = (uint8_t)(eight >> (8 * t));
+                                    break;
+                            }
+                        }
+                    } else if (EXTRAS == 1 && (PACKONLY || pcodes)) {      // the warp's 32 * V codes are V * b whole words of the bit string
                         const uint32_t lane = threadIdx.x & 31;
                         const uint32_t nb = (uint32_t)(V * code_bits);
                         const int64_t row_e = e0 + k0 + (int64_t)(j * kThreads + (threadIdx.x & ~31u)) * V;
@@ -715,6 +758,17 @@ cudaError_t quant_flat_t(const QuantIO& io, const Geom& g, int bits, const float
                         aligned16(io.gy) && aligned16(io.y) && aligned16(io.gx) && ((uintptr_t)io.codes % 4 == 0) &&
                         ((uintptr_t)io.mask % 4 == 0);
     if constexpr (MODE == MODE_FWD) {
+        if ((vec || ragged) && pack_only && g.E % 32 == 0) {       // whole words of codes: the byte-wise writer
+            if (vec)
+                quant_flat_kernel<T, VF, MODE, 3, true><<<grid, kThreads, 0, st>>>(
+                    (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
+                    io.code_bits, f, qmax, lo, hi);
+            else
+                quant_flat_kernel<T, VF, MODE, 3, true, true><<<grid, kThreads, 0, st>>>(
+                    (const T*)io.x, (const T*)io.gy, (T*)io.y, (T*)io.gx, io.codes, io.mask, io.pmask, io.dist, io.pcodes,
+                    io.code_bits, f, qmax, lo, hi);
+            return cudaGetLastError();
+        }
         if ((vec || ragged) && pack_only) {
             if (vec)
                 quant_flat_kernel<T, VF, MODE, 1, true><<<grid, kThreads, 0, st>>>(
