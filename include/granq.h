@@ -286,6 +286,37 @@ int granq_fakequant_weights(const granq_weight_desc* descs, int n_tensors, int d
                             size_t workspace_bytes, uint32_t flags, void* cuda_stream);
 
 /*
+ * The fused call (Algorithm 1, range step through pre-scale step, + STE backward) for a LIST of activation
+ * tensors in one host call: a layer stack's tensors of one training step (the ResNet-20 mix has 19 of 1-17 MB
+ * each, where the host's per-call cost, not the GPU, sets the pace).  Tensor i is processed exactly as
+ * granq_fakequant_fused(descs[i].x, descs[i].gy_opt, dtype, descs[i].dims, channel_axis, group, descs[i].bits,
+ * ..., NULL codes, NULL mask, ..., flags, cuda_stream) would, in order, on the same stream; the results are
+ * bit for bit those of the single calls.
+ *   descs       HOST array of n_tensors descriptors; pointers inside are DEVICE memory, owned by the caller;
+ *               every tensor has its own workspace of granq_workspace_bytes() (they may not share one: the
+ *               kernels of consecutive tensors overlap on the GPU)
+ *   failed_opt  HOST int or NULL: receives the index of the tensor whose call failed (-1 if none)
+ * Returns the first non-OK status; the tensors before the failing one have been enqueued, none after it.
+ */
+typedef struct granq_fused_desc {
+    const void* x;
+    const void* gy_opt;
+    void* y;
+    void* gx_opt;
+    float* min_out;
+    float* max_out;
+    float* scale_opt;
+    float* zp_opt;
+    void* workspace;
+    size_t workspace_bytes;
+    int64_t dims[4];
+    int32_t bits;
+    int32_t reserved;
+} granq_fused_desc;
+int granq_fakequant_fused_batch(const granq_fused_desc* descs, int n_tensors, int dtype, int channel_axis, int group,
+                                uint32_t flags, void* cuda_stream, int* failed_opt);
+
+/*
  * Integer codes as a packed bit string (Eq. 1 yields b-bit integers; Eq. 6 and the accumulation of
  * Algorithm 1 consume them together with the per-group scale and zero-point).  Element e occupies bits
  * [e*b, (e+1)*b) of a little-endian bit string (bit k of the string = bit k % 32 of word k / 32);

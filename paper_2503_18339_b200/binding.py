@@ -39,7 +39,7 @@ EXPORTS = [
     "granq_host_arena_status", "granq_distortion", "granq_fakequant_fused_stats",
     "granq_weights_workspace_bytes", "granq_fakequant_weights", "granq_packed_codes_bytes",
     "granq_quantize_packed", "granq_dequantize_packed", "granq_cluster_geometry", "granq_distortion_stats",
-    "granq_accumulate_workspace_bytes", "granq_accumulate_codes",
+    "granq_accumulate_workspace_bytes", "granq_accumulate_codes", "granq_fakequant_fused_batch",
 ]
 NOALLOC_MAX_GROUPS = 32768
 
@@ -59,6 +59,15 @@ class WeightDesc(ctypes.Structure):
                 ("gx_opt", ctypes.c_void_p), ("min_out", ctypes.c_void_p), ("max_out", ctypes.c_void_p),
                 ("scale_opt", ctypes.c_void_p), ("zp_opt", ctypes.c_void_p), ("channels", ctypes.c_int64),
                 ("group_elems", ctypes.c_int64), ("bits", ctypes.c_int32), ("reserved", ctypes.c_int32)]
+
+
+class FusedDesc(ctypes.Structure):
+    """granq_fused_desc of include/granq.h."""
+    _fields_ = [("x", ctypes.c_void_p), ("gy_opt", ctypes.c_void_p), ("y", ctypes.c_void_p),
+                ("gx_opt", ctypes.c_void_p), ("min_out", ctypes.c_void_p), ("max_out", ctypes.c_void_p),
+                ("scale_opt", ctypes.c_void_p), ("zp_opt", ctypes.c_void_p), ("workspace", ctypes.c_void_p),
+                ("workspace_bytes", ctypes.c_size_t), ("dims", ctypes.c_int64 * 4), ("bits", ctypes.c_int32),
+                ("reserved", ctypes.c_int32)]
 
 
 def lib() -> ctypes.CDLL:
@@ -101,6 +110,9 @@ def lib() -> ctypes.CDLL:
         L.granq_distortion_stats.restype = ci
         L.granq_distortion_stats.argtypes = [ctypes.POINTER(ctypes.c_double), ctypes.POINTER(ctypes.c_double),
                                              ctypes.POINTER(ctypes.c_double)]
+        L.granq_fakequant_fused_batch.restype = ci
+        L.granq_fakequant_fused_batch.argtypes = [ctypes.POINTER(FusedDesc), ci, ci, ci, ci, u32, vp,
+                                                  ctypes.POINTER(ci)]
         L.granq_accumulate_workspace_bytes.restype = sz
         L.granq_accumulate_workspace_bytes.argtypes = [i64p, ci, ctypes.c_int64]
         L.granq_accumulate_codes.restype = ci
@@ -406,6 +418,56 @@ def granq_fakequant_bwd_packmask(gy: torch.Tensor, packed_mask: torch.Tensor, gx
                                               _dims(gy.shape), _dev(gx, "gx"), flags, _stream(stream)),
            "granq_fakequant_bwd_packmask")
     return gx
+
+
+class FusedBatch:
+    """A list of tensors for granq_fakequant_fused_batch(): descriptors are marshalled once, run() is one C call.
+    items: (x, bits, gy or None) triples of one dtype; outputs are allocated here (or taken from `outs`)."""
+
+    def __init__(self, items, channel_axis: int = 1, group: int = GROUP_CHANNEL, outs=None, want_params: bool = False,
+                 zeroed: bool = False):
+        if not items:
+            raise ValueError("no tensors")
+        self.channel_axis, self.group = channel_axis, group
+        self.dtype = _dtype(items[0][0])
+        self.items = list(items)
+        self.outs = []
+        self.flags = FLAG_WORKSPACE_ZEROED if zeroed else 0
+        self._descs = (FusedDesc * len(self.items))()
+        for i, (x, bits, gy) in enumerate(self.items):
+            if _dtype(x) != self.dtype:
+                raise ValueError("all tensors of a batch have one dtype")
+            o = outs[i] if outs is not None else FakeQuantOut()
+            G = num_groups(x.shape, channel_axis, group)
+            if o.y is None:
+                o.y = _new_like(x)
+            if gy is not None and o.gx is None:
+                o.gx = _new_like(x)
+            if o.lo is None:
+                o.lo = _new(G, torch.float32, x.device)
+            if o.hi is None:
+                o.hi = _new(G, torch.float32, x.device)
+            if want_params and o.s is None:
+                o.s = _new(G, torch.float32, x.device)
+                o.z = _new(G, torch.float32, x.device)
+            if o.workspace is None:
+                o.workspace = make_workspace(x, channel_axis, group, zeroed=zeroed)
+            d = self._descs[i]
+            d.x, d.gy_opt, d.y, d.gx_opt = _dev(x, "x"), _dev(gy, "gy"), _dev(o.y, "y"), _dev(o.gx, "gx")
+            d.min_out, d.max_out, d.scale_opt, d.zp_opt = _dev(o.lo, "lo"), _dev(o.hi, "hi"), _dev(o.s, "s"), _dev(o.z, "z")
+            d.workspace, d.workspace_bytes = _dev(o.workspace, "workspace"), o.workspace.numel()
+            for k in range(4):
+                d.dims[k] = int(x.shape[k])
+            d.bits = int(bits)
+            self.outs.append(o)
+
+    def run(self, stream=None, flags: int = 0):
+        failed = ctypes.c_int(-1)
+        rc = lib().granq_fakequant_fused_batch(self._descs, len(self.items), self.dtype, self.channel_axis, self.group,
+                                               self.flags | flags, _stream(stream), ctypes.byref(failed))
+        if rc != OK:
+            raise GranqError(rc, f"granq_fakequant_fused_batch (tensor {failed.value})")
+        return self.outs
 
 
 def granq_fakequant_fused_fwd_packmask(x: torch.Tensor, bits: int, channel_axis: int = 1,

@@ -331,6 +331,23 @@ int granq_fakequant_fused_fwd_packmask(const void* x, int dtype, const int64_t d
     return cuda_status(e);
 }
 
+int granq_fakequant_fused_batch(const granq_fused_desc* descs, int n_tensors, int dtype, int channel_axis, int group,
+                                uint32_t flags, void* cuda_stream, int* failed_opt) {
+    if (failed_opt) *failed_opt = -1;
+    if (!descs || n_tensors < 0) return GRANQ_ERR_INVALID_ARG;
+    for (int i = 0; i < n_tensors; ++i) {
+        const granq_fused_desc& d = descs[i];
+        const int rc = granq_fakequant_fused(d.x, d.gy_opt, dtype, d.dims, channel_axis, group, d.bits, d.y, d.gx_opt,
+                                             d.min_out, d.max_out, nullptr, nullptr, d.scale_opt, d.zp_opt, d.workspace,
+                                             d.workspace_bytes, flags, cuda_stream);
+        if (rc != GRANQ_OK) {
+            if (failed_opt) *failed_opt = i;
+            return rc;
+        }
+    }
+    return GRANQ_OK;
+}
+
 int granq_distortion(const void* x, const void* q, int dtype, const int64_t dims[4], double* sums_out,
                      uint32_t flags, void* cuda_stream) {
     (void)flags;
