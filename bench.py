@@ -696,7 +696,7 @@ def main():
                 flops = 2.0 * pix * s.shape[1] * oc * 2                          # two bf16 halves of the weights
                 rows.append({"tensor": s.name, "out_channels": oc, "us": round(ta, 1),
                              "frac_measured_hbm": round(alg / ta / 1e3 / peak, 3), "tflops": round(flops / ta / 1e6, 1),
-                             "note": "three launches: weights, codes -> bf16 channels-last, contraction"})
+                             "note": "two launches: weights (scale folded in, hi / lo halves, bias), then code expansion + contraction + epilogue in one persistent kernel"})
             sub["accumulate_codes"] = rows
             # ---- all weight tensors of a network in one launch against one fused call per tensor ----
             rows = []
