@@ -389,8 +389,9 @@ __device__ __forceinline__ void a_tmem_ld16(uint32_t taddr, uint32_t (&v)[16]) {
 //                  it is warps, not issue slots, that are short);
 //   warp  16       one thread loads both weight halves for all K blocks once (TMA) and issues every MMA
 //                  (4 per K block);
-//   warps 17 .. 24 read a finished accumulator out of tensor memory (a warp reads the 32 lanes of its quarter,
-//                  warp % 4, and one half of the columns), subtract the bias and store y.
+//   warps 17 .. 24 two groups of four warps take the finished accumulators in turn (a warp reads the 32 lanes of
+//                  its quarter, warp % 4, 16 columns of each half at a time), add the halves, subtract the bias and
+//                  store y; while one group stores, the other reads tensor memory.
 // Both weight halves sit one after the other in shared memory and are multiplied as ONE operand of 2 BN columns
 // (an MMA of 128 x 64 x 16 spends its time fetching the 128 x 16 code operand, not computing: with both halves
 // behind one fetch the tensor core is busy half as long); the epilogue adds the two column blocks.
@@ -438,7 +439,7 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
         }
         for (int b = 0; b < kAcc; ++b) {
             a_mbar_init(&bars.acc_full[b], 1);
-            a_mbar_init(&bars.acc_empty[b], kPEpilogue / 32);     // one arrival per epilogue warp
+            a_mbar_init(&bars.acc_empty[b], 4);     // one arrival per warp of the epilogue group that reads it out
         }
         a_mbar_init(&bars.b_full, 1);
         s_abort = 0;
@@ -698,10 +699,10 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
         }
         __syncwarp();
     } else {
-        // ---- epilogue: a warp reads lanes 32 q .. 32 q + 31 (q = warp % 4) and one half of the columns ----
+        // ---- epilogue: a warp reads lanes 32 q .. 32 q + 31 (q = warp % 4) of every second accumulator ----
         const uint32_t q = warp & 3u;
-        const int chalf = (int)((warp - (kPProducers / 32 + 1)) >> 2) * (BN / 2);
-        for (int t = 0; t < my_tiles; ++t) {
+        const int egroup = (int)((warp - (kPProducers / 32 + 1)) >> 2);      // two groups of four warps, tiles in turn
+        for (int t = egroup; t < my_tiles; t += 2) {
             const uint32_t buf = (uint32_t)(t % kAcc);
             if (!warp_wait(&bars.acc_full[buf], (uint32_t)((t / kAcc) & 1))) break;
             asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -712,13 +713,13 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
             float* const yrow = NHWC ? a.y + (size_t)gp * (size_t)a.O + col0
                                      : a.y + ((size_t)n * (size_t)a.O + col0) * (size_t)a.P + p;
 #pragma unroll 1
-            for (int c = chalf; c < chalf + BN / 2; c += 16) {
+            for (int c = 0; c < BN; c += 16) {
                 uint32_t vh[16], vl[16];
                 const uint32_t taddr = tmem + ((q * 32u) << 16) + buf * (2 * BN) + (uint32_t)c;
                 a_tmem_ld16(taddr, vh);              // the hi half's sums
                 a_tmem_ld16(taddr + BN, vl);         // the lo half's
                 asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
-                if (c + 16 >= chalf + BN / 2) {          // this warp's part is in registers: hand the accumulator back
+                if (c + 16 >= BN) {          // this warp's part is in registers: hand the accumulator back
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
                     __syncwarp();
                     if (lane == 0) a_mbar_arrive(&bars.acc_empty[buf]);
