@@ -554,7 +554,21 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
                             r.shifts |= (uint64_t)a_codes8_load(a.packed, bit, (uint32_t)r.keep, a.nwords, r.w0[i], r.w1[i],
                                                                 r.w2[i])
                                         << (5 * i);
-                        } else {                                 // a sample boundary or the end of the batch inside
+                        } else if (P32 >= 8) {
+                            // a sample boundary or the end of the batch inside: the rows up to the boundary are one run of
+                            // this channel's codes in sample n0, the rest the first codes of the channel in sample n0 + 1
+                            const uint32_t live = min(8u, rows32 - gp0), first = min(live, P32 - p0), rest = live - first;
+                            uint32_t x0, x1, x2;
+                            uint32_t sh = a_codes8_load(a.packed, bit, first * (uint32_t)bits, a.nwords, x0, x1, x2);
+                            uint64_t v = a_codes8_finish(x0, x1, x2, sh, (int)first * bits);
+                            if (rest) {
+                                const uint64_t bit2 = (((uint64_t)(n0 + 1) * C32 + c) * P32) * (uint32_t)bits;
+                                sh = a_codes8_load(a.packed, bit2, rest * (uint32_t)bits, a.nwords, x0, x1, x2);
+                                v |= a_codes8_finish(x0, x1, x2, sh, (int)rest * bits) << (first * (uint32_t)bits);
+                            }
+                            r.w0[i] = (uint32_t)v;
+                            r.w1[i] = (uint32_t)(v >> 32);
+                        } else {                                 // planes of fewer than 8 pixels: code by code
                             uint64_t v = 0;
                             for (uint32_t j = 0; j < 8; ++j) {
                                 const uint32_t gp = gp0 + j;
