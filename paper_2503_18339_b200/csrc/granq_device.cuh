@@ -97,6 +97,16 @@ struct Pack<float> {
     uint4 raw;
     __device__ __forceinline__ float get(int i) const { return __uint_as_float((&raw.x)[i]); }
     __device__ __forceinline__ void set(int i, float v) { (&raw.x)[i] = __float_as_uint(v); }
+    __device__ __forceinline__ void set_all(const float (&v)[4]) {
+        raw = make_uint4(__float_as_uint(v[0]), __float_as_uint(v[1]), __float_as_uint(v[2]), __float_as_uint(v[3]));
+    }
+    // element i of g where bit i of `keep` is set, +0 elsewhere (the straight-through gradient)
+    __device__ __forceinline__ void select(const Pack& g, uint32_t keep) {
+        raw.x = (keep & 1u) ? g.raw.x : 0u;
+        raw.y = (keep & 2u) ? g.raw.y : 0u;
+        raw.z = (keep & 4u) ? g.raw.z : 0u;
+        raw.w = (keep & 8u) ? g.raw.w : 0u;
+    }
 };
 
 template <>
@@ -112,6 +122,22 @@ struct Pack<__nv_bfloat16> {
         uint32_t h = (uint32_t)__bfloat16_as_ushort(__float2bfloat16_rn(v));
         uint32_t& w = (&raw.x)[i >> 1];
         w = (i & 1) ? ((w & 0x0000FFFFu) | (h << 16)) : ((w & 0xFFFF0000u) | h);
+    }
+    // eight floats -> eight bf16 (round to nearest even), two per conversion instruction
+    __device__ __forceinline__ void set_all(const float (&v)[8]) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const __nv_bfloat162 h = __floats2bfloat162_rn(v[2 * k], v[2 * k + 1]);      // .x, the low half, = the first
+            (&raw.x)[k] = *reinterpret_cast<const uint32_t*>(&h);
+        }
+    }
+    // element i of g where bit i of `keep` is set, +0 elsewhere: on the raw halves, nothing is converted
+    __device__ __forceinline__ void select(const Pack& g, uint32_t keep) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const uint32_t m = ((keep >> (2 * k)) & 1u ? 0x0000FFFFu : 0u) | ((keep >> (2 * k + 1)) & 1u ? 0xFFFF0000u : 0u);
+            (&raw.x)[k] = (&g.raw.x)[k] & m;
+        }
     }
 };
 
@@ -274,11 +300,13 @@ __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& 
         cb[i] = 0;
         mb[i] = 0;
     }
+    float yv[V];
+    uint32_t keep = 0;                                          // bit i: the clamp was inactive for element i
     auto finish = [&](int i, float r, float s, float z) {      // r: the rounded value, within [-1, qmax + 1]
         const float q = fminf(fmaxf(r, 0.0f), qmax);
         const bool in = (r == q);
-        py.set(i, __fmul_rn(s, __fsub_rn(q, z)));
-        if constexpr (BWD) pgx.set(i, in ? pg.get(i) : 0.0f);
+        yv[i] = __fmul_rn(s, __fsub_rn(q, z));
+        if constexpr (BWD) keep |= in ? (1u << i) : 0u;
         if constexpr (EXTRAS == 1) {
             cb[i / 4] |= (uint32_t)q << (8 * (i % 4));
             mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
@@ -316,6 +344,8 @@ __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& 
             finish(i, exact_round(__fdiv_rn(px.get(i), s), z), s, z);
         }
     }
+    py.set_all(yv);
+    if constexpr (BWD) pgx.select(pg, keep);
 }
 
 // Quantize one pack whose V elements belong to V different groups (channels-last rows), the range being the
@@ -332,6 +362,8 @@ __device__ __forceinline__ void quantize_pack_each(const Pack<T>& px, const Pack
         cb[i] = 0;
         mb[i] = 0;
     }
+    float yv[V];
+    uint32_t keep = 0;
 #pragma unroll
     for (int i = 0; i < V; ++i) {
         const float s = g[i].s, z = g[i].z, rc = g[i].r, x = px.get(i);
@@ -351,13 +383,15 @@ __device__ __forceinline__ void quantize_pack_each(const Pack<T>& px, const Pack
         }
         const float q = fminf(fmaxf(r, 0.0f), qmax);
         const bool in = (r == q);
-        py.set(i, __fmul_rn(s, __fsub_rn(q, z)));
-        if constexpr (BWD) pgx.set(i, in ? pg.get(i) : 0.0f);
+        yv[i] = __fmul_rn(s, __fsub_rn(q, z));
+        if constexpr (BWD) keep |= in ? (1u << i) : 0u;
         if constexpr (EXTRAS) {
             cb[i / 4] |= (uint32_t)q << (8 * (i % 4));
             mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
         }
     }
+    py.set_all(yv);
+    if constexpr (BWD) pgx.select(pg, keep);
 }
 
 // per-lane min / max of elements [first, last) of one pack

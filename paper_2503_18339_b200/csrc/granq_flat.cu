@@ -598,8 +598,7 @@ __global__ void __launch_bounds__(kThreads) bwd_packmask_kernel(const T* __restr
                 store_scalar(gx + e[j], (bits & 1u) ? sg[j] : 0.0f);
             } else {
                 Pack<T> out;
-#pragma unroll
-                for (int i = 0; i < V; ++i) out.set(i, ((bits >> i) & 1u) ? pg[j].get(i) : 0.0f);
+                out.select(pg[j], bits);
                 st_stream_16(gx + e[j], out.raw);
             }
         }
