@@ -306,7 +306,10 @@ __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& 
         const float q = fminf(fmaxf(r, 0.0f), qmax);
         const bool in = (r == q);
         yv[i] = __fmul_rn(s, __fsub_rn(q, z));
-        if constexpr (BWD) keep |= in ? (1u << i) : 0u;
+        if constexpr (BWD) {
+            if constexpr (V == 4) pgx.set(i, in ? pg.get(i) : 0.0f);      // fp32: a select per element is all it takes
+            else keep |= in ? (1u << i) : 0u;                              // bf16: on the raw halves, below
+        }
         if constexpr (EXTRAS == 1) {
             cb[i / 4] |= (uint32_t)q << (8 * (i % 4));
             mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
@@ -345,7 +348,7 @@ __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& 
         }
     }
     py.set_all(yv);
-    if constexpr (BWD) pgx.select(pg, keep);
+    if constexpr (BWD && V != 4) pgx.select(pg, keep);
 }
 
 // Quantize one pack whose V elements belong to V different groups (channels-last rows), the range being the
@@ -384,14 +387,17 @@ __device__ __forceinline__ void quantize_pack_each(const Pack<T>& px, const Pack
         const float q = fminf(fmaxf(r, 0.0f), qmax);
         const bool in = (r == q);
         yv[i] = __fmul_rn(s, __fsub_rn(q, z));
-        if constexpr (BWD) keep |= in ? (1u << i) : 0u;
+        if constexpr (BWD) {
+            if constexpr (V == 4) pgx.set(i, in ? pg.get(i) : 0.0f);
+            else keep |= in ? (1u << i) : 0u;
+        }
         if constexpr (EXTRAS) {
             cb[i / 4] |= (uint32_t)q << (8 * (i % 4));
             mb[i / 4] |= (in ? 1u : 0u) << (8 * (i % 4));
         }
     }
     py.set_all(yv);
-    if constexpr (BWD) pgx.select(pg, keep);
+    if constexpr (BWD && V != 4) pgx.select(pg, keep);
 }
 
 // per-lane min / max of elements [first, last) of one pack
