@@ -418,6 +418,12 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
     constexpr uint32_t kABytes = kABm * kABk * 2, kBBytes = BN * kABk * 2;
     constexpr int kAcc = kPTmemCols / (2 * BN);    // accumulators (each: BN columns for the hi half, BN for the lo half)
     static_assert(kAcc <= 8, "barriers for at most 8 accumulators");
+    // A parity wait tells "the phase before the current one" from "two phases before" no more than a clock tells
+    // noon from midnight: whoever waits for completion k of a barrier must know that completion k - 1 has
+    // happened.  With an even number of accumulators and two epilogue groups taking tiles in turn every
+    // accumulator is read out by one group only, which has itself seen its previous completion; the producers,
+    // who share stages between groups, cannot get a whole turn of the ring ahead of the MMAs they wait for.
+    static_assert(kAcc % 2 == 0 && kPEpilogue == 256, "each accumulator belongs to one of the two epilogue groups");
     extern __shared__ __align__(1024) unsigned char a_smem[];
     __shared__ __align__(8) PBars bars;
     __shared__ float s_bias[BN];

@@ -66,6 +66,9 @@ SHAPES = [   # (N, C, H, W, O)
     (32, 64, 56, 56, 64),     # 784 pixel tiles: a persistent CTA takes five or six, both accumulators and every
                               # stage of the ring come round several times
     (9, 72, 28, 28, 40),      # 56 tiles, 2 K blocks each (the second one 8 channels wide)
+    (40, 128, 56, 56, 128),   # 980 tiles with the 128-channel tile: only two accumulators, which the two epilogue
+                              # groups take in turn six or seven times per CTA (a wait that mistook an earlier
+                              # completion of a barrier for the one it needs would read a stale accumulator here)
 ]
 
 
