@@ -676,8 +676,12 @@ def main():
                                                                        stream=stream), 3, reps=2)
                 td, _ = sustained_us(lambda k: b.granq_dequantize_packed(pc, x.shape, x.dtype, bits, q.s, q.z, y=out.y,
                                                                          stream=stream), 3, reps=2)
+                fo = b.granq_quantize_packed_fused(x, bits, packed_codes=pc, stream=stream)
+                tf, _ = sustained_us(lambda k: b.granq_quantize_packed_fused(x, bits, out=fo, stream=stream), 3, reps=2)
                 rows.append({"tensor": s.name, "bits": bits, "quantize_us": round(tq, 1),
                              "quantize_frac_measured": round(frac(s.numel, 4 + bits / 8, tq), 3),
+                             "fused_range_and_quantize_us": round(tf, 1),
+                             "fused_frac_measured": round(frac(s.numel, 4 + bits / 8, tf), 3),
                              "dequantize_us": round(td, 1), "dequantize_frac_measured": round(frac(s.numel, 4 + bits / 8, td), 3)})
             sub["packed_codes"] = rows
             # ---- the accumulation over the codes on the tensor cores (Eq. 6 left-hand side, pointwise case) ----

@@ -328,6 +328,14 @@ int granq_fakequant_fused_batch(const granq_fused_desc* descs, int n_tensors, in
  *                            NULL, also receives the dequantized values as granq_fakequant_fwd() would.
  * granq_dequantize_packed(): Eq. 6, y = s * (code - z), from the packed codes; bit for bit the y of
  *                            granq_fakequant_fwd() for the same range.
+ * granq_quantize_packed_fused(): the producer of the integer pipeline in one call (Algorithm 1, range step
+ *                            through quantize step): range of x itself -> scale / zero-point -> packed codes; x is
+ *                            read from HBM once where a single-read plan fits (cluster-local kernel, column
+ *                            walk: groups of 8 codes must not straddle slabs and the tensor is a multiple of 32
+ *                            elements), else a range pass, the parameters and an elementwise pass.  The codes
+ *                            are bit for bit those of granq_range() + granq_quantize_packed().  workspace and
+ *                            flags (GRANQ_FLAG_WORKSPACE_ZEROED, GRANQ_FLAG_FORCE_TWO_PASS / _COLWALK / _CLUSTER) as
+ *                            for granq_fakequant_fused().
  */
 size_t granq_packed_codes_bytes(const int64_t dims[4], int bits);
 int granq_quantize_packed(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group, int bits,
@@ -336,6 +344,9 @@ int granq_quantize_packed(const void* x, int dtype, const int64_t dims[4], int c
 int granq_dequantize_packed(const uint32_t* packed_codes, int dtype, const int64_t dims[4], int channel_axis,
                             int group, int bits, const float* scale_in, const float* zp_in, void* y, uint32_t flags,
                             void* cuda_stream);
+int granq_quantize_packed_fused(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group, int bits,
+                                uint32_t* packed_codes, float* min_out, float* max_out, float* scale_out, float* zp_out,
+                                void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream);
 
 /*
  * The accumulation over the integer codes, pointwise (1 x 1) case: Eq. 6 left-hand side and the output

@@ -40,6 +40,7 @@ EXPORTS = [
     "granq_weights_workspace_bytes", "granq_fakequant_weights", "granq_packed_codes_bytes",
     "granq_quantize_packed", "granq_dequantize_packed", "granq_cluster_geometry", "granq_distortion_stats",
     "granq_accumulate_workspace_bytes", "granq_accumulate_codes", "granq_fakequant_fused_batch",
+    "granq_quantize_packed_fused",
 ]
 NOALLOC_MAX_GROUPS = 32768
 
@@ -139,6 +140,8 @@ def lib() -> ctypes.CDLL:
         L.granq_packed_codes_bytes.argtypes = [i64p, ci]
         L.granq_quantize_packed.restype = ci
         L.granq_quantize_packed.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, u32, vp]
+        L.granq_quantize_packed_fused.restype = ci
+        L.granq_quantize_packed_fused.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, vp, vp, vp, sz, u32, vp]
         L.granq_dequantize_packed.restype = ci
         L.granq_dequantize_packed.argtypes = [vp, ci, i64p, ci, ci, ci, vp, vp, vp, u32, vp]
         L.granq_packmask_bytes.restype = sz
@@ -628,6 +631,30 @@ def granq_dequantize_packed(packed_codes: torch.Tensor, shape, dtype: torch.dtyp
 
 def accumulate_workspace_bytes(shape, channel_axis: int, out_channels: int) -> int:
     return int(lib().granq_accumulate_workspace_bytes(_dims(shape), channel_axis, out_channels))
+
+
+def granq_quantize_packed_fused(x: torch.Tensor, bits: int, channel_axis: int = 1, group: int = GROUP_CHANNEL,
+                                packed_codes: torch.Tensor = None, out: FakeQuantOut = None, flags: int = 0,
+                                stream=None) -> FakeQuantOut:
+    """Range of x itself -> scale / zero-point -> integer codes as a bit string, in one call (lo, hi, s, z and
+    packed_codes of the returned record are filled)."""
+    G = num_groups(x.shape, channel_axis, group)
+    o = out if out is not None else FakeQuantOut()
+    dev = x.device
+    for name in ("lo", "hi", "s", "z"):
+        if getattr(o, name) is None:
+            setattr(o, name, _new(G, torch.float32, dev))
+    if packed_codes is not None:
+        o.packed_codes = packed_codes
+    if o.packed_codes is None:
+        o.packed_codes = _new(packed_codes_bytes(x.shape, bits) // 4, torch.int32, dev)
+    if o.workspace is None:
+        o.workspace = make_workspace(x, channel_axis, group)
+    _check(lib().granq_quantize_packed_fused(
+        _dev(x, "x"), _dtype(x), _dims(x.shape), channel_axis, group, bits, _dev(o.packed_codes, "packed_codes"),
+        _dev(o.lo, "lo"), _dev(o.hi, "hi"), _dev(o.s, "s"), _dev(o.z, "z"), _dev(o.workspace, "workspace"),
+        o.workspace.numel(), flags, _stream(stream)), "granq_quantize_packed_fused")
+    return o
 
 
 def granq_accumulate_codes(packed_codes: torch.Tensor, shape, bits: int, s: torch.Tensor, z: torch.Tensor,

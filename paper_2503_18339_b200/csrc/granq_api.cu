@@ -461,6 +461,53 @@ int granq_quantize_packed(const void* x, int dtype, const int64_t dims[4], int c
     return cuda_status(e);
 }
 
+int granq_quantize_packed_fused(const void* x, int dtype, const int64_t dims[4], int channel_axis, int group, int bits,
+                                uint32_t* packed_codes, float* min_out, float* max_out, float* scale_out, float* zp_out,
+                                void* workspace, size_t workspace_bytes, uint32_t flags, void* cuda_stream) {
+    Geom g;
+    int64_t G;
+    if (!x || !packed_codes || !min_out || !max_out || !scale_out || !zp_out || bits < 1 || bits > 8 ||
+        !dtype_ok(dtype) || !make_geom(dims, channel_axis, group, g, G) || ((uintptr_t)packed_codes & 3))
+        return GRANQ_ERR_INVALID_ARG;
+    if (G >= (1ll << 31)) return GRANQ_ERR_UNSUPPORTED;
+    const size_t nb = (size_t)g.E * elt_size(dtype), cbytes = (size_t)((g.E * bits + 31) / 32) * 4;
+    if (overlaps(x, nb, packed_codes, cbytes)) return GRANQ_ERR_INVALID_ARG;
+    if (int rc = check_workspace(workspace, workspace_bytes, G)) return rc;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    QuantIO io{x, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, nullptr, packed_codes, bits};
+    // the cluster-local kernel where a run of whole groups of 8 codes fits one cluster, the column walk where
+    // slabs and waves are such groups, else range pass, parameters, elementwise pass
+    ColPlan cp{};
+    ClusterPlan kp{};
+    const bool two_pass = (flags & GRANQ_FLAG_FORCE_TWO_PASS) != 0;
+    if (!two_pass && !(flags & GRANQ_FLAG_FORCE_COLWALK)) kp = plan_cluster(dtype, g, io, false, g_tune);
+    if ((flags & GRANQ_FLAG_FORCE_CLUSTER) && !kp.ok) return GRANQ_ERR_UNSUPPORTED;
+    if (!two_pass && !kp.ok) cp = plan_colwalk(dtype, g, io, g_tune);
+    if ((flags & GRANQ_FLAG_FORCE_COLWALK) && !cp.ok) return GRANQ_ERR_UNSUPPORTED;
+    Workspace ws = carve_workspace(workspace, G);
+    const bool zeroed = (flags & GRANQ_FLAG_WORKSPACE_ZEROED) != 0;
+    cudaError_t e = cudaSuccess;
+    if (kp.ok) {
+        if (!zeroed) e = cudaMemsetAsync(workspace, 0, sizeof(uint32_t), st);      // the status word
+        if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+        return cuda_status(launch_cluster(kp, io, MODE_FWD, dtype, g, bits, ws, min_out, max_out, scale_out, zp_out,
+                                          g_tune, st));
+    }
+    if (!(zeroed && cp.ok)) e = cudaMemsetAsync(workspace, 0, ws.clear_bytes, st);
+    if (e != cudaSuccess) return GRANQ_ERR_CUDA;
+    if (cp.ok) {
+        e = launch_colwalk(cp, io, MODE_FWD, dtype, g, bits, ws, min_out, max_out, scale_out, zp_out, g_tune, st);
+    } else {
+        e = launch_range_flat(x, dtype, g, ws.kmin, ws.kmax, st);
+        if (e == cudaSuccess)
+            e = launch_finalize_range(ws.kmin, ws.kmax, G, min_out, max_out, bits, scale_out, zp_out, st);
+        if (e == cudaSuccess) e = launch_quant_flat(io, MODE_FWD, dtype, g, bits, min_out, max_out, st);
+        if (e == cudaSuccess && zeroed)
+            e = cudaMemsetAsync((char*)workspace + sizeof(uint32_t), 0, ws.clear_bytes - sizeof(uint32_t), st);
+    }
+    return cuda_status(e);
+}
+
 int granq_dequantize_packed(const uint32_t* packed_codes, int dtype, const int64_t dims[4], int channel_axis,
                             int group, int bits, const float* scale_in, const float* zp_in, void* y, uint32_t flags,
                             void* cuda_stream) {

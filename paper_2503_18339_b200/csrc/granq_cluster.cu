@@ -43,6 +43,8 @@ struct KArgs {
     uint8_t* codes;
     uint8_t* mask;
     uint32_t* pmask;       // the STE mask at one bit per element, or null (forward plans with whole mask bytes per run)
+    uint32_t* pcodes;      // the codes as a bit string of code_bits each, or null (forward plans; y is then not written)
+    int code_bits;
     double* dist;          // four running sums of Table 2's statistics, or null
     uint32_t* status;
     float* lo;
@@ -438,7 +440,13 @@ __global__ void __launch_bounds__(kKMaxThreads, 2) cluster_kernel(const KArgs a)
         auto emit = [&](const Pack<T>& px, const Pack<T>& pg, size_t at) {
             Pack<T> py, pgx;
             uint32_t cb[V / 4], mb[V / 4];
-            quantize_pack<T, kBwd, !ALIGNED, EXTRAS, true>(px, pg, g1, g2, ne, qmax, py, pgx, cb, mb);
+            quantize_pack<T, kBwd, !ALIGNED, EXTRAS, true>(px, pg, g1, g2, ne, qmax, py, pgx, cb, mb, EXTRAS == 3 ? a.code_bits : 8);
+            if constexpr (EXTRAS == 3) {
+                // the packed codes are the only output: 8 codes = b bytes per pair of fp32 lanes (per bf16 lane); the
+                // planner has made every run and slab whole groups of 8 elements, so both lanes of a pair are here
+                store_code_bytes<V>(a.pcodes, (gbase + at) * V, code_string_of<V>(cb, a.code_bits), a.code_bits, tid & 31);
+                return;
+            }
             st_hint_16(yg + at, py.raw, drop);
             if constexpr (kBwd) st_hint_16(gxg + at, pgx.raw, drop);
             if constexpr (EXTRAS != 0) {
@@ -559,7 +567,7 @@ cudaError_t k_launch_t(const KArgs& args, const ClusterPlan& plan, uint32_t grid
         cfg.numAttrs = plan.early_launch ? 2 : 1;
         return cudaLaunchKernelEx(&cfg, kern, args);
     };
-    if constexpr (EXTRAS == 2) {      // the packed mask alone: forward plans with per-thread copies or plain loads
+    if constexpr (EXTRAS == 2 || EXTRAS == 3) {      // packed mask or packed codes alone: forward plans with per-thread copies or plain loads
         if (plan.load == K_LOAD_ASYNC_X) return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_ASYNC_X, 4, 2>);
         return launch(cluster_kernel<T, MODE, ALIGNED, EXTRAS, K_LOAD_PLAIN, 4, 2>);
     } else {
@@ -579,6 +587,8 @@ cudaError_t k_launch_mode(const KArgs& a, const ClusterPlan& p, bool aligned, in
     if constexpr (MODE == MODE_FWD) {
         if (extras == 2)
             return aligned ? k_launch_t<T, MODE, true, 2>(a, p, grid, st) : k_launch_t<T, MODE, false, 2>(a, p, grid, st);
+        if (extras == 3)
+            return aligned ? k_launch_t<T, MODE, true, 3>(a, p, grid, st) : k_launch_t<T, MODE, false, 3>(a, p, grid, st);
     }
     if (aligned)
         return extras ? k_launch_t<T, MODE, true, 1>(a, p, grid, st) : k_launch_t<T, MODE, true, 0>(a, p, grid, st);
@@ -595,8 +605,11 @@ ClusterPlan plan_cluster(int dtype, const Geom& g, const QuantIO& io, bool backw
     ClusterPlan p{};
     p.ok = false;
     const uint32_t V = dtype == 0 ? 4 : 8, esize = 16 / V;
-    if (io.pcodes) return p;
-    if (io.pmask && (g.C * g.inner) % 8 != 0) return p;
+    // packed codes: forward only, nothing else beside them, whole words of codes (no padding to clear)
+    if (io.pcodes && (backward || io.codes || io.mask || io.pmask || io.dist || ((uintptr_t)io.pcodes & 3) ||
+                      io.code_bits < 1 || io.code_bits > 8 || g.E % 32 != 0))
+        return p;
+    if ((io.pmask || io.pcodes) && (g.C * g.inner) % 8 != 0) return p;
     if (!k_aligned16(io.x) || !k_aligned16(io.gy) || !k_aligned16(io.y) || !k_aligned16(io.gx)) return p;
     if (((uintptr_t)io.codes & 3) || ((uintptr_t)io.mask & 3)) return p;
     if (g.inner < (int64_t)V || g.inner >= (1ll << 24) || g.C >= (1ll << 28) || g.outer >= (1ll << 24)) return p;
@@ -608,7 +621,7 @@ ClusterPlan plan_cluster(int dtype, const Geom& g, const QuantIO& io, bool backw
     // bf16 halves the bytes per element, and reading gy in the quantize walk measured faster).
     const uint64_t limit = tune.cl_tile_kb > 0 ? (uint64_t)tune.cl_tile_kb * 1024 : 112ull * 1024;   // two CTAs per SM
     // a run is whole 16-byte units; with a packed mask also whole bytes of mask (8 elements)
-    const uint32_t unit = io.pmask ? 8u : V;
+    const uint32_t unit = (io.pmask || io.pcodes) ? 8u : V;
     const uint64_t group_bytes = (uint64_t)g.outer * (unit / k_gcd((uint32_t)g.inner, unit)) * g.inner * esize;
     switch (tune.cl_load) {
         case 1: p.load = K_LOAD_BULK_X; break;
@@ -621,7 +634,7 @@ ClusterPlan plan_cluster(int dtype, const Geom& g, const QuantIO& io, bool backw
             break;
     }
     // the two lanes that assemble a byte of mask must both be there: only the variants without a give-up path qualify
-    if (io.pmask && p.load != K_LOAD_ASYNC_X && p.load != K_LOAD_ASYNC_XG && p.load != K_LOAD_PLAIN) return p;
+    if ((io.pmask || io.pcodes) && p.load != K_LOAD_ASYNC_X && p.load != K_LOAD_ASYNC_XG && p.load != K_LOAD_PLAIN) return p;
     const uint64_t tiles = (p.load == K_LOAD_BULK_XG || p.load == K_LOAD_ASYNC_XG) ? 2 : 1;   // staged tiles per CTA
     const uint32_t k0 = unit / k_gcd(inner, unit);
     const uint64_t target = std::min<uint64_t>(limit, 64ull * 1024);
@@ -692,6 +705,8 @@ cudaError_t launch_cluster(const ClusterPlan& plan, const QuantIO& io, int mode,
     a.codes = io.codes;
     a.mask = io.mask;
     a.pmask = io.pmask;
+    a.pcodes = io.pcodes;
+    a.code_bits = io.code_bits;
     a.dist = io.dist;
     a.status = ws.status;
     a.lo = lo;
@@ -714,7 +729,7 @@ cudaError_t launch_cluster(const ClusterPlan& plan, const QuantIO& io, int mode,
     const uint32_t grid = nruns * plan.R;
     const bool aligned = (a.inner % V) == 0;
     // 1: codes / mask bytes / sums compiled in; 2: the packed mask alone (a leaner instantiation of the forward kernel)
-    const int extras = (io.codes != nullptr || io.mask != nullptr || io.dist != nullptr) ? 1 : (io.pmask != nullptr ? 2 : 0);
+    const int extras = (io.codes != nullptr || io.mask != nullptr || io.dist != nullptr) ? 1 : (io.pmask != nullptr ? 2 : (io.pcodes != nullptr ? 3 : 0));
     if (dtype == 0) {
         if (mode == MODE_FWD) return k_launch_mode<float, MODE_FWD>(a, plan, aligned, extras, grid, st);
         return k_launch_mode<float, MODE_BOTH>(a, plan, aligned, extras, grid, st);

@@ -52,6 +52,8 @@ struct CArgs {
     uint8_t* codes;
     uint8_t* mask;
     uint32_t* pmask;       // mask at one bit per element, or null
+    uint32_t* pcodes;      // the codes as a bit string of code_bits each, or null (forward calls; y is then not written)
+    int code_bits;
     double* dist;          // four running sums of Table 2's statistics, or null
     uint32_t* status;
     uint32_t* kmin;
@@ -307,7 +309,13 @@ __global__ void __launch_bounds__(kCThreads, 4) colwalk_kernel(const CArgs a) {
             auto emit = [&](const Pack<T>& px, const Pack<T>& pg, size_t at) {
                 Pack<T> py, pgx;
                 uint32_t cb[V / 4], mb[V / 4];
-                quantize_pack<T, kBwd, !ALIGNED, EXTRAS, true>(px, pg, g1, g2, it.ne, qmax, py, pgx, cb, mb);
+                quantize_pack<T, kBwd, !ALIGNED, EXTRAS, true>(px, pg, g1, g2, it.ne, qmax, py, pgx, cb, mb, EXTRAS == 3 ? a.code_bits : 8);
+                if constexpr (EXTRAS == 3) {
+                    // the packed codes are the only output: 8 codes = b bytes per pair of fp32 lanes (per bf16 lane);
+                    // the planner has made every slab and wave whole groups of 8 elements
+                    store_code_bytes<V>(a.pcodes, at * V, code_string_of<V>(cb, a.code_bits), a.code_bits, lane);
+                    return;
+                }
                 st_hint_16(yg + at, py.raw, drop);
                 if constexpr (kBwd) st_hint_16(gxg + at, pgx.raw, drop);
                 if constexpr (EXTRAS != 0) {
@@ -463,6 +471,8 @@ cudaError_t c_launch_mode(CArgs& a, bool aligned, int extras, int sms, int cap, 
     if constexpr (MODE == MODE_FWD) {
         if (extras == 2)       // the packed mask alone: a leaner instantiation of the forward kernel
             return aligned ? c_launch_t<T, MODE, true, 2>(a, sms, cap, st) : c_launch_t<T, MODE, false, 2>(a, sms, cap, st);
+        if (extras == 3)       // the packed codes alone
+            return aligned ? c_launch_t<T, MODE, true, 3>(a, sms, cap, st) : c_launch_t<T, MODE, false, 3>(a, sms, cap, st);
     }
     if (aligned)
         return extras ? c_launch_t<T, MODE, true, 1>(a, sms, cap, st) : c_launch_t<T, MODE, true, 0>(a, sms, cap, st);
@@ -488,7 +498,12 @@ ColPlan plan_colwalk(int dtype, const Geom& g, const QuantIO& io, const StagedTu
     const uint32_t inner = (uint32_t)g.inner, C = (uint32_t)g.C;
     // waves are whole 16-byte units; with a packed mask also whole 32-element mask words
     if (io.pmask && (((uintptr_t)io.pmask & 3) || (g.C * g.inner) % 32 != 0)) return p;
-    const uint32_t q = io.pmask ? 32 / c_gcd(inner, 32) : V / c_gcd(inner, V);
+    // packed codes: nothing else beside them, slabs and waves of whole groups of 8 elements, whole words of codes
+    if (io.pcodes && (io.gy || io.codes || io.mask || io.pmask || io.dist || ((uintptr_t)io.pcodes & 3) ||
+                      io.code_bits < 1 || io.code_bits > 8 || (g.C * g.inner) % 8 != 0 || g.E % 32 != 0))
+        return p;
+    const uint32_t q = io.pmask ? 32 / c_gcd(inner, 32) : io.pcodes ? std::max(8 / c_gcd(inner, 8), V / c_gcd(inner, V))
+                                                                    : V / c_gcd(inner, V);
     // x bytes of a wave: 32 MB with a gradient (gy and gx stream through the L2 beside the wave), 64 MB without
     // (measured: 3-6 % faster forward-only; larger waves lose to eviction either way)
     const uint64_t target = (tune.l2_wave_kb > 0 ? (uint64_t)tune.l2_wave_kb : (io.gy ? 32ull : 64ull) * 1024) * 1024;
@@ -568,6 +583,8 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
     a.codes = io.codes;
     a.mask = io.mask;
     a.pmask = io.pmask;
+    a.pcodes = io.pcodes;
+    a.code_bits = io.code_bits;
     a.dist = io.dist;
     a.status = ws.status;
     a.kmin = ws.kmin;
@@ -607,7 +624,7 @@ cudaError_t launch_colwalk(const ColPlan& plan, const QuantIO& io, int mode, int
     }
     a.div_plane = make_fastdiv(aligned ? inner / V : inner);
     // 1: codes / mask bytes / sums compiled in; 2: the packed mask alone
-    const int extras = (io.codes != nullptr || io.mask != nullptr || io.dist != nullptr) ? 1 : (io.pmask != nullptr ? 2 : 0);
+    const int extras = (io.codes != nullptr || io.mask != nullptr || io.dist != nullptr) ? 1 : (io.pmask != nullptr ? 2 : (io.pcodes != nullptr ? 3 : 0));
     const int cap = tune.l2_ctas_per_sm;
     if (dtype == 0) {
         if (mode == MODE_FWD) return c_launch_mode<float, MODE_FWD>(a, aligned, extras, sms, cap, st);

@@ -285,14 +285,16 @@ __device__ __forceinline__ float tie_threshold(float z) {
 // g2 (n1 = V when the pack lies in one group).  EXTRAS = 1 also packs the codes and the mask
 // (one byte per element); EXTRAS = 2 leaves the codes out and returns the mask as V bits in mb[0]
 // (bit i: the clamp was inactive for element i), which is all the packed mask needs; EXTRAS = 3 returns
-// only the codes, one byte per element, taken from the low mantissa bits of code + 2^23 instead of a
-// float-to-integer conversion (packed-code output).  SELF: the range is that of the tensor itself, so x / s + z lies within
+// only the codes, code_bits each (cb[h] = the four codes of half h as a string of 4 * code_bits bits; bytes for
+// the default of 8), taken from the low mantissa bits of code + 2^23 instead of a float-to-integer conversion
+// (packed-code output).  SELF: the range is that of the tensor itself, so x / s + z lies within
 // [-1, qmax + 1] already (x in [lo, hi] gives RN(x / s) - round(RN(lo / s)) >= -1/2, and at most qmax plus a few
 // units in the last place of hi / s < 2^33 above that) and the clamp before the rounding can go.
 template <typename T, bool BWD, bool SPLIT, int EXTRAS, bool SELF = false>
 __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& pg, const GroupParam& g1,
                                               const GroupParam& g2, int n1, float qmax, Pack<T>& py, Pack<T>& pgx,
-                                              uint32_t (&cb)[Pack<T>::V / 4], uint32_t (&mb)[Pack<T>::V / 4]) {
+                                              uint32_t (&cb)[Pack<T>::V / 4], uint32_t (&mb)[Pack<T>::V / 4],
+                                              int code_bits = 8) {
     constexpr int V = Pack<T>::V;
     const float kMagic = 12582912.0f;  // 1.5 * 2^23
 #pragma unroll
@@ -316,7 +318,7 @@ __device__ __forceinline__ void quantize_pack(const Pack<T>& px, const Pack<T>& 
         } else if constexpr (EXTRAS == 2) {
             mb[0] |= in ? (1u << i) : 0u;
         } else if constexpr (EXTRAS == 3) {
-            cb[i / 4] |= (__float_as_uint(__fadd_rn(q, 8388608.0f)) & 0xFFu) << (8 * (i % 4));
+            cb[i / 4] |= (__float_as_uint(__fadd_rn(q, 8388608.0f)) & 0xFFu) << ((i % 4) * code_bits);
         }
     };
     auto exact_round = [&](float t, float z) -> float {        // t = RN(x / s): the sequence as defined
@@ -437,6 +439,45 @@ __device__ __forceinline__ void store_mask_byte(uint32_t* pmask, size_t first, u
     } else {
         static_assert(V == 8, "a pack is 4 or 8 elements");
         reinterpret_cast<uint8_t*>(pmask)[first >> 3] = (uint8_t)bits;
+    }
+}
+
+// The codes of one pack as a string of V * b bits, from the half strings of quantize_pack<EXTRAS = 3>(.., code_bits).
+template <int V>
+__device__ __forceinline__ uint64_t code_string_of(const uint32_t (&cb)[V / 4], int code_bits) {
+    uint64_t str = cb[0];
+    if constexpr (V == 8) str |= (uint64_t)cb[1] << (4 * code_bits);
+    return str;
+}
+
+// Store the packed codes 8 codes = b bytes at a time: `str` is the code string of the pack that starts at element
+// `first` (a multiple of V); byte (first / 8) * b of the bit string is where the 8 codes of an aligned group of 8
+// elements begin.  For V = 4 the even lane of a pair holds the first half and stores; both lanes of the pair must
+// call this together with neighbouring packs.  The buffer is only known to be 4-byte aligned.
+template <int V>
+__device__ __forceinline__ void store_code_bytes(uint32_t* pcodes, size_t first, uint64_t str, int code_bits, uint32_t lane) {
+    uint64_t eight = str;
+    if constexpr (V == 4) {
+        const uint32_t other = __shfl_xor_sync(3u << (lane & ~1u), (uint32_t)str, 1);
+        if (lane & 1) return;
+        eight |= (uint64_t)other << (4 * code_bits);
+    }
+    uint8_t* dst = reinterpret_cast<uint8_t*>(pcodes) + (first >> 3) * (size_t)code_bits;
+    switch (code_bits) {
+        case 8:
+            reinterpret_cast<uint32_t*>(dst)[0] = (uint32_t)eight;
+            reinterpret_cast<uint32_t*>(dst)[1] = (uint32_t)(eight >> 32);
+            break;
+        case 4: *reinterpret_cast<uint32_t*>(dst) = (uint32_t)eight; break;
+        case 2: *reinterpret_cast<uint16_t*>(dst) = (uint16_t)eight; break;
+        case 6:
+            reinterpret_cast<uint16_t*>(dst)[0] = (uint16_t)eight;
+            reinterpret_cast<uint16_t*>(dst)[1] = (uint16_t)(eight >> 16);
+            reinterpret_cast<uint16_t*>(dst)[2] = (uint16_t)(eight >> 32);
+            break;
+        default:
+            for (int t = 0; t < code_bits; ++t) dst[t] = (uint8_t)(eight >> (8 * t));
+            break;
     }
 }
 

@@ -408,21 +408,9 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                             }
                         }
                     }
-                    quantize_pack<T, kBwd, RAGGED, EXTRAS>(px[j], pg[j], gp, gp2, n1, qmax, py, pgx, cb, mb);
+                    quantize_pack<T, kBwd, RAGGED, EXTRAS>(px[j], pg[j], gp, gp2, n1, qmax, py, pgx, cb, mb, EXTRAS == 3 ? code_bits : 8);
                     if constexpr (EXTRAS == 3) {
-                        // V codes of b bits from V bytes (32-bit arithmetic while the string fits one word)
-                        if (code_bits == 8) {
-                            code_string = cb[0];
-                            if constexpr (V == 8) code_string |= (uint64_t)cb[1] << 32;
-                        } else {
-#pragma unroll
-                            for (int h = 0; h < V / 4; ++h) {
-                                uint32_t four = 0;
-#pragma unroll
-                                for (int i = 0; i < 4; ++i) four |= ((cb[h] >> (8 * i)) & 0xFFu) << (i * code_bits);
-                                code_string |= (uint64_t)four << (h * 4 * code_bits);
-                            }
-                        }
+                        code_string = code_string_of<V>(cb, code_bits);
                     } else if constexpr (EXTRAS != 0) {
                         if constexpr (!PACKONLY) inside_bits = mask_bits_of<V, EXTRAS>(mb);
                         if constexpr (kFwd && EXTRAS == 1) {
@@ -472,31 +460,11 @@ __global__ void __launch_bounds__(kThreads) quant_flat_kernel(const T* __restric
                         }
                     }
                     if constexpr (EXTRAS == 3) {
-                        // 8 consecutive codes are b whole bytes of the bit string, at byte (first element / 8) * b
-                        const uint32_t lane = threadIdx.x & 31;
-                        uint64_t eight = code_string;
-                        if constexpr (V == 4) {
-                            const uint32_t next = __shfl_down_sync(kFullMask, (uint32_t)code_string, 1);
-                            eight |= (uint64_t)next << (4 * code_bits);
-                        }
-                        if (valid && (V == 8 || !(lane & 1))) {
-                            uint8_t* dst = reinterpret_cast<uint8_t*>(pcodes) + ((e0 + k[j]) >> 3) * code_bits;
-                            switch (code_bits) {
-                                case 8:          // (the buffer is only known to be 4-byte aligned)
-                                    reinterpret_cast<uint32_t*>(dst)[0] = (uint32_t)eight;
-                                    reinterpret_cast<uint32_t*>(dst)[1] = (uint32_t)(eight >> 32);
-                                    break;
-                                case 4: *reinterpret_cast<uint32_t*>(dst) = (uint32_t)eight; break;
-                                case 2: *reinterpret_cast<uint16_t*>(dst) = (uint16_t)eight; break;
-                                case 6:
-                                    reinterpret_cast<uint16_t*>(dst)[0] = (uint16_t)eight;
-                                    reinterpret_cast<uint16_t*>(dst)[1] = (uint16_t)(eight >> 16);
-                                    reinterpret_cast<uint16_t*>(dst)[2] = (uint16_t)(eight >> 32);
-                                    break;
-                                default:
-                                    for (int t = 0; t < code_bits; ++t) dst[t] = (uint8_t)(eight >> (8 * t));
-                                    break;
-                            }
+                        // 8 consecutive codes are b whole bytes of the bit string (the tensor is a multiple of 32
+                        // elements, so the lanes of a pair are valid or not together, and a lane without a pack has
+                        // nothing to say)
+                        if constexpr (V > 1) {
+                            if (valid) store_code_bytes<V>(pcodes, (size_t)(e0 + k[j]), code_string, code_bits, threadIdx.x & 31);
                         }
                     } else if (EXTRAS == 1 && (PACKONLY || pcodes)) {      // the warp's 32 * V codes are V * b whole words of the bit string
                         const uint32_t lane = threadIdx.x & 31;

@@ -68,3 +68,51 @@ def test_packed_codes_reject_bad_arguments(b):
         b.granq_quantize_packed(x, 4, lo, hi, packed_codes=buf[1:])
     assert err.value.status == b.ERR_INVALID_ARG
     assert b.packed_codes_bytes((1, 1, 1, 33), 3) == 16 and b.packed_codes_bytes((1, 1, 1, 32), 9) == 0
+
+
+FUSED_SHAPES = [(2, 2, 2, 2), (3, 5, 7, 7), (4, 16, 14, 14), (16, 32, 7, 7), (16, 8, 7, 7), (9, 24, 12, 12), (8, 4, 8, 8),
+                (32, 6, 40, 28), (5, 7, 3, 11), (12, 10, 16, 16)]
+
+
+@pytest.mark.parametrize("shape", FUSED_SHAPES, ids=lambda s: "x".join(map(str, s)))
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_quantize_packed_fused(b, shape, dtype):
+    """Range of the tensor itself -> parameters -> packed codes in one call, on every plan that takes the geometry
+    (cluster-local kernel, column walk, range pass + flat pass), every bit-width, both group modes with planes."""
+    x, _ = make_case(shape, seed=sum(shape) + 21, dtype=dtype, relu=(shape[1] % 2 == 0))
+    taken = set()
+    for mode in (orc.GROUP_CHANNEL, orc.GROUP_SAMPLE_CHANNEL):
+        for bits in range(1, 9):
+            ref = orc.fused(x, bits, group_mode=mode, want_codes=True)
+            want = padded(orc.pack_codes(ref.codes, bits), b.packed_codes_bytes(shape, bits))
+            for flags in (0, b.FLAG_FORCE_TWO_PASS, b.FLAG_FORCE_COLWALK, b.FLAG_FORCE_CLUSTER):
+                try:
+                    got = b.granq_quantize_packed_fused(to_dev(x), bits, group=mode, flags=flags)
+                except b.GranqError as err:
+                    assert flags in (b.FLAG_FORCE_COLWALK, b.FLAG_FORCE_CLUSTER) and err.status == b.ERR_UNSUPPORTED
+                    continue
+                taken.add(flags)
+                assert b.workspace_status(got.workspace) == b.OK
+                assert np.array_equal(got.packed_codes.cpu().numpy().view(np.uint8), want), \
+                    f"bit string differs (mode {mode}, b = {bits}, flags {flags})"
+                assert same_bits(to_np(got.lo), ref.lo) and same_bits(to_np(got.hi), ref.hi)
+                assert same_bits(to_np(got.s), ref.s) and same_bits(to_np(got.z), ref.z)
+    e = int(np.prod(shape))
+    if e % 32 == 0 and (shape[1] * shape[2] * shape[3]) % 8 == 0 and shape[2] * shape[3] >= 8:
+        assert b.FLAG_FORCE_CLUSTER in taken, "the cluster-local kernel must take whole groups of 8 codes"
+        if shape[0] >= 8:
+            assert b.FLAG_FORCE_COLWALK in taken
+
+
+@pytest.mark.parametrize("spec", [wl.config_tensors(3)[1], wl.config_tensors(3)[4], wl.config_tensors(4)[3]],
+                         ids=lambda s: s.name)
+def test_quantize_packed_fused_full_size(b, spec):
+    """Every code of three benchmarked tensors (column walk, cluster-local with 7x7 planes, cluster-local with 28x28)."""
+    x = wl.make_activation(spec)
+    for bits in (3, 4, 5):
+        ref = orc.fused(x, bits, want_codes=True)
+        got = b.granq_quantize_packed_fused(to_dev(x), bits)
+        want = orc.pack_codes(ref.codes, bits)
+        assert b.workspace_status(got.workspace) == b.OK
+        assert np.array_equal(got.packed_codes.cpu().numpy().view(np.uint8)[:want.size], want)
+        assert same_bits(to_np(got.s), ref.s) and same_bits(to_np(got.z), ref.z)
