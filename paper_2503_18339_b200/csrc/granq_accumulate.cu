@@ -405,7 +405,8 @@ constexpr int kPGroups = 4;                // groups of 128 threads that expand 
 constexpr int kPProducers = 128 * kPGroups;
 constexpr int kPEpilogue = 256;           // threads that read accumulators out and store y
 constexpr int kPThreads = kPProducers + 32 + kPEpilogue;
-constexpr size_t kPWeightBytes = 128 * 1024;      // resident weight halves at most
+constexpr size_t kPWeightBytes = 128 * 1024;      // resident weight halves at most (channels-last: 16 KB less,
+                                                  // which the epilogue's staging tiles take)
 
 struct PBars {
     uint64_t a_full[kPStages], a_empty[kPStages], acc_full[8], acc_empty[8], b_full;
@@ -428,6 +429,7 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
     __shared__ __align__(8) PBars bars;
     __shared__ float s_bias[BN];
     __shared__ uint32_t s_tmem, s_abort;
+    __shared__ __align__(16) float4 s_stage[NHWC ? kPEpilogue / 32 : 1][NHWC ? 128 : 1];      // channels-last epilogue
     const uint32_t tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     unsigned char* ring = a_smem + ((1024u - (a_smem_u32(a_smem) & 1023u)) & 1023u);
     unsigned char* wts = ring + (size_t)kPStages * kABytes;          // per K block: hi half, lo half
@@ -748,19 +750,36 @@ accumulate_persistent_kernel(const __grid_constant__ CUtensorMap map_hi, const _
 #pragma unroll
                 for (int j = 0; j < 16; ++j)
                     f[j] = __fsub_rn(__fadd_rn(__uint_as_float(vh[j]), __uint_as_float(vl[j])), s_bias[c + j]);
-                if (live) {
-                    if constexpr (NHWC) {
-                        float* out = yrow + c;
-                        if ((a.O & 3) == 0 && col0 + c + 16 <= a.O && ((uintptr_t)a.y & 15) == 0) {      // 16-byte aligned rows
+                if constexpr (NHWC) {
+                    // channels-last: a thread's 16 values are 64 contiguous bytes of its pixel's row, but the rows of
+                    // neighbouring lanes lie O floats apart: stored straight from the registers, every instruction
+                    // would touch 32 lines.  The warp passes the chunk through a 2 KB staging tile (quads swizzled
+                    // by the row so that neither side has bank conflicts worth naming) and stores 8 rows x 64
+                    // bytes per instruction instead.
+                    const bool vec = (a.O & 3) == 0 && col0 + c + 16 <= a.O && ((uintptr_t)a.y & 15) == 0;      // same for the warp
+                    if (vec) {
+                        float4* stg = s_stage[warp - (kPProducers / 32 + 1)];
+                        __syncwarp();                                   // the previous chunk has been read out
 #pragma unroll
-                            for (int j = 0; j < 16; j += 4)
-                                *reinterpret_cast<float4*>(out + j) = make_float4(f[j], f[j + 1], f[j + 2], f[j + 3]);
-                        } else {
+                        for (int j = 0; j < 4; ++j)
+                            stg[lane * 4 + (j ^ (lane & 3))] = make_float4(f[4 * j], f[4 * j + 1], f[4 * j + 2], f[4 * j + 3]);
+                        __syncwarp();
+                        const uint32_t gp_first = gp - lane, quad = lane & 3;
 #pragma unroll
-                            for (int j = 0; j < 16; ++j)
-                                if (col0 + c + j < a.O) out[j] = f[j];
+                        for (int i = 0; i < 4; ++i) {
+                            const uint32_t row = 8u * i + (lane >> 2);
+                            const float4 v = stg[row * 4 + (quad ^ (row & 3))];
+                            if (gp_first + row < (uint32_t)a.rows)
+                                *reinterpret_cast<float4*>(a.y + (size_t)(gp_first + row) * (size_t)a.O + col0 + c + 4 * quad) = v;
                         }
-                    } else {
+                    } else if (live) {
+                        float* out = yrow + c;
+#pragma unroll
+                        for (int j = 0; j < 16; ++j)
+                            if (col0 + c + j < a.O) out[j] = f[j];
+                    }
+                } else if (live) {
+                    {
                         float* out = yrow + (size_t)c * (size_t)a.P;
                         const int left = (int)a.O - col0 - c;          // channels of this chunk that exist
 #pragma unroll
@@ -921,7 +940,8 @@ extern "C" int granq_accumulate_codes(const uint32_t* packed_codes, const int64_
     // Output channels per tile: 128 when there are more than 64 of them, unless only the narrower tile lets the
     // weight halves of all K blocks stay resident in shared memory (the persistent kernel's condition).
     const int kblocks = (int)((L.Cpad + kABk - 1) / kABk);
-    auto resident = [&](int bn) { return (size_t)kblocks * 2 * bn * kABk * 2 <= kPWeightBytes; };
+    const size_t weight_room = kPWeightBytes - (channel_axis == 3 ? 16 * 1024 : 0);
+    auto resident = [&](int bn) { return (size_t)kblocks * 2 * bn * kABk * 2 <= weight_room; };
     const bool one_tile_per_cta = (flags & GRANQ_FLAG_FORCE_TWO_PASS) != 0;
     int BN = out_channels <= 64 ? 64 : 128;
     if (!one_tile_per_cta && BN == 128 && !resident(128) && resident(64)) BN = 64;
